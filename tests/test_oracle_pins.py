@@ -1,0 +1,459 @@
+"""Pins for the CPU oracle: it is checked here against things other than itself --
+values the paper prints, textbook constants, invariants, brute force in pure Python
+on tiny inputs, and special cases that reduce to a library routine.  CPU only."""
+import math
+import os
+import struct
+
+import numpy as np
+import pytest
+
+from oracle import evaluator as E
+from pn_workloads import configs as C
+from pn_workloads import descriptor as D
+from pn_workloads.descriptor import GraphBuilder, Imm
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _gold(name):
+    rows = []
+    with open(os.path.join(GOLD, name)) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                rows.append(line.split())
+    return rows
+
+
+def run1(op, arrays, dtypes, out_dtype, out_dims, imms=(), attr=(0, 0), extra_imm=()):
+    """Evaluate a one-node graph through the oracle's public entry point."""
+    g = GraphBuilder()
+    ids = [g.input(dt, a.shape) for a, dt in zip(arrays, dtypes)]
+    ins = list(ids) + [Imm(v) for v in imms]
+    o = g.op(op, ins, out_dtype, out_dims, attr=attr, extra_imm=extra_imm)
+    g.mark_output(o)
+    return E.evaluate(g.build(), arrays)[0]
+
+
+def f32(*v):
+    return np.array(v, dtype=np.float32)
+
+
+# ---------------------------------------------------------------------------
+# descriptor format
+# ---------------------------------------------------------------------------
+def test_parser_reads_what_the_writer_wrote():
+    w = C.c5(M=3, N=8)
+    g = E.parse(w.desc)
+    assert [g.tensors[i].dims for i in g.input_ids] == [(3, 8), (3, 8), (1, 8), (3, 1)]
+    assert [n.op for n in g.nodes][-4:] == ["gt", "cast", "mean", "var"]
+    gt = [n for n in g.nodes if n.op == "gt"][0]
+    assert gt.ins[1] == ("imm", 0.0)
+    # hand-assembled bytes for a one-node graph: neg(f32[2]) -> f32[2]
+    raw = struct.pack("<IHHII", 0x31474E50, 1, 0, 2, 1)
+    raw += struct.pack("<BBBBI4q", 0, 1, 1, 0, 0, 2, 0, 0, 0)
+    raw += struct.pack("<BBBBI4q", 0, 2, 1, 0, 0, 2, 0, 0, 0)
+    raw += struct.pack("<HBB4I3I2d2q", 1, 1, 1, 0, 0, 0, 0, 1, 0, 0, 0.0, 0.0, 0, 0)
+    out = E.evaluate(raw, [f32(1.5, -2.0)])[0]
+    assert out.tolist() == [-1.5, 2.0]
+
+
+@pytest.mark.parametrize("mutate", ["short", "magic", "length", "opcode", "operand"])
+def test_parser_rejects_malformed(mutate):
+    good = bytearray(C.c1(M=2, N=4).desc)
+    if mutate == "short":
+        bad = good[:10]
+    elif mutate == "magic":
+        bad = good[:]; bad[0] ^= 0xFF
+    elif mutate == "length":
+        bad = good + b"\0"
+    elif mutate == "opcode":
+        bad = good[:]; struct.pack_into("<H", bad, 16 + 40 * 8, 999)
+    else:
+        bad = good[:]; struct.pack_into("<I", bad, 16 + 40 * 8 + 4, 77)
+    with pytest.raises(ValueError):
+        E.evaluate(bytes(bad), C.c1(M=2, N=4).inputs)
+
+
+# ---------------------------------------------------------------------------
+# activations: textbook constants, symmetries, libm
+# ---------------------------------------------------------------------------
+def test_activation_known_points():
+    x = f32(0.0, 1.0, -1.0, 2.0)
+    ge = run1("gelu_erf", [x], [D.F32], D.F32, (4,))
+    # gelu_erf(1) = Phi(1), the standard normal CDF at one standard deviation
+    assert ge[0] == 0.0 and abs(ge[1] - 0.8413447460685429) < 1e-15
+    assert abs(ge[2] - (-(1 - 0.8413447460685429))) < 1e-15
+    gt = run1("gelu_tanh", [x], [D.F32], D.F32, (4,))
+    assert gt[0] == 0.0
+    assert abs(gt[1] - 0.8411919906082768) < 1e-15
+    assert abs(gt[2] + 0.15880800939172324) < 1e-15
+    assert abs(gt[3] - 1.954597694087775) < 1e-15
+    si = run1("silu", [x], [D.F32], D.F32, (4,))
+    # silu(1) = 1/(1+1/e)
+    assert si[0] == 0.0 and abs(si[1] - 0.7310585786300049) < 1e-15
+    assert abs(si[2] + 0.2689414213699951) < 1e-15
+    sg = run1("sigmoid", [x], [D.F32], D.F32, (4,))
+    assert sg[0] == 0.5 and abs(sg[1] - 0.7310585786300049) < 1e-15
+
+
+def test_activation_symmetries():
+    rng = np.random.default_rng(1)
+    x = rng.standard_normal(257).astype(np.float32) * 3
+    xm = (-x).astype(np.float32)
+    for op in ("gelu_tanh", "gelu_erf", "silu"):
+        a = run1(op, [x], [D.F32], D.F32, x.shape)
+        b = run1(op, [xm], [D.F32], D.F32, x.shape)
+        # f(x) = x * s(x) with s(x) + s(-x) = 1  =>  f(x) - f(-x) = x
+        np.testing.assert_allclose(a - b, x.astype(np.float64), rtol=0, atol=1e-14)
+    s = run1("sigmoid", [x], [D.F32], D.F32, x.shape) + run1("sigmoid", [xm], [D.F32], D.F32, x.shape)
+    np.testing.assert_allclose(s, 1.0, atol=1e-15)
+    # gelu_erf through the complementary error function of libm
+    ge = run1("gelu_erf", [x], [D.F32], D.F32, x.shape)
+    ref = [0.5 * float(v) * math.erfc(-float(v) / math.sqrt(2)) for v in x]
+    np.testing.assert_allclose(ge, ref, rtol=1e-13, atol=1e-15)
+    # tanh through exponentials
+    th = run1("tanh", [x], [D.F32], D.F32, x.shape)
+    ref = [(math.exp(2 * float(v)) - 1) / (math.exp(2 * float(v)) + 1) for v in x]
+    np.testing.assert_allclose(th, ref, rtol=1e-13, atol=1e-15)
+
+
+def test_unary_binary_against_libm_scalars():
+    x = f32(0.25, 1.0, 2.5, 9.0)
+    table = {"exp": math.exp, "log": math.log, "sqrt": math.sqrt, "neg": lambda v: -v,
+             "recip": lambda v: 1 / v, "rsqrt": lambda v: 1 / math.sqrt(v), "abs": abs,
+             "square": lambda v: v * v, "erf": math.erf, "relu": lambda v: max(v, 0.0)}
+    for op, fn in table.items():
+        for arr in (x, (-x).astype(np.float32)) if op in ("neg", "abs", "relu", "erf", "square") else (x,):
+            got = run1(op, [arr], [D.F32], D.F32, arr.shape)
+            np.testing.assert_allclose(got, [fn(float(v)) for v in arr], rtol=1e-15)
+    a, b = f32(3.0, -2.0, 0.5, 7.0), f32(2.0, 4.0, -0.5, 7.0)
+    bt = {"add": lambda p, q: p + q, "sub": lambda p, q: p - q, "mul": lambda p, q: p * q,
+          "div": lambda p, q: p / q, "max": max, "min": min}
+    for op, fn in bt.items():
+        got = run1(op, [a, b], [D.F32, D.F32], D.F32, (4,))
+        assert got.tolist() == [fn(float(p), float(q)) for p, q in zip(a, b)]
+    ct = {"gt": [1, 0, 1, 0], "ge": [1, 0, 1, 1], "lt": [0, 1, 0, 0], "le": [0, 1, 0, 1],
+          "eq": [0, 0, 0, 1], "ne": [1, 1, 1, 0]}
+    for op, want in ct.items():
+        got = run1(op, [a, b], [D.F32, D.F32], D.BOOL, (4,))
+        assert got.dtype == np.int64 and got.tolist() == want
+    # sub is not commutative, div neither: operand order matters
+    assert run1("sub", [a], [D.F32], D.F32, (4,), imms=[1.0]).tolist() == [2.0, -3.0, -0.5, 6.0]
+    assert run1("fma", [a, b, a], [D.F32] * 3, D.F32, (4,)).tolist() == [9.0, -10.0, 0.25, 56.0]
+    assert run1("clamp", [a], [D.F32], D.F32, (4,), imms=[0.0, 3.0]).tolist() == [3.0, 0.0, 0.5, 3.0]
+
+
+def test_where_and_signed_zero():
+    c = np.array([1, 0, -3, 0], dtype=np.int8)
+    a, b = f32(1, 2, 3, 4), f32(-1, -2, -3, -4)
+    assert run1("where", [c, a, b], [D.I8, D.F32, D.F32], D.F32, (4,)).tolist() == [1, -2, 3, -4]
+    z = f32(-0.0, 0.0, 1e-30, -1e-30)
+    assert run1("gt", [z], [D.F32], D.BOOL, (4,), imms=[0.0]).tolist() == [0, 0, 1, 0]
+
+
+# ---------------------------------------------------------------------------
+# reductions and composites
+# ---------------------------------------------------------------------------
+def test_softmax_invariants_and_brute_force():
+    rng = np.random.default_rng(2)
+    x = (np.rint(rng.standard_normal((7, 33)) * 2 * 1024) / 1024).astype(np.float32)   # multiples of 2^-10
+    y = run1("softmax", [x], [D.F32], D.F32, x.shape)
+    np.testing.assert_allclose(y.sum(-1), 1.0, atol=1e-12)
+    assert (y >= 0).all() and (y <= 1).all()
+    # brute force without the max shift (inputs are well scaled)
+    for i in range(x.shape[0]):
+        ex = [math.exp(float(v)) for v in x[i]]
+        tot = math.fsum(ex)
+        np.testing.assert_allclose(y[i], [e / tot for e in ex], rtol=1e-13)
+    # shift invariance, with a shift that is exact in fp32 for these magnitudes
+    xs = (x + np.float32(8.0)).astype(np.float32)
+    assert np.array_equal(xs.astype(np.float64) - 8.0, x.astype(np.float64))
+    np.testing.assert_allclose(run1("softmax", [xs], [D.F32], D.F32, x.shape), y, rtol=1e-12)
+    # the row maximum is subtracted first: inputs near 1000 would overflow e^x otherwise
+    xb = (x + np.float32(1000.0)).astype(np.float32)
+    assert np.array_equal(xb.astype(np.float64) - 1000.0, x.astype(np.float64))
+    np.testing.assert_allclose(run1("softmax", [xb], [D.F32], D.F32, x.shape), y, rtol=1e-12)
+    # masked entries are exactly zero; a fully masked row is NaN
+    xm = x.copy(); xm[:, 5:] = -np.inf; xm[3, :] = -np.inf
+    ym = run1("softmax", [xm], [D.F32], D.F32, x.shape)
+    assert (ym[[0, 1, 2, 4, 5, 6], 5:] == 0).all() and np.isnan(ym[3]).all()
+    np.testing.assert_allclose(ym[0, :5].sum(), 1.0, atol=1e-13)
+
+
+def test_c2_structure():
+    w = C.c2(B=2, Q=9, K=9)
+    y = E.evaluate(w.desc, w.inputs)[0]
+    for q in range(9):
+        assert (np.count_nonzero(y[:, q, :], axis=-1) == q + 1).all()   # causal: k <= q
+        assert (y[:, q, q + 1:] == 0).all()
+    assert (y[:, 0, 0] == 1.0).all()
+    np.testing.assert_allclose(y.sum(-1), 1.0, atol=1e-12)
+    # row q = 1: two survivors, closed form 1/(1+e^{(s1-s0)/8})
+    s = E.widen(w.inputs[0], D.BF16)
+    want = 1.0 / (1.0 + np.exp((s[:, 1, 1] - s[:, 1, 0]) * 0.125))
+    np.testing.assert_allclose(y[:, 1, 0], want, rtol=1e-13)
+
+
+def test_logsumexp_pins():
+    rng = np.random.default_rng(3)
+    x = (np.rint(rng.standard_normal((5, 41)) * 3 * 1024) / 1024).astype(np.float32)   # multiples of 2^-10
+    l = run1("logsumexp", [x], [D.F32], D.F32, (5,))
+    for i in range(5):
+        m = max(float(v) for v in x[i])
+        ref = m + math.log(math.fsum(math.exp(float(v) - m) for v in x[i]))
+        assert abs(l[i] - ref) < 1e-13
+        assert m <= l[i] <= m + math.log(41)
+    c = np.full((2, 16), 1.25, dtype=np.float32)
+    np.testing.assert_allclose(run1("logsumexp", [c], [D.F32], D.F32, (2,)), 1.25 + math.log(16), rtol=1e-15)
+    xs = (x + np.float32(4.0)).astype(np.float32)
+    assert np.array_equal(xs.astype(np.float64) - 4.0, x.astype(np.float64))
+    np.testing.assert_allclose(run1("logsumexp", [xs], [D.F32], D.F32, (5,)), l + 4.0, rtol=1e-13)
+    inf = np.full((1, 4), -np.inf, dtype=np.float32)
+    assert run1("logsumexp", [inf], [D.F32], D.F32, (1,))[0] == -np.inf
+    inf[0, 2] = np.inf
+    assert run1("logsumexp", [inf], [D.F32], D.F32, (1,))[0] == np.inf
+    # keepdim form of the declared shape is honoured
+    assert run1("logsumexp", [x], [D.F32], D.F32, (5, 1)).shape == (5, 1)
+    # relation to softmax: log(softmax) = x - lse
+    ls = run1("log_softmax", [x], [D.F32], D.F32, x.shape)
+    sm = run1("softmax", [x], [D.F32], D.F32, x.shape)
+    np.testing.assert_allclose(ls, np.log(sm), rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(ls, x.astype(np.float64) - l[:, None], rtol=1e-13, atol=1e-13)
+
+
+def test_c4_closed_form():
+    w = C.c4(M=4, N=50000)
+    x = w.inputs[0]
+    lse, idx = E.evaluate(w.desc, w.inputs)
+    assert idx.dtype == np.int64
+    for i in range(4):
+        hits = [j for j in range(x.shape[1]) if x[i, j] == np.float32(30.0)]
+        assert len(hits) >= 2                       # ties exist; lowest index must win
+        assert idx[i] == hits[0]
+        # the other entries are N(0, var 4): they add less than 1e-6 to the sum
+        assert 0 <= lse[i] - (30.0 + math.log(len(hits))) < 1e-6 / len(hits) * 50
+
+
+def test_argmax_argmin_brute_force_and_nan():
+    rng = np.random.default_rng(4)
+    x = rng.integers(-3, 4, size=(20, 17)).astype(np.float32)      # many ties
+    am = run1("argmax", [x], [D.F32], D.I64, (20,))
+    an = run1("argmin", [x], [D.F32], D.I64, (20,))
+    for i in range(20):
+        best = 0
+        worst = 0
+        for j in range(17):
+            if x[i, j] > x[i, best]:
+                best = j
+            if x[i, j] < x[i, worst]:
+                worst = j
+        assert am[i] == best and an[i] == worst
+    xn = x.copy(); xn[2, 9] = np.nan; xn[2, 12] = np.nan
+    assert run1("argmax", [xn], [D.F32], D.I64, (20,))[2] == 9
+    assert run1("argmin", [xn], [D.F32], D.I64, (20,))[2] == 9
+    assert np.isnan(run1("amax", [xn], [D.F32], D.F32, (20,))[2])
+    assert run1("amax", [x], [D.F32], D.F32, (20,)).tolist() == [float(max(r)) for r in x]
+    assert run1("amin", [x], [D.F32], D.F32, (20,)).tolist() == [float(min(r)) for r in x]
+
+
+def test_mean_var_pins():
+    v = np.arange(1, 9, dtype=np.float32)[None, :]               # 1..8: mean 4.5, var 5.25 / 6
+    assert run1("mean", [v], [D.F32], D.F32, (1,))[0] == 4.5
+    assert run1("sum", [v], [D.F32], D.F32, (1,))[0] == 36.0
+    assert run1("var", [v], [D.F32], D.F32, (1,), attr=(0, 0))[0] == 5.25
+    assert run1("var", [v], [D.F32], D.F32, (1,), attr=(1, 0))[0] == 6.0
+    c = np.full((3, 10), -2.5, dtype=np.float32)
+    assert (run1("var", [c], [D.F32], D.F32, (3,))[...] == 0).all()
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal((6, 29)).astype(np.float32)
+    var = run1("var", [x], [D.F32], D.F32, (6,))
+    for i in range(6):
+        xs = [float(t) for t in x[i]]
+        ex2 = math.fsum(t * t for t in xs) / 29
+        ex = math.fsum(xs) / 29
+        assert abs(var[i] - (ex2 - ex * ex)) < 1e-13
+
+
+def test_layer_norm_pins():
+    gold = dict((k, float(v)) for k, v in _gold("layernorm_case.txt"))
+    v = np.arange(1, 9, dtype=np.float32)[None, :]
+    g = GraphBuilder()
+    x = g.input(D.F32, (1, 8)); ga = g.input(D.F32, (8,)); be = g.input(D.F32, (8,))
+    y, mean, rstd = g.node("layer_norm", [x, ga, be], [D.F32] * 3, [(1, 8), (1,), (1,)],
+                           extra_imm=[gold["eps"]])
+    for t in (y, mean, rstd):
+        g.mark_output(t)
+    yo, mo, ro = E.evaluate(g.build(), [v, np.full(8, 2, np.float32), np.full(8, -1, np.float32)])
+    assert mo[0] == gold["mean"]
+    assert abs(1.0 / ro[0] ** 2 - (gold["biased_var"] + gold["eps"])) < 1e-12
+    want = [(j - 4.5) / math.sqrt(5.25 + 1e-5) * 2 - 1 for j in range(1, 9)]
+    np.testing.assert_allclose(yo[0], want, rtol=1e-14)
+    # invariants on random rows with gamma = 1, beta = 0
+    rng = np.random.default_rng(6)
+    xr = (rng.standard_normal((9, 64)) * 1.5 + 0.3).astype(np.float32)
+    g = GraphBuilder(); x = g.input(D.F32, (9, 64))
+    y, mean, rstd = g.node("layer_norm", [x], [D.F32] * 3, [(9, 64), (9,), (9,)], extra_imm=[1e-5])
+    for t in (y, mean, rstd):
+        g.mark_output(t)
+    yo, mo, ro = E.evaluate(g.build(), [xr])
+    np.testing.assert_allclose(yo.mean(-1), 0, atol=1e-12)
+    var = xr.astype(np.float64).var(-1)
+    np.testing.assert_allclose(yo.var(-1), var / (var + 1e-5), rtol=1e-12)      # "1" up to eps
+    np.testing.assert_allclose(ro ** 2 * (var + 1e-5), 1.0, rtol=1e-13)
+    # affine part
+    ga = rng.uniform(0.5, 1.5, 64).astype(np.float32); be = rng.standard_normal(64).astype(np.float32)
+    g = GraphBuilder(); x = g.input(D.F32, (9, 64)); a = g.input(D.F32, (64,)); b = g.input(D.F32, (64,))
+    g.mark_output(g.node("layer_norm", [x, a, b], [D.F32], [(9, 64)], extra_imm=[1e-5])[0])
+    np.testing.assert_allclose(E.evaluate(g.build(), [xr, ga, be])[0],
+                               yo * ga.astype(np.float64) + be.astype(np.float64), rtol=1e-14, atol=1e-15)
+    # rms_norm: unit gamma gives rows whose mean square is ms/(ms+eps)
+    yr = run1("rms_norm", [xr], [D.F32], D.F32, xr.shape, extra_imm=[1e-6])
+    ms = (xr.astype(np.float64) ** 2).mean(-1)
+    np.testing.assert_allclose((yr ** 2).mean(-1), ms / (ms + 1e-6), rtol=1e-12)
+    assert np.sign(yr[0, 0]) == np.sign(xr[0, 0])
+
+
+def test_clamped_divide_of_masked_mean_pooling():
+    # out = sum(h*m) / max(sum(m), 1e-9): the epilogue of the paper's pooling kernel
+    floor = dict((k, float(v)) for k, v in _gold("layernorm_case.txt"))["clamp_floor"]
+    h = f32(1, 2, 3, 4, 5, 6).reshape(2, 3)
+    m = f32(1, 0, 1, 0, 0, 0).reshape(2, 3)
+    g = GraphBuilder()
+    hi = g.input(D.F32, (2, 3)); mi = g.input(D.F32, (2, 3))
+    p = g.op("mul", [hi, mi], D.F32, (2, 3))
+    s = g.op("sum", [p], D.F32, (2, 1)); c = g.op("sum", [mi], D.F32, (2, 1))
+    cc = g.op("clamp", [c, Imm(floor), Imm(math.inf)], D.F32, (2, 1))
+    g.mark_output(g.op("div", [s, cc], D.F32, (2, 1)))
+    assert E.evaluate(g.build(), [h, m])[0].ravel().tolist() == [2.0, 0.0]
+
+
+# ---------------------------------------------------------------------------
+# broadcasting and casts
+# ---------------------------------------------------------------------------
+def test_broadcasting_matches_explicit_materialisation():
+    rng = np.random.default_rng(7)
+    a = rng.standard_normal((2, 3, 1, 5)).astype(np.float32)
+    b = rng.standard_normal((3, 4, 1)).astype(np.float32)
+    got = run1("mul", [a, b], [D.F32, D.F32], D.F32, (2, 3, 4, 5))
+    full_a = np.empty((2, 3, 4, 5)); full_b = np.empty((2, 3, 4, 5))
+    for i in range(2):
+        for j in range(3):
+            for k in range(4):
+                for l in range(5):
+                    full_a[i, j, k, l] = a[i, j, 0, l]; full_b[i, j, k, l] = b[j, k, 0]
+    assert np.array_equal(got, full_a * full_b)
+
+
+def test_bf16_widen_exhaustive_and_narrow_ties():
+    bits = np.arange(65536, dtype=np.uint16)
+    got = E.widen(bits, D.BF16)
+    ref = np.array([struct.unpack("<f", struct.pack("<I", int(b) << 16))[0] for b in bits])
+    assert np.array_equal(got[~np.isnan(ref)], ref[~np.isnan(ref)]) and np.isnan(got[np.isnan(ref)]).all()
+    # every bf16 value rounds to itself
+    fin = np.isfinite(ref)
+    assert np.array_equal(E.round_to_bf16(ref[fin]), ref[fin])
+    # ties to even: 1 + 2^-8 is halfway between 1 and 1 + 2^-7 -> 1; 1 + 3*2^-8 -> 1 + 2^-6
+    r = E.round_to_bf16(np.array([1 + 2.0 ** -8, 1 + 3 * 2.0 ** -8, 1 + 2.0 ** -8 + 2.0 ** -30,
+                                  -(1 + 2.0 ** -8), 3.4e38, 2.0 ** -133 * 1.5, 1e-45]))
+    assert r.tolist() == [1.0, 1 + 2.0 ** -6, 1 + 2.0 ** -7, -1.0, np.inf, 2.0 ** -132, 0.0]
+    # the midpoint of two neighbours always lands on the one with the even mantissa
+    pos = np.sort(ref[fin & (ref > 0)])
+    mids = (pos[:-1] + pos[1:]) / 2
+    rm = E.round_to_bf16(mids)
+    lo_bits = np.arange(1, len(pos))            # bit pattern of pos[k] is k+1
+    want = np.where(lo_bits % 2 == 0, pos[:-1], pos[1:])
+    assert np.array_equal(rm, want)
+    # Table 2's accepted bf16 "max diff" is one spacing of bf16 in [4, 8)
+    name, printed, lo, hi = _gold("sparkle_max_diff.txt")[0]
+    sp = E.round_to_bf16(np.array([float(lo) + 1e-9 + 2.0 ** -6])) - float(lo)
+    assert sp[0] == 2.0 ** -5 and round(float(sp[0]), 3) == float(printed)
+    # fp16 narrowing agrees with the IEEE half type
+    assert E.round_to_f16(np.array([1 + 2.0 ** -11, 65520.0])).tolist() == [1.0, np.inf]
+
+
+def test_declared_narrow_intermediate_is_rounded_for_consumers_only():
+    x = f32(1.00390625 * 3)                      # 3.01171875 is not a bf16 value
+    g = GraphBuilder()
+    xi = g.input(D.F32, (1,))
+    nb = g.op("cast", [xi], D.BF16, (1,))        # declared bf16, consumed below
+    d = g.op("sub", [nb, xi], D.F32, (1,))
+    g.mark_output(nb); g.mark_output(d)
+    out_nb, out_d = E.evaluate(g.build(), [x])
+    assert out_nb[0] == float(x[0])              # outputs are reported unrounded
+    assert out_d[0] == 3.015625 - float(x[0])    # the consumer saw the rounded value
+    # float -> int truncates toward zero; int8 -> float is exact
+    assert run1("cast", [f32(2.9, -2.9)], [D.F32], D.I32, (2,)).tolist() == [2, -2]
+    assert run1("cast", [np.array([-128, 127], np.int8)], [D.I8], D.F32, (2,)).tolist() == [-128.0, 127.0]
+
+
+# ---------------------------------------------------------------------------
+# whole graphs: a third restatement in pure Python on tiny shapes
+# ---------------------------------------------------------------------------
+def _bf(a):
+    return E.widen(a, D.BF16)
+
+
+def test_c1_restated():
+    w = C.c1(M=3, N=5)
+    x, ww, b, r = [a.astype(np.float64) for a in w.inputs]
+    y = E.evaluate(w.desc, w.inputs)[0]
+    for i in range(3):
+        for j in range(5):
+            u = x[i, j] * ww[j] + b[j]
+            ref = 0.5 * u * (1 + math.tanh(math.sqrt(2 / math.pi) * (u + 0.044715 * u ** 3))) + r[i, j]
+            assert abs(y[i, j] - ref) < 1e-14
+
+
+def test_c3_restated():
+    w = C.c3(M=4, N=12, also_output_sum=True)
+    x, res = _bf(w.inputs[0]), _bf(w.inputs[1])
+    ga, be = w.inputs[2].astype(np.float64), w.inputs[3].astype(np.float64)
+    out = dict(zip(w.output_names, E.evaluate(w.desc, w.inputs)))
+    for i in range(4):
+        h = [x[i, j] + res[i, j] for j in range(12)]
+        mu = math.fsum(h) / 12
+        var = math.fsum((t - mu) ** 2 for t in h) / 12
+        rs = 1 / math.sqrt(var + 1e-5)
+        assert abs(out["mean"][i] - mu) < 1e-14 and abs(out["rstd"][i] - rs) < 1e-13
+        for j in range(12):
+            assert abs(out["y"][i, j] - ((h[j] - mu) * rs * ga[j] + be[j])) < 1e-13
+            assert out["h"][i, j] == h[j]
+
+
+def test_c5_restated_and_mask_identity():
+    w = C.c5(M=5, N=24)
+    a, gt, col, row = [_bf(t) for t in w.inputs]
+    h, mask, mean, var = E.evaluate(w.desc, w.inputs)
+    assert mask.dtype == np.int64 and np.array_equal(mask, (a > 0).astype(np.int64))
+    for i in range(5):
+        hr = [a[i, j] * (1 / (1 + math.exp(-gt[i, j]))) * col[0, j] * row[i, 0] for j in range(24)]
+        np.testing.assert_allclose(h[i], hr, rtol=1e-14)
+        mu = math.fsum(hr) / 24
+        assert abs(mean[i] - mu) < 1e-14
+        assert abs(var[i] - math.fsum((t - mu) ** 2 for t in hr) / 24) < 1e-14
+
+
+# ---------------------------------------------------------------------------
+# the comparison rule
+# ---------------------------------------------------------------------------
+def test_tolerance_rule_matches_the_papers_ladder():
+    rows = {r[0]: r for r in _gold("tolerance_ladder.txt")}
+    # bf16 rtol used here is the paper's printed t = -5 value, itself 10^(-1.796) to two digits
+    k = float(rows["bfloat16"][1])
+    assert float(f"{10 ** (-5 * k / 5):.1e}") == float(rows["bfloat16"][2]) == E.TOLERANCES[D.BF16][0]
+    assert float(rows["float16"][2]) == E.TOLERANCES[D.F16][0] and float(rows["float16"][3]) == E.TOLERANCES[D.F16][1]
+    assert float(f"{10 ** (-float(rows['float32'][1])):.1e}") == float(rows["float32"][2])
+    assert float(rows["others"][2]) == 0.0       # integers and booleans: exact
+    ref = np.array([1.0, 100.0, 0.0, np.inf, np.nan])
+    ok = E.compare(ref * (1 + 9e-6) + np.array([0, 0, 9e-7, 0, 0]), ref, D.F32)
+    assert ok["ok"] and ok["violations"] == 0
+    assert not E.compare(ref * (1 + 2e-5), ref, D.F32)["ok"]
+    assert not E.compare(np.array([1.0, 100.0, 0.0, -np.inf, np.nan]), ref, D.F32)["ok"]
+    assert not E.compare(np.array([1.0, 100.0, 0.0, np.inf, 0.0]), ref, D.F32)["ok"]
+    assert not E.compare(np.array([1.0, np.nan, 0.0, np.inf, np.nan]), ref, D.F32)["ok"]
+    assert E.compare(np.array([1.015]), np.array([1.0]), D.BF16)["ok"]
+    assert not E.compare(np.array([1.02]), np.array([1.0]), D.BF16)["ok"]
+    assert not E.compare(np.array([1, 2, 4]), np.array([1, 2, 3]), D.I64)["ok"]
+    assert E.compare(np.array([1, 2, 3], np.int8), np.array([1, 2, 3]), D.I8)["ok"]
