@@ -1,0 +1,161 @@
+/*
+ * pn.h -- C ABI of the fused-subgraph executor for NVIDIA B200 (sm_100a).
+ *
+ * The library runs a "long-tail fusible subgraph" -- a DAG of pointwise operators
+ * with broadcasting, optional reductions over the last dimension, and a
+ * normalisation / scaling epilogue -- as ONE pass over HBM instead of one kernel
+ * per operator.  The input is the paper's computational graph G = (V, E, tau, sigma)
+ * (Definition 3.1: operator nodes, data dependencies, an operator type per node and a
+ * static output shape per node), serialised as a descriptor.  What a handle computes
+ * is f_G; a fused execution is acceptable when it equals the per-operator evaluation
+ * within a tolerance (Definition 3.2, Eq. 1).  One handle serves one shape / dtype
+ * instance of a graph, as in the paper's task formulation (Section 3.1).
+ *
+ * All functions are thread-safe with respect to different handles.  Nothing throws
+ * or aborts across this boundary: every failure is a negative pn_status, with a
+ * thread-local detail message available from pn_last_error().
+ *
+ * Descriptor format, version 1 (little-endian):
+ *   header  16 B : u32 magic 0x31474E50 ('PNG1') | u16 version = 1 | u16 0
+ *                  | u32 n_tensors | u32 n_nodes
+ *   tensor  40 B : u8 dtype | u8 role (bit0 graph input, bit1 graph output) | u8 rank (<= 4)
+ *                  | u8 0 | u32 0 | i64 dims[4]
+ *   node    64 B : u16 opcode | u8 n_in (<= 4) | u8 n_out (1..3) | u32 in[4] | u32 out[3]
+ *                  | f64 imm[2] | i64 attr[2]
+ * Tensor ids are table positions.  Graph inputs / outputs are the tensors carrying the
+ * role bit, in table order: that order is the order of the pointer arrays passed to
+ * pn_graph_run.  An operand slot equal to 0xFFFFFFFF / 0xFFFFFFFE names imm[0] / imm[1].
+ * Nodes are listed in topological order.  All tensors are dense, row-major, last
+ * dimension contiguous; operands broadcast by NumPy's size-1 rules.  Reductions and
+ * composites act over the last dimension; their per-row results have the input's
+ * shape with the last dimension dropped or kept as 1.
+ *
+ * Opcodes: 1 neg, 2 abs, 3 exp, 4 log, 5 sqrt, 6 rsqrt, 7 recip, 8 tanh, 9 sigmoid,
+ * 10 silu, 11 gelu_tanh, 12 gelu_erf, 13 relu, 14 cast (to the output tensor's dtype),
+ * 15 square, 16 erf; 32 add, 33 sub, 34 mul, 35 div, 36 max, 37 min, 38 gt, 39 ge,
+ * 40 lt, 41 le, 42 eq, 43 ne; 64 where(c, a, b), 65 clamp(x, lo, hi), 66 fma(a, b, c);
+ * 96 sum, 97 mean, 98 var (attr[0] = correction), 99 amax, 100 amin, 101 argmax,
+ * 102 argmin (lowest index on ties; i32 / i64 result), 103 logsumexp; 128 softmax,
+ * 129 log_softmax, 130 layer_norm(x[, gamma[, beta]]) -> y[, mean, rstd] with
+ * imm[0] = eps, 131 rms_norm(x[, gamma]) with imm[0] = eps.
+ * Arithmetic is fp32 in registers whatever the storage types; integer and boolean
+ * tensors take part as exact small integers / predicates; a node whose declared
+ * output dtype is bf16 / f16 is rounded to it (nearest even) for its consumers.
+ */
+#ifndef PN_H_
+#define PN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct pn_graph pn_graph_t; /* opaque handle */
+typedef int pn_status;
+
+enum {
+  PN_OK = 0,
+  PN_ERR_INVALID_ARG = -1,    /* null pointer, bad enum, bad size                       */
+  PN_ERR_BAD_DESCRIPTOR = -2, /* malformed bytes, ids out of range, not topological     */
+  PN_ERR_UNSUPPORTED_OP = -3, /* unknown opcode, or an operator / dtype mix not lowered */
+  PN_ERR_SHAPE = -4,          /* broadcast mismatch, reduction result of the wrong shape */
+  PN_ERR_TOO_LARGE = -5,      /* exceeds the bytecode, register, I/O or stage budget    */
+  PN_ERR_ALIGNMENT = -6,      /* a device pointer is less aligned than the plan needs   */
+  PN_ERR_COUNT = -7,          /* n_inputs / n_outputs differ from the descriptor        */
+  PN_ERR_DEVICE = -8,         /* no such device, or not an sm_100 part                  */
+  PN_ERR_CUDA = -9            /* a CUDA call failed; text in pn_last_error()            */
+};
+
+/* dtype codes of the descriptor */
+enum { PN_F32 = 0, PN_F16 = 1, PN_BF16 = 2, PN_I8 = 3, PN_BOOL = 4, PN_I32 = 5, PN_I64 = 6 };
+
+/* create-time flags */
+enum {
+  PN_FLAG_UNFUSED = 1u << 0,      /* one kernel per node, intermediates in a workspace   */
+  PN_FLAG_PLAN_ONLY = 1u << 1,    /* no CUDA call at all: lower for a B200, allow query  */
+  PN_FLAG_FORCE_WARP = 1u << 4,   /* row kernels: one warp per row                        */
+  PN_FLAG_FORCE_BLOCK = 1u << 5,  /* row kernels: one thread block per row                */
+  PN_FLAG_FORCE_CLUSTER = 1u << 6,/* row kernels: one thread-block cluster per row        */
+  PN_FLAG_FORCE_SCALAR = 1u << 7, /* element-wise (unvectorised) memory accesses          */
+  PN_FLAG_FORCE_MULTICHUNK = 1u << 8 /* smallest tile: rows span several chunks per thread */
+};
+
+/* pn_graph_query selectors; each writes int64 values into `out` */
+enum {
+  PN_Q_N_INPUTS = 1,        /* 1 value                                                   */
+  PN_Q_N_OUTPUTS = 2,       /* 1 value                                                   */
+  PN_Q_INPUT_META = 3,      /* per input 6 values: dtype, rank, dims[4]                  */
+  PN_Q_OUTPUT_META = 4,     /* per output 6 values                                       */
+  PN_Q_COMPULSORY_BYTES = 5,/* 1 value: every input read once + every output written once */
+  PN_Q_N_KERNELS = 6,       /* 1 value: launches per pn_graph_run (1 when fused)         */
+  PN_Q_N_NODES = 7,         /* 1 value: operator nodes in the descriptor                 */
+  PN_Q_WORKSPACE_BYTES = 8, /* 1 value: device memory owned by the handle                */
+  PN_Q_KERNEL_INFO = 9      /* per kernel 12 values: family (0 pointwise, 1 warp-per-row,
+                               2 block-per-row, 3 cluster-per-row), grid, block, cluster,
+                               dynamic smem bytes, vector length, groups per tile, chunks
+                               per row slice, bytecode words, stages, rows, row length   */
+};
+
+/*
+ * pn_graph_create -- parse, validate and lower a graph (the host side of running G of
+ * Definition 3.1; the lowering picks a kernel family per shape, which is the hardware
+ * cost model whose absence the paper lists as a failure mode, Section 4.4).
+ *   desc, desc_bytes : HOST pointer to the descriptor; copied, caller may free it.
+ *   device           : CUDA device ordinal the handle is bound to.
+ *   flags            : PN_FLAG_* bits.
+ *   out              : receives the handle; set to NULL on failure.
+ * Allocates device memory only for PN_FLAG_UNFUSED (the intermediates) -- owned by the
+ * handle and released by pn_graph_destroy.  Launches no kernel.
+ */
+pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsigned flags,
+                          pn_graph_t** out);
+
+/*
+ * pn_graph_run -- enqueue one evaluation of f_G (Definition 3.1) on `stream`.
+ *   inputs  : HOST array of n_inputs DEVICE pointers, descriptor input order; read-only.
+ *   outputs : HOST array of n_outputs DEVICE pointers, descriptor output order; every
+ *             element of every output is overwritten.
+ *   stream  : a cudaStream_t (NULL = the default stream).
+ * Asynchronous: returns after the launch(es).  No allocation, no host synchronisation.
+ * Pointers must be aligned to 16 bytes unless the handle was created with
+ * PN_FLAG_FORCE_SCALAR (then to the element size); otherwise PN_ERR_ALIGNMENT.  Inputs
+ * and outputs must not overlap.  The library never retains or frees user memory.  Runs on
+ * one PN_FLAG_UNFUSED handle share its workspace and must be stream-ordered by the caller.
+ * A graph any of whose inputs or outputs has zero elements runs as a no-op.
+ */
+pn_status pn_graph_run(pn_graph_t* g, const void* const* inputs, int n_inputs,
+                       void* const* outputs, int n_outputs, void* stream);
+
+/*
+ * pn_graph_run_host -- the same evaluation of f_G (Definition 3.1) for callers whose
+ * tensors live in HOST memory: copies each input to the device, runs, copies each output
+ * back and waits.  `inputs` / `outputs` are HOST arrays of HOST pointers to dense buffers
+ * of the sizes the descriptor states (pinned memory lets the copies run at full speed).
+ * Staging buffers are allocated on first use and owned by the handle.
+ */
+pn_status pn_graph_run_host(pn_graph_t* g, const void* const* inputs, int n_inputs,
+                            void* const* outputs, int n_outputs, void* stream);
+
+/* pn_graph_destroy -- release the handle and what it owns; NULL is accepted. */
+pn_status pn_graph_destroy(pn_graph_t* g);
+
+/*
+ * pn_graph_query -- introspection for tests and benchmarks (the kernel count is the
+ * paper's "kernels N -> 1" figure of Table 2).  Writes int64 values as listed beside
+ * each PN_Q_* selector into `out` (HOST memory, out_bytes large enough, else
+ * PN_ERR_INVALID_ARG).
+ */
+pn_status pn_graph_query(const pn_graph_t* g, int what, void* out, size_t out_bytes);
+
+/* Static text for a status code. */
+const char* pn_status_string(pn_status s);
+
+/* Detail of the calling thread's most recent failure ("" if none). */
+const char* pn_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PN_H_ */

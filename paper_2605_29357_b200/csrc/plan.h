@@ -1,0 +1,126 @@
+// plan.h -- what the host lowering hands to the kernels: a tile bytecode program, the
+// addressing of every graph input / output, and the launch shape.  Plain structs only;
+// included by host (.cpp) and device (.cu) code.
+#pragma once
+#include <stdint.h>
+
+namespace pn {
+
+constexpr int kMaxIo = 12;      // graph inputs + outputs of one kernel
+constexpr int kMaxCode = 224;   // 32-bit bytecode words of one kernel
+constexpr int kMaxStages = 4;   // reduction-separated stages
+constexpr int kMaxRed = 4;      // reductions accumulated in one stage
+constexpr int kMaxSlots = 24;   // per-row scalar slots
+constexpr int kMaxStash = 6;    // tile values parked in shared memory across stages
+
+// Storage types (same numbering as the descriptor).
+enum DType : uint8_t { kF32 = 0, kF16 = 1, kBF16 = 2, kI8 = 3, kBool = 4, kI32 = 5, kI64 = 6 };
+
+// Tile bytecode.  One instruction acts on the whole register tile of a thread.  The
+// machine has an accumulator tile `acc`, K tile registers, a per-tile scalar `ts`, and
+// reads per-row scalars from shared-memory slots.  Word layout: op | a<<8 | b<<16 | c<<24;
+// an immediate operand occupies the following word (fp32 bits).
+enum Op : uint8_t {
+  OP_END = 0,
+  // memory
+  OP_LDRAW,   // a = io, b = reg (K = acc): issue the loads of a tile, storage bits as they are
+  OP_WIDEN,   // a = io (for its dtype), b = reg: storage bits -> fp32 in place
+  OP_LDBC,    // a = io, b = reg: last-dim-broadcast operand, one element splat over the tile
+  OP_LD,      // acc = reg[a]
+  OP_ST,      // reg[a] = acc
+  OP_STOUT,   // a = io: narrow acc and store it
+  // unary on acc
+  OP_NEG, OP_ABS, OP_EXP, OP_LOG, OP_SQRT, OP_RSQRT, OP_RECIP, OP_TANH, OP_SIGMOID, OP_SILU,
+  OP_GELU_TANH, OP_GELU_ERF, OP_RELU, OP_SQUARE, OP_ERF,
+  OP_RND_BF16, OP_RND_F16,  // round to a narrow float and back (a declared narrow intermediate)
+  OP_TRUNC,                 // float -> integer value, toward zero
+  OP_NEZ,                   // x != 0 -> 1 / 0
+  OP_I2F,                   // value holding int32 bits -> float (scalar programs)
+  // binary: acc = acc (op) src, src = operand(a, kind b)
+  OP_ADD, OP_SUB, OP_RSUB, OP_MUL, OP_DIV, OP_RDIV, OP_MAX, OP_MIN,
+  OP_GT, OP_GE, OP_LT, OP_LE, OP_EQ, OP_NE,
+  OP_LSEFIN,  // acc = isinf(acc) ? acc : acc + log(src)
+  // ternary: X = operand(a, kind c&15), Y = operand(b, kind c>>4)
+  OP_WHERE,   // acc = acc != 0 ? X : Y
+  OP_FMA,     // acc = acc * X + Y
+  // reductions over the tile into the thread's partial state
+  OP_RED,      // a = RedKind, b = reduction index within the stage
+  OP_SCALE_TS, // acc *= exp(ts - slot[a]) * slot[b]   (softmax epilogue)
+  // parking tile values in shared memory across stages (rows of several chunks per thread)
+  OP_SPILL, OP_FILL,        // a = reg (K = acc), b = stash index
+  OP_SPILL_TS, OP_FILL_TS,  // b = stash index
+  // scalar programs only
+  OP_SLD,     // acc = slot[a]
+  OP_SST,     // slot[a] = acc
+  OP_STOUT_I, // a = io: store the int32 bits held in acc as an integer (argmax / argmin)
+  OP_COUNT_
+};
+
+enum OperandKind : uint8_t { OPK_REG = 0, OPK_IMM = 1, OPK_SLOT = 2 };
+
+// Reductions.  Each keeps a 3-float partial (a, b, c) per thread and combines associatively.
+enum RedKind : uint8_t {
+  RED_SUM = 0,     // a = sum
+  RED_MAX,         // a = max                     (NaN wins)
+  RED_MIN,         // a = min
+  RED_ARGMAX,      // a = max, b = int bits of its lowest column
+  RED_ARGMIN,
+  RED_LSE,         // a = running max M, b = sum of exp(x - M)
+  RED_SOFTMAX,     // as RED_LSE; also leaves exp(x - m_tile) in acc and m_tile in ts
+  RED_MEANVAR      // a = count, b = mean, c = sum of squared deviations
+};
+
+enum Family : int32_t { FAM_POINTWISE = 0, FAM_WARP = 1, FAM_BLOCK = 2, FAM_CLUSTER = 3 };
+
+struct IoDesc {
+  void* base;              // device pointer; filled in per run
+  int64_t lead_stride[3];  // elements per step of each collapsed leading dim; 0 = broadcast
+  int32_t col_stride;      // 1, or 0 when the last dim is broadcast
+  uint8_t dtype;
+  uint8_t is_row_scalar;   // per-row result tensor (one element per row)
+  uint8_t pad[2];
+};
+
+struct RedDesc {
+  uint8_t kind;
+  uint8_t slot;   // first of the 3 slots receiving the combined (a, b, c)
+};
+
+struct StageDesc {
+  uint16_t elem_begin, elem_end;   // tile program [begin, end) in code[]
+  uint16_t scal_begin, scal_end;   // per-row scalar program run after the stage's combine
+  uint8_t n_red;
+  uint8_t pad[3];
+  RedDesc red[kMaxRed];
+};
+
+struct KernelParams {
+  IoDesc io[kMaxIo];
+  int32_t n_io;
+  int32_t n_stages;
+  uint32_t lead_dim[3];    // collapsed leading dims of the iteration space (unused = 1)
+  int64_t rows;            // product of the leading dims
+  int32_t row_len;         // N
+  int32_t slice_len;       // columns one CTA covers (N unless a cluster splits the row)
+  int32_t chunks;          // chunks per slice: ceil(slice_len / (team_threads * VL * NG))
+  int32_t split_chunks;    // pointwise graphs: every (row, chunk) is its own work item
+  int32_t cluster;         // CTAs per cluster (1 unless FAM_CLUSTER)
+  int32_t stash_floats;    // floats of parked tile values per CTA
+  // shared-memory layout, byte offsets into dynamic shared memory
+  int32_t sm_rowoff, sm_part, sm_wpart, sm_slots, sm_ctapart, sm_stash;
+  StageDesc stage[kMaxStages];
+  uint32_t code[kMaxCode];
+};
+
+// One kernel launch as planned by the lowering.
+struct LaunchPlan {
+  KernelParams p;
+  int32_t family;
+  int32_t vl, ng, k;       // template instance: vector length, groups per tile, tile registers
+  int32_t grid, block, smem_bytes;
+  int32_t code_words;
+  int32_t io_tensor[kMaxIo];   // tensor id behind each io entry
+  int32_t io_is_output[kMaxIo];
+};
+
+}  // namespace pn
