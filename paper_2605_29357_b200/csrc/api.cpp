@@ -1,0 +1,324 @@
+// api.cpp -- the exported C ABI (see include/pn.h): handle life cycle, pointer checks,
+// launches, the unfused one-kernel-per-node path, and the host-memory convenience call.
+#include <cuda_runtime.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/pn.h"
+#include "graph.h"
+
+namespace pn {
+cudaError_t launch_plan(const LaunchPlan& lp, cudaStream_t stream);   // kernels.cu
+}
+
+using namespace pn;
+
+namespace {
+
+thread_local std::string g_last_error;
+
+int fail(int status, const std::string& msg) { g_last_error = msg; return status; }
+
+// where the pointer behind one io entry of one launch comes from
+struct IoSource { int kind; int64_t index; };   // kind 0 user input, 1 user output, 2 workspace offset
+
+struct PlannedLaunch {
+  LaunchPlan plan;
+  std::vector<IoSource> src;
+};
+
+}  // namespace
+
+struct pn_graph {
+  Graph g;
+  unsigned flags = 0;
+  int device = 0;
+  bool plan_only = false;
+  std::vector<PlannedLaunch> launches;
+  void* workspace = nullptr;
+  size_t workspace_bytes = 0;
+  int64_t compulsory_bytes = 0;
+  std::vector<void*> stage_in, stage_out;   // device staging of pn_graph_run_host
+};
+
+namespace {
+
+int64_t tensor_bytes(const Tensor& t) { return t.numel() * dtype_bytes(t.dtype); }
+
+bool any_empty(const Graph& g) {
+  for (const Tensor& t : g.tensors) if (t.numel() == 0) return true;
+  return false;
+}
+
+// The single-node graph executed by one launch of the unfused path.
+void node_subgraph(const Graph& g, const Node& n, Graph& sub, std::vector<int>& orig_of_sub) {
+  sub = Graph();
+  orig_of_sub.clear();
+  Node m = n;
+  auto add = [&](int orig, uint8_t role) {
+    for (size_t i = 0; i < orig_of_sub.size(); ++i) if (orig_of_sub[i] == orig) return (int)i;
+    Tensor t = g.tensors[orig];
+    t.role = role; t.producer = -1;
+    sub.tensors.push_back(t);
+    orig_of_sub.push_back(orig);
+    return (int)sub.tensors.size() - 1;
+  };
+  for (int k = 0; k < n.n_in; ++k) {
+    if (n.in[k] == kImm0 || n.in[k] == kImm1) continue;
+    m.in[k] = (uint32_t)add((int)n.in[k], 1);
+  }
+  for (int k = 0; k < n.n_out; ++k) {
+    m.out[k] = (uint32_t)add((int)n.out[k], 2);
+    sub.tensors[m.out[k]].producer = 0;
+  }
+  sub.nodes.push_back(m);
+  for (size_t i = 0; i < sub.tensors.size(); ++i) {
+    if (sub.tensors[i].role & 1) sub.inputs.push_back((int)i);
+    if (sub.tensors[i].role & 2) sub.outputs.push_back((int)i);
+  }
+}
+
+pn_status check_counts(const pn_graph* h, const void* const* inputs, int n_inputs, void* const* outputs, int n_outputs) {
+  if (!h || (!inputs && n_inputs > 0) || !outputs) return fail(PN_ERR_INVALID_ARG, "null argument");
+  if (h->plan_only) return fail(PN_ERR_DEVICE, "handle was created with PN_FLAG_PLAN_ONLY");
+  if (n_inputs != (int)h->g.inputs.size() || n_outputs != (int)h->g.outputs.size())
+    return fail(PN_ERR_COUNT, "expected " + std::to_string(h->g.inputs.size()) + " inputs and " +
+                                  std::to_string(h->g.outputs.size()) + " outputs");
+  return PN_OK;
+}
+
+}  // namespace
+
+extern "C" {
+#pragma GCC visibility push(default)
+
+pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsigned flags, pn_graph_t** out) {
+  if (out) *out = nullptr;
+  if (!desc || !out) return fail(PN_ERR_INVALID_ARG, "null argument");
+  pn_graph* h = new (std::nothrow) pn_graph();
+  if (!h) return fail(PN_ERR_INVALID_ARG, "out of host memory");
+  std::string err;
+  int st = parse_descriptor(desc, desc_bytes, h->g, err);
+  if (st != PN_OK) { delete h; return fail(st, err); }
+  h->flags = flags;
+  h->device = device;
+  h->plan_only = (flags & PN_FLAG_PLAN_ONLY) != 0;
+
+  DeviceModel dev;
+  if (!h->plan_only) {
+    int count = 0;
+    cudaError_t e = cudaGetDeviceCount(&count);
+    if (e != cudaSuccess || device < 0 || device >= count) { delete h; return fail(PN_ERR_DEVICE, "no such CUDA device"); }
+    cudaDeviceProp prop;
+    e = cudaGetDeviceProperties(&prop, device);
+    if (e != cudaSuccess) { delete h; return fail(PN_ERR_CUDA, cudaGetErrorString(e)); }
+    if (prop.major != 10) { delete h; return fail(PN_ERR_DEVICE, "the kernels are built for sm_100a only"); }
+    e = cudaSetDevice(device);
+    if (e != cudaSuccess) { delete h; return fail(PN_ERR_CUDA, cudaGetErrorString(e)); }
+    dev.sm_count = prop.multiProcessorCount;
+    dev.max_smem_per_block = (int)prop.sharedMemPerBlockOptin;
+    dev.have_device = true;
+  }
+
+  const Graph& g = h->g;
+  for (int t : g.inputs) h->compulsory_bytes += tensor_bytes(g.tensors[t]);
+  for (int t : g.outputs) h->compulsory_bytes += tensor_bytes(g.tensors[t]);
+  if (any_empty(g)) { *out = h; return PN_OK; }   // nothing to compute: runs are no-ops
+
+  if (!(flags & PN_FLAG_UNFUSED)) {
+    PlannedLaunch pl;
+    st = lower_graph(g, flags, dev, pl.plan, err);
+    if (st != PN_OK) { delete h; return fail(st, err); }
+    for (int q = 0; q < pl.plan.p.n_io; ++q) {
+      const int t = pl.plan.io_tensor[q];
+      IoSource s{pl.plan.io_is_output[q] ? 1 : 0, 0};
+      const std::vector<int>& list = pl.plan.io_is_output[q] ? g.outputs : g.inputs;
+      for (size_t i = 0; i < list.size(); ++i) if (list[i] == t) s.index = (int64_t)i;
+      pl.src.push_back(s);
+    }
+    h->launches.push_back(pl);
+  } else {
+    // one launch per node; intermediates live in a workspace in their declared dtype
+    std::vector<int64_t> ws_off(g.tensors.size(), -1);
+    size_t ws = 0;
+    for (size_t t = 0; t < g.tensors.size(); ++t) {
+      if (g.tensors[t].role != 0 || g.tensors[t].producer < 0) continue;
+      ws_off[t] = (int64_t)ws;
+      ws += ((size_t)tensor_bytes(g.tensors[t]) + 255) / 256 * 256;
+    }
+    for (size_t ni = 0; ni < g.nodes.size(); ++ni) {
+      Graph sub;
+      std::vector<int> orig;
+      node_subgraph(g, g.nodes[ni], sub, orig);
+      PlannedLaunch pl;
+      st = lower_graph(sub, flags, dev, pl.plan, err);
+      if (st != PN_OK) { delete h; return fail(st, "node " + std::to_string(ni) + " (unfused): " + err); }
+      for (int q = 0; q < pl.plan.p.n_io; ++q) {
+        const int t = orig[pl.plan.io_tensor[q]];
+        IoSource s{2, ws_off[t]};
+        for (size_t i = 0; i < g.inputs.size(); ++i) if (g.inputs[i] == t) s = IoSource{0, (int64_t)i};
+        for (size_t i = 0; i < g.outputs.size(); ++i) if (g.outputs[i] == t) s = IoSource{1, (int64_t)i};
+        pl.src.push_back(s);
+      }
+      h->launches.push_back(pl);
+    }
+    h->workspace_bytes = ws;
+    if (!h->plan_only && ws > 0) {
+      cudaError_t e = cudaMalloc(&h->workspace, ws);
+      if (e != cudaSuccess) { delete h; return fail(PN_ERR_CUDA, std::string("workspace: ") + cudaGetErrorString(e)); }
+    }
+  }
+  *out = h;
+  return PN_OK;
+}
+
+pn_status pn_graph_run(pn_graph_t* h, const void* const* inputs, int n_inputs, void* const* outputs,
+                       int n_outputs, void* stream) {
+  pn_status st = check_counts(h, inputs, n_inputs, outputs, n_outputs);
+  if (st != PN_OK) return st;
+  const Graph& g = h->g;
+  if (any_empty(g)) return PN_OK;   // nothing to compute
+  const bool scalar = (h->flags & PN_FLAG_FORCE_SCALAR) != 0;
+  for (int i = 0; i < n_inputs; ++i) {
+    if (!inputs[i]) return fail(PN_ERR_INVALID_ARG, "input " + std::to_string(i) + " is null");
+    const uintptr_t m = scalar ? (uintptr_t)(dtype_bytes(g.tensors[g.inputs[i]].dtype) - 1) : 15;
+    if ((uintptr_t)inputs[i] & m) return fail(PN_ERR_ALIGNMENT, "input " + std::to_string(i) + " is not aligned");
+  }
+  for (int i = 0; i < n_outputs; ++i) {
+    if (!outputs[i]) return fail(PN_ERR_INVALID_ARG, "output " + std::to_string(i) + " is null");
+    const uintptr_t m = scalar ? (uintptr_t)(dtype_bytes(g.tensors[g.outputs[i]].dtype) - 1) : 15;
+    if ((uintptr_t)outputs[i] & m) return fail(PN_ERR_ALIGNMENT, "output " + std::to_string(i) + " is not aligned");
+  }
+  // inputs go through the read-only data path: none may overlap an output; outputs are
+  // written independently: none may overlap another
+  for (int o = 0; o < n_outputs; ++o) {
+    const char* b0 = (const char*)outputs[o];
+    const char* b1 = b0 + tensor_bytes(g.tensors[g.outputs[o]]);
+    for (int i = 0; i < n_inputs; ++i) {
+      const char* a0 = (const char*)inputs[i];
+      const char* a1 = a0 + tensor_bytes(g.tensors[g.inputs[i]]);
+      if (a0 < b1 && b0 < a1) return fail(PN_ERR_INVALID_ARG, "input " + std::to_string(i) + " overlaps output " + std::to_string(o));
+    }
+    for (int i = 0; i < o; ++i) {
+      const char* a0 = (const char*)outputs[i];
+      const char* a1 = a0 + tensor_bytes(g.tensors[g.outputs[i]]);
+      if (a0 < b1 && b0 < a1) return fail(PN_ERR_INVALID_ARG, "outputs " + std::to_string(i) + " and " + std::to_string(o) + " overlap");
+    }
+  }
+  for (PlannedLaunch& pl : h->launches) {
+    for (int q = 0; q < pl.plan.p.n_io; ++q) {
+      const IoSource& s = pl.src[q];
+      pl.plan.p.io[q].base = s.kind == 0 ? const_cast<void*>(inputs[s.index])
+                           : s.kind == 1 ? outputs[s.index]
+                                         : (void*)((char*)h->workspace + s.index);
+    }
+    cudaError_t e = launch_plan(pl.plan, (cudaStream_t)stream);
+    if (e != cudaSuccess) return fail(PN_ERR_CUDA, std::string("launch: ") + cudaGetErrorString(e));
+  }
+  return PN_OK;
+}
+
+pn_status pn_graph_run_host(pn_graph_t* h, const void* const* inputs, int n_inputs, void* const* outputs,
+                            int n_outputs, void* stream) {
+  pn_status st = check_counts(h, inputs, n_inputs, outputs, n_outputs);
+  if (st != PN_OK) return st;
+  const Graph& g = h->g;
+  if (any_empty(g)) return PN_OK;
+  cudaStream_t s = (cudaStream_t)stream;
+  cudaError_t e;
+  if (h->stage_in.empty() && h->stage_out.empty()) {
+    for (int pass = 0; pass < 2; ++pass)
+      for (int t : pass == 0 ? g.inputs : g.outputs) {
+        void* p = nullptr;
+        e = cudaMalloc(&p, std::max<size_t>((size_t)tensor_bytes(g.tensors[t]), 16));
+        if (e != cudaSuccess) return fail(PN_ERR_CUDA, std::string("staging: ") + cudaGetErrorString(e));
+        (pass == 0 ? h->stage_in : h->stage_out).push_back(p);
+      }
+  }
+  for (int i = 0; i < n_inputs; ++i) {
+    if (!inputs[i]) return fail(PN_ERR_INVALID_ARG, "input " + std::to_string(i) + " is null");
+    e = cudaMemcpyAsync(h->stage_in[i], inputs[i], (size_t)tensor_bytes(g.tensors[g.inputs[i]]), cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return fail(PN_ERR_CUDA, std::string("copy in: ") + cudaGetErrorString(e));
+  }
+  st = pn_graph_run(h, (const void* const*)h->stage_in.data(), n_inputs, h->stage_out.data(), n_outputs, stream);
+  if (st != PN_OK) return st;
+  for (int i = 0; i < n_outputs; ++i) {
+    if (!outputs[i]) return fail(PN_ERR_INVALID_ARG, "output " + std::to_string(i) + " is null");
+    e = cudaMemcpyAsync(outputs[i], h->stage_out[i], (size_t)tensor_bytes(g.tensors[g.outputs[i]]), cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return fail(PN_ERR_CUDA, std::string("copy out: ") + cudaGetErrorString(e));
+  }
+  e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return fail(PN_ERR_CUDA, std::string("sync: ") + cudaGetErrorString(e));
+  return PN_OK;
+}
+
+pn_status pn_graph_destroy(pn_graph_t* h) {
+  if (!h) return PN_OK;
+  if (!h->plan_only) {
+    if (h->workspace) cudaFree(h->workspace);
+    for (void* p : h->stage_in) cudaFree(p);
+    for (void* p : h->stage_out) cudaFree(p);
+  }
+  delete h;
+  return PN_OK;
+}
+
+pn_status pn_graph_query(const pn_graph_t* h, int what, void* out, size_t out_bytes) {
+  if (!h || !out) return fail(PN_ERR_INVALID_ARG, "null argument");
+  const Graph& g = h->g;
+  std::vector<int64_t> v;
+  auto meta = [&](const std::vector<int>& ids) {
+    for (int t : ids) {
+      const Tensor& T = g.tensors[t];
+      v.push_back(T.dtype); v.push_back(T.rank);
+      for (int d = 0; d < 4; ++d) v.push_back(d < T.rank ? T.dims[d] : 0);
+    }
+  };
+  switch (what) {
+    case PN_Q_N_INPUTS: v.push_back((int64_t)g.inputs.size()); break;
+    case PN_Q_N_OUTPUTS: v.push_back((int64_t)g.outputs.size()); break;
+    case PN_Q_INPUT_META: meta(g.inputs); break;
+    case PN_Q_OUTPUT_META: meta(g.outputs); break;
+    case PN_Q_COMPULSORY_BYTES: v.push_back(h->compulsory_bytes); break;
+    case PN_Q_N_KERNELS: v.push_back((int64_t)h->launches.size()); break;
+    case PN_Q_N_NODES: v.push_back((int64_t)g.nodes.size()); break;
+    case PN_Q_WORKSPACE_BYTES: v.push_back((int64_t)h->workspace_bytes); break;
+    case PN_Q_KERNEL_INFO:
+      for (const PlannedLaunch& pl : h->launches) {
+        const LaunchPlan& p = pl.plan;
+        const int64_t row[12] = {p.family, p.grid, p.block, p.p.cluster, p.smem_bytes, p.vl, p.ng, p.p.chunks,
+                                 p.code_words, p.p.n_stages, p.p.rows, p.p.row_len};
+        v.insert(v.end(), row, row + 12);
+      }
+      break;
+    default: return fail(PN_ERR_INVALID_ARG, "unknown query");
+  }
+  if (out_bytes < v.size() * sizeof(int64_t)) return fail(PN_ERR_INVALID_ARG, "query buffer too small");
+  if (!v.empty()) memcpy(out, v.data(), v.size() * sizeof(int64_t));
+  return PN_OK;
+}
+
+const char* pn_status_string(pn_status s) {
+  switch (s) {
+    case PN_OK: return "ok";
+    case PN_ERR_INVALID_ARG: return "invalid argument";
+    case PN_ERR_BAD_DESCRIPTOR: return "malformed descriptor";
+    case PN_ERR_UNSUPPORTED_OP: return "unsupported operator or combination";
+    case PN_ERR_SHAPE: return "shape error";
+    case PN_ERR_TOO_LARGE: return "graph exceeds a kernel budget";
+    case PN_ERR_ALIGNMENT: return "pointer alignment";
+    case PN_ERR_COUNT: return "wrong number of inputs or outputs";
+    case PN_ERR_DEVICE: return "device error";
+    case PN_ERR_CUDA: return "CUDA error";
+    default: return "unknown status";
+  }
+}
+
+const char* pn_last_error(void) { return g_last_error.c_str(); }
+
+#pragma GCC visibility pop
+}  // extern "C"

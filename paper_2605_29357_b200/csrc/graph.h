@@ -1,0 +1,68 @@
+// graph.h -- host-side representation of a parsed descriptor, and the lowering entry points.
+#pragma once
+#include <stddef.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "plan.h"
+
+namespace pn {
+
+// opcodes of descriptor format version 1
+enum NodeOp : uint16_t {
+  N_NEG = 1, N_ABS, N_EXP, N_LOG, N_SQRT, N_RSQRT, N_RECIP, N_TANH, N_SIGMOID, N_SILU,
+  N_GELU_TANH, N_GELU_ERF, N_RELU, N_CAST, N_SQUARE, N_ERF,
+  N_ADD = 32, N_SUB, N_MUL, N_DIV, N_MAX, N_MIN, N_GT, N_GE, N_LT, N_LE, N_EQ, N_NE,
+  N_WHERE = 64, N_CLAMP, N_FMA,
+  N_SUM = 96, N_MEAN, N_VAR, N_AMAX, N_AMIN, N_ARGMAX, N_ARGMIN, N_LOGSUMEXP,
+  N_SOFTMAX = 128, N_LOG_SOFTMAX, N_LAYER_NORM, N_RMS_NORM
+};
+
+constexpr uint32_t kImm0 = 0xFFFFFFFFu, kImm1 = 0xFFFFFFFEu;
+
+struct Tensor {
+  uint8_t dtype = 0;
+  uint8_t role = 0;        // bit0 input, bit1 output
+  int rank = 0;
+  int64_t dims[4] = {1, 1, 1, 1};
+  int producer = -1;       // node index, -1 for graph inputs
+  int64_t numel() const { int64_t n = 1; for (int i = 0; i < rank; ++i) n *= dims[i]; return n; }
+};
+
+struct Node {
+  uint16_t op = 0;
+  int n_in = 0, n_out = 0;
+  uint32_t in[4] = {0, 0, 0, 0};
+  uint32_t out[3] = {0, 0, 0};
+  double imm[2] = {0, 0};
+  int64_t attr[2] = {0, 0};
+};
+
+struct Graph {
+  std::vector<Tensor> tensors;
+  std::vector<Node> nodes;
+  std::vector<int> inputs, outputs;   // tensor ids in pointer-array order
+};
+
+inline int dtype_bytes(int dt) {
+  switch (dt) { case kF32: case kI32: return 4; case kF16: case kBF16: return 2; case kI64: return 8; default: return 1; }
+}
+inline bool dtype_is_float(int dt) { return dt == kF32 || dt == kF16 || dt == kBF16; }
+inline bool is_reduction(uint16_t op) { return op >= N_SUM && op <= N_LOGSUMEXP; }
+inline bool is_composite(uint16_t op) { return op >= N_SOFTMAX && op <= N_RMS_NORM; }
+
+// Returns a pn_status value (see pn.h).
+int parse_descriptor(const void* desc, size_t bytes, Graph& g, std::string& err);
+
+struct DeviceModel {      // what the lowering needs to know about the GPU
+  int sm_count = 148;
+  int max_smem_per_block = 227 * 1024;
+  bool have_device = false;   // occupancy queries allowed
+};
+
+// Lower a whole graph into one fused launch.  Returns a pn_status value.
+int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPlan& out, std::string& err);
+
+}  // namespace pn

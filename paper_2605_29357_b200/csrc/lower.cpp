@@ -1,0 +1,787 @@
+// lower.cpp -- host lowering of a validated graph into one fused launch.
+//
+// Steps: (1) shape analysis: the iteration space [rows, N] (N = last dim), which tensors
+// are tile values (one element per column) and which are per-row scalars (results of
+// last-dim reductions); (2) expansion of every node into tile / reduction / scalar
+// micro-operations, split into stages at reduction boundaries; (3) choice of the kernel
+// family and tile shape from (rows, N, dtypes, SM count) -- the per-shape cost model whose
+// absence the paper names as a failure mode ("static tiling across varying shapes",
+// Section 4.4); (4) accumulator-machine code generation with register allocation;
+// (5) shared-memory layout and grid.
+#include <math.h>
+#include <string.h>
+
+#include <algorithm>
+#include <map>
+#include <string>
+#include <vector>
+
+#include "../../include/pn.h"
+#include "graph.h"
+
+namespace pn {
+
+int instance_occupancy(int vl, int ng, int k, int block, int smem_bytes);  // kernels.cu
+
+namespace {
+
+enum ValKind { VK_E, VK_S, VK_IMM };
+
+struct Val {
+  ValKind kind = VK_E;
+  int stage = 0;
+  int io = -1;          // tile value that is a graph input not loaded yet
+  bool bcast = false;   // that input has col_stride 0
+  bool streamed = false;// that input has one element per element of the iteration space
+  float imm = 0.f;
+  int slot = -1;        // per-row scalar: its shared-memory slot
+  bool int_bits = false;// slot holds int32 bits (argmax / argmin)
+  bool has_ts = false;  // exp(x - m_tile) of a softmax: travels with the tile scalar
+  bool integral = false;// known to hold integer / 0-1 values
+  int uses = 0;
+};
+
+struct MOp {
+  int op = OP_END;      // VM opcode
+  int stage = 0;
+  bool scalar = false;
+  int nin = 0;
+  int in[3] = {-1, -1, -1};
+  int out = -1;
+  int aux0 = 0, aux1 = 0;
+};
+
+struct Shape4 { int64_t d[4]; };
+
+Shape4 align4(const Tensor& t) {
+  Shape4 s{{1, 1, 1, 1}};
+  for (int i = 0; i < t.rank; ++i) s.d[4 - t.rank + i] = t.dims[i];
+  return s;
+}
+
+bool bcast_into(Shape4& acc, const Shape4& s) {
+  for (int i = 0; i < 4; ++i) {
+    if (acc.d[i] == s.d[i] || s.d[i] == 1) continue;
+    if (acc.d[i] == 1) { acc.d[i] = s.d[i]; continue; }
+    return false;
+  }
+  return true;
+}
+
+int vm_unary(uint16_t op) {
+  switch (op) {
+    case N_NEG: return OP_NEG; case N_ABS: return OP_ABS; case N_EXP: return OP_EXP; case N_LOG: return OP_LOG;
+    case N_SQRT: return OP_SQRT; case N_RSQRT: return OP_RSQRT; case N_RECIP: return OP_RECIP;
+    case N_TANH: return OP_TANH; case N_SIGMOID: return OP_SIGMOID; case N_SILU: return OP_SILU;
+    case N_GELU_TANH: return OP_GELU_TANH; case N_GELU_ERF: return OP_GELU_ERF; case N_RELU: return OP_RELU;
+    case N_SQUARE: return OP_SQUARE; case N_ERF: return OP_ERF;
+  }
+  return -1;
+}
+int vm_binary(uint16_t op) {
+  switch (op) {
+    case N_ADD: return OP_ADD; case N_SUB: return OP_SUB; case N_MUL: return OP_MUL; case N_DIV: return OP_DIV;
+    case N_MAX: return OP_MAX; case N_MIN: return OP_MIN; case N_GT: return OP_GT; case N_GE: return OP_GE;
+    case N_LT: return OP_LT; case N_LE: return OP_LE; case N_EQ: return OP_EQ; case N_NE: return OP_NE;
+  }
+  return -1;
+}
+// opcode computing op(y, x) when acc holds y instead of x
+int swapped(int op) {
+  switch (op) {
+    case OP_SUB: return OP_RSUB; case OP_RSUB: return OP_SUB; case OP_DIV: return OP_RDIV; case OP_RDIV: return OP_DIV;
+    case OP_GT: return OP_LT; case OP_LT: return OP_GT; case OP_GE: return OP_LE; case OP_LE: return OP_GE;
+    default: return op;  // commutative
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// code generation for one program (tile program of a stage, or a per-row scalar program)
+// ---------------------------------------------------------------------------------------
+struct Gen {
+  std::vector<uint32_t>& code;
+  std::vector<Val>& vals;
+  const bool scalar;
+  const int K;
+  const bool multichunk;
+  int accv = -1;
+  std::vector<int> regv;
+  std::vector<char> regraw;
+  std::map<int, int>& stash_of;   // value -> stash index (shared over the stages)
+  int& n_stash;
+  std::string err;
+
+  Gen(std::vector<uint32_t>& c, std::vector<Val>& v, bool sc, int k, bool mc, std::map<int, int>& so, int& ns)
+      : code(c), vals(v), scalar(sc), K(k), multichunk(mc), regv(k, -1), regraw(k, 0), stash_of(so), n_stash(ns) {}
+
+  void emit(int op, int a = 0, int b = 0, int c = 0) {
+    code.push_back((uint32_t)op | ((uint32_t)a << 8) | ((uint32_t)b << 16) | ((uint32_t)c << 24));
+  }
+  void emit_f(float f) { uint32_t u; memcpy(&u, &f, 4); code.push_back(u); }
+  int find_reg(int v) const { for (int k = 0; k < K; ++k) if (regv[k] == v) return k; return -1; }
+  int free_reg() {
+    for (int k = 0; k < K; ++k) if (regv[k] < 0) return k;
+    for (int k = 0; k < K; ++k) if (vals[regv[k]].uses <= 0) { regv[k] = -1; regraw[k] = 0; return k; }
+    err = "expression needs more tile registers than the kernel instance has";
+    return -1;
+  }
+  int n_free() const { int n = 0; for (int k = 0; k < K; ++k) n += regv[k] < 0; return n; }
+  void widen_if_raw(int k) { if (regraw[k]) { emit(OP_WIDEN, vals[regv[k]].io, k); regraw[k] = 0; } }
+  void drop_dead() {
+    for (int k = 0; k < K; ++k) if (regv[k] >= 0 && vals[regv[k]].uses <= 0) { regv[k] = -1; regraw[k] = 0; }
+    if (accv >= 0 && vals[accv].uses <= 0) accv = -1;
+  }
+  bool save_acc() {   // acc is about to be overwritten
+    if (accv < 0 || vals[accv].uses <= 0 || find_reg(accv) >= 0) return true;
+    if (vals[accv].kind != VK_E) return true;   // scalars live in their slots
+    const int k = free_reg();
+    if (k < 0) return false;
+    emit(OP_ST, k); regv[k] = accv; regraw[k] = 0;
+    return true;
+  }
+  void load_input(int v, int target) {   // target = K names acc
+    const Val& x = vals[v];
+    if (x.bcast) emit(OP_LDBC, x.io, target);
+    else { emit(OP_LDRAW, x.io, target); emit(OP_WIDEN, x.io, target); }
+  }
+  bool place_in_acc(int v) {
+    if (accv == v) return true;
+    if (!save_acc()) return false;
+    const Val& x = vals[v];
+    if (x.kind == VK_S) { emit(OP_SLD, x.slot); accv = v; return true; }
+    if (x.kind == VK_IMM) { err = "constant-only subexpression is not lowered"; return false; }
+    const int k = find_reg(v);
+    if (k >= 0) { widen_if_raw(k); emit(OP_LD, k); }
+    else if (stash_of.count(v)) { emit(OP_FILL, K, stash_of[v]); if (x.has_ts) emit(OP_FILL_TS, 0, stash_of[v] + 1); }
+    else if (x.io >= 0) load_input(v, K);
+    else { err = "internal: tile value has no location"; return false; }
+    accv = v;
+    return true;
+  }
+  struct Src { int idx = 0, kind = OPK_REG; float imm = 0.f; };
+  bool src_operand(int v, Src& s) {
+    const Val& x = vals[v];
+    if (x.kind == VK_IMM) { s.kind = OPK_IMM; s.imm = x.imm; return true; }
+    if (x.kind == VK_S) { s.kind = OPK_SLOT; s.idx = x.slot; return true; }
+    int k = find_reg(v);
+    if (k >= 0) { widen_if_raw(k); s.idx = k; return true; }
+    k = free_reg();
+    if (k < 0) return false;
+    if (accv == v) emit(OP_ST, k);
+    else if (stash_of.count(v)) emit(OP_FILL, k, stash_of[v]);
+    else if (x.io >= 0) load_input(v, k);
+    else { err = "internal: tile operand has no location"; return false; }
+    regv[k] = v; regraw[k] = 0; s.idx = k;
+    return true;
+  }
+  // after an op consumed `v` from acc: keep a copy if others still need it
+  bool keep_if_live(int v) {
+    if (vals[v].kind != VK_E || vals[v].uses <= 0 || find_reg(v) >= 0 || stash_of.count(v)) return true;
+    const int k = free_reg();
+    if (k < 0) return false;
+    emit(OP_ST, k); regv[k] = v; regraw[k] = 0;
+    return true;
+  }
+  void result(int r) {
+    accv = r;
+    if (scalar && r >= 0 && vals[r].kind == VK_S) emit(OP_SST, vals[r].slot);
+    drop_dead();
+  }
+  bool is_tile(int v) const { return vals[v].kind == (scalar ? VK_S : VK_E); }
+
+  bool gen(const MOp& m) {
+    switch (m.op) {
+      case OP_STOUT: case OP_STOUT_I: {
+        if (!place_in_acc(m.in[0])) return false;
+        vals[m.in[0]].uses--;
+        emit(m.op, m.aux0);
+        drop_dead();
+        return true;
+      }
+      case OP_RED: {
+        if (!place_in_acc(m.in[0])) return false;
+        vals[m.in[0]].uses--;
+        if (m.aux0 == RED_SOFTMAX) {
+          if (!keep_if_live(m.in[0])) return false;
+          emit(OP_RED, m.aux0, m.aux1);
+          result(m.out);
+        } else {
+          emit(OP_RED, m.aux0, m.aux1);
+          drop_dead();
+        }
+        return true;
+      }
+      case OP_SCALE_TS: {
+        if (!place_in_acc(m.in[0])) return false;
+        vals[m.in[0]].uses--;
+        if (!keep_if_live(m.in[0])) return false;
+        emit(OP_SCALE_TS, m.aux0, m.aux1);
+        result(m.out);
+        return true;
+      }
+      case OP_WHERE: case OP_FMA: {
+        int x = m.in[0], X = m.in[1], Y = m.in[2];
+        if (m.op == OP_FMA && !is_tile(x) && is_tile(X)) std::swap(x, X);
+        if (vals[x].kind == VK_IMM) { err = "where / fma with a constant first operand is not lowered"; return false; }
+        if (!place_in_acc(x)) return false;
+        Src sx, sy;
+        if (!src_operand(X, sx) || !src_operand(Y, sy)) return false;
+        vals[x].uses--; vals[X].uses--; vals[Y].uses--;
+        if (!keep_if_live(x)) return false;
+        emit(m.op, sx.idx, sy.idx, sx.kind | (sy.kind << 4));
+        if (sx.kind == OPK_IMM) emit_f(sx.imm);
+        if (sy.kind == OPK_IMM) emit_f(sy.imm);
+        result(m.out);
+        return true;
+      }
+      default: break;
+    }
+    if (m.nin == 1) {   // unary
+      if (!place_in_acc(m.in[0])) return false;
+      vals[m.in[0]].uses--;
+      if (!keep_if_live(m.in[0])) return false;
+      emit(m.op);
+      result(m.out);
+      return true;
+    }
+    // binary
+    int op = m.op, x = m.in[0], y = m.in[1];
+    const bool xt = is_tile(x), yt = is_tile(y);
+    if ((!xt && yt) || (xt && yt && accv == y && accv != x)) { std::swap(x, y); op = swapped(op); }
+    if (vals[x].kind == VK_IMM) { err = "constant-only subexpression is not lowered"; return false; }
+    if (!place_in_acc(x)) return false;
+    Src s;
+    if (!src_operand(y, s)) return false;
+    vals[x].uses--; vals[y].uses--;
+    if (!keep_if_live(x)) return false;
+    emit(op, s.idx, s.kind);
+    if (s.kind == OPK_IMM) emit_f(s.imm);
+    result(m.out);
+    return true;
+  }
+
+  // Issue the loads of this stage's inputs before any arithmetic, so that they are all in
+  // flight together; the large (streamed) operands first.
+  void hoist_loads(const std::vector<MOp>& ops, int stage) {
+    if (scalar) return;
+    for (int pass = 0; pass < 2; ++pass)
+      for (const MOp& m : ops) {
+        if (m.stage != stage || m.scalar) continue;
+        for (int i = 0; i < m.nin; ++i) {
+          const int v = m.in[i];
+          if (v < 0 || vals[v].kind != VK_E || vals[v].io < 0 || vals[v].bcast) continue;
+          if (vals[v].streamed != (pass == 0)) continue;
+          if (find_reg(v) >= 0 || accv == v || stash_of.count(v)) continue;
+          if (n_free() <= 1) return;
+          const int k = free_reg();
+          emit(OP_LDRAW, vals[v].io, k);
+          regv[k] = v; regraw[k] = 1;
+        }
+      }
+  }
+
+  // End of a stage: tile values still needed later stay in registers (one chunk per thread)
+  // or are parked in shared memory (several chunks per thread).
+  bool end_stage() {
+    if (scalar) { accv = -1; return true; }
+    if (!multichunk) return save_acc();
+    auto park = [&](int v, int k) {
+      stash_of[v] = n_stash; emit(OP_SPILL, k, n_stash); n_stash++;
+      if (vals[v].has_ts) { emit(OP_SPILL_TS, 0, n_stash); n_stash++; }
+    };
+    if (accv >= 0 && vals[accv].uses > 0 && vals[accv].kind == VK_E && find_reg(accv) < 0 && !stash_of.count(accv))
+      park(accv, K);
+    for (int k = 0; k < K; ++k) {
+      const int v = regv[k];
+      if (v >= 0 && vals[v].uses > 0 && !stash_of.count(v)) { widen_if_raw(k); park(v, k); }
+      regv[k] = -1; regraw[k] = 0;
+    }
+    accv = -1;
+    return true;
+  }
+};
+
+struct Config { int family, vl, ng, k, block, cluster, chunks, slice_len; bool multichunk; };
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------
+int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPlan& lp, std::string& err) {
+  const int nt = (int)g.tensors.size();
+  std::vector<char> is_s(nt, 0);
+  std::vector<int> n_consumers(nt, 0);
+  bool has_red = false;
+
+  // ---- (1) shapes ---------------------------------------------------------------------
+  for (const Node& n : g.nodes) {
+    if (is_reduction(n.op) || is_composite(n.op)) has_red = true;
+    for (int k = 0; k < n.n_in; ++k) if (n.in[k] < (uint32_t)nt) n_consumers[n.in[k]]++;
+  }
+  for (const Node& n : g.nodes) {   // per-row scalars
+    if (is_reduction(n.op)) is_s[n.out[0]] = 1;
+    else if (n.op == N_LAYER_NORM) { for (int k = 1; k < n.n_out; ++k) is_s[n.out[k]] = 1; }
+    else if (!is_composite(n.op)) {
+      bool any_t = false, all_s = true;
+      for (int k = 0; k < n.n_in; ++k) {
+        if (n.in[k] >= (uint32_t)nt) continue;
+        any_t = true;
+        all_s = all_s && is_s[n.in[k]];
+      }
+      if (!any_t) { err = "a node with only constant operands is not lowered"; return PN_ERR_UNSUPPORTED_OP; }
+      if (all_s) is_s[n.out[0]] = 1;
+    }
+  }
+  Shape4 F{{1, 1, 1, 1}};
+  bool have_full = false;
+  for (const Node& n : g.nodes) {
+    if (is_reduction(n.op) || is_composite(n.op)) {
+      const Shape4 s = align4(g.tensors[n.in[0]]);
+      if (!have_full) { F = s; have_full = true; }
+      else if (memcmp(&F, &s, sizeof(s)) != 0) { err = "all reductions of a graph must act on the same shape"; return PN_ERR_SHAPE; }
+    }
+  }
+  for (int t = 0; t < nt; ++t) {
+    if (is_s[t]) continue;
+    const Shape4 s = align4(g.tensors[t]);
+    if (has_red) {
+      for (int i = 0; i < 4; ++i)
+        if (s.d[i] != 1 && s.d[i] != F.d[i]) { err = "tensor " + std::to_string(t) + " does not broadcast into the iteration space"; return PN_ERR_SHAPE; }
+    } else if (!bcast_into(F, s)) { err = "tensor " + std::to_string(t) + ": shapes do not broadcast"; return PN_ERR_SHAPE; }
+  }
+  const int64_t rows = F.d[0] * F.d[1] * F.d[2];
+  const int64_t N = F.d[3];
+  if (N <= 0) { err = "the last dimension is empty"; return PN_ERR_SHAPE; }
+  if (N >= (int64_t(1) << 30)) { err = "last dimension too long"; return PN_ERR_TOO_LARGE; }
+  for (size_t ni = 0; ni < g.nodes.size(); ++ni) {   // per-node shape rules
+    const Node& n = g.nodes[ni];
+    const std::string where = "node " + std::to_string(ni) + ": ";
+    auto row_shaped = [&](const Tensor& t, const Tensor& src) {
+      if (t.rank == src.rank - 1) { for (int i = 0; i < t.rank; ++i) if (t.dims[i] != src.dims[i]) return false; return true; }
+      if (t.rank == src.rank) { for (int i = 0; i + 1 < t.rank; ++i) if (t.dims[i] != src.dims[i]) return false; return t.rank > 0 && t.dims[t.rank - 1] == 1; }
+      return false;
+    };
+    if (is_reduction(n.op) || is_composite(n.op)) {
+      const Tensor& src = g.tensors[n.in[0]];
+      if (src.rank < 1) { err = where + "reduction of a rank-0 tensor"; return PN_ERR_SHAPE; }
+      if (is_s[n.in[0]]) { err = where + "reduction of a per-row result"; return PN_ERR_UNSUPPORTED_OP; }
+      if (is_reduction(n.op)) {
+        if (!row_shaped(g.tensors[n.out[0]], src)) { err = where + "result must have the input's shape with the last dim dropped or 1"; return PN_ERR_SHAPE; }
+        if ((n.op == N_ARGMAX || n.op == N_ARGMIN) && g.tensors[n.out[0]].dtype != kI64 && g.tensors[n.out[0]].dtype != kI32) {
+          err = where + "argmax / argmin results must be i32 or i64"; return PN_ERR_UNSUPPORTED_OP;
+        }
+      } else {
+        const Tensor& y = g.tensors[n.out[0]];
+        if (y.rank != src.rank || memcmp(y.dims, src.dims, sizeof(int64_t) * 4) != 0) { err = where + "output shape differs from the input's"; return PN_ERR_SHAPE; }
+        for (int k = 1; k < n.n_out; ++k)
+          if (!row_shaped(g.tensors[n.out[k]], src)) { err = where + "mean / rstd must have the per-row shape"; return PN_ERR_SHAPE; }
+      }
+    } else {
+      Shape4 b{{1, 1, 1, 1}};
+      for (int k = 0; k < n.n_in; ++k)
+        if (n.in[k] < (uint32_t)nt && !bcast_into(b, align4(g.tensors[n.in[k]]))) { err = where + "operands do not broadcast"; return PN_ERR_SHAPE; }
+      const Shape4 o = align4(g.tensors[n.out[0]]);
+      if (memcmp(&b, &o, sizeof(o)) != 0) { err = where + "declared output shape is not the broadcast of the operands"; return PN_ERR_SHAPE; }
+    }
+  }
+  for (int o : g.outputs) {
+    if (is_s[o]) continue;
+    const Shape4 s = align4(g.tensors[o]);
+    if (memcmp(&s, &F, sizeof(s)) != 0) { err = "output tensor " + std::to_string(o) + " must have the full iteration shape or be a per-row result"; return PN_ERR_UNSUPPORTED_OP; }
+  }
+
+  // ---- io table ------------------------------------------------------------------------
+  memset(&lp, 0, sizeof(lp));
+  KernelParams& P = lp.p;
+  const int n_io = (int)(g.inputs.size() + g.outputs.size());
+  if (n_io > kMaxIo) { err = "more graph inputs + outputs than one kernel takes (" + std::to_string(kMaxIo) + ")"; return PN_ERR_TOO_LARGE; }
+  P.n_io = n_io;
+  std::vector<int> io_of_tensor(nt, -1);
+  std::vector<char> io_streamed(n_io, 0);
+  {
+    int idx = 0;
+    auto add_io = [&](int t, bool is_out) {
+      IoDesc& io = P.io[idx];
+      const Tensor& T = g.tensors[t];
+      io.dtype = T.dtype;
+      if (is_s[t]) {   // one element per row, dense over the leading dims
+        io.is_row_scalar = 1; io.col_stride = 0;
+        io.lead_stride[2] = 1; io.lead_stride[1] = F.d[2]; io.lead_stride[0] = F.d[2] * F.d[1];
+      } else {
+        const Shape4 s = align4(T);
+        int64_t st = 1, strides[4];
+        bool full = true;
+        for (int i = 3; i >= 0; --i) { strides[i] = (s.d[i] == 1 && F.d[i] != 1) ? 0 : st; st *= s.d[i]; full = full && s.d[i] == F.d[i]; }
+        for (int i = 0; i < 3; ++i) io.lead_stride[i] = F.d[i] == 1 ? 0 : strides[i];
+        io.col_stride = (s.d[3] == 1 && N != 1) ? 0 : 1;
+        io_streamed[idx] = full;
+      }
+      lp.io_tensor[idx] = t; lp.io_is_output[idx] = is_out;
+      io_of_tensor[t] = idx++;
+    };
+    for (int t : g.inputs) add_io(t, false);
+    for (int t : g.outputs) add_io(t, true);
+  }
+  // collapse leading dims that every io walks contiguously (or broadcasts) together
+  int64_t lead_dim[3] = {F.d[0], F.d[1], F.d[2]};
+  for (int pass = 0; pass < 2; ++pass) {
+    for (int i = 1; i >= 0; --i) {   // try merging dim i into dim i+1
+      if (lead_dim[i] == 1) continue;
+      bool ok = true;
+      if (lead_dim[i + 1] != 1)
+        for (int q = 0; q < n_io && ok; ++q) ok = P.io[q].lead_stride[i] == P.io[q].lead_stride[i + 1] * lead_dim[i + 1];
+      if (!ok) continue;
+      for (int q = 0; q < n_io; ++q) {
+        IoDesc& io = P.io[q];
+        if (lead_dim[i + 1] == 1) io.lead_stride[i + 1] = io.lead_stride[i];
+        io.lead_stride[i] = 0;
+      }
+      lead_dim[i + 1] *= lead_dim[i]; lead_dim[i] = 1;
+    }
+  }
+  for (int i = 0; i < 3; ++i) if (lead_dim[i] > 0xFFFFFFFFll) { err = "leading dimension too large"; return PN_ERR_TOO_LARGE; }
+  int64_t eff_rows = rows, eff_N = N;
+  // a purely pointwise graph whose tensors all have the full shape is one long row
+  if (!has_red && rows > 1 && rows * N < (int64_t(1) << 30) && lead_dim[0] == 1 && lead_dim[1] == 1) {
+    bool flat = true;
+    for (int q = 0; q < n_io; ++q) flat = flat && P.io[q].col_stride == 1 && P.io[q].lead_stride[2] == N;
+    if (flat) { eff_N = rows * N; eff_rows = 1; lead_dim[2] = 1; for (int q = 0; q < n_io; ++q) P.io[q].lead_stride[2] = 0; }
+  }
+  for (int i = 0; i < 3; ++i) P.lead_dim[i] = (uint32_t)std::max<int64_t>(lead_dim[i], 1);
+  P.rows = eff_rows;
+  P.row_len = (int32_t)eff_N;
+
+  // ---- (2) micro-operations --------------------------------------------------------------
+  std::vector<Val> vals;
+  std::vector<MOp> ops;
+  std::vector<int> tval(nt, -1);
+  int n_slots = 0;
+  std::vector<std::vector<RedDesc>> stage_reds(kMaxStages);
+  std::map<std::pair<int, int>, int> red_cache;   // (kind, value) -> first slot
+  auto new_val = [&](ValKind k, int stage) { Val v; v.kind = k; v.stage = stage; vals.push_back(v); return (int)vals.size() - 1; };
+  auto new_slot = [&](int n) { int s = n_slots; n_slots += n; return s; };
+  auto add_op = [&](int op, int stage, bool scalar, std::initializer_list<int> in, int out, int a0 = 0, int a1 = 0) {
+    MOp m; m.op = op; m.stage = stage; m.scalar = scalar; m.nin = 0;
+    for (int v : in) m.in[m.nin++] = v;
+    m.out = out; m.aux0 = a0; m.aux1 = a1; ops.push_back(m);
+  };
+  for (int t : g.inputs) {
+    const int v = new_val(VK_E, 0);
+    const int q = io_of_tensor[t];
+    vals[v].io = q;
+    vals[v].bcast = P.io[q].col_stride == 0;
+    vals[v].streamed = io_streamed[q];
+    vals[v].integral = !dtype_is_float(g.tensors[t].dtype);
+    tval[t] = v;
+  }
+  std::vector<char> feeds_var(nt, 0);
+  for (const Node& n : g.nodes) if (n.op == N_VAR) feeds_var[n.in[0]] = 1;
+
+  auto pointwise = [&](int vmop, std::initializer_list<int> in, bool integral) -> int {
+    bool any_e = false; int stage = 0;
+    for (int v : in) { any_e |= vals[v].kind == VK_E; stage = std::max(stage, vals[v].stage); }
+    const bool sc = !any_e;
+    const int r = new_val(sc ? VK_S : VK_E, stage);
+    vals[r].integral = integral;
+    if (sc) vals[r].slot = new_slot(1);
+    add_op(vmop, sc ? stage - 1 : stage, sc, in, r);
+    return r;
+  };
+  auto slot_val = [&](int slot, int stage, bool int_bits) { const int v = new_val(VK_S, stage); vals[v].slot = slot; vals[v].int_bits = int_bits; return v; };
+  auto imm_val = [&](double x) { const int v = new_val(VK_IMM, 0); vals[v].imm = (float)x; return v; };
+  // reduction of tile value x; returns the first of its 3 slots, -1 / -2 when a budget is hit
+  auto reduce = [&](int kind, int x, int* e_out) -> int {
+    const int s = vals[x].stage;
+    auto key = std::make_pair(kind, x);
+    if (kind != RED_SOFTMAX && red_cache.count(key)) return red_cache[key];
+    if (s >= kMaxStages - 1) return -1;
+    if ((int)stage_reds[s].size() >= kMaxRed) return -2;
+    const int base = new_slot(3);
+    RedDesc rd; rd.kind = (uint8_t)kind; rd.slot = (uint8_t)base;
+    const int ridx = (int)stage_reds[s].size();
+    stage_reds[s].push_back(rd);
+    int e = -1;
+    if (kind == RED_SOFTMAX) { e = new_val(VK_E, s); vals[e].has_ts = true; }
+    add_op(OP_RED, s, false, {x}, e, kind, ridx);
+    if (e_out) *e_out = e;
+    red_cache[key] = base;
+    return base;
+  };
+
+  int softmax_count = 0;
+  for (size_t ni = 0; ni < g.nodes.size(); ++ni) {
+    const Node& n = g.nodes[ni];
+    const std::string where = "node " + std::to_string(ni) + ": ";
+    int in[4] = {-1, -1, -1, -1};
+    for (int k = 0; k < n.n_in; ++k) {
+      if (n.in[k] == kImm0) in[k] = imm_val(n.imm[0]);
+      else if (n.in[k] == kImm1) in[k] = imm_val(n.imm[1]);
+      else in[k] = tval[n.in[k]];
+    }
+    int res[3] = {-1, -1, -1};
+    const Tensor& T0 = g.tensors[n.out[0]];
+    const double Nd = (double)N;
+    if (vm_unary(n.op) >= 0) {
+      if (vals[in[0]].int_bits) in[0] = pointwise(OP_I2F, {in[0]}, true);
+      res[0] = pointwise(vm_unary(n.op), {in[0]}, false);
+    } else if (n.op == N_CAST) {
+      const bool src_int = vals[in[0]].integral;
+      if (vals[in[0]].int_bits) {   // an index held as int32 bits
+        res[0] = dtype_is_float(T0.dtype) ? pointwise(OP_I2F, {in[0]}, true) : in[0];
+        if (T0.dtype == kBool) res[0] = pointwise(OP_NEZ, {pointwise(OP_I2F, {in[0]}, true)}, true);
+      }
+      else if (dtype_is_float(T0.dtype)) res[0] = in[0];
+      else if (T0.dtype == kBool) res[0] = (src_int && g.tensors[n.in[0]].dtype == kBool) ? in[0] : pointwise(OP_NEZ, {in[0]}, true);
+      else res[0] = src_int ? in[0] : pointwise(OP_TRUNC, {in[0]}, true);
+    } else if (vm_binary(n.op) >= 0) {
+      for (int k = 0; k < 2; ++k) if (vals[in[k]].int_bits) in[k] = pointwise(OP_I2F, {in[k]}, true);
+      res[0] = pointwise(vm_binary(n.op), {in[0], in[1]}, n.op >= N_GT);
+    } else if (n.op == N_WHERE || n.op == N_FMA) {
+      for (int k = 0; k < 3; ++k) if (vals[in[k]].int_bits) in[k] = pointwise(OP_I2F, {in[k]}, true);
+      res[0] = pointwise(n.op == N_WHERE ? OP_WHERE : OP_FMA, {in[0], in[1], in[2]}, false);
+    } else if (n.op == N_CLAMP) {
+      for (int k = 0; k < 3; ++k) if (vals[in[k]].int_bits) in[k] = pointwise(OP_I2F, {in[k]}, true);
+      const int lo = pointwise(OP_MAX, {in[0], in[1]}, false);
+      res[0] = pointwise(OP_MIN, {lo, in[2]}, false);
+    } else if (is_reduction(n.op) || is_composite(n.op)) {
+      const int x = in[0];
+      if (vals[x].kind != VK_E) { err = where + "reduction of a per-row value"; return PN_ERR_UNSUPPORTED_OP; }
+      const int s1 = vals[x].stage + 1;
+      int base = 0;
+      auto bad = [&](int b) {
+        if (b == -1) { err = where + "more reduction-dependent stages than the kernel takes"; return true; }
+        if (b == -2) { err = where + "more reductions in one stage than the kernel takes"; return true; }
+        return false;
+      };
+      switch (n.op) {
+        case N_SUM: base = reduce(RED_SUM, x, nullptr); if (bad(base)) return PN_ERR_TOO_LARGE; res[0] = slot_val(base, s1, false); break;
+        case N_AMAX: base = reduce(RED_MAX, x, nullptr); if (bad(base)) return PN_ERR_TOO_LARGE; res[0] = slot_val(base, s1, false); break;
+        case N_AMIN: base = reduce(RED_MIN, x, nullptr); if (bad(base)) return PN_ERR_TOO_LARGE; res[0] = slot_val(base, s1, false); break;
+        case N_ARGMAX: base = reduce(RED_ARGMAX, x, nullptr); if (bad(base)) return PN_ERR_TOO_LARGE; res[0] = slot_val(base + 1, s1, true); break;
+        case N_ARGMIN: base = reduce(RED_ARGMIN, x, nullptr); if (bad(base)) return PN_ERR_TOO_LARGE; res[0] = slot_val(base + 1, s1, true); break;
+        case N_MEAN:
+          if (feeds_var[n.in[0]]) { base = reduce(RED_MEANVAR, x, nullptr); if (bad(base)) return PN_ERR_TOO_LARGE; res[0] = slot_val(base + 1, s1, false); }
+          else { base = reduce(RED_SUM, x, nullptr); if (bad(base)) return PN_ERR_TOO_LARGE; res[0] = pointwise(OP_DIV, {slot_val(base, s1, false), imm_val(Nd)}, false); }
+          break;
+        case N_VAR: {
+          base = reduce(RED_MEANVAR, x, nullptr); if (bad(base)) return PN_ERR_TOO_LARGE;
+          res[0] = pointwise(OP_DIV, {slot_val(base + 2, s1, false), imm_val(Nd - (double)n.attr[0])}, false);
+          break;
+        }
+        case N_LOGSUMEXP: case N_LOG_SOFTMAX: {
+          base = reduce(RED_LSE, x, nullptr); if (bad(base)) return PN_ERR_TOO_LARGE;
+          const int lse = pointwise(OP_LSEFIN, {slot_val(base, s1, false), slot_val(base + 1, s1, false)}, false);
+          res[0] = n.op == N_LOGSUMEXP ? lse : pointwise(OP_SUB, {x, lse}, false);
+          break;
+        }
+        case N_SOFTMAX: {
+          if (++softmax_count > 1) { err = where + "more than one softmax per graph is not lowered"; return PN_ERR_UNSUPPORTED_OP; }
+          int e = -1;
+          base = reduce(RED_SOFTMAX, x, &e); if (bad(base)) return PN_ERR_TOO_LARGE;
+          const int inv = pointwise(OP_RECIP, {slot_val(base + 1, s1, false)}, false);
+          const int r = new_val(VK_E, s1);
+          add_op(OP_SCALE_TS, s1, false, {e}, r, base, vals[inv].slot);
+          res[0] = r;
+          break;
+        }
+        case N_LAYER_NORM: {
+          base = reduce(RED_MEANVAR, x, nullptr); if (bad(base)) return PN_ERR_TOO_LARGE;
+          const int mean = slot_val(base + 1, s1, false);
+          const int var = pointwise(OP_DIV, {slot_val(base + 2, s1, false), imm_val(Nd)}, false);
+          const int ve = pointwise(OP_ADD, {var, imm_val(n.imm[0])}, false);
+          const int rstd = pointwise(OP_RSQRT, {ve}, false);
+          int y = pointwise(OP_SUB, {x, mean}, false);
+          y = pointwise(OP_MUL, {y, rstd}, false);
+          if (n.n_in > 1) y = pointwise(OP_MUL, {y, in[1]}, false);
+          if (n.n_in > 2) y = pointwise(OP_ADD, {y, in[2]}, false);
+          res[0] = y; res[1] = mean; res[2] = rstd;
+          break;
+        }
+        case N_RMS_NORM: {
+          const int sq = pointwise(OP_SQUARE, {x}, false);
+          base = reduce(RED_SUM, sq, nullptr); if (bad(base)) return PN_ERR_TOO_LARGE;
+          const int ms = pointwise(OP_DIV, {slot_val(base, s1, false), imm_val(Nd)}, false);
+          const int me = pointwise(OP_ADD, {ms, imm_val(n.imm[0])}, false);
+          const int r = pointwise(OP_RSQRT, {me}, false);
+          int y = pointwise(OP_MUL, {x, r}, false);
+          if (n.n_in > 1) y = pointwise(OP_MUL, {y, in[1]}, false);
+          res[0] = y;
+          break;
+        }
+      }
+    } else { err = where + "opcode not lowered"; return PN_ERR_UNSUPPORTED_OP; }
+
+    for (int k = 0; k < n.n_out; ++k) {
+      const int t = n.out[k];
+      const Tensor& T = g.tensors[t];
+      int v = res[k];
+      if (v < 0) { err = where + "internal: missing result"; return PN_ERR_UNSUPPORTED_OP; }
+      if (vals[v].stage >= kMaxStages) { err = where + "more reduction-dependent stages than the kernel takes"; return PN_ERR_TOO_LARGE; }
+      // a declared 16-bit float intermediate is rounded for its consumers
+      if ((T.dtype == kBF16 || T.dtype == kF16) && n_consumers[t] > 0 && !vals[v].integral && vals[v].kind != VK_IMM)
+        v = pointwise(T.dtype == kBF16 ? OP_RND_BF16 : OP_RND_F16, {v}, false);
+      tval[t] = v;
+      if (T.role & 2) {
+        if (vals[v].kind == VK_IMM) { err = where + "constant output"; return PN_ERR_UNSUPPORTED_OP; }
+        if (vals[v].int_bits && dtype_is_float(T.dtype)) v = pointwise(OP_I2F, {v}, true);
+        const bool sc = vals[v].kind == VK_S;
+        if (vals[v].int_bits && T.dtype != kI64 && T.dtype != kI32) { err = where + "index results must be stored as i32 or i64"; return PN_ERR_UNSUPPORTED_OP; }
+        add_op(vals[v].int_bits ? OP_STOUT_I : OP_STOUT, sc ? vals[v].stage - 1 : vals[v].stage, sc, {v}, -1, io_of_tensor[t]);
+      }
+    }
+  }
+  if (n_slots > kMaxSlots) { err = "more per-row scalars than the kernel takes"; return PN_ERR_TOO_LARGE; }
+  for (const MOp& m : ops) for (int i = 0; i < m.nin; ++i) vals[m.in[i]].uses++;
+  int n_stages = 1;
+  for (const MOp& m : ops) n_stages = std::max(n_stages, m.stage + 1);
+  if (n_stages > kMaxStages) { err = "more reduction-dependent stages than the kernel takes"; return PN_ERR_TOO_LARGE; }
+
+  // ---- (3) family and tile shape ---------------------------------------------------------
+  int min_esize = 8;
+  bool vec8 = true, vec4 = true;
+  for (int q = 0; q < n_io; ++q) {
+    const IoDesc& io = P.io[q];
+    if (io.is_row_scalar || io.col_stride == 0) continue;
+    if (io_streamed[q]) min_esize = std::min(min_esize, dtype_bytes(io.dtype));
+    for (int vl : {8, 4}) {
+      bool ok = eff_N % vl == 0;
+      for (int i = 0; i < 3; ++i) ok = ok && io.lead_stride[i] % vl == 0;
+      if (vl == 8) vec8 = vec8 && ok; else vec4 = vec4 && ok;
+    }
+  }
+  int VL = (min_esize <= 2 && vec8) ? 8 : (vec4 ? 4 : 1);
+  if (flags & PN_FLAG_FORCE_SCALAR) VL = 1;
+  std::vector<std::pair<int, int>> ng_opts;   // (NG, K): the 8-element tile first
+  if (VL == 8) ng_opts = {{1, 4}, {2, 2}};
+  else if (VL == 4) ng_opts = {{2, 4}, {4, 2}};
+  else ng_opts = {{8, 4}};
+
+  std::vector<Config> cands;
+  const int sms = dev.sm_count;
+  auto chunks_of = [&](int64_t len, int T, int ng) { const int64_t cap = (int64_t)T * VL * ng; return (int)((len + cap - 1) / cap); };
+  if (!has_red) {
+    for (auto o : ng_opts) cands.push_back(Config{FAM_POINTWISE, VL, o.first, o.second, 256, 1, chunks_of(eff_N, 32, o.first), (int)eff_N, false});
+  } else {
+    const bool fw = flags & PN_FLAG_FORCE_WARP, fb = flags & PN_FLAG_FORCE_BLOCK, fc = flags & PN_FLAG_FORCE_CLUSTER;
+    const bool fm = flags & PN_FLAG_FORCE_MULTICHUNK;
+    const bool any_force = fw || fb || fc;
+    const bool few_rows = eff_rows < 2ll * sms;
+    auto tile_ok = [&](int T, int ng) { return !(T > 256 && VL * ng > 8); };   // 16-element tiles: <= 256 threads
+    // one chunk per thread: the smallest team that holds the row
+    if (!fm && !fc) {
+      for (int T : {32, 64, 128, 256, 512}) {
+        if ((fw && T != 32) || (fb && T == 32)) continue;
+        for (auto o : ng_opts)
+          if (tile_ok(T, o.first) && (int64_t)T * VL * o.first >= eff_N)
+            cands.push_back(Config{T == 32 ? FAM_WARP : FAM_BLOCK, VL, o.first, o.second, T == 32 ? 256 : T, 1, 1, (int)eff_N, false});
+      }
+    }
+    // several chunks per thread
+    if (fw)
+      for (auto o : ng_opts) {
+        const int ch = chunks_of(eff_N, 32, o.first);
+        cands.push_back(Config{FAM_WARP, VL, o.first, o.second, 256, 1, ch, (int)eff_N, ch > 1});
+      }
+    if ((!any_force && !few_rows) || fb) {
+      std::vector<Config> mc;
+      for (int T : fm ? std::vector<int>{64} : std::vector<int>{256, 512})
+        for (auto o : ng_opts) {
+          if (!tile_ok(T, o.first)) continue;
+          const int ch = chunks_of(eff_N, T, o.first);
+          mc.push_back(Config{FAM_BLOCK, VL, o.first, o.second, T, 1, ch, (int)eff_N, ch > 1});
+        }
+      std::stable_sort(mc.begin(), mc.end(), [&](const Config& a, const Config& b) {
+        return (int64_t)a.chunks * a.block * a.vl * a.ng < (int64_t)b.chunks * b.block * b.vl * b.ng;   // least padding first
+      });
+      cands.insert(cands.end(), mc.begin(), mc.end());
+    }
+    if ((!any_force && few_rows) || fc || cands.empty()) {
+      for (int C : {8, 4, 2})
+        for (auto o : ng_opts) {
+          const int T = fm ? 64 : 256;
+          int64_t slice = (eff_N + C - 1) / C;
+          slice = (slice + VL - 1) / VL * VL;
+          if (slice * (C - 1) >= eff_N) continue;                              // a CTA would get no columns
+          if (!fc && !fm && slice < (int64_t)T * VL * o.first) continue;     // keep every CTA busy
+          const int ch = chunks_of(slice, T, o.first);
+          cands.push_back(Config{FAM_CLUSTER, VL, o.first, o.second, T, C, ch, (int)slice, ch > 1});
+        }
+      for (auto o : ng_opts) {   // rows too short to split: plain blocks
+        const int ch = chunks_of(eff_N, 256, o.first);
+        cands.push_back(Config{FAM_BLOCK, VL, o.first, o.second, 256, 1, ch, (int)eff_N, ch > 1});
+      }
+    }
+  }
+
+  // ---- (4) code generation: first candidate whose program fits -----------------------------
+  std::string gen_err = "no kernel configuration fits this graph";
+  for (const Config& cf : cands) {
+    std::vector<Val> v2 = vals;
+    std::vector<uint32_t> code;
+    std::map<int, int> stash_of;
+    int n_stash = 0;
+    StageDesc stages[kMaxStages];
+    memset(stages, 0, sizeof(stages));
+    bool ok = true;
+    Gen ge(code, v2, false, cf.k, cf.multichunk, stash_of, n_stash);
+    for (int s = 0; s < n_stages && ok; ++s) {
+      stages[s].elem_begin = (uint16_t)code.size();
+      ge.hoist_loads(ops, s);
+      for (const MOp& m : ops) {
+        if (m.stage != s || m.scalar) continue;
+        if (!ge.gen(m)) { ok = false; gen_err = ge.err; break; }
+      }
+      if (ok && !ge.end_stage()) { ok = false; gen_err = ge.err; }
+      stages[s].elem_end = (uint16_t)code.size();
+      stages[s].scal_begin = (uint16_t)code.size();
+      Gen gs(code, v2, true, 4, false, stash_of, n_stash);
+      for (const MOp& m : ops) {
+        if (m.stage != s || !m.scalar || !ok) continue;
+        if (!gs.gen(m)) { ok = false; gen_err = gs.err; }
+      }
+      stages[s].scal_end = (uint16_t)code.size();
+      stages[s].n_red = (uint8_t)stage_reds[s].size();
+      for (size_t r = 0; r < stage_reds[s].size(); ++r) stages[s].red[r] = stage_reds[s][r];
+    }
+    if (!ok) continue;
+    if ((int)code.size() > kMaxCode) { gen_err = "bytecode longer than the kernel takes"; continue; }
+    if (n_stash > kMaxStash) { gen_err = "too many tile values cross a reduction"; continue; }
+
+    // ---- (5) shared memory and grid ------------------------------------------------------
+    const int teams = cf.family <= FAM_WARP ? cf.block / 32 : 1;
+    int off = 0;
+    auto take = [&](int bytes) { const int o = off; off += (bytes + 15) / 16 * 16; return o; };
+    P.sm_rowoff = take(teams * kMaxIo * 8);
+    P.sm_slots = take(teams * kMaxSlots * 4);
+    P.sm_part = take(has_red ? kMaxRed * 3 * cf.block * 4 : 0);
+    P.sm_wpart = take(has_red ? 32 * kMaxRed * 3 * 4 : 0);
+    P.sm_ctapart = take(cf.cluster > 1 ? 2 * kMaxRed * 3 * 4 : 0);
+    const int64_t stash_floats = (int64_t)n_stash * cf.chunks * cf.vl * cf.ng * cf.block;
+    if (off + stash_floats * 4 > dev.max_smem_per_block) { gen_err = "the row does not fit in shared memory for its epilogue"; continue; }
+    P.sm_stash = take((int)(stash_floats * 4));
+    P.stash_floats = (int32_t)stash_floats;
+    P.n_stages = n_stages;
+    memcpy(P.stage, stages, sizeof(stages));
+    memset(P.code, 0, sizeof(P.code));
+    memcpy(P.code, code.data(), code.size() * 4);
+    P.slice_len = cf.slice_len;
+    P.chunks = cf.chunks;
+    P.split_chunks = cf.family == FAM_POINTWISE;
+    P.cluster = cf.cluster;
+    lp.family = cf.family; lp.vl = cf.vl; lp.ng = cf.ng; lp.k = cf.k;
+    lp.block = cf.block; lp.smem_bytes = off; lp.code_words = (int)code.size();
+    int occ = dev.have_device ? instance_occupancy(cf.vl, cf.ng, cf.k, cf.block, off) : 0;
+    if (occ <= 0) occ = std::max(1, 512 / cf.block);
+    const int64_t items = P.split_chunks ? eff_rows * cf.chunks : eff_rows;
+    const int64_t resident = (int64_t)sms * occ;
+    int64_t grid;
+    if (cf.family <= FAM_WARP) grid = std::min<int64_t>((items + teams - 1) / teams, resident * 8);
+    else if (cf.family == FAM_BLOCK) grid = std::min<int64_t>(items, resident * 8);
+    else grid = std::min<int64_t>(items, std::max<int64_t>(1, resident * 8 / cf.cluster)) * cf.cluster;
+    lp.grid = (int)std::max<int64_t>(grid, cf.cluster);
+    return PN_OK;
+  }
+  err = gen_err;
+  return PN_ERR_TOO_LARGE;
+}
+
+}  // namespace pn
