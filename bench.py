@@ -1,0 +1,344 @@
+#!/usr/bin/env python
+"""Benchmark of the fused-subgraph path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-sweep]
+
+A step is one pass of the whole fused path (one pn_graph_run) over one batch of the masked
+scaled softmax workload (bf16 scores [512,512,512], int8 causal mask, fp32 math): the
+workload the headline metric is quoted on.  The metric is effective HBM GB/s on compulsory
+bytes (every graph input read once + every output written once).  With N > 1 every rank
+runs its own batch (rows are independent: no collective on the data path), so scaling is
+weak and the value is the sum over ranks divided by the slowest rank's time.
+
+One JSON line is printed by rank 0.  Beside the base keys it carries `roofline` (the fused
+kernel against the measured HBM copy rate), `e2e` (the same metric through
+pn_graph_run_host on pinned host buffers, copies inside the timed region),
+`cpu_baseline` (the CPU oracle timed on a bounded sample of the same workload) and, at
+N = 1 unless --no-sweep, `sweep`: the other four benchmark subgraphs, fused and unfused.
+
+--impl reference times the CPU oracle itself, as it stands, on the host cores.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from pn_workloads import configs as C  # noqa: E402
+from pn_workloads import descriptor as D  # noqa: E402
+
+METRIC = "fused-subgraph effective HBM GB/s on compulsory bytes"
+WORKLOAD = "c2 masked scaled softmax: bf16 scores [512,512,512], int8 causal mask [512,512], fp32 math, bf16 out"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (earlier pool measurement)"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 6:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def nbytes_of(meta):
+    return [D.DTYPE_BYTES[dt] * int(np.prod(dims, dtype=np.int64)) for dt, dims in meta]
+
+
+def device_sets(torch, w, n_sets):
+    """n_sets distinct copies of the inputs and outputs on the device."""
+    sets = []
+    host = [np.ascontiguousarray(a).reshape(-1).view(np.uint8) for a in w.inputs]
+    for _ in range(n_sets):
+        d_in = [torch.from_numpy(h).cuda() for h in host]
+        d_out = [torch.full((s,), 0xFF, dtype=torch.uint8, device="cuda") for s in nbytes_of(w.output_meta)]
+        sets.append((d_in, d_out))
+    return sets
+
+
+def time_graph(torch, g, sets, steps, warmup, flush=None):
+    """W untimed + K timed launches rotating over the buffer sets.  Returns (total ms over the
+    K steps by CUDA events on the launch stream, per-step ms list)."""
+    stream = torch.cuda.current_stream()
+    ptrs = [([t.data_ptr() for t in a], [t.data_ptr() for t in b]) for a, b in sets]
+    for i in range(warmup):
+        g.run(*ptrs[i % len(ptrs)], stream.cuda_stream)
+    torch.cuda.synchronize()
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    evs[0].record(stream)
+    for i in range(steps):
+        if flush is not None:
+            flush.add_(1)
+        g.run(*ptrs[i % len(ptrs)], stream.cuda_stream)
+        evs[i + 1].record(stream)
+    torch.cuda.synchronize()
+    per = [evs[i].elapsed_time(evs[i + 1]) for i in range(steps)]
+    return evs[0].elapsed_time(evs[steps]), per
+
+
+def stats(per):
+    a = np.sort(np.asarray(per))
+    q1, med, q3 = np.percentile(a, [25, 50, 75])
+    return {"median_ms": float(med), "min_ms": float(a[0]), "iqr_ms": float(q3 - q1)}
+
+
+def oracle_sample(rows_b):
+    """A bounded sample of the benchmark workload for the CPU oracle: rows_b of the 512 batches."""
+    return C.c2(B=rows_b)
+
+
+def time_oracle(sample, repeats):
+    from oracle import evaluator as E
+    best = None
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        E.evaluate(sample.desc, sample.inputs)
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    return best
+
+
+def oracle_threads():
+    """Threads the oracle uses: its NumPy elementwise loops and reductions run on one core."""
+    return 1
+
+
+def run_reference(args, rank):
+    """--impl reference: the CPU oracle, as it stands, on a bounded sample per step."""
+    if rank != 0:
+        return
+    sample = oracle_sample(8)
+    for _ in range(min(args.warmup, 3)):
+        time_oracle(sample, 1)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        time_oracle(sample, 1)
+    dt = (time.perf_counter() - t0) / args.steps
+    gbs = sample.compulsory_bytes / dt / 1e9
+    line = {"impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": min(args.warmup, 3), "ms_per_step": dt * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "sample": "8 of the 512 batches per step (2.1 M elements)"},
+            "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": oracle_threads(), "kind": "oracle",
+                             "sample": "8 of 512 batches per step"},
+            "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--workload", default="c2", choices=list(C.CONFIGS))
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        if args.steps > 20:
+            args.steps = 20
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_2605_29357_b200 as pn
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    warmup = max(args.warmup, 3)
+
+    # ---- the benchmark workload: one batch per rank, seed = rank ---------------------------
+    w = C.CONFIGS[args.workload](seed=rank)
+    g = pn.Graph(w.desc, local_rank, 0)
+    info = g.kernel_info[0]
+    cbytes = g.compulsory_bytes
+    l2 = torch.cuda.get_device_properties(local_rank).L2_cache_size
+    n_sets = 1 if cbytes > 2 * l2 else int(2 * l2 // cbytes) + 2
+    sets = device_sets(torch, w, n_sets)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    time_graph(torch, g, sets, 3, warmup)     # warm-up (and first-launch costs)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    total_ms, per = time_graph(torch, g, sets, args.steps, 0)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * cbytes / (ms_per_step * 1e-3) / 1e9
+
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region -----
+    pin_in = [torch.from_numpy(np.ascontiguousarray(a).reshape(-1).view(np.uint8)).pin_memory() for a in w.inputs]
+    pin_out = [torch.empty(s, dtype=torch.uint8).pin_memory() for s in nbytes_of(w.output_meta)]
+    e2e_steps = max(3, min(args.steps, 10))
+    stream = torch.cuda.current_stream().cuda_stream
+    for _ in range(2):
+        g.run_host([t_.data_ptr() for t_ in pin_in], [t_.data_ptr() for t_ in pin_out], stream)
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        g.run_host([t_.data_ptr() for t_ in pin_in], [t_.data_ptr() for t_ in pin_out], stream)
+    torch.cuda.synchronize()
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_s = float(t.item())
+    h2d = int(sum(a.nbytes for a in w.inputs))
+    d2h = int(sum(nbytes_of(w.output_meta)))
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_src = measured_peak()
+    st = stats(per)
+    achieved = cbytes / (np.mean(per) * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": WORKLOAD if args.workload == "c2" else w.name, "compulsory_bytes": cbytes,
+                   "l2": "inputs larger than L2" if n_sets == 1 else f"{n_sets} rotating buffer sets larger than 2x L2",
+                   "family": pn.FAMILY_NAMES[info["family"]], "grid": info["grid"], "block": info["block"],
+                   "cluster": info["cluster"], "tile": [info["vl"], info["ng"]], "kernels": g.n_kernels,
+                   "nodes": g.n_nodes, "per_step": st, "pct_of_8000": 100 * value / world / 8000.0},
+        "clocks": clocks,
+        "gpu_launches": args.steps * g.n_kernels,
+        "e2e": {"value": world * cbytes / e2e_s / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s * 1e3, "steps": e2e_steps},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": None, "peak_source": peak_src, "kernel": f"fused_kernel<{info['vl']},{info['ng']}>",
+                     "algorithmic_bytes_per_launch": cbytes},
+    }
+
+    # ---- the unfused path of the same library on the same workload ---------------------------
+    try:
+        gu = pn.Graph(w.desc, local_rank, pn.FLAG_UNFUSED)
+        _, per_u = time_graph(torch, gu, sets, max(5, args.steps // 5), 3)
+        su = stats(per_u)
+        line["unfused"] = {"kernels": gu.n_kernels, "median_ms": su["median_ms"],
+                           "speedup_fused_over_unfused": su["median_ms"] / st["median_ms"]}
+        gu.close()
+    except Exception as e:  # report, do not hide
+        line["unfused"] = {"error": str(e)}
+    del sets
+    torch.cuda.empty_cache()
+
+    # ---- the other benchmark subgraphs (N = 1 only) ------------------------------------------
+    if world == 1 and not args.no_sweep:
+        sweep = {}
+        for name in C.CONFIGS:
+            if name == args.workload:
+                continue
+            wi = C.CONFIGS[name]()
+            gi = pn.Graph(wi.desc, local_rank, 0)
+            cb = gi.compulsory_bytes
+            ns = 1 if cb > 2 * l2 else int(2 * l2 // cb) + 2
+            si = device_sets(torch, wi, ns)
+            _, pi = time_graph(torch, gi, si, args.steps, warmup)
+            sti = stats(pi)
+            ki = gi.kernel_info[0]
+            entry = {"compulsory_bytes": cb, "median_ms": sti["median_ms"], "min_ms": sti["min_ms"],
+                     "iqr_ms": sti["iqr_ms"], "gbs": cb / (sti["median_ms"] * 1e-3) / 1e9,
+                     "frac_of_measured_peak": cb / (sti["median_ms"] * 1e-3) / 1e9 / peak,
+                     "family": pn.FAMILY_NAMES[ki["family"]], "buffer_sets": ns}
+            try:
+                gui = pn.Graph(wi.desc, local_rank, pn.FLAG_UNFUSED)
+                _, pu = time_graph(torch, gui, si, max(5, args.steps // 5), 3)
+                entry["unfused_kernels"] = gui.n_kernels
+                entry["unfused_median_ms"] = stats(pu)["median_ms"]
+                entry["speedup_fused_over_unfused"] = entry["unfused_median_ms"] / sti["median_ms"]
+                gui.close()
+            except Exception as e:
+                entry["unfused_error"] = str(e)
+            sweep[name] = entry
+            gi.close()
+            del si
+            torch.cuda.empty_cache()
+        line["sweep"] = sweep
+
+    # ---- the CPU oracle on a bounded sample of the same workload ------------------------------
+    sample = oracle_sample(32)
+    t_or = time_oracle(sample, 3)
+    line["cpu_baseline"] = {"value": sample.compulsory_bytes / t_or / 1e9, "unit": "GB/s", "cores": oracle_threads(),
+                            "kind": "oracle", "sample": "32 of the 512 batches (8.4 M elements), best of 3",
+                            "seconds": t_or}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,158 @@
+"""ctypes binding of the C-ABI library (include/pn.h): argument marshalling only.
+
+Every step of the computation runs in the CUDA kernels of libpn.so.  There is no CPU
+fallback: if the library is missing it is built with nvcc, and if that fails the import
+raises.  torch is used by callers for device memory and streams; this module itself only
+needs raw device pointers.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Sequence, Tuple
+
+from . import _build
+
+# status codes and flags (numerically as in pn.h)
+PN_OK = 0
+FLAG_UNFUSED = 1 << 0
+FLAG_PLAN_ONLY = 1 << 1
+FLAG_FORCE_WARP = 1 << 4
+FLAG_FORCE_BLOCK = 1 << 5
+FLAG_FORCE_CLUSTER = 1 << 6
+FLAG_FORCE_SCALAR = 1 << 7
+FLAG_FORCE_MULTICHUNK = 1 << 8
+
+Q_N_INPUTS, Q_N_OUTPUTS, Q_INPUT_META, Q_OUTPUT_META, Q_COMPULSORY_BYTES = 1, 2, 3, 4, 5
+Q_N_KERNELS, Q_N_NODES, Q_WORKSPACE_BYTES, Q_KERNEL_INFO = 6, 7, 8, 9
+
+FAMILY_NAMES = {0: "pointwise", 1: "warp-per-row", 2: "block-per-row", 3: "cluster-per-row"}
+EXPORTS = ["pn_graph_create", "pn_graph_run", "pn_graph_run_host", "pn_graph_destroy",
+           "pn_graph_query", "pn_status_string", "pn_last_error"]
+
+
+class PnError(RuntimeError):
+    def __init__(self, status: int, what: str, detail: str):
+        super().__init__(f"{what}: {detail} (status {status})")
+        self.status = status
+        self.detail = detail
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def load_library() -> ctypes.CDLL:
+    """Load libpn.so, building it first if it is not there.  Raises when neither works."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_build.LIB):
+        _build.build_library()
+    lib = ctypes.CDLL(_build.LIB)
+    vp, vpp = ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p)
+    lib.pn_graph_create.restype = ctypes.c_int
+    lib.pn_graph_create.argtypes = [ctypes.c_char_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_uint, vpp]
+    for fn in (lib.pn_graph_run, lib.pn_graph_run_host):
+        fn.restype = ctypes.c_int
+        fn.argtypes = [vp, vpp, ctypes.c_int, vpp, ctypes.c_int, vp]
+    lib.pn_graph_destroy.restype = ctypes.c_int
+    lib.pn_graph_destroy.argtypes = [vp]
+    lib.pn_graph_query.restype = ctypes.c_int
+    lib.pn_graph_query.argtypes = [vp, ctypes.c_int, vp, ctypes.c_size_t]
+    lib.pn_status_string.restype = ctypes.c_char_p
+    lib.pn_status_string.argtypes = [ctypes.c_int]
+    lib.pn_last_error.restype = ctypes.c_char_p
+    lib.pn_last_error.argtypes = []
+    _lib = lib
+    return lib
+
+
+def _check(status: int, what: str) -> None:
+    if status != PN_OK:
+        lib = load_library()
+        raise PnError(status, what + ": " + lib.pn_status_string(status).decode(), lib.pn_last_error().decode())
+
+
+class Graph:
+    """One lowered graph (pn_graph_t).  ``desc`` is a serialized descriptor."""
+
+    def __init__(self, desc: bytes, device: int = 0, flags: int = 0):
+        self._lib = load_library()
+        self._h = ctypes.c_void_p()
+        _check(self._lib.pn_graph_create(desc, len(desc), device, flags, ctypes.byref(self._h)), "pn_graph_create")
+        self.n_inputs = self._query(Q_N_INPUTS, 1)[0]
+        self.n_outputs = self._query(Q_N_OUTPUTS, 1)[0]
+
+    # -- pn_graph_query -----------------------------------------------------
+    def _query(self, what: int, n: int) -> List[int]:
+        buf = (ctypes.c_int64 * max(n, 1))()
+        _check(self._lib.pn_graph_query(self._h, what, buf, ctypes.sizeof(buf)), "pn_graph_query")
+        return list(buf[:n])
+
+    def _meta(self, what: int, n: int) -> List[Tuple[int, tuple]]:
+        v = self._query(what, 6 * n)
+        return [(v[6 * i], tuple(v[6 * i + 2: 6 * i + 2 + v[6 * i + 1]])) for i in range(n)]
+
+    @property
+    def input_meta(self):
+        return self._meta(Q_INPUT_META, self.n_inputs)
+
+    @property
+    def output_meta(self):
+        return self._meta(Q_OUTPUT_META, self.n_outputs)
+
+    @property
+    def compulsory_bytes(self) -> int:
+        return self._query(Q_COMPULSORY_BYTES, 1)[0]
+
+    @property
+    def n_kernels(self) -> int:
+        return self._query(Q_N_KERNELS, 1)[0]
+
+    @property
+    def n_nodes(self) -> int:
+        return self._query(Q_N_NODES, 1)[0]
+
+    @property
+    def workspace_bytes(self) -> int:
+        return self._query(Q_WORKSPACE_BYTES, 1)[0]
+
+    @property
+    def kernel_info(self) -> List[dict]:
+        n = self.n_kernels
+        v = self._query(Q_KERNEL_INFO, 12 * n)
+        keys = ["family", "grid", "block", "cluster", "smem_bytes", "vl", "ng", "chunks",
+                "code_words", "stages", "rows", "row_len"]
+        return [dict(zip(keys, v[12 * i: 12 * i + 12])) for i in range(n)]
+
+    # -- pn_graph_run / pn_graph_run_host -------------------------------------
+    @staticmethod
+    def _ptr_array(ptrs: Sequence[int]):
+        return (ctypes.c_void_p * max(len(ptrs), 1))(*[ctypes.c_void_p(int(p)) for p in ptrs])
+
+    def run(self, input_ptrs: Sequence[int], output_ptrs: Sequence[int], stream: int = 0) -> None:
+        """Enqueue one evaluation on device pointers (integers) and a cudaStream_t handle."""
+        _check(self._lib.pn_graph_run(self._h, self._ptr_array(input_ptrs), len(input_ptrs),
+                                      self._ptr_array(output_ptrs), len(output_ptrs),
+                                      ctypes.c_void_p(stream)), "pn_graph_run")
+
+    def run_host(self, input_ptrs: Sequence[int], output_ptrs: Sequence[int], stream: int = 0) -> None:
+        """Evaluate on HOST buffers (addresses): copy in, run, copy out, wait."""
+        _check(self._lib.pn_graph_run_host(self._h, self._ptr_array(input_ptrs), len(input_ptrs),
+                                           self._ptr_array(output_ptrs), len(output_ptrs),
+                                           ctypes.c_void_p(stream)), "pn_graph_run_host")
+
+    def close(self) -> None:
+        if getattr(self, "_h", None) is not None and self._h:
+            self._lib.pn_graph_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
