@@ -308,7 +308,7 @@ struct TileCtx {
   bool leader;              // this thread performs per-row scalar stores
 };
 
-// Run the statements with `r` bound to tile register k (k >= K names the accumulator).
+// Run the statements with `r` bound to tile register k (kAccReg names the accumulator).
 // A macro, so that every case is straight-line code on statically indexed registers.
 #define PN_CASE_REG(n, ...) \
   case n: if constexpr (K > n) { float(&r)[V] = reg[n]; __VA_ARGS__ } break;

@@ -139,7 +139,7 @@ struct Gen {
     emit(OP_ST, k); regv[k] = accv; regraw[k] = 0;
     return true;
   }
-  void load_input(int v, int target) {   // target = K names acc
+  void load_input(int v, int target) {   // target = kAccReg names acc
     const Val& x = vals[v];
     if (x.bcast) emit(OP_LDBC, x.io, target);
     else { emit(OP_LDRAW, x.io, target); emit(OP_WIDEN, x.io, target); }
@@ -152,8 +152,8 @@ struct Gen {
     if (x.kind == VK_IMM) { err = "constant-only subexpression is not lowered"; return false; }
     const int k = find_reg(v);
     if (k >= 0) { widen_if_raw(k); emit(OP_LD, k); }
-    else if (stash_of.count(v)) { emit(OP_FILL, K, stash_of[v]); if (x.has_ts) emit(OP_FILL_TS, 0, stash_of[v] + 1); }
-    else if (x.io >= 0) load_input(v, K);
+    else if (stash_of.count(v)) { emit(OP_FILL, kAccReg, stash_of[v]); if (x.has_ts) emit(OP_FILL_TS, 0, stash_of[v] + 1); }
+    else if (x.io >= 0) load_input(v, kAccReg);
     else { err = "internal: tile value has no location"; return false; }
     accv = v;
     return true;
@@ -290,7 +290,7 @@ struct Gen {
       if (vals[v].has_ts) { emit(OP_SPILL_TS, 0, n_stash); n_stash++; }
     };
     if (accv >= 0 && vals[accv].uses > 0 && vals[accv].kind == VK_E && find_reg(accv) < 0 && !stash_of.count(accv))
-      park(accv, K);
+      park(accv, kAccReg);
     for (int k = 0; k < K; ++k) {
       const int v = regv[k];
       if (v >= 0 && vals[v].uses > 0 && !stash_of.count(v)) { widen_if_raw(k); park(v, k); }

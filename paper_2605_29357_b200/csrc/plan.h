@@ -12,6 +12,7 @@ constexpr int kMaxStages = 4;   // reduction-separated stages
 constexpr int kMaxRed = 4;      // reductions accumulated in one stage
 constexpr int kMaxSlots = 24;   // per-row scalar slots
 constexpr int kMaxStash = 6;    // tile values parked in shared memory across stages
+constexpr int kAccReg = 7;      // register operand id that names the accumulator tile
 
 // Storage types (same numbering as the descriptor).
 enum DType : uint8_t { kF32 = 0, kF16 = 1, kBF16 = 2, kI8 = 3, kBool = 4, kI32 = 5, kI64 = 6 };
@@ -23,7 +24,7 @@ enum DType : uint8_t { kF32 = 0, kF16 = 1, kBF16 = 2, kI8 = 3, kBool = 4, kI32 =
 enum Op : uint8_t {
   OP_END = 0,
   // memory
-  OP_LDRAW,   // a = io, b = reg (K = acc): issue the loads of a tile, storage bits as they are
+  OP_LDRAW,   // a = io, b = reg (kAccReg = acc): issue the loads of a tile, storage bits as they are
   OP_WIDEN,   // a = io (for its dtype), b = reg: storage bits -> fp32 in place
   OP_LDBC,    // a = io, b = reg: last-dim-broadcast operand, one element splat over the tile
   OP_LD,      // acc = reg[a]
@@ -47,7 +48,7 @@ enum Op : uint8_t {
   OP_RED,      // a = RedKind, b = reduction index within the stage
   OP_SCALE_TS, // acc *= exp(ts - slot[a]) * slot[b]   (softmax epilogue)
   // parking tile values in shared memory across stages (rows of several chunks per thread)
-  OP_SPILL, OP_FILL,        // a = reg (K = acc), b = stash index
+  OP_SPILL, OP_FILL,        // a = reg (kAccReg = acc), b = stash index
   OP_SPILL_TS, OP_FILL_TS,  // b = stash index
   // scalar programs only
   OP_SLD,     // acc = slot[a]
