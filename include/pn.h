@@ -79,7 +79,9 @@ enum {
   PN_FLAG_FORCE_BLOCK = 1u << 5,  /* row kernels: one thread block per row                */
   PN_FLAG_FORCE_CLUSTER = 1u << 6,/* row kernels: one thread-block cluster per row        */
   PN_FLAG_FORCE_SCALAR = 1u << 7, /* element-wise (unvectorised) memory accesses          */
-  PN_FLAG_FORCE_MULTICHUNK = 1u << 8 /* smallest tile: rows span several chunks per thread */
+  PN_FLAG_FORCE_MULTICHUNK = 1u << 8,/* smallest tile: rows span several chunks per thread */
+  PN_FLAG_INTERPRET = 1u << 9     /* run the bytecode on the interpreter kernels built into the
+                                     library instead of a kernel specialised for the graph */
 };
 
 /* pn_graph_query selectors; each writes int64 values into `out` */
@@ -92,10 +94,11 @@ enum {
   PN_Q_N_KERNELS = 6,       /* 1 value: launches per pn_graph_run (1 when fused)         */
   PN_Q_N_NODES = 7,         /* 1 value: operator nodes in the descriptor                 */
   PN_Q_WORKSPACE_BYTES = 8, /* 1 value: device memory owned by the handle                */
-  PN_Q_KERNEL_INFO = 9      /* per kernel 12 values: family (0 pointwise, 1 warp-per-row,
+  PN_Q_KERNEL_INFO = 9      /* per kernel 13 values: family (0 pointwise, 1 warp-per-row,
                                2 block-per-row, 3 cluster-per-row), grid, block, cluster,
                                dynamic smem bytes, vector length, groups per tile, chunks
-                               per row slice, bytecode words, stages, rows, row length   */
+                               per row slice, bytecode words, stages, rows, row length,
+                               specialised (1) or interpreted (0)                        */
 };
 
 /*
@@ -108,6 +111,10 @@ enum {
  *   out              : receives the handle; set to NULL on failure.
  * Allocates device memory only for PN_FLAG_UNFUSED (the intermediates) -- owned by the
  * handle and released by pn_graph_destroy.  Launches no kernel.
+ * Unless PN_FLAG_INTERPRET is given, the bytecode of each launch is also translated into a
+ * kernel of its own and compiled for sm_100a with NVRTC (a few hundred ms per distinct
+ * kernel; loaded kernels are cached for the life of the process).  If NVRTC or the driver
+ * library cannot be opened the handle runs on the interpreter; PN_Q_KERNEL_INFO tells which.
  */
 pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsigned flags,
                           pn_graph_t** out);
@@ -148,6 +155,18 @@ pn_status pn_graph_destroy(pn_graph_t* g);
  * PN_ERR_INVALID_ARG).
  */
 pn_status pn_graph_query(const pn_graph_t* g, int what, void* out, size_t out_bytes);
+
+/*
+ * pn_graph_codegen -- the CUDA source generated for launch `kernel` of a handle (the
+ * translation of its bytecode; the device library it is compiled against is not repeated).
+ * Copies at most out_bytes - 1 characters plus a terminator into `out` (HOST memory; may be
+ * NULL with out_bytes 0) and stores the full length in *needed if that is not NULL.  With
+ * compile != 0 the source is also compiled for sm_100a with NVRTC, without loading it: this
+ * needs no GPU and returns PN_ERR_CUDA with the compiler's log on failure.  The paper has no
+ * counterpart: an aid for tests and for reading what the specialiser made of a graph.
+ */
+pn_status pn_graph_codegen(const pn_graph_t* g, int kernel, int compile, char* out, size_t out_bytes,
+                           size_t* needed);
 
 /* Static text for a status code. */
 const char* pn_status_string(pn_status s);

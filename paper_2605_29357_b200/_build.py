@@ -14,8 +14,9 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 OBJ = os.path.join(CSRC, "_build")
 LIB = os.path.join(HERE, "libpn.so")
-SOURCES = ["kernels.cu", "lower.cpp", "descriptor.cpp", "api.cpp"]
-HEADERS = [os.path.join(CSRC, "plan.h"), os.path.join(CSRC, "graph.h"), os.path.join(INCLUDE, "pn.h")]
+SOURCES = ["kernels.cu", "lower.cpp", "descriptor.cpp", "spec.cpp", "api.cpp"]
+HEADERS = [os.path.join(CSRC, "plan.h"), os.path.join(CSRC, "graph.h"), os.path.join(CSRC, "spec.h"),
+           os.path.join(CSRC, "device_lib.cuh"), os.path.join(INCLUDE, "pn.h")]
 FLAGS = ["-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
          "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
 
@@ -27,8 +28,24 @@ def _nvcc() -> str:
     raise RuntimeError("nvcc not found: the CUDA toolkit is needed to build libpn.so")
 
 
+def _embed_device_source() -> None:
+    """plan.h + device_lib.cuh as one C++ raw string literal: the text that the kernels
+    specialised at run time are compiled from."""
+    text = ""
+    for name in ("plan.h", "device_lib.cuh"):
+        with open(os.path.join(CSRC, name)) as f:
+            text += "".join(line for line in f if not line.startswith("#pragma once"))
+    assert ')PNSRC"' not in text
+    out = os.path.join(OBJ, "device_src.inc")
+    new = 'R"PNSRC(' + text + ')PNSRC"\n'
+    if not os.path.exists(out) or open(out).read() != new:
+        with open(out, "w") as f:
+            f.write(new)
+
+
 def build_library(force: bool = False, verbose: bool = False) -> str:
     os.makedirs(OBJ, exist_ok=True)
+    _embed_device_source()
     nvcc = _nvcc()
     newest_header = max(os.path.getmtime(h) for h in HEADERS)
     objs, relink = [], force or not os.path.exists(LIB)

@@ -22,13 +22,14 @@ FLAG_FORCE_BLOCK = 1 << 5
 FLAG_FORCE_CLUSTER = 1 << 6
 FLAG_FORCE_SCALAR = 1 << 7
 FLAG_FORCE_MULTICHUNK = 1 << 8
+FLAG_INTERPRET = 1 << 9
 
 Q_N_INPUTS, Q_N_OUTPUTS, Q_INPUT_META, Q_OUTPUT_META, Q_COMPULSORY_BYTES = 1, 2, 3, 4, 5
 Q_N_KERNELS, Q_N_NODES, Q_WORKSPACE_BYTES, Q_KERNEL_INFO = 6, 7, 8, 9
 
 FAMILY_NAMES = {0: "pointwise", 1: "warp-per-row", 2: "block-per-row", 3: "cluster-per-row"}
 EXPORTS = ["pn_graph_create", "pn_graph_run", "pn_graph_run_host", "pn_graph_destroy",
-           "pn_graph_query", "pn_status_string", "pn_last_error"]
+           "pn_graph_query", "pn_graph_codegen", "pn_status_string", "pn_last_error"]
 
 
 class PnError(RuntimeError):
@@ -63,6 +64,9 @@ def load_library() -> ctypes.CDLL:
     lib.pn_graph_destroy.argtypes = [vp]
     lib.pn_graph_query.restype = ctypes.c_int
     lib.pn_graph_query.argtypes = [vp, ctypes.c_int, vp, ctypes.c_size_t]
+    lib.pn_graph_codegen.restype = ctypes.c_int
+    lib.pn_graph_codegen.argtypes = [vp, ctypes.c_int, ctypes.c_int, ctypes.c_char_p, ctypes.c_size_t,
+                                     ctypes.POINTER(ctypes.c_size_t)]
     lib.pn_status_string.restype = ctypes.c_char_p
     lib.pn_status_string.argtypes = [ctypes.c_int]
     lib.pn_last_error.restype = ctypes.c_char_p
@@ -124,10 +128,19 @@ class Graph:
     @property
     def kernel_info(self) -> List[dict]:
         n = self.n_kernels
-        v = self._query(Q_KERNEL_INFO, 12 * n)
+        v = self._query(Q_KERNEL_INFO, 13 * n)
         keys = ["family", "grid", "block", "cluster", "smem_bytes", "vl", "ng", "chunks",
-                "code_words", "stages", "rows", "row_len"]
-        return [dict(zip(keys, v[12 * i: 12 * i + 12])) for i in range(n)]
+                "code_words", "stages", "rows", "row_len", "specialised"]
+        return [dict(zip(keys, v[13 * i: 13 * i + 13])) for i in range(n)]
+
+    def codegen(self, kernel: int = 0, compile: bool = False) -> str:
+        """Generated CUDA source of one launch; with compile=True also compiled by NVRTC."""
+        need = ctypes.c_size_t()
+        _check(self._lib.pn_graph_codegen(self._h, kernel, 0, None, 0, ctypes.byref(need)), "pn_graph_codegen")
+        buf = ctypes.create_string_buffer(need.value + 1)
+        _check(self._lib.pn_graph_codegen(self._h, kernel, 1 if compile else 0, buf, need.value + 1, None),
+               "pn_graph_codegen")
+        return buf.value.decode()
 
     # -- pn_graph_run / pn_graph_run_host -------------------------------------
     @staticmethod

@@ -10,6 +10,7 @@
 
 #include "../../include/pn.h"
 #include "graph.h"
+#include "spec.h"
 
 namespace pn {
 cudaError_t launch_plan(const LaunchPlan& lp, cudaStream_t stream);   // kernels.cu
@@ -29,6 +30,7 @@ struct IoSource { int kind; int64_t index; };   // kind 0 user input, 1 user out
 struct PlannedLaunch {
   LaunchPlan plan;
   std::vector<IoSource> src;
+  SpecKernel spec;   // fn == nullptr: run the plan on the interpreter
 };
 
 }  // namespace
@@ -172,6 +174,15 @@ pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsig
       if (e != cudaSuccess) { delete h; return fail(PN_ERR_CUDA, std::string("workspace: ") + cudaGetErrorString(e)); }
     }
   }
+  // a kernel of its own for every launch, unless the interpreter was asked for
+  if (!h->plan_only && !(flags & PN_FLAG_INTERPRET) && spec_available(nullptr)) {
+    cudaFree(0);   // makes the device's primary context current for the driver calls
+    for (PlannedLaunch& pl : h->launches)
+      if (!spec_compile(pl.plan, device, dev.sm_count, pl.spec, err)) {
+        pn_graph_destroy(h);
+        return fail(PN_ERR_CUDA, err);
+      }
+  }
   *out = h;
   return PN_OK;
 }
@@ -216,8 +227,13 @@ pn_status pn_graph_run(pn_graph_t* h, const void* const* inputs, int n_inputs, v
                            : s.kind == 1 ? outputs[s.index]
                                          : (void*)((char*)h->workspace + s.index);
     }
-    cudaError_t e = launch_plan(pl.plan, (cudaStream_t)stream);
-    if (e != cudaSuccess) return fail(PN_ERR_CUDA, std::string("launch: ") + cudaGetErrorString(e));
+    if (pl.spec.fn) {
+      std::string err;
+      if (!spec_launch(pl.spec, pl.plan, stream, err)) return fail(PN_ERR_CUDA, err);
+    } else {
+      cudaError_t e = launch_plan(pl.plan, (cudaStream_t)stream);
+      if (e != cudaSuccess) return fail(PN_ERR_CUDA, std::string("launch: ") + cudaGetErrorString(e));
+    }
   }
   return PN_OK;
 }
@@ -290,15 +306,33 @@ pn_status pn_graph_query(const pn_graph_t* h, int what, void* out, size_t out_by
     case PN_Q_KERNEL_INFO:
       for (const PlannedLaunch& pl : h->launches) {
         const LaunchPlan& p = pl.plan;
-        const int64_t row[12] = {p.family, p.grid, p.block, p.p.cluster, p.smem_bytes, p.vl, p.ng, p.p.chunks,
-                                 p.code_words, p.p.n_stages, p.p.rows, p.p.row_len};
-        v.insert(v.end(), row, row + 12);
+        const int64_t row[13] = {p.family, p.grid, p.block, p.p.cluster, p.smem_bytes, p.vl, p.ng, p.p.chunks,
+                                 p.code_words, p.p.n_stages, p.p.rows, p.p.row_len, p.specialised};
+        v.insert(v.end(), row, row + 13);
       }
       break;
     default: return fail(PN_ERR_INVALID_ARG, "unknown query");
   }
   if (out_bytes < v.size() * sizeof(int64_t)) return fail(PN_ERR_INVALID_ARG, "query buffer too small");
   if (!v.empty()) memcpy(out, v.data(), v.size() * sizeof(int64_t));
+  return PN_OK;
+}
+
+pn_status pn_graph_codegen(const pn_graph_t* h, int kernel, int compile, char* out, size_t out_bytes, size_t* needed) {
+  if (!h) return fail(PN_ERR_INVALID_ARG, "null argument");
+  if (kernel < 0 || kernel >= (int)h->launches.size()) return fail(PN_ERR_INVALID_ARG, "no such kernel");
+  const LaunchPlan& lp = h->launches[kernel].plan;
+  const std::string src = spec_source(lp);
+  if (needed) *needed = src.size();
+  if (out && out_bytes > 0) {
+    const size_t n = std::min(src.size(), out_bytes - 1);
+    memcpy(out, src.data(), n);
+    out[n] = '\0';
+  }
+  if (compile) {
+    std::string err;
+    if (!spec_check(lp, err)) return fail(PN_ERR_CUDA, err);
+  }
   return PN_OK;
 }
 

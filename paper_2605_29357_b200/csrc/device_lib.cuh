@@ -1,0 +1,769 @@
+// device_lib.cuh -- device side of the fused kernels (sm_100a), self-contained: it includes
+// no header, so that the same text serves the kernels compiled into the library (the bytecode
+// interpreter) and the kernels specialised per graph at create time (NVRTC).  plan.h must
+// precede it.
+//
+// A *team* of threads (a warp, a thread block, or the thread blocks of a cluster) owns one
+// row of the iteration space at a time; each thread holds a register tile of NG groups of VL
+// consecutive elements.  Loads widen to fp32 in registers, the pointwise DAG runs in
+// registers, reductions fold the tile into a 3-float partial that is combined thread -> warp
+// (shuffles) -> block (shared memory) -> cluster (distributed shared memory), per-row scalar
+// programs run on the combined values, and the epilogue narrows and stores.  Every graph
+// input is read once and every output written once.
+//
+// A program (class Prog) supplies the tile code and the scalar code of each stage: either by
+// interpreting the bytecode (Interp) or as straight-line code generated from the same
+// bytecode.  Both are built from the op_* functions below: one definition of every operation.
+//
+// No spin-waits anywhere: cross-thread hand-offs are __syncwarp / __syncthreads / cluster
+// barriers only.  Nothing traps.
+#pragma once
+
+namespace pn {
+
+#define PN_DEV __device__ __forceinline__
+#define PN_UNROLL _Pragma("unroll")
+#define PN_INF __int_as_float(0x7f800000)
+#define PN_NAN __int_as_float(0x7fffffff)
+
+PN_DEV float bits_f(uint32_t u) { return __uint_as_float(u); }
+PN_DEV uint32_t f_bits(float f) { return __float_as_uint(f); }
+
+PN_DEV int dtype_size(int dt) {
+  switch (dt) {
+    case kF32: case kI32: return 4;
+    case kF16: case kBF16: return 2;
+    case kI64: return 8;
+    default: return 1;
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// conversions (PTX, so that no header is needed)
+// ---------------------------------------------------------------------------------------
+PN_DEV float half_to_float(uint32_t h16) {
+  float f;
+  asm("{ .reg .b16 t; cvt.u16.u32 t, %1; cvt.f32.f16 %0, t; }" : "=f"(f) : "r"(h16));
+  return f;
+}
+PN_DEV uint32_t pack_bf16x2(float lo, float hi) {   // round to nearest even
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+PN_DEV uint32_t pack_f16x2(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+PN_DEV float round_bf16(float x) { return bits_f(pack_bf16x2(x, 0.f) << 16); }
+PN_DEV float round_f16(float x) { return half_to_float(pack_f16x2(x, 0.f) & 0xFFFFu); }
+
+// ---------------------------------------------------------------------------------------
+// global memory access: BYTES contiguous bytes, aligned to min(BYTES, 16)
+// ---------------------------------------------------------------------------------------
+template <int BYTES>
+PN_DEV void load_words(const char* p, uint32_t* w) {
+  if constexpr (BYTES >= 16) {
+    PN_UNROLL for (int i = 0; i < BYTES / 16; ++i) {
+      const uint4 v = __ldg(reinterpret_cast<const uint4*>(p) + i);
+      w[4 * i] = v.x; w[4 * i + 1] = v.y; w[4 * i + 2] = v.z; w[4 * i + 3] = v.w;
+    }
+  } else if constexpr (BYTES == 8) {
+    const uint2 v = __ldg(reinterpret_cast<const uint2*>(p));
+    w[0] = v.x; w[1] = v.y;
+  } else if constexpr (BYTES == 4) {
+    w[0] = __ldg(reinterpret_cast<const unsigned int*>(p));
+  } else if constexpr (BYTES == 2) {
+    w[0] = __ldg(reinterpret_cast<const unsigned short*>(p));
+  } else {
+    w[0] = __ldg(reinterpret_cast<const unsigned char*>(p));
+  }
+}
+
+template <int BYTES>
+PN_DEV void store_words(char* p, const uint32_t* w) {
+  if constexpr (BYTES >= 16) {
+    PN_UNROLL for (int i = 0; i < BYTES / 16; ++i)
+      reinterpret_cast<uint4*>(p)[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+  } else if constexpr (BYTES == 8) {
+    *reinterpret_cast<uint2*>(p) = make_uint2(w[0], w[1]);
+  } else if constexpr (BYTES == 4) {
+    *reinterpret_cast<unsigned int*>(p) = w[0];
+  } else if constexpr (BYTES == 2) {
+    *reinterpret_cast<unsigned short*>(p) = static_cast<unsigned short>(w[0]);
+  } else {
+    *reinterpret_cast<unsigned char*>(p) = static_cast<unsigned char>(w[0]);
+  }
+}
+
+PN_DEV float widen_scalar(const char* p, int dt) {
+  switch (dt) {
+    case kF32: return __ldg(reinterpret_cast<const float*>(p));
+    case kF16: return half_to_float(__ldg(reinterpret_cast<const unsigned short*>(p)));
+    case kBF16: return bits_f(static_cast<uint32_t>(__ldg(reinterpret_cast<const unsigned short*>(p))) << 16);
+    case kI8: return static_cast<float>(__ldg(reinterpret_cast<const signed char*>(p)));
+    case kBool: return __ldg(reinterpret_cast<const unsigned char*>(p)) ? 1.f : 0.f;
+    case kI32: return static_cast<float>(__ldg(reinterpret_cast<const int*>(p)));
+    default: return static_cast<float>(__ldg(reinterpret_cast<const long long*>(p)));
+  }
+}
+
+// Storage bits of one group of VL elements -> VL floats, in place.
+template <int VL>
+PN_DEV void widen_group(float* g, int dt) {
+  uint32_t w[VL];
+  PN_UNROLL for (int i = 0; i < VL; ++i) w[i] = f_bits(g[i]);
+  switch (dt) {
+    case kF32: case kI64: break;  // i64 operands are converted at load time
+    case kBF16:
+      PN_UNROLL for (int i = 0; i < VL; ++i) g[i] = bits_f((i & 1) ? (w[i >> 1] & 0xFFFF0000u) : (w[i >> 1] << 16));
+      break;
+    case kF16:
+      PN_UNROLL for (int i = 0; i < VL; ++i) g[i] = half_to_float((w[i >> 1] >> ((i & 1) * 16)) & 0xFFFFu);
+      break;
+    case kI8:
+      PN_UNROLL for (int i = 0; i < VL; ++i)
+        g[i] = static_cast<float>(static_cast<signed char>((w[i >> 2] >> ((i & 3) * 8)) & 0xFF));
+      break;
+    case kBool:
+      PN_UNROLL for (int i = 0; i < VL; ++i) g[i] = ((w[i >> 2] >> ((i & 3) * 8)) & 0xFF) ? 1.f : 0.f;
+      break;
+    case kI32:
+      PN_UNROLL for (int i = 0; i < VL; ++i) g[i] = static_cast<float>(static_cast<int>(w[i]));
+      break;
+  }
+}
+
+template <int VL>
+PN_DEV void load_group_raw(const char* base, long long elem, int dt, float* g) {
+  uint32_t w[VL];
+  PN_UNROLL for (int i = 0; i < VL; ++i) w[i] = 0;
+  switch (dt) {
+    case kF32: case kI32: load_words<VL * 4>(base + elem * 4, w); break;
+    case kF16: case kBF16: load_words<VL * 2>(base + elem * 2, w); break;
+    case kI8: case kBool: load_words<VL>(base + elem, w); break;
+    default:  // i64: converted here, widening is then a no-op
+      PN_UNROLL for (int i = 0; i < VL; ++i)
+        w[i] = f_bits(static_cast<float>(__ldg(reinterpret_cast<const long long*>(base) + elem + i)));
+      break;
+  }
+  PN_UNROLL for (int i = 0; i < VL; ++i) g[i] = bits_f(w[i]);
+}
+
+template <int VL>
+PN_DEV void store_group(char* base, long long elem, int dt, const float* g) {
+  uint32_t w[VL];
+  switch (dt) {
+    case kF32:
+      PN_UNROLL for (int i = 0; i < VL; ++i) w[i] = f_bits(g[i]);
+      store_words<VL * 4>(base + elem * 4, w);
+      break;
+    case kI32:
+      PN_UNROLL for (int i = 0; i < VL; ++i) w[i] = static_cast<uint32_t>(__float2int_rz(g[i]));
+      store_words<VL * 4>(base + elem * 4, w);
+      break;
+    case kBF16:
+      if constexpr (VL == 1) { w[0] = pack_bf16x2(g[0], 0.f) & 0xFFFFu; }
+      else { PN_UNROLL for (int i = 0; i < VL / 2; ++i) w[i] = pack_bf16x2(g[2 * i], g[2 * i + 1]); }
+      store_words<VL * 2>(base + elem * 2, w);
+      break;
+    case kF16:
+      if constexpr (VL == 1) { w[0] = pack_f16x2(g[0], 0.f) & 0xFFFFu; }
+      else { PN_UNROLL for (int i = 0; i < VL / 2; ++i) w[i] = pack_f16x2(g[2 * i], g[2 * i + 1]); }
+      store_words<VL * 2>(base + elem * 2, w);
+      break;
+    case kI8: case kBool: {
+      PN_UNROLL for (int i = 0; i < (VL + 3) / 4; ++i) w[i] = 0;
+      PN_UNROLL for (int i = 0; i < VL; ++i) {
+        const uint32_t b = dt == kBool ? (g[i] != 0.f ? 1u : 0u)
+                                       : (static_cast<uint32_t>(__float2int_rz(g[i])) & 0xFFu);
+        w[i >> 2] |= b << ((i & 3) * 8);
+      }
+      store_words<VL>(base + elem, w);
+      break;
+    }
+    default:  // i64
+      PN_UNROLL for (int i = 0; i < VL; ++i)
+        reinterpret_cast<long long*>(base)[elem + i] = static_cast<long long>(__float2int_rz(g[i]));
+      break;
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// scalar math (fp32).  The fp32 outputs are held to rtol 1e-5, so the special-function
+// unit's approximations are used only where a correction keeps the error near 1e-7.
+// ---------------------------------------------------------------------------------------
+// e^x = 2^(x*log2 e).  The product is split into its rounded value t and the rounding
+// residual r (recovered exactly by an fma, plus the low part of log2 e); 2^t comes from the
+// hardware exponential and the residual is applied as a first-order factor.  Overflow gives
+// +inf, large negative arguments 0, NaN stays NaN.
+PN_DEV float f_exp(float x) {
+  const float L2E_HI = 1.4426950216293335f, L2E_LO = 1.9259629911266175e-8f, LN2 = 0.6931471805599453f;
+  const float t = x * L2E_HI;
+  float r = fmaf(x, L2E_HI, -t);
+  r = fmaf(x, L2E_LO, r);
+  const float e = exp2f(t);
+  return (fabsf(x) < 100.f) ? fmaf(e, r * LN2, e) : e;   // no correction at inf / overflow
+}
+PN_DEV float f_sigmoid(float x) { return __fdividef(1.f, 1.f + f_exp(-x)); }
+// 0.5 x (1 + tanh u) = x / (1 + e^(-2u)),  u = sqrt(2/pi) (x + 0.044715 x^3)
+PN_DEV float f_gelu_tanh(float x) {
+  const float k0 = 0.7978845608028654f, k1 = 0.044715f;
+  const float u = k0 * fmaf(k1 * x * x, x, x);
+  return x * f_sigmoid(2.f * u);
+}
+PN_DEV float f_gelu_erf(float x) { return 0.5f * x * (1.f + erff(x * 0.7071067811865476f)); }
+PN_DEV float f_max_nan(float a, float b) { return (a != a || b != b) ? PN_NAN : fmaxf(a, b); }
+PN_DEV float f_min_nan(float a, float b) { return (a != a || b != b) ? PN_NAN : fminf(a, b); }
+
+template <int OP>
+PN_DEV float un(float x) {
+  if constexpr (OP == OP_NEG) return -x;
+  else if constexpr (OP == OP_ABS) return fabsf(x);
+  else if constexpr (OP == OP_EXP) return f_exp(x);
+  else if constexpr (OP == OP_LOG) return logf(x);
+  else if constexpr (OP == OP_SQRT) return sqrtf(x);
+  else if constexpr (OP == OP_RSQRT) return 1.f / sqrtf(x);
+  else if constexpr (OP == OP_RECIP) return 1.f / x;
+  else if constexpr (OP == OP_TANH) return tanhf(x);
+  else if constexpr (OP == OP_SIGMOID) return f_sigmoid(x);
+  else if constexpr (OP == OP_SILU) return x * f_sigmoid(x);
+  else if constexpr (OP == OP_GELU_TANH) return f_gelu_tanh(x);
+  else if constexpr (OP == OP_GELU_ERF) return f_gelu_erf(x);
+  else if constexpr (OP == OP_RELU) return (x != x) ? x : fmaxf(x, 0.f);
+  else if constexpr (OP == OP_SQUARE) return x * x;
+  else if constexpr (OP == OP_ERF) return erff(x);
+  else if constexpr (OP == OP_RND_BF16) return round_bf16(x);
+  else if constexpr (OP == OP_RND_F16) return round_f16(x);
+  else if constexpr (OP == OP_TRUNC) return truncf(x);
+  else if constexpr (OP == OP_NEZ) return x != 0.f ? 1.f : 0.f;
+  else if constexpr (OP == OP_I2F) return static_cast<float>(static_cast<int>(f_bits(x)));
+  else return x;
+}
+
+template <int OP>
+PN_DEV float bin(float x, float y) {
+  if constexpr (OP == OP_ADD) return x + y;
+  else if constexpr (OP == OP_SUB) return x - y;
+  else if constexpr (OP == OP_RSUB) return y - x;
+  else if constexpr (OP == OP_MUL) return x * y;
+  else if constexpr (OP == OP_DIV) return x / y;
+  else if constexpr (OP == OP_RDIV) return y / x;
+  else if constexpr (OP == OP_MAX) return f_max_nan(x, y);
+  else if constexpr (OP == OP_MIN) return f_min_nan(x, y);
+  else if constexpr (OP == OP_GT) return x > y ? 1.f : 0.f;
+  else if constexpr (OP == OP_GE) return x >= y ? 1.f : 0.f;
+  else if constexpr (OP == OP_LT) return x < y ? 1.f : 0.f;
+  else if constexpr (OP == OP_LE) return x <= y ? 1.f : 0.f;
+  else if constexpr (OP == OP_EQ) return x == y ? 1.f : 0.f;
+  else if constexpr (OP == OP_NE) return x != y ? 1.f : 0.f;
+  else if constexpr (OP == OP_LSEFIN) return (fabsf(x) == PN_INF) ? x : x + logf(y);
+  else return x;
+}
+
+// ---------------------------------------------------------------------------------------
+// reduction partials
+// ---------------------------------------------------------------------------------------
+struct Part { float a, b, c; };
+
+PN_DEV Part red_identity(int kind) {
+  switch (kind) {
+    case RED_MAX: return {-PN_INF, 0.f, 0.f};
+    case RED_MIN: return {PN_INF, 0.f, 0.f};
+    case RED_ARGMAX: return {-PN_INF, bits_f(0x7FFFFFFFu), 0.f};
+    case RED_ARGMIN: return {PN_INF, bits_f(0x7FFFFFFFu), 0.f};
+    case RED_LSE: case RED_SOFTMAX: return {-PN_INF, 0.f, 0.f};
+    default: return {0.f, 0.f, 0.f};
+  }
+}
+
+// true when (v2, i2) should replace (v1, i1): larger value, NaN above everything, and on
+// equal values (or both NaN) the lower column
+PN_DEV bool arg_better(float v2, int i2, float v1, int i1, bool want_max) {
+  const bool n1 = v1 != v1, n2 = v2 != v2;
+  if (n1 || n2) return n2 && (!n1 || i2 < i1);
+  if (v2 == v1) return i2 < i1;
+  return want_max ? v2 > v1 : v2 < v1;
+}
+
+PN_DEV Part red_combine(int kind, Part x, Part y) {
+  switch (kind) {
+    case RED_SUM: x.a += y.a; break;
+    case RED_MAX: x.a = f_max_nan(x.a, y.a); break;
+    case RED_MIN: x.a = f_min_nan(x.a, y.a); break;
+    case RED_ARGMAX: case RED_ARGMIN:
+      if (arg_better(y.a, (int)f_bits(y.b), x.a, (int)f_bits(x.b), kind == RED_ARGMAX)) x = y;
+      break;
+    case RED_LSE: case RED_SOFTMAX: {
+      const float m = fmaxf(x.a, y.a);
+      if (m == -PN_INF) { x.b = 0.f; }
+      else { x.b = x.b * f_exp(x.a - m) + y.b * f_exp(y.a - m); }
+      x.a = m;
+      break;
+    }
+    default: {  // RED_MEANVAR: pairwise update of (count, mean, M2)
+      const float n = x.a + y.a;
+      if (n > 0.f) {
+        const float d = y.b - x.b, r = y.a / n;
+        x.c = x.c + y.c + d * d * x.a * r;
+        x.b = fmaf(d, r, x.b);
+      }
+      x.a = n;
+      break;
+    }
+  }
+  return x;
+}
+
+PN_DEV Part warp_combine(int kind, Part v) {
+  PN_UNROLL for (int o = 16; o > 0; o >>= 1) {
+    Part w;
+    w.a = __shfl_xor_sync(0xFFFFFFFFu, v.a, o);
+    w.b = __shfl_xor_sync(0xFFFFFFFFu, v.b, o);
+    w.c = __shfl_xor_sync(0xFFFFFFFFu, v.c, o);
+    // fixed operand order (lower lane first): both partners compute the same value
+    v = (threadIdx.x & o) ? red_combine(kind, w, v) : red_combine(kind, v, w);
+  }
+  return v;
+}
+
+// ---------------------------------------------------------------------------------------
+// cluster primitives (PTX)
+// ---------------------------------------------------------------------------------------
+PN_DEV uint32_t cluster_ctarank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+PN_DEV void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// read a float at the same shared-memory offset in the CTA of the given cluster rank
+PN_DEV float ld_shared_cluster(const float* local_smem_ptr, uint32_t rank) {
+  const uint32_t a = static_cast<uint32_t>(__cvta_generic_to_shared(local_smem_ptr));
+  uint32_t ra; float v;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(a), "r"(rank));
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(ra) : "memory");
+  return v;
+}
+
+// ---------------------------------------------------------------------------------------
+// tile operations: one function per bytecode instruction
+// ---------------------------------------------------------------------------------------
+struct TileCtx {
+  const long long* rowoff;  // shared: element offset of this row for every io entry
+  float* part;              // shared: this thread's partials, part[(r*3+q)*part_stride]
+  float* slots;             // shared: per-row scalar slots of this team
+  float* stash;             // shared: parked tile values (already offset by threadIdx.x)
+  int part_stride;          // threads per CTA
+  int col0;                 // column of (group 0, element 0)
+  int gstride;              // columns between consecutive groups
+  int col_end;              // one past the last valid column of this slice
+  int chunk, chunks;        // position within the slice (chunk 0 starts a reduction)
+  bool leader;              // this thread performs per-row scalar stores
+};
+
+template <int VL, int NG>
+PN_DEV void op_ldraw(const KernelParams& p, const TileCtx& cx, int io, int dt, float (&r)[VL * NG]) {
+  const char* base = static_cast<const char*>(p.io[io].base);
+  const long long off = cx.rowoff[io];
+  PN_UNROLL for (int j = 0; j < NG; ++j) {
+    const int col = cx.col0 + j * cx.gstride;
+    if (col < cx.col_end) {
+      load_group_raw<VL>(base, off + col, dt, &r[j * VL]);
+    } else {
+      PN_UNROLL for (int i = 0; i < VL; ++i) r[j * VL + i] = 0.f;
+    }
+  }
+}
+template <int VL, int NG>
+PN_DEV void op_widen(int dt, float (&r)[VL * NG]) {
+  if (dt != kF32 && dt != kI64) { PN_UNROLL for (int j = 0; j < NG; ++j) widen_group<VL>(&r[j * VL], dt); }
+}
+template <int V>
+PN_DEV void op_ldbc(const KernelParams& p, const TileCtx& cx, int io, int dt, float (&r)[V]) {
+  const float v = widen_scalar(static_cast<const char*>(p.io[io].base) + cx.rowoff[io] * dtype_size(dt), dt);
+  PN_UNROLL for (int e = 0; e < V; ++e) r[e] = v;
+}
+template <int V>
+PN_DEV void op_mov(float (&d)[V], const float (&s)[V]) { PN_UNROLL for (int e = 0; e < V; ++e) d[e] = s[e]; }
+template <int VL, int NG>
+PN_DEV void op_stout(const KernelParams& p, const TileCtx& cx, int io, int dt, const float (&acc)[VL * NG]) {
+  char* base = static_cast<char*>(p.io[io].base);
+  const long long off = cx.rowoff[io];
+  PN_UNROLL for (int j = 0; j < NG; ++j) {
+    const int col = cx.col0 + j * cx.gstride;
+    if (col < cx.col_end) store_group<VL>(base, off + col, dt, &acc[j * VL]);
+  }
+}
+// per-row scalar stores (leader thread only)
+PN_DEV void op_stout_scalar(const KernelParams& p, const TileCtx& cx, int io, int dt, float v) {
+  if (cx.leader) store_group<1>(static_cast<char*>(p.io[io].base), cx.rowoff[io], dt, &v);
+}
+PN_DEV void op_stout_index(const KernelParams& p, const TileCtx& cx, int io, int dt, float v) {
+  if (cx.leader) {
+    const int i = static_cast<int>(f_bits(v));
+    if (dt == kI64) static_cast<long long*>(p.io[io].base)[cx.rowoff[io]] = i;
+    else static_cast<int*>(p.io[io].base)[cx.rowoff[io]] = i;
+  }
+}
+template <int OP, int V>
+PN_DEV void op_unary(float (&acc)[V]) { PN_UNROLL for (int e = 0; e < V; ++e) acc[e] = un<OP>(acc[e]); }
+template <int OP, int V>
+PN_DEV void op_binary(float (&acc)[V], const float (&r)[V]) { PN_UNROLL for (int e = 0; e < V; ++e) acc[e] = bin<OP>(acc[e], r[e]); }
+template <int OP, int V>
+PN_DEV void op_binary_s(float (&acc)[V], float y) { PN_UNROLL for (int e = 0; e < V; ++e) acc[e] = bin<OP>(acc[e], y); }
+// acc = acc != 0 ? x : y   /   acc = acc * x + y
+template <int OP, int V>
+PN_DEV void op_ternary(float (&acc)[V], const float (&x)[V], const float (&y)[V]) {
+  PN_UNROLL for (int e = 0; e < V; ++e)
+    acc[e] = (OP == OP_WHERE) ? (acc[e] != 0.f ? x[e] : y[e]) : fmaf(acc[e], x[e], y[e]);
+}
+template <int V>
+PN_DEV void op_splat(float (&t)[V], float v) { PN_UNROLL for (int e = 0; e < V; ++e) t[e] = v; }
+
+// Fold the valid elements of the tile (in element order) into the thread's partial of
+// reduction `ridx`; RED_SOFTMAX also turns acc into exp(x - m_tile) and leaves m_tile in ts.
+template <int VL, int NG>
+PN_DEV void op_red(const TileCtx& cx, int kind, int ridx, float (&acc)[VL * NG], float& ts) {
+  Part t = red_identity(kind);
+  if (kind == RED_SUM) {
+    PN_UNROLL for (int j = 0; j < NG; ++j)
+      if (cx.col0 + j * cx.gstride < cx.col_end) {
+        PN_UNROLL for (int i = 0; i < VL; ++i) t.a += acc[j * VL + i];
+      }
+  } else if (kind == RED_MAX || kind == RED_MIN) {
+    PN_UNROLL for (int j = 0; j < NG; ++j)
+      if (cx.col0 + j * cx.gstride < cx.col_end) {
+        PN_UNROLL for (int i = 0; i < VL; ++i)
+          t.a = kind == RED_MAX ? f_max_nan(t.a, acc[j * VL + i]) : f_min_nan(t.a, acc[j * VL + i]);
+      }
+  } else if (kind == RED_ARGMAX || kind == RED_ARGMIN) {
+    int bi = 0x7FFFFFFF;
+    float bv = t.a;
+    PN_UNROLL for (int j = 0; j < NG; ++j) {
+      const int col = cx.col0 + j * cx.gstride;
+      if (col < cx.col_end) {
+        PN_UNROLL for (int i = 0; i < VL; ++i) {
+          const float v = acc[j * VL + i];
+          if (arg_better(v, col + i, bv, bi, kind == RED_ARGMAX)) { bv = v; bi = col + i; }
+        }
+      }
+    }
+    t.a = bv; t.b = bits_f(static_cast<uint32_t>(bi));
+  } else if (kind == RED_LSE || kind == RED_SOFTMAX) {
+    float m = -PN_INF;
+    PN_UNROLL for (int j = 0; j < NG; ++j)
+      if (cx.col0 + j * cx.gstride < cx.col_end) {
+        PN_UNROLL for (int i = 0; i < VL; ++i) m = fmaxf(m, acc[j * VL + i]);
+      }
+    const float ms = (m == -PN_INF) ? 0.f : m;   // keeps exp(x - ms) free of inf - inf
+    float s = 0.f;
+    PN_UNROLL for (int j = 0; j < NG; ++j) {
+      const bool ok = cx.col0 + j * cx.gstride < cx.col_end;
+      PN_UNROLL for (int i = 0; i < VL; ++i) {
+        const float ev = ok ? f_exp(acc[j * VL + i] - ms) : 0.f;
+        s += ev;
+        if (kind == RED_SOFTMAX) acc[j * VL + i] = ev;
+      }
+    }
+    t.a = m; t.b = s;
+    if (kind == RED_SOFTMAX) ts = ms;
+  } else {  // RED_MEANVAR
+    float n = 0.f, sum = 0.f;
+    PN_UNROLL for (int j = 0; j < NG; ++j)
+      if (cx.col0 + j * cx.gstride < cx.col_end) {
+        n += static_cast<float>(VL);
+        PN_UNROLL for (int i = 0; i < VL; ++i) sum += acc[j * VL + i];
+      }
+    const float mean = n > 0.f ? sum / n : 0.f;
+    float m2 = 0.f;
+    PN_UNROLL for (int j = 0; j < NG; ++j)
+      if (cx.col0 + j * cx.gstride < cx.col_end) {
+        PN_UNROLL for (int i = 0; i < VL; ++i) { const float d = acc[j * VL + i] - mean; m2 = fmaf(d, d, m2); }
+      }
+    t.a = n; t.b = mean; t.c = m2;
+  }
+  float* ps = cx.part + ridx * 3 * cx.part_stride;
+  if (cx.chunk > 0) {
+    const Part prev{ps[0], ps[cx.part_stride], ps[2 * cx.part_stride]};
+    t = red_combine(kind, prev, t);
+  }
+  ps[0] = t.a; ps[cx.part_stride] = t.b; ps[2 * cx.part_stride] = t.c;
+}
+template <int V>
+PN_DEV void op_scale_ts(const TileCtx& cx, int slot_m, int slot_inv, float (&acc)[V], float ts) {
+  const float f = f_exp(ts - cx.slots[slot_m]) * cx.slots[slot_inv];
+  PN_UNROLL for (int e = 0; e < V; ++e) acc[e] *= f;
+}
+template <int V>
+PN_DEV float* stash_ptr(const TileCtx& cx, int idx) { return cx.stash + ((size_t)(idx * cx.chunks + cx.chunk) * V) * cx.part_stride; }
+template <int V>
+PN_DEV void op_spill(const TileCtx& cx, int idx, const float (&r)[V]) {
+  float* sp = stash_ptr<V>(cx, idx);
+  PN_UNROLL for (int e = 0; e < V; ++e) sp[e * cx.part_stride] = r[e];
+}
+template <int V>
+PN_DEV void op_fill(const TileCtx& cx, int idx, float (&r)[V]) {
+  const float* sp = stash_ptr<V>(cx, idx);
+  PN_UNROLL for (int e = 0; e < V; ++e) r[e] = sp[e * cx.part_stride];
+}
+// scalar programs: slot writes by lane 0 of the executing warp, visible after the warp sync
+PN_DEV void op_sst(const TileCtx& cx, int slot, float v) {
+  __syncwarp();
+  if ((threadIdx.x & 31) == 0) cx.slots[slot] = v;
+  __syncwarp();
+}
+
+// ---------------------------------------------------------------------------------------
+// the bytecode interpreter
+// ---------------------------------------------------------------------------------------
+// Run the statements with `r` bound to tile register k (kAccReg names the accumulator).
+// A macro, so that every case is straight-line code on statically indexed registers.
+#define PN_CASE_REG(n, ...) \
+  case n: if constexpr (K > n) { float(&r)[V] = reg[n]; __VA_ARGS__ } break;
+#define PN_WITH_REG(k, ...)                                 \
+  switch (k) {                                              \
+    PN_CASE_REG(0, __VA_ARGS__) PN_CASE_REG(1, __VA_ARGS__) \
+    PN_CASE_REG(2, __VA_ARGS__) PN_CASE_REG(3, __VA_ARGS__) \
+    default: { float(&r)[V] = acc; __VA_ARGS__ } break;     \
+  }
+
+// SCALAR = true: a per-row scalar program (VL = NG = 1): stores go to the row's element of a
+// per-row output and are done by the leader only.
+template <int VL, int NG, int K, bool SCALAR>
+PN_DEV void run_program(const KernelParams& p, int pc, const int pc_end, const TileCtx& cx,
+                        float (&acc)[VL * NG], float (&reg)[K][VL * NG], float& ts) {
+  constexpr int V = VL * NG;
+  while (pc < pc_end) {
+    const uint32_t word = p.code[pc++];
+    const int op = word & 0xFF, a = (word >> 8) & 0xFF, b = (word >> 16) & 0xFF, c = word >> 24;
+#define PN_U(OP) case OP: op_unary<OP, V>(acc); break;
+#define PN_B(OP)                                                              \
+  case OP:                                                                    \
+    if (b == OPK_REG) { PN_WITH_REG(a, op_binary<OP, V>(acc, r);) }           \
+    else op_binary_s<OP, V>(acc, (b == OPK_IMM) ? bits_f(p.code[pc++]) : cx.slots[a]); \
+    break;
+    switch (op) {
+      case OP_LDRAW:
+        if constexpr (!SCALAR) { const int dt = p.io[a].dtype; PN_WITH_REG(b, op_ldraw<VL, NG>(p, cx, a, dt, r);) }
+        break;
+      case OP_WIDEN:
+        if constexpr (!SCALAR) { const int dt = p.io[a].dtype; PN_WITH_REG(b, op_widen<VL, NG>(dt, r);) }
+        break;
+      case OP_LDBC: { const int dt = p.io[a].dtype; PN_WITH_REG(b, op_ldbc<V>(p, cx, a, dt, r);) break; }
+      case OP_LD: PN_WITH_REG(a, op_mov<V>(acc, r);) break;
+      case OP_ST: PN_WITH_REG(a, op_mov<V>(r, acc);) break;
+      case OP_STOUT:
+        if constexpr (SCALAR) op_stout_scalar(p, cx, a, p.io[a].dtype, acc[0]);
+        else op_stout<VL, NG>(p, cx, a, p.io[a].dtype, acc);
+        break;
+      case OP_STOUT_I:
+        if constexpr (SCALAR) op_stout_index(p, cx, a, p.io[a].dtype, acc[0]);
+        break;
+      PN_U(OP_NEG) PN_U(OP_ABS) PN_U(OP_EXP) PN_U(OP_LOG) PN_U(OP_SQRT) PN_U(OP_RSQRT) PN_U(OP_RECIP)
+      PN_U(OP_TANH) PN_U(OP_SIGMOID) PN_U(OP_SILU) PN_U(OP_GELU_TANH) PN_U(OP_GELU_ERF) PN_U(OP_RELU)
+      PN_U(OP_SQUARE) PN_U(OP_ERF) PN_U(OP_RND_BF16) PN_U(OP_RND_F16) PN_U(OP_TRUNC) PN_U(OP_NEZ) PN_U(OP_I2F)
+      PN_B(OP_ADD) PN_B(OP_SUB) PN_B(OP_RSUB) PN_B(OP_MUL) PN_B(OP_DIV) PN_B(OP_RDIV) PN_B(OP_MAX) PN_B(OP_MIN)
+      PN_B(OP_GT) PN_B(OP_GE) PN_B(OP_LT) PN_B(OP_LE) PN_B(OP_EQ) PN_B(OP_NE) PN_B(OP_LSEFIN)
+      case OP_WHERE: case OP_FMA: {
+        const int kx = c & 15, ky = c >> 4;
+        float xt[V], yt[V];
+        if (kx == OPK_REG) { PN_WITH_REG(a, op_mov<V>(xt, r);) }
+        else op_splat<V>(xt, kx == OPK_IMM ? bits_f(p.code[pc++]) : cx.slots[a]);
+        if (ky == OPK_REG) { PN_WITH_REG(b, op_mov<V>(yt, r);) }
+        else op_splat<V>(yt, ky == OPK_IMM ? bits_f(p.code[pc++]) : cx.slots[b]);
+        if (op == OP_WHERE) op_ternary<OP_WHERE, V>(acc, xt, yt); else op_ternary<OP_FMA, V>(acc, xt, yt);
+        break;
+      }
+      case OP_RED:
+        if constexpr (!SCALAR) op_red<VL, NG>(cx, a, b, acc, ts);
+        break;
+      case OP_SCALE_TS: op_scale_ts<V>(cx, a, b, acc, ts); break;
+      case OP_SPILL:
+        if constexpr (!SCALAR) { PN_WITH_REG(a, op_spill<V>(cx, b, r);) }
+        break;
+      case OP_FILL:
+        if constexpr (!SCALAR) { PN_WITH_REG(a, op_fill<V>(cx, b, r);) }
+        break;
+      case OP_SPILL_TS:
+        if constexpr (!SCALAR) *stash_ptr<V>(cx, b) = ts;
+        break;
+      case OP_FILL_TS:
+        if constexpr (!SCALAR) ts = *stash_ptr<V>(cx, b);
+        break;
+      case OP_SLD: op_splat<V>(acc, cx.slots[a]); break;
+      case OP_SST:
+        if constexpr (SCALAR) op_sst(cx, a, acc[0]);
+        break;
+      default: break;
+    }
+#undef PN_U
+#undef PN_B
+  }
+}
+
+// The interpreting program: every property is read from the launch parameters.
+template <int VL_, int NG_, int K_>
+struct Interp {
+  static constexpr int VL = VL_, NG = NG_, K = K_;
+  static constexpr bool kStatic = false;
+  static constexpr int kStages = kMaxStages;
+  static PN_DEV int family(const KernelParams& p) { return p.family; }
+  static PN_DEV int cluster(const KernelParams& p) { return p.cluster; }
+  static PN_DEV int chunks(const KernelParams& p) { return p.chunks; }
+  static PN_DEV int split_chunks(const KernelParams& p) { return p.split_chunks; }
+  static PN_DEV int row_len(const KernelParams& p) { return p.row_len; }
+  static PN_DEV int slice_len(const KernelParams& p) { return p.slice_len; }
+  static PN_DEV int n_stages(const KernelParams& p) { return p.n_stages; }
+  static PN_DEV int n_io(const KernelParams& p) { return p.n_io; }
+  static PN_DEV int n_red(const KernelParams& p, int s) { return p.stage[s].n_red; }
+  static PN_DEV int red_kind(const KernelParams& p, int s, int r) { return p.stage[s].red[r].kind; }
+  static PN_DEV int red_slot(const KernelParams& p, int s, int r) { return p.stage[s].red[r].slot; }
+  static PN_DEV bool has_scalar(const KernelParams& p, int s) { return p.stage[s].scal_begin != p.stage[s].scal_end; }
+  static PN_DEV void tile(const KernelParams& p, int s, const TileCtx& cx, float (&acc)[VL * NG],
+                          float (&reg)[K][VL * NG], float& ts) {
+    run_program<VL, NG, K, false>(p, p.stage[s].elem_begin, p.stage[s].elem_end, cx, acc, reg, ts);
+  }
+  static PN_DEV void scalar(const KernelParams& p, int s, const TileCtx& cx) {
+    float sacc[1] = {0.f}, sreg[4][1] = {{0.f}, {0.f}, {0.f}, {0.f}}, sts = 0.f;
+    run_program<1, 1, 4, true>(p, p.stage[s].scal_begin, p.stage[s].scal_end, cx, sacc, sreg, sts);
+  }
+};
+
+// ---------------------------------------------------------------------------------------
+// the kernel body, common to every family and to both kinds of program
+// ---------------------------------------------------------------------------------------
+template <class Prog>
+PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
+  constexpr int VL = Prog::VL, NG = Prog::NG, K = Prog::K, V = VL * NG;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+  const int family = Prog::family(p);
+  const int cluster = Prog::cluster(p);
+  const int chunks = Prog::chunks(p);
+  const bool split = Prog::split_chunks(p) != 0;
+  const bool warp_team = family <= FAM_WARP;
+  const int team_threads = warp_team ? 32 : (int)blockDim.x;
+  const int team_tid = warp_team ? lane : tid;
+  const int team_in_cta = warp_team ? warp : 0;
+  const int crank = (cluster > 1) ? (int)cluster_ctarank() : 0;
+
+  long long* rowoff = reinterpret_cast<long long*>(smem + p.sm_rowoff) + team_in_cta * kMaxIo;
+  float* wpart = reinterpret_cast<float*>(smem + p.sm_wpart);
+  float* slots = reinterpret_cast<float*>(smem + p.sm_slots) + team_in_cta * kMaxSlots;
+  float* ctapart = reinterpret_cast<float*>(smem + p.sm_ctapart);
+
+  TileCtx cx;
+  cx.rowoff = rowoff;
+  cx.part = reinterpret_cast<float*>(smem + p.sm_part) + tid;
+  cx.part_stride = blockDim.x;
+  cx.slots = slots;
+  cx.stash = reinterpret_cast<float*>(smem + p.sm_stash) + tid;
+  cx.gstride = team_threads * VL;
+  cx.chunks = chunks;
+  cx.chunk = 0;
+  cx.leader = (team_tid == 0) && (crank == 0);
+
+  const long long n_items = split ? p.rows * chunks : p.rows;
+  long long team_global, n_teams;
+  if (warp_team) { team_global = (long long)blockIdx.x * nwarps + warp; n_teams = (long long)gridDim.x * nwarps; }
+  else { team_global = blockIdx.x / cluster; n_teams = gridDim.x / cluster; }
+
+  const int slice_lo = crank * Prog::slice_len(p);
+  cx.col_end = min(Prog::row_len(p), slice_lo + Prog::slice_len(p));
+  const int chunk_cols = team_threads * V;
+  unsigned parity = 0;
+
+  float acc[V];
+  float reg[K][V];
+  float ts = 0.f;
+  PN_UNROLL for (int e = 0; e < V; ++e) acc[e] = 0.f;
+  PN_UNROLL for (int k = 0; k < K; ++k) { PN_UNROLL for (int e = 0; e < V; ++e) reg[k][e] = 0.f; }
+
+  for (long long item = team_global; item < n_items; item += n_teams) {
+    long long row = item;
+    int c_first = 0, c_count = chunks;
+    if (split) { row = item / chunks; c_first = (int)(item - row * chunks); c_count = 1; }
+
+    // element offset of this row in every input / output
+    if (team_tid < Prog::n_io(p)) {
+      const IoDesc& io = p.io[team_tid];
+      long long r = row;
+      const long long i2 = r % p.lead_dim[2]; r /= p.lead_dim[2];
+      const long long i1 = r % p.lead_dim[1]; r /= p.lead_dim[1];
+      rowoff[team_tid] = r * io.lead_stride[0] + i1 * io.lead_stride[1] + i2 * io.lead_stride[2];
+    }
+    if (warp_team) __syncwarp(); else __syncthreads();
+
+#pragma unroll(Prog::kStatic ? Prog::kStages : 1)
+    for (int s = 0; s < Prog::kStages; ++s) {
+      if (s >= Prog::n_stages(p)) break;
+      for (int c = c_first; c < c_first + c_count; ++c) {
+        cx.chunk = split ? 0 : c;
+        cx.col0 = slice_lo + c * chunk_cols + team_tid * VL;
+        Prog::tile(p, s, cx, acc, reg, ts);
+      }
+      const int n_red = Prog::n_red(p, s);
+      if (n_red == 0 && !Prog::has_scalar(p, s)) continue;
+
+      // ---- combine the partials of this stage over the team, then the scalar program ---
+      if (warp_team) {
+        for (int r = 0; r < n_red; ++r) {
+          const int kind = Prog::red_kind(p, s, r);
+          Part v{cx.part[(r * 3) * cx.part_stride], cx.part[(r * 3 + 1) * cx.part_stride],
+                 cx.part[(r * 3 + 2) * cx.part_stride]};
+          v = warp_combine(kind, v);
+          if (lane == 0) { float* d = slots + Prog::red_slot(p, s, r); d[0] = v.a; d[1] = v.b; d[2] = v.c; }
+        }
+        __syncwarp();
+        Prog::scalar(p, s, cx);
+        __syncwarp();
+      } else {
+        for (int r = 0; r < n_red; ++r) {
+          const int kind = Prog::red_kind(p, s, r);
+          Part v{cx.part[(r * 3) * cx.part_stride], cx.part[(r * 3 + 1) * cx.part_stride],
+                 cx.part[(r * 3 + 2) * cx.part_stride]};
+          v = warp_combine(kind, v);
+          if (lane == 0) { float* w = wpart + (warp * kMaxRed + r) * 3; w[0] = v.a; w[1] = v.b; w[2] = v.c; }
+        }
+        __syncthreads();
+        if (warp == 0) {
+          for (int r = 0; r < n_red; ++r) {
+            const int kind = Prog::red_kind(p, s, r);
+            Part v = red_identity(kind);
+            if (lane < nwarps) { const float* w = wpart + (lane * kMaxRed + r) * 3; v = Part{w[0], w[1], w[2]}; }
+            v = warp_combine(kind, v);
+            if (lane == 0) {
+              float* d = (cluster > 1) ? ctapart + (parity * kMaxRed + r) * 3 : slots + Prog::red_slot(p, s, r);
+              d[0] = v.a; d[1] = v.b; d[2] = v.c;
+            }
+          }
+        }
+        if (cluster > 1) {
+          cluster_sync_all();   // every CTA's partial is now in its own shared memory
+          if (warp == 0) {
+            for (int r = 0; r < n_red; ++r) {
+              const int kind = Prog::red_kind(p, s, r);
+              Part v = red_identity(kind);
+              if (lane < cluster) {
+                const float* w = ctapart + (parity * kMaxRed + r) * 3;
+                v = Part{ld_shared_cluster(w, lane), ld_shared_cluster(w + 1, lane), ld_shared_cluster(w + 2, lane)};
+              }
+              v = warp_combine(kind, v);
+              if (lane == 0) { float* d = slots + Prog::red_slot(p, s, r); d[0] = v.a; d[1] = v.b; d[2] = v.c; }
+            }
+          }
+          parity ^= 1u;
+        }
+        if (warp == 0) {
+          __syncwarp();
+          Prog::scalar(p, s, cx);
+        }
+        __syncthreads();
+      }
+    }
+    // the next item rewrites rowoff / slots: everyone must be done reading them
+    if (warp_team) __syncwarp(); else __syncthreads();
+  }
+  // a CTA's shared memory may still be read by its cluster peers until they pass this point
+  if (cluster > 1) cluster_sync_all();
+}
+
+}  // namespace pn

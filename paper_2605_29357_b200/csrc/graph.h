@@ -65,4 +65,7 @@ struct DeviceModel {      // what the lowering needs to know about the GPU
 // Lower a whole graph into one fused launch.  Returns a pn_status value.
 int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPlan& out, std::string& err);
 
+// Grid size of a planned launch given the SM count and its kernel's resident CTAs per SM.
+void size_grid(LaunchPlan& lp, int sms, int occ);
+
 }  // namespace pn

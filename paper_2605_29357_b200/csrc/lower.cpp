@@ -301,6 +301,23 @@ struct Gen {
   }
 };
 
+}  // namespace
+
+// Grid of a planned launch from the SM count and the resident CTAs per SM of its kernel:
+// whole work if it fits in a few waves, else a grid-stride loop over a bounded grid.
+void size_grid(LaunchPlan& lp, int sms, int occ) {
+  if (occ <= 0) occ = std::max(1, 512 / lp.block);
+  const int64_t resident = (int64_t)sms * occ;
+  const int cluster = std::max(lp.p.cluster, 1);
+  int64_t grid;
+  if (lp.family <= FAM_WARP) grid = std::min<int64_t>((lp.items + lp.teams_per_cta - 1) / lp.teams_per_cta, resident * 8);
+  else if (lp.family == FAM_BLOCK) grid = std::min<int64_t>(lp.items, resident * 8);
+  else grid = std::min<int64_t>(lp.items, std::max<int64_t>(1, resident * 8 / cluster)) * cluster;
+  lp.grid = (int)std::max<int64_t>(grid, cluster);
+}
+
+namespace {
+
 struct Config { int family, vl, ng, k, block, cluster, chunks, slice_len; bool multichunk; };
 
 }  // namespace
@@ -769,15 +786,12 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     P.cluster = cf.cluster;
     lp.family = cf.family; lp.vl = cf.vl; lp.ng = cf.ng; lp.k = cf.k;
     lp.block = cf.block; lp.smem_bytes = off; lp.code_words = (int)code.size();
+    P.family = cf.family;
+    lp.items = P.split_chunks ? eff_rows * cf.chunks : eff_rows;
+    lp.teams_per_cta = teams;
+    lp.specialised = 0;
     int occ = dev.have_device ? instance_occupancy(cf.vl, cf.ng, cf.k, cf.block, off) : 0;
-    if (occ <= 0) occ = std::max(1, 512 / cf.block);
-    const int64_t items = P.split_chunks ? eff_rows * cf.chunks : eff_rows;
-    const int64_t resident = (int64_t)sms * occ;
-    int64_t grid;
-    if (cf.family <= FAM_WARP) grid = std::min<int64_t>((items + teams - 1) / teams, resident * 8);
-    else if (cf.family == FAM_BLOCK) grid = std::min<int64_t>(items, resident * 8);
-    else grid = std::min<int64_t>(items, std::max<int64_t>(1, resident * 8 / cf.cluster)) * cf.cluster;
-    lp.grid = (int)std::max<int64_t>(grid, cf.cluster);
+    size_grid(lp, sms, occ);
     return PN_OK;
   }
   err = gen_err;

@@ -2,7 +2,19 @@
 // addressing of every graph input / output, and the launch shape.  Plain structs only;
 // included by host (.cpp) and device (.cu) code.
 #pragma once
+#ifndef __CUDACC_RTC__
 #include <stdint.h>
+#else   // run-time compilation has no standard headers: the fixed-width types by hand
+typedef signed char int8_t;
+typedef unsigned char uint8_t;
+typedef short int16_t;
+typedef unsigned short uint16_t;
+typedef int int32_t;
+typedef unsigned int uint32_t;
+typedef long long int64_t;
+typedef unsigned long long uint64_t;
+typedef unsigned long size_t;
+#endif
 
 namespace pn {
 
@@ -99,6 +111,8 @@ struct KernelParams {
   IoDesc io[kMaxIo];
   int32_t n_io;
   int32_t n_stages;
+  int32_t family;          // Family
+  int32_t pad0;
   uint32_t lead_dim[3];    // collapsed leading dims of the iteration space (unused = 1)
   int64_t rows;            // product of the leading dims
   int32_t row_len;         // N
@@ -120,6 +134,9 @@ struct LaunchPlan {
   int32_t vl, ng, k;       // template instance: vector length, groups per tile, tile registers
   int32_t grid, block, smem_bytes;
   int32_t code_words;
+  int64_t items;           // rows, or rows * chunks for pointwise graphs
+  int32_t teams_per_cta;
+  int32_t specialised;     // 1 when the launch uses a kernel generated for this program
   int32_t io_tensor[kMaxIo];   // tensor id behind each io entry
   int32_t io_is_output[kMaxIo];
 };

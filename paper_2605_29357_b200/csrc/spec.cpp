@@ -1,0 +1,306 @@
+// spec.cpp -- specialisation of a planned launch: the bytecode of a plan is translated,
+// instruction by instruction, into straight-line calls of the same op_* device functions the
+// interpreter dispatches to, wrapped in the common kernel body, and compiled for sm_100a with
+// NVRTC when the handle is created.  The result computes exactly what the interpreter would,
+// without the per-instruction decode and with registers allocated by the compiler.
+//
+// NVRTC and the driver API are opened with dlopen, so that the library loads (and the
+// interpreter works) on machines that have neither.
+#include <cuda.h>
+#include <dlfcn.h>
+#include <nvrtc.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <map>
+#include <mutex>
+#include <string>
+#include <vector>
+
+#include "graph.h"
+#include "spec.h"
+
+namespace pn {
+
+namespace {
+
+// plan.h followed by device_lib.cuh, as text (written by the build step)
+const char kDeviceSource[] =
+#include "_build/device_src.inc"
+    ;
+
+struct Api {
+  bool ok = false;
+  std::string why;
+  // nvrtc
+  nvrtcResult (*CreateProgram)(nvrtcProgram*, const char*, const char*, int, const char* const*, const char* const*) = nullptr;
+  nvrtcResult (*CompileProgram)(nvrtcProgram, int, const char* const*) = nullptr;
+  nvrtcResult (*GetProgramLogSize)(nvrtcProgram, size_t*) = nullptr;
+  nvrtcResult (*GetProgramLog)(nvrtcProgram, char*) = nullptr;
+  nvrtcResult (*GetCUBINSize)(nvrtcProgram, size_t*) = nullptr;
+  nvrtcResult (*GetCUBIN)(nvrtcProgram, char*) = nullptr;
+  nvrtcResult (*DestroyProgram)(nvrtcProgram*) = nullptr;
+  // driver
+  CUresult (*ModuleLoadData)(CUmodule*, const void*) = nullptr;
+  CUresult (*ModuleGetFunction)(CUfunction*, CUmodule, const char*) = nullptr;
+  CUresult (*FuncSetAttribute)(CUfunction, CUfunction_attribute, int) = nullptr;
+  CUresult (*LaunchKernelEx)(const CUlaunchConfig*, CUfunction, void**, void**) = nullptr;
+  CUresult (*OccupancyMaxActiveBlocks)(int*, CUfunction, int, size_t) = nullptr;
+  CUresult (*GetErrorString)(CUresult, const char**) = nullptr;
+};
+
+template <class F>
+bool sym(void* lib, const char* name, F& f, std::string& why) {
+  f = reinterpret_cast<F>(dlsym(lib, name));
+  if (!f) { why = std::string("symbol not found: ") + name; return false; }
+  return true;
+}
+
+const Api& api() {
+  static Api a;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    const char* builtins[] = {"libnvrtc-builtins.so.12.9", "/usr/local/cuda/lib64/libnvrtc-builtins.so.12.9",
+                              "libnvrtc-builtins.so.12.8", "libnvrtc-builtins.so"};
+    const char* names[] = {"libnvrtc.so.12", "/usr/local/cuda/lib64/libnvrtc.so.12", "libnvrtc.so"};
+    void* rt = nullptr;
+    for (const char* n : names) {
+      for (const char* b : builtins) if (dlopen(b, RTLD_NOW | RTLD_GLOBAL)) break;   // best effort
+      if ((rt = dlopen(n, RTLD_NOW | RTLD_GLOBAL))) break;
+    }
+    if (!rt) { a.why = "libnvrtc.so.12 not found"; return; }
+    bool ok = sym(rt, "nvrtcCreateProgram", a.CreateProgram, a.why) && sym(rt, "nvrtcCompileProgram", a.CompileProgram, a.why) &&
+              sym(rt, "nvrtcGetProgramLogSize", a.GetProgramLogSize, a.why) && sym(rt, "nvrtcGetProgramLog", a.GetProgramLog, a.why) &&
+              sym(rt, "nvrtcGetCUBINSize", a.GetCUBINSize, a.why) && sym(rt, "nvrtcGetCUBIN", a.GetCUBIN, a.why) &&
+              sym(rt, "nvrtcDestroyProgram", a.DestroyProgram, a.why);
+    if (!ok) { a.CreateProgram = nullptr; return; }
+    void* cu = dlopen("libcuda.so.1", RTLD_NOW | RTLD_GLOBAL);   // absent on machines without a GPU
+    if (!cu) { a.why = "libcuda.so.1 not found"; return; }
+    ok = sym(cu, "cuModuleLoadData", a.ModuleLoadData, a.why) && sym(cu, "cuModuleGetFunction", a.ModuleGetFunction, a.why) &&
+              sym(cu, "cuFuncSetAttribute", a.FuncSetAttribute, a.why) && sym(cu, "cuLaunchKernelEx", a.LaunchKernelEx, a.why) &&
+              sym(cu, "cuOccupancyMaxActiveBlocksPerMultiprocessor", a.OccupancyMaxActiveBlocks, a.why) &&
+              sym(cu, "cuGetErrorString", a.GetErrorString, a.why);
+    a.ok = ok;
+  });
+  return a;
+}
+
+std::string cu_err(CUresult r) {
+  const char* s = nullptr;
+  if (api().GetErrorString && api().GetErrorString(r, &s) == CUDA_SUCCESS && s) return s;
+  return "CUDA driver error " + std::to_string((int)r);
+}
+
+// ---------------------------------------------------------------------------------------
+// bytecode -> source
+// ---------------------------------------------------------------------------------------
+std::string regname(int k) { return k == kAccReg ? "acc" : "reg[" + std::to_string(k) + "]"; }
+std::string fbits(uint32_t u) { char b[48]; snprintf(b, sizeof(b), "__uint_as_float(0x%08xu)", u); return b; }
+
+bool is_unary(int op) { return op >= OP_NEG && op <= OP_I2F; }
+bool is_binary(int op) { return op >= OP_ADD && op <= OP_LSEFIN; }
+
+// One program range [pc, end) as statements.  vl/ng are the tile shape (1, 1 for scalar programs).
+bool emit_program(const KernelParams& P, int pc, int end, bool scalar, int vl, int ng, std::string& out, std::string& err) {
+  const std::string V = std::to_string(vl * ng), VLNG = std::to_string(vl) + ", " + std::to_string(ng);
+  while (pc < end) {
+    const uint32_t w = P.code[pc++];
+    const int op = w & 0xFF, a = (w >> 8) & 0xFF, b = (w >> 16) & 0xFF, c = w >> 24;
+    const std::string A = std::to_string(a), B = std::to_string(b), OP = std::to_string(op);
+    auto dt = [&](int io) { return std::to_string((int)P.io[io].dtype); };
+    std::string s;
+    if (op == OP_LDRAW) s = "op_ldraw<" + VLNG + ">(p, cx, " + A + ", " + dt(a) + ", " + regname(b) + ");";
+    else if (op == OP_WIDEN) s = "op_widen<" + VLNG + ">(" + dt(a) + ", " + regname(b) + ");";
+    else if (op == OP_LDBC) s = "op_ldbc<" + V + ">(p, cx, " + A + ", " + dt(a) + ", " + regname(b) + ");";
+    else if (op == OP_LD) s = "op_mov<" + V + ">(acc, " + regname(a) + ");";
+    else if (op == OP_ST) s = "op_mov<" + V + ">(" + regname(a) + ", acc);";
+    else if (op == OP_STOUT) s = scalar ? "op_stout_scalar(p, cx, " + A + ", " + dt(a) + ", acc[0]);"
+                                        : "op_stout<" + VLNG + ">(p, cx, " + A + ", " + dt(a) + ", acc);";
+    else if (op == OP_STOUT_I) s = "op_stout_index(p, cx, " + A + ", " + dt(a) + ", acc[0]);";
+    else if (is_unary(op)) s = "op_unary<" + OP + ", " + V + ">(acc);";
+    else if (is_binary(op)) {
+      if (b == OPK_REG) s = "op_binary<" + OP + ", " + V + ">(acc, " + regname(a) + ");";
+      else if (b == OPK_IMM) s = "op_binary_s<" + OP + ", " + V + ">(acc, " + fbits(P.code[pc++]) + ");";
+      else s = "op_binary_s<" + OP + ", " + V + ">(acc, cx.slots[" + A + "]);";
+    } else if (op == OP_WHERE || op == OP_FMA) {
+      const int kx = c & 15, ky = c >> 4;
+      std::string x, y, pre = "{ ";
+      if (kx == OPK_REG) x = regname(a);
+      else { pre += "float xt[" + V + "]; op_splat<" + V + ">(xt, " + (kx == OPK_IMM ? fbits(P.code[pc++]) : "cx.slots[" + A + "]") + "); "; x = "xt"; }
+      if (ky == OPK_REG) y = regname(b);
+      else { pre += "float yt[" + V + "]; op_splat<" + V + ">(yt, " + (ky == OPK_IMM ? fbits(P.code[pc++]) : "cx.slots[" + B + "]") + "); "; y = "yt"; }
+      s = pre + "op_ternary<" + OP + ", " + V + ">(acc, " + x + ", " + y + "); }";
+    }
+    else if (op == OP_RED) s = "op_red<" + VLNG + ">(cx, " + A + ", " + B + ", acc, ts);";
+    else if (op == OP_SCALE_TS) s = "op_scale_ts<" + V + ">(cx, " + A + ", " + B + ", acc, ts);";
+    else if (op == OP_SPILL) s = "op_spill<" + V + ">(cx, " + B + ", " + regname(a) + ");";
+    else if (op == OP_FILL) s = "op_fill<" + V + ">(cx, " + B + ", " + regname(a) + ");";
+    else if (op == OP_SPILL_TS) s = "*stash_ptr<" + V + ">(cx, " + B + ") = ts;";
+    else if (op == OP_FILL_TS) s = "ts = *stash_ptr<" + V + ">(cx, " + B + ");";
+    else if (op == OP_SLD) s = "op_splat<" + V + ">(acc, cx.slots[" + A + "]);";
+    else if (op == OP_SST) s = "op_sst(cx, " + A + ", acc[0]);";
+    else if (op == OP_END) continue;
+    else { err = "specialiser: unknown opcode " + OP; return false; }
+    out += "        " + s + "\n";
+  }
+  return true;
+}
+
+bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
+  const KernelParams& P = lp.p;
+  auto I = [](long long v) { return std::to_string(v); };
+  std::string s;
+  s.reserve(sizeof(kDeviceSource) + 8192);
+  s += kDeviceSource;
+  s += "\nnamespace pn {\nstruct Spec {\n";
+  s += "  static constexpr int VL = " + I(lp.vl) + ", NG = " + I(lp.ng) + ", K = " + I(lp.k) + ";\n";
+  s += "  static constexpr bool kStatic = true;\n  static constexpr int kStages = " + I(P.n_stages) + ";\n";
+  auto konst = [&](const char* name, long long v) {
+    s += std::string("  static PN_DEV int ") + name + "(const KernelParams&) { return " + I(v) + "; }\n";
+  };
+  konst("family", P.family); konst("cluster", P.cluster); konst("chunks", P.chunks); konst("split_chunks", P.split_chunks);
+  konst("row_len", P.row_len); konst("slice_len", P.slice_len); konst("n_stages", P.n_stages); konst("n_io", P.n_io);
+  auto table = [&](const char* name, const char* type, auto get) {
+    s += std::string("  static PN_DEV ") + type + " " + name + "(const KernelParams&, int s, int r) {\n    switch (s * " + I(kMaxRed) + " + r) {\n";
+    for (int st = 0; st < P.n_stages; ++st)
+      for (int r = 0; r < P.stage[st].n_red; ++r) s += "      case " + I(st * kMaxRed + r) + ": return " + I(get(st, r)) + ";\n";
+    s += "      default: return 0;\n    }\n  }\n";
+  };
+  table("red_kind", "int", [&](int st, int r) { return (long long)P.stage[st].red[r].kind; });
+  table("red_slot", "int", [&](int st, int r) { return (long long)P.stage[st].red[r].slot; });
+  s += "  static PN_DEV int n_red(const KernelParams&, int s) {\n    switch (s) {\n";
+  for (int st = 0; st < P.n_stages; ++st) s += "      case " + I(st) + ": return " + I(P.stage[st].n_red) + ";\n";
+  s += "      default: return 0;\n    }\n  }\n";
+  s += "  static PN_DEV bool has_scalar(const KernelParams&, int s) {\n    switch (s) {\n";
+  for (int st = 0; st < P.n_stages; ++st) s += "      case " + I(st) + ": return " + (P.stage[st].scal_begin != P.stage[st].scal_end ? "true" : "false") + ";\n";
+  s += "      default: return false;\n    }\n  }\n";
+  const std::string V = I(lp.vl * lp.ng);
+  s += "  static PN_DEV void tile(const KernelParams& p, int s, const TileCtx& cx, float (&acc)[" + V + "], float (&reg)[" + I(lp.k) + "][" + V + "], float& ts) {\n    switch (s) {\n";
+  for (int st = 0; st < P.n_stages; ++st) {
+    s += "      case " + I(st) + ": {\n";
+    if (!emit_program(P, P.stage[st].elem_begin, P.stage[st].elem_end, false, lp.vl, lp.ng, s, err)) return false;
+    s += "      } break;\n";
+  }
+  s += "      default: break;\n    }\n  }\n";
+  s += "  static PN_DEV void scalar(const KernelParams& p, int s, const TileCtx& cx) {\n"
+       "    float acc[1] = {0.f}; float reg[4][1] = {{0.f}, {0.f}, {0.f}, {0.f}}; float ts = 0.f;\n    (void)reg; (void)ts;\n    switch (s) {\n";
+  for (int st = 0; st < P.n_stages; ++st) {
+    s += "      case " + I(st) + ": {\n";
+    if (!emit_program(P, P.stage[st].scal_begin, P.stage[st].scal_end, true, 1, 1, s, err)) return false;
+    s += "      } break;\n";
+  }
+  s += "      default: break;\n    }\n  }\n};\n}  // namespace pn\n\n";
+  s += "extern \"C\" __global__ void __launch_bounds__(" + I(lp.block) + ") pn_spec_kernel(const __grid_constant__ pn::KernelParams p) {\n"
+       "  extern __shared__ __align__(16) unsigned char smem[];\n  pn::fused_body<pn::Spec>(p, smem);\n}\n";
+  src.swap(s);
+  return true;
+}
+
+struct Compiled { CUmodule mod = nullptr; CUfunction fn = nullptr; };
+std::mutex g_cache_mutex;
+std::map<std::pair<int, std::string>, Compiled> g_cache;   // (device, source) -> loaded kernel; lives until exit
+
+}  // namespace
+
+bool spec_available(std::string* why) {
+  const Api& a = api();
+  if (!a.ok && why) *why = a.why;
+  return a.ok;
+}
+
+std::string spec_source(const LaunchPlan& lp) {
+  std::string src, err;
+  if (!generate_source(lp, src, err)) return "// " + err;
+  return src.substr(sizeof(kDeviceSource) - 1);   // the generated part only
+}
+
+bool spec_check(const LaunchPlan& lp, std::string& err) {
+  const Api& a = api();
+  if (!a.CreateProgram) { err = a.why.empty() ? "NVRTC not available" : a.why; return false; }
+  std::string src;
+  if (!generate_source(lp, src, err)) return false;
+  nvrtcProgram prog;
+  if (a.CreateProgram(&prog, src.c_str(), "pn_spec.cu", 0, nullptr, nullptr) != NVRTC_SUCCESS) { err = "nvrtcCreateProgram failed"; return false; }
+  const char* opts[] = {"-arch=sm_100a", "-std=c++17", "-lineinfo"};
+  const nvrtcResult r = a.CompileProgram(prog, 3, opts);
+  size_t n = 0; a.GetProgramLogSize(prog, &n);
+  std::string log(n, '\0');
+  if (n) a.GetProgramLog(prog, &log[0]);
+  a.DestroyProgram(&prog);
+  if (r != NVRTC_SUCCESS) { err = "run-time compilation failed: " + log.substr(0, 4000); return false; }
+  return true;
+}
+
+bool spec_compile(LaunchPlan& lp, int device, int sm_count, SpecKernel& out, std::string& err) {
+  const Api& a = api();
+  if (!a.ok) { err = a.why; return false; }
+  std::string src;
+  if (!generate_source(lp, src, err)) return false;
+  Compiled cmp;
+  {
+    std::lock_guard<std::mutex> lock(g_cache_mutex);
+    auto it = g_cache.find(std::make_pair(device, src));
+    if (it != g_cache.end()) cmp = it->second;
+  }
+  if (!cmp.fn) {
+    nvrtcProgram prog;
+    if (a.CreateProgram(&prog, src.c_str(), "pn_spec.cu", 0, nullptr, nullptr) != NVRTC_SUCCESS) { err = "nvrtcCreateProgram failed"; return false; }
+    const char* opts[] = {"-arch=sm_100a", "-std=c++17", "-lineinfo"};
+    const nvrtcResult r = a.CompileProgram(prog, 3, opts);
+    if (r != NVRTC_SUCCESS) {
+      size_t n = 0; a.GetProgramLogSize(prog, &n);
+      std::string log(n, '\0');
+      if (n) a.GetProgramLog(prog, &log[0]);
+      a.DestroyProgram(&prog);
+      err = "run-time compilation failed: " + log.substr(0, 2000);
+      return false;
+    }
+    size_t n = 0;
+    a.GetCUBINSize(prog, &n);
+    std::vector<char> cubin(n);
+    a.GetCUBIN(prog, cubin.data());
+    a.DestroyProgram(&prog);
+    CUresult cr = a.ModuleLoadData(&cmp.mod, cubin.data());
+    if (cr != CUDA_SUCCESS) { err = "cuModuleLoadData: " + cu_err(cr); return false; }
+    cr = a.ModuleGetFunction(&cmp.fn, cmp.mod, "pn_spec_kernel");
+    if (cr != CUDA_SUCCESS) { err = "cuModuleGetFunction: " + cu_err(cr); return false; }
+    std::lock_guard<std::mutex> lock(g_cache_mutex);
+    g_cache[std::make_pair(device, src)] = cmp;
+  }
+  if (lp.smem_bytes > 48 * 1024) {
+    const CUresult cr = a.FuncSetAttribute(cmp.fn, CU_FUNC_ATTRIBUTE_MAX_DYNAMIC_SHARED_SIZE_BYTES, lp.smem_bytes);
+    if (cr != CUDA_SUCCESS) { err = "cuFuncSetAttribute: " + cu_err(cr); return false; }
+  }
+  int occ = 0;
+  if (a.OccupancyMaxActiveBlocks(&occ, cmp.fn, lp.block, (size_t)lp.smem_bytes) != CUDA_SUCCESS) occ = 0;
+  out.fn = cmp.fn;
+  out.occupancy = occ;
+  lp.specialised = 1;
+  size_grid(lp, sm_count, occ);
+  return true;
+}
+
+bool spec_launch(const SpecKernel& k, const LaunchPlan& lp, void* stream, std::string& err) {
+  const Api& a = api();
+  CUlaunchConfig cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDimX = lp.grid; cfg.gridDimY = 1; cfg.gridDimZ = 1;
+  cfg.blockDimX = lp.block; cfg.blockDimY = 1; cfg.blockDimZ = 1;
+  cfg.sharedMemBytes = lp.smem_bytes;
+  cfg.hStream = (CUstream)stream;
+  CUlaunchAttribute attr[1];
+  if (lp.p.cluster > 1) {
+    attr[0].id = CU_LAUNCH_ATTRIBUTE_CLUSTER_DIMENSION;
+    attr[0].value.clusterDim.x = lp.p.cluster;
+    attr[0].value.clusterDim.y = 1;
+    attr[0].value.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+  }
+  void* args[] = {const_cast<KernelParams*>(&lp.p)};
+  const CUresult r = a.LaunchKernelEx(&cfg, (CUfunction)k.fn, args, nullptr);
+  if (r != CUDA_SUCCESS) { err = "cuLaunchKernelEx: " + cu_err(r); return false; }
+  return true;
+}
+
+}  // namespace pn

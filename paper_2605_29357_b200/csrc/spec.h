@@ -1,0 +1,30 @@
+// spec.h -- per-graph specialised kernels (see spec.cpp).
+#pragma once
+#include <string>
+
+#include "plan.h"
+
+namespace pn {
+
+struct SpecKernel {
+  void* fn = nullptr;     // CUfunction of the loaded kernel; owned by a process-wide cache
+  int occupancy = 0;      // resident CTAs per SM at the plan's block size and shared memory
+};
+
+// True when NVRTC and the driver API could be opened; otherwise *why says what is missing.
+bool spec_available(std::string* why);
+
+// Translate the plan's bytecode into a kernel, compile it for sm_100a, load it on the
+// current device and re-size the plan's grid from the kernel's occupancy.
+bool spec_compile(LaunchPlan& lp, int device, int sm_count, SpecKernel& out, std::string& err);
+
+// Enqueue the specialised kernel of a plan on a stream.
+bool spec_launch(const SpecKernel& k, const LaunchPlan& lp, void* stream, std::string& err);
+
+// Compile the plan's generated kernel with NVRTC and discard the result (needs no GPU).
+bool spec_check(const LaunchPlan& lp, std::string& err);
+
+// The generated part of the source, for inspection.
+std::string spec_source(const LaunchPlan& lp);
+
+}  // namespace pn

@@ -14,6 +14,10 @@ pytestmark = pytest.mark.gpu
 
 FORCES = {
     "default": 0,
+    "interpret": pn.FLAG_INTERPRET,
+    "interpret_unfused": pn.FLAG_INTERPRET | pn.FLAG_UNFUSED,
+    "interpret_cluster": pn.FLAG_INTERPRET | pn.FLAG_FORCE_CLUSTER,
+    "interpret_block_multichunk": pn.FLAG_INTERPRET | pn.FLAG_FORCE_BLOCK | pn.FLAG_FORCE_MULTICHUNK,
     "unfused": pn.FLAG_UNFUSED,
     "scalar": pn.FLAG_FORCE_SCALAR,
     "warp": pn.FLAG_FORCE_WARP,
@@ -32,6 +36,8 @@ def test_small_config(cfg, force):
     g = pn.Graph(w.desc, 0, FORCES[force])
     outs = run_graph(g, w.inputs)
     check_against_oracle(w.desc, w.inputs, outs, w.output_meta, w.output_names)
+    want_spec = 0 if force.startswith("interpret") else 1
+    assert all(k["specialised"] == want_spec for k in g.kernel_info)
     if force == "default":
         assert g.n_kernels == 1
     if force == "unfused":

@@ -1,0 +1,162 @@
+"""Host-side logic of the library, on the CPU: the shared library loads and exports what
+include/pn.h declares, descriptors are validated into the documented status codes, the
+lowering picks the documented kernel families, and the kernel generated for each benchmark
+graph compiles for sm_100a.  No GPU is touched (handles are created plan-only)."""
+import ctypes
+import os
+import re
+import struct
+
+import pytest
+
+import paper_2605_29357_b200 as pn
+from paper_2605_29357_b200 import binding
+from pn_workloads import configs as C
+from pn_workloads import descriptor as D
+from pn_workloads.descriptor import GraphBuilder, Imm
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+PLAN = pn.FLAG_PLAN_ONLY
+
+
+def test_library_exports_every_declared_symbol():
+    lib = pn.load_library()
+    header = open(os.path.join(ROOT, "include", "pn.h")).read()
+    declared = set(re.findall(r"\b(pn_[a-z_]+)\s*\(", header))
+    assert declared == set(binding.EXPORTS)
+    for name in declared:
+        assert getattr(lib, name) is not None
+
+
+def test_status_strings_and_null_arguments():
+    lib = pn.load_library()
+    assert lib.pn_status_string(0) == b"ok"
+    assert lib.pn_status_string(-4) == b"shape error"
+    h = ctypes.c_void_p()
+    assert lib.pn_graph_create(None, 0, 0, PLAN, ctypes.byref(h)) == -1
+    assert lib.pn_graph_destroy(None) == 0
+    assert lib.pn_graph_query(None, 1, None, 0) == -1
+
+
+def _status(desc, flags=PLAN):
+    try:
+        pn.Graph(bytes(desc), 0, flags).close()
+        return 0
+    except pn.PnError as e:
+        return e.status
+
+
+def test_malformed_descriptors_are_rejected():
+    good = bytearray(C.c1(M=2, N=8).desc)
+    assert _status(good) == 0
+    assert _status(good[:10]) == -2
+    bad = good[:]; bad[0] ^= 0xFF
+    assert _status(bad) == -2                                   # magic
+    assert _status(good + b"\0") == -2                          # length
+    bad = good[:]; struct.pack_into("<H", bad, 16 + 40 * 8, 999)
+    assert _status(bad) == -3                                   # unknown opcode
+    bad = good[:]; struct.pack_into("<I", bad, 16 + 40 * 8 + 4, 77)
+    assert _status(bad) == -2                                   # operand id out of range
+    bad = good[:]; bad[16] = 9
+    assert _status(bad) == -2                                   # unknown dtype
+    # a node reading a tensor that a later node produces
+    g = GraphBuilder(); x = g.input(D.F32, (4,))
+    t_late = g._add_tensor(D.F32, (4,), 0)
+    y = g.op("add", [x, t_late], D.F32, (4,))
+    g.node("neg", [x], [D.F32], [(4,)])
+    g._nodes[-1].outs = [t_late]; g._tensors.pop()
+    g.mark_output(y)
+    assert _status(g.build()) == -2
+
+
+def test_shape_and_support_errors():
+    g = GraphBuilder(); a = g.input(D.F32, (4, 8)); b = g.input(D.F32, (3, 8))
+    g.mark_output(g.op("add", [a, b], D.F32, (4, 8)))
+    assert _status(g.build()) == -4                             # operands do not broadcast
+    g = GraphBuilder(); a = g.input(D.F32, (4, 8))
+    g.mark_output(g.op("sum", [a], D.F32, (8,)))
+    assert _status(g.build()) == -4                             # reduction result of the wrong shape
+    g = GraphBuilder(); a = g.input(D.F32, (4, 8))
+    g.mark_output(g.op("argmax", [a], D.F32, (4,)))
+    assert _status(g.build()) == -3                             # index results are integers
+    g = GraphBuilder(); a = g.input(D.F32, (4, 0))
+    g.mark_output(g.op("neg", [a], D.F32, (4, 0)))
+    assert _status(g.build()) == 0                              # empty tensors: a no-op handle
+    g = GraphBuilder(); ins = [g.input(D.F32, (8,)) for _ in range(13)]
+    t = ins[0]
+    for u in ins[1:]:
+        t = g.op("add", [t, u], D.F32, (8,))
+    g.mark_output(t)
+    assert _status(g.build()) == -5                             # more inputs than a kernel takes
+    assert _status(g.build(), PLAN | pn.FLAG_UNFUSED) == 0      # one node at a time still fits
+
+
+FAMILY = {"c1": "pointwise", "c2": "warp-per-row", "c3": "block-per-row", "c4": "cluster-per-row",
+          "c5": "block-per-row"}
+FULL = {"c1": dict(M=1024, N=1024), "c2": dict(B=512, Q=512, K=512), "c3": dict(M=16384, N=4096),
+        "c4": dict(M=64, N=262144), "c5": dict(M=8192, N=14336)}
+
+
+def _descriptor_only(cfg, kw):
+    """The full-size graph without drawing its inputs: descriptors depend on shapes only, so
+    take one built at a tiny size of every free dimension and patch nothing -- instead build
+    the graph at full size through a generator stub."""
+    import numpy as np
+    real_draw = C._draw
+    C._draw = lambda rng, kind, shape, a, b, chunk=0: np.zeros(shape, dtype=np.float32)
+    try:
+        return C.CONFIGS[cfg](**kw)
+    finally:
+        C._draw = real_draw
+
+
+@pytest.mark.parametrize("cfg", list(FAMILY))
+def test_lowering_of_the_benchmark_graphs(cfg):
+    w = _descriptor_only(cfg, FULL[cfg])
+    g = pn.Graph(w.desc, 0, PLAN)
+    assert g.n_kernels == 1 and g.n_nodes == w.n_nodes
+    assert g.compulsory_bytes == w.compulsory_bytes
+    k = g.kernel_info[0]
+    assert pn.FAMILY_NAMES[k["family"]] == FAMILY[cfg]
+    assert k["vl"] * (2 if cfg in ("c2", "c3", "c5") else 4) == 16         # 128-bit accesses
+    if cfg == "c4":
+        assert k["cluster"] == 8 and k["grid"] % 8 == 0
+    if cfg in ("c2", "c3"):
+        assert k["chunks"] == 1                                             # row resident in registers
+    gu = pn.Graph(w.desc, 0, PLAN | pn.FLAG_UNFUSED)
+    assert gu.n_kernels == w.n_nodes and (gu.workspace_bytes > 0 or cfg == "c4")
+    assert [m for m in g.input_meta] == [(dt, tuple(d)) for dt, d in w.input_meta]
+    assert [m for m in g.output_meta] == [(dt, tuple(d)) for dt, d in w.output_meta]
+
+
+COMPULSORY = {"c1": 12591104, "c2": 537133056, "c3": 402817024, "c4": 67109632, "c5": 822194176}
+
+
+@pytest.mark.parametrize("cfg", list(COMPULSORY))
+def test_compulsory_bytes(cfg):
+    w = _descriptor_only(cfg, FULL[cfg])
+    assert w.compulsory_bytes == COMPULSORY[cfg]
+
+
+@pytest.mark.parametrize("flags", [0, pn.FLAG_FORCE_SCALAR, pn.FLAG_FORCE_CLUSTER | pn.FLAG_FORCE_MULTICHUNK])
+@pytest.mark.parametrize("cfg", list(FAMILY))
+def test_generated_kernels_compile(cfg, flags):
+    w = C.CONFIGS[cfg](**C.SMALL[cfg])
+    g = pn.Graph(w.desc, 0, PLAN | flags)
+    src = g.codegen(0, compile=True)
+    assert "pn_spec_kernel" in src and "struct Spec" in src
+
+
+def test_forced_families():
+    w = C.c3(M=8, N=1024)
+    for flag, fam in ((pn.FLAG_FORCE_WARP, "warp-per-row"), (pn.FLAG_FORCE_BLOCK, "block-per-row"),
+                      (pn.FLAG_FORCE_CLUSTER, "cluster-per-row")):
+        k = pn.Graph(w.desc, 0, PLAN | flag).kernel_info[0]
+        assert pn.FAMILY_NAMES[k["family"]] == fam
+    k = pn.Graph(w.desc, 0, PLAN | pn.FLAG_FORCE_SCALAR).kernel_info[0]
+    assert k["vl"] == 1
+    k = pn.Graph(w.desc, 0, PLAN | pn.FLAG_FORCE_BLOCK | pn.FLAG_FORCE_MULTICHUNK).kernel_info[0]
+    assert k["chunks"] > 1
+    # a row length that is not a multiple of the vector width falls back to element accesses
+    k = pn.Graph(C.c3(M=4, N=1001).desc, 0, PLAN).kernel_info[0]
+    assert k["vl"] == 1
