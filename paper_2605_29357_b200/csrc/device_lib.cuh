@@ -206,6 +206,14 @@ PN_DEV float f_exp(float x) {
   const float e = exp2f(t);
   return (fabsf(x) < 100.f) ? fmaf(e, r * LN2, e) : e;   // no correction at inf / overflow
 }
+// e^x for the shifted arguments of softmax / logsumexp (x <= 0 up to rounding): 2^(x*log2 e)
+// straight from the hardware exponential.  The rounding of the product costs a relative
+// error of about |x| * 6e-8 (5e-6 at the underflow edge x = -87), on values that are at most 1.
+PN_DEV float f_exp_neg(float x) {
+  float e;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(x * 1.4426950408889634f));
+  return e;
+}
 PN_DEV float f_sigmoid(float x) { return __fdividef(1.f, 1.f + f_exp(-x)); }
 // 0.5 x (1 + tanh u) = x / (1 + e^(-2u)),  u = sqrt(2/pi) (x + 0.044715 x^3)
 PN_DEV float f_gelu_tanh(float x) {
@@ -298,7 +306,7 @@ PN_DEV Part red_combine(int kind, Part x, Part y) {
     case RED_LSE: case RED_SOFTMAX: {
       const float m = fmaxf(x.a, y.a);
       if (m == -PN_INF) { x.b = 0.f; }
-      else { x.b = x.b * f_exp(x.a - m) + y.b * f_exp(y.a - m); }
+      else { x.b = x.b * f_exp_neg(x.a - m) + y.b * f_exp_neg(y.a - m); }
       x.a = m;
       break;
     }
@@ -349,8 +357,8 @@ PN_DEV float ld_shared_cluster(const float* local_smem_ptr, uint32_t rank) {
 // ---------------------------------------------------------------------------------------
 struct TileCtx {
   const long long* rowoff;  // shared: element offset of this row for every io entry
-  float* part;              // shared: this thread's partials, part[(r*3+q)*part_stride]
-  float* slots;             // shared: per-row scalar slots of this team
+  float* part;              // shared: this thread's partials, part[(r*3+q)*part_stride] (interpreter)
+  float* slots;             // per-row scalar slots of this team (shared memory, or registers)
   float* stash;             // shared: parked tile values (already offset by threadIdx.x)
   int part_stride;          // threads per CTA
   int col0;                 // column of (group 0, element 0)
@@ -360,13 +368,14 @@ struct TileCtx {
   bool leader;              // this thread performs per-row scalar stores
 };
 
-template <int VL, int NG>
+// FULL: every group of every tile lies inside the row (no validity tests needed).
+template <int VL, int NG, bool FULL = false>
 PN_DEV void op_ldraw(const KernelParams& p, const TileCtx& cx, int io, int dt, float (&r)[VL * NG]) {
   const char* base = static_cast<const char*>(p.io[io].base);
   const long long off = cx.rowoff[io];
   PN_UNROLL for (int j = 0; j < NG; ++j) {
     const int col = cx.col0 + j * cx.gstride;
-    if (col < cx.col_end) {
+    if (FULL || col < cx.col_end) {
       load_group_raw<VL>(base, off + col, dt, &r[j * VL]);
     } else {
       PN_UNROLL for (int i = 0; i < VL; ++i) r[j * VL + i] = 0.f;
@@ -384,13 +393,13 @@ PN_DEV void op_ldbc(const KernelParams& p, const TileCtx& cx, int io, int dt, fl
 }
 template <int V>
 PN_DEV void op_mov(float (&d)[V], const float (&s)[V]) { PN_UNROLL for (int e = 0; e < V; ++e) d[e] = s[e]; }
-template <int VL, int NG>
+template <int VL, int NG, bool FULL = false>
 PN_DEV void op_stout(const KernelParams& p, const TileCtx& cx, int io, int dt, const float (&acc)[VL * NG]) {
   char* base = static_cast<char*>(p.io[io].base);
   const long long off = cx.rowoff[io];
   PN_UNROLL for (int j = 0; j < NG; ++j) {
     const int col = cx.col0 + j * cx.gstride;
-    if (col < cx.col_end) store_group<VL>(base, off + col, dt, &acc[j * VL]);
+    if (FULL || col < cx.col_end) store_group<VL>(base, off + col, dt, &acc[j * VL]);
   }
 }
 // per-row scalar stores (leader thread only)
@@ -419,19 +428,19 @@ PN_DEV void op_ternary(float (&acc)[V], const float (&x)[V], const float (&y)[V]
 template <int V>
 PN_DEV void op_splat(float (&t)[V], float v) { PN_UNROLL for (int e = 0; e < V; ++e) t[e] = v; }
 
-// Fold the valid elements of the tile (in element order) into the thread's partial of
-// reduction `ridx`; RED_SOFTMAX also turns acc into exp(x - m_tile) and leaves m_tile in ts.
-template <int VL, int NG>
-PN_DEV void op_red(const TileCtx& cx, int kind, int ridx, float (&acc)[VL * NG], float& ts) {
+// Fold the valid elements of the tile (in element order) into the thread's partial `st` of a
+// reduction; RED_SOFTMAX also turns acc into exp(x - m_tile) and leaves m_tile in ts.
+template <int VL, int NG, bool FULL = false>
+PN_DEV void op_red(const TileCtx& cx, int kind, Part& st, float (&acc)[VL * NG], float& ts) {
   Part t = red_identity(kind);
   if (kind == RED_SUM) {
     PN_UNROLL for (int j = 0; j < NG; ++j)
-      if (cx.col0 + j * cx.gstride < cx.col_end) {
+      if (FULL || cx.col0 + j * cx.gstride < cx.col_end) {
         PN_UNROLL for (int i = 0; i < VL; ++i) t.a += acc[j * VL + i];
       }
   } else if (kind == RED_MAX || kind == RED_MIN) {
     PN_UNROLL for (int j = 0; j < NG; ++j)
-      if (cx.col0 + j * cx.gstride < cx.col_end) {
+      if (FULL || cx.col0 + j * cx.gstride < cx.col_end) {
         PN_UNROLL for (int i = 0; i < VL; ++i)
           t.a = kind == RED_MAX ? f_max_nan(t.a, acc[j * VL + i]) : f_min_nan(t.a, acc[j * VL + i]);
       }
@@ -440,7 +449,7 @@ PN_DEV void op_red(const TileCtx& cx, int kind, int ridx, float (&acc)[VL * NG],
     float bv = t.a;
     PN_UNROLL for (int j = 0; j < NG; ++j) {
       const int col = cx.col0 + j * cx.gstride;
-      if (col < cx.col_end) {
+      if (FULL || col < cx.col_end) {
         PN_UNROLL for (int i = 0; i < VL; ++i) {
           const float v = acc[j * VL + i];
           if (arg_better(v, col + i, bv, bi, kind == RED_ARGMAX)) { bv = v; bi = col + i; }
@@ -451,15 +460,15 @@ PN_DEV void op_red(const TileCtx& cx, int kind, int ridx, float (&acc)[VL * NG],
   } else if (kind == RED_LSE || kind == RED_SOFTMAX) {
     float m = -PN_INF;
     PN_UNROLL for (int j = 0; j < NG; ++j)
-      if (cx.col0 + j * cx.gstride < cx.col_end) {
+      if (FULL || cx.col0 + j * cx.gstride < cx.col_end) {
         PN_UNROLL for (int i = 0; i < VL; ++i) m = fmaxf(m, acc[j * VL + i]);
       }
     const float ms = (m == -PN_INF) ? 0.f : m;   // keeps exp(x - ms) free of inf - inf
     float s = 0.f;
     PN_UNROLL for (int j = 0; j < NG; ++j) {
-      const bool ok = cx.col0 + j * cx.gstride < cx.col_end;
+      const bool ok = FULL || cx.col0 + j * cx.gstride < cx.col_end;
       PN_UNROLL for (int i = 0; i < VL; ++i) {
-        const float ev = ok ? f_exp(acc[j * VL + i] - ms) : 0.f;
+        const float ev = ok ? f_exp_neg(acc[j * VL + i] - ms) : 0.f;
         s += ev;
         if (kind == RED_SOFTMAX) acc[j * VL + i] = ev;
       }
@@ -469,28 +478,23 @@ PN_DEV void op_red(const TileCtx& cx, int kind, int ridx, float (&acc)[VL * NG],
   } else {  // RED_MEANVAR
     float n = 0.f, sum = 0.f;
     PN_UNROLL for (int j = 0; j < NG; ++j)
-      if (cx.col0 + j * cx.gstride < cx.col_end) {
+      if (FULL || cx.col0 + j * cx.gstride < cx.col_end) {
         n += static_cast<float>(VL);
         PN_UNROLL for (int i = 0; i < VL; ++i) sum += acc[j * VL + i];
       }
     const float mean = n > 0.f ? sum / n : 0.f;
     float m2 = 0.f;
     PN_UNROLL for (int j = 0; j < NG; ++j)
-      if (cx.col0 + j * cx.gstride < cx.col_end) {
+      if (FULL || cx.col0 + j * cx.gstride < cx.col_end) {
         PN_UNROLL for (int i = 0; i < VL; ++i) { const float d = acc[j * VL + i] - mean; m2 = fmaf(d, d, m2); }
       }
     t.a = n; t.b = mean; t.c = m2;
   }
-  float* ps = cx.part + ridx * 3 * cx.part_stride;
-  if (cx.chunk > 0) {
-    const Part prev{ps[0], ps[cx.part_stride], ps[2 * cx.part_stride]};
-    t = red_combine(kind, prev, t);
-  }
-  ps[0] = t.a; ps[cx.part_stride] = t.b; ps[2 * cx.part_stride] = t.c;
+  st = (cx.chunk > 0) ? red_combine(kind, st, t) : t;
 }
 template <int V>
 PN_DEV void op_scale_ts(const TileCtx& cx, int slot_m, int slot_inv, float (&acc)[V], float ts) {
-  const float f = f_exp(ts - cx.slots[slot_m]) * cx.slots[slot_inv];
+  const float f = f_exp_neg(ts - cx.slots[slot_m]) * cx.slots[slot_inv];
   PN_UNROLL for (int e = 0; e < V; ++e) acc[e] *= f;
 }
 template <int V>
@@ -505,11 +509,17 @@ PN_DEV void op_fill(const TileCtx& cx, int idx, float (&r)[V]) {
   const float* sp = stash_ptr<V>(cx, idx);
   PN_UNROLL for (int e = 0; e < V; ++e) r[e] = sp[e * cx.part_stride];
 }
-// scalar programs: slot writes by lane 0 of the executing warp, visible after the warp sync
+// scalar programs: slots in shared memory are written by lane 0 of the executing warp and
+// visible after the warp sync; slots kept in registers (every lane holds the same values) are
+// plain assignments
+template <bool REG_SLOTS = false>
 PN_DEV void op_sst(const TileCtx& cx, int slot, float v) {
-  __syncwarp();
-  if ((threadIdx.x & 31) == 0) cx.slots[slot] = v;
-  __syncwarp();
+  if constexpr (REG_SLOTS) { cx.slots[slot] = v; }
+  else {
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) cx.slots[slot] = v;
+    __syncwarp();
+  }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -574,7 +584,12 @@ PN_DEV void run_program(const KernelParams& p, int pc, const int pc_end, const T
         break;
       }
       case OP_RED:
-        if constexpr (!SCALAR) op_red<VL, NG>(cx, a, b, acc, ts);
+        if constexpr (!SCALAR) {
+          float* ps = cx.part + b * 3 * cx.part_stride;
+          Part st{ps[0], ps[cx.part_stride], ps[2 * cx.part_stride]};
+          op_red<VL, NG>(cx, a, st, acc, ts);
+          ps[0] = st.a; ps[cx.part_stride] = st.b; ps[2 * cx.part_stride] = st.c;
+        }
         break;
       case OP_SCALE_TS: op_scale_ts<V>(cx, a, b, acc, ts); break;
       case OP_SPILL:
@@ -591,7 +606,7 @@ PN_DEV void run_program(const KernelParams& p, int pc, const int pc_end, const T
         break;
       case OP_SLD: op_splat<V>(acc, cx.slots[a]); break;
       case OP_SST:
-        if constexpr (SCALAR) op_sst(cx, a, acc[0]);
+        if constexpr (SCALAR) op_sst<false>(cx, a, acc[0]);
         break;
       default: break;
     }
@@ -604,8 +619,11 @@ PN_DEV void run_program(const KernelParams& p, int pc, const int pc_end, const T
 template <int VL_, int NG_, int K_>
 struct Interp {
   static constexpr int VL = VL_, NG = NG_, K = K_;
-  static constexpr bool kStatic = false;
+  static constexpr bool kStatic = false;   // properties are launch parameters, not constants
   static constexpr int kStages = kMaxStages;
+  static constexpr int kFamily = -1, kNumIo = kMaxIo;
+  static PN_DEV unsigned lead_dim(const KernelParams& p, int i) { return p.lead_dim[i]; }
+  static PN_DEV long long lead_stride(const KernelParams& p, int io, int i) { return p.io[io].lead_stride[i]; }
   static PN_DEV int family(const KernelParams& p) { return p.family; }
   static PN_DEV int cluster(const KernelParams& p) { return p.cluster; }
   static PN_DEV int chunks(const KernelParams& p) { return p.chunks; }
@@ -619,7 +637,7 @@ struct Interp {
   static PN_DEV int red_slot(const KernelParams& p, int s, int r) { return p.stage[s].red[r].slot; }
   static PN_DEV bool has_scalar(const KernelParams& p, int s) { return p.stage[s].scal_begin != p.stage[s].scal_end; }
   static PN_DEV void tile(const KernelParams& p, int s, const TileCtx& cx, float (&acc)[VL * NG],
-                          float (&reg)[K][VL * NG], float& ts) {
+                          float (&reg)[K][VL * NG], float& ts, Part (&)[kMaxRed]) {
     run_program<VL, NG, K, false>(p, p.stage[s].elem_begin, p.stage[s].elem_end, cx, acc, reg, ts);
   }
   static PN_DEV void scalar(const KernelParams& p, int s, const TileCtx& cx) {
@@ -634,6 +652,10 @@ struct Interp {
 template <class Prog>
 PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
   constexpr int VL = Prog::VL, NG = Prog::NG, K = Prog::K, V = VL * NG;
+  // a generated program for warp teams keeps row offsets, partials and per-row scalars in
+  // registers (every lane computes the same values); otherwise they live in shared memory
+  constexpr bool kRegSlots = Prog::kStatic && Prog::kFamily <= FAM_WARP;
+  constexpr bool kRegRowoff = Prog::kStatic;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
   const int family = Prog::family(p);
   const int cluster = Prog::cluster(p);
@@ -645,13 +667,15 @@ PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
   const int team_in_cta = warp_team ? warp : 0;
   const int crank = (cluster > 1) ? (int)cluster_ctarank() : 0;
 
-  long long* rowoff = reinterpret_cast<long long*>(smem + p.sm_rowoff) + team_in_cta * kMaxIo;
+  long long rowoff_reg[kRegRowoff ? Prog::kNumIo : 1];
+  float slots_reg[kRegSlots ? kMaxSlots : 1];
+  long long* rowoff_sm = reinterpret_cast<long long*>(smem + p.sm_rowoff) + team_in_cta * kMaxIo;
   float* wpart = reinterpret_cast<float*>(smem + p.sm_wpart);
-  float* slots = reinterpret_cast<float*>(smem + p.sm_slots) + team_in_cta * kMaxSlots;
+  float* slots = kRegSlots ? slots_reg : reinterpret_cast<float*>(smem + p.sm_slots) + team_in_cta * kMaxSlots;
   float* ctapart = reinterpret_cast<float*>(smem + p.sm_ctapart);
 
   TileCtx cx;
-  cx.rowoff = rowoff;
+  cx.rowoff = kRegRowoff ? rowoff_reg : rowoff_sm;
   cx.part = reinterpret_cast<float*>(smem + p.sm_part) + tid;
   cx.part_stride = blockDim.x;
   cx.slots = slots;
@@ -674,8 +698,10 @@ PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
   float acc[V];
   float reg[K][V];
   float ts = 0.f;
+  Part parts[kMaxRed];
   PN_UNROLL for (int e = 0; e < V; ++e) acc[e] = 0.f;
   PN_UNROLL for (int k = 0; k < K; ++k) { PN_UNROLL for (int e = 0; e < V; ++e) reg[k][e] = 0.f; }
+  PN_UNROLL for (int r = 0; r < kMaxRed; ++r) parts[r] = Part{0.f, 0.f, 0.f};
 
   for (long long item = team_global; item < n_items; item += n_teams) {
     long long row = item;
@@ -683,14 +709,25 @@ PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
     if (split) { row = item / chunks; c_first = (int)(item - row * chunks); c_count = 1; }
 
     // element offset of this row in every input / output
-    if (team_tid < Prog::n_io(p)) {
-      const IoDesc& io = p.io[team_tid];
-      long long r = row;
-      const long long i2 = r % p.lead_dim[2]; r /= p.lead_dim[2];
-      const long long i1 = r % p.lead_dim[1]; r /= p.lead_dim[1];
-      rowoff[team_tid] = r * io.lead_stride[0] + i1 * io.lead_stride[1] + i2 * io.lead_stride[2];
+    if constexpr (kRegRowoff) {
+      const unsigned long long r0 = (unsigned long long)row;
+      const unsigned d2 = Prog::lead_dim(p, 2), d1 = Prog::lead_dim(p, 1);
+      const unsigned long long q2 = r0 / d2;
+      const long long i2 = (long long)(r0 - q2 * d2);
+      const unsigned long long q1 = q2 / d1;
+      const long long i1 = (long long)(q2 - q1 * d1);
+      PN_UNROLL for (int q = 0; q < Prog::kNumIo; ++q)
+        rowoff_reg[q] = (long long)q1 * Prog::lead_stride(p, q, 0) + i1 * Prog::lead_stride(p, q, 1) + i2 * Prog::lead_stride(p, q, 2);
+    } else {
+      if (team_tid < Prog::n_io(p)) {
+        const IoDesc& io = p.io[team_tid];
+        long long r = row;
+        const long long i2 = r % p.lead_dim[2]; r /= p.lead_dim[2];
+        const long long i1 = r % p.lead_dim[1]; r /= p.lead_dim[1];
+        rowoff_sm[team_tid] = r * io.lead_stride[0] + i1 * io.lead_stride[1] + i2 * io.lead_stride[2];
+      }
+      if (warp_team) __syncwarp(); else __syncthreads();
     }
-    if (warp_team) __syncwarp(); else __syncthreads();
 
 #pragma unroll(Prog::kStatic ? Prog::kStages : 1)
     for (int s = 0; s < Prog::kStages; ++s) {
@@ -698,30 +735,36 @@ PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
       for (int c = c_first; c < c_first + c_count; ++c) {
         cx.chunk = split ? 0 : c;
         cx.col0 = slice_lo + c * chunk_cols + team_tid * VL;
-        Prog::tile(p, s, cx, acc, reg, ts);
+        Prog::tile(p, s, cx, acc, reg, ts, parts);
       }
       const int n_red = Prog::n_red(p, s);
       if (n_red == 0 && !Prog::has_scalar(p, s)) continue;
 
       // ---- combine the partials of this stage over the team, then the scalar program ---
       if (warp_team) {
-        for (int r = 0; r < n_red; ++r) {
-          const int kind = Prog::red_kind(p, s, r);
-          Part v{cx.part[(r * 3) * cx.part_stride], cx.part[(r * 3 + 1) * cx.part_stride],
-                 cx.part[(r * 3 + 2) * cx.part_stride]};
-          v = warp_combine(kind, v);
-          if (lane == 0) { float* d = slots + Prog::red_slot(p, s, r); d[0] = v.a; d[1] = v.b; d[2] = v.c; }
+        PN_UNROLL for (int r = 0; r < kMaxRed; ++r) {
+          if (r < n_red) {
+            const int kind = Prog::red_kind(p, s, r);
+            Part v = Prog::kStatic ? parts[r]
+                                   : Part{cx.part[(r * 3) * cx.part_stride], cx.part[(r * 3 + 1) * cx.part_stride],
+                                          cx.part[(r * 3 + 2) * cx.part_stride]};
+            v = warp_combine(kind, v);
+            if (kRegSlots || lane == 0) { float* d = slots + Prog::red_slot(p, s, r); d[0] = v.a; d[1] = v.b; d[2] = v.c; }
+          }
         }
-        __syncwarp();
+        if constexpr (!kRegSlots) __syncwarp();
         Prog::scalar(p, s, cx);
-        __syncwarp();
+        if constexpr (!kRegSlots) __syncwarp();
       } else {
-        for (int r = 0; r < n_red; ++r) {
-          const int kind = Prog::red_kind(p, s, r);
-          Part v{cx.part[(r * 3) * cx.part_stride], cx.part[(r * 3 + 1) * cx.part_stride],
-                 cx.part[(r * 3 + 2) * cx.part_stride]};
-          v = warp_combine(kind, v);
-          if (lane == 0) { float* w = wpart + (warp * kMaxRed + r) * 3; w[0] = v.a; w[1] = v.b; w[2] = v.c; }
+        PN_UNROLL for (int r = 0; r < kMaxRed; ++r) {
+          if (r < n_red) {
+            const int kind = Prog::red_kind(p, s, r);
+            Part v = Prog::kStatic ? parts[r]
+                                   : Part{cx.part[(r * 3) * cx.part_stride], cx.part[(r * 3 + 1) * cx.part_stride],
+                                          cx.part[(r * 3 + 2) * cx.part_stride]};
+            v = warp_combine(kind, v);
+            if (lane == 0) { float* w = wpart + (warp * kMaxRed + r) * 3; w[0] = v.a; w[1] = v.b; w[2] = v.c; }
+          }
         }
         __syncthreads();
         if (warp == 0) {
@@ -759,8 +802,8 @@ PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
         __syncthreads();
       }
     }
-    // the next item rewrites rowoff / slots: everyone must be done reading them
-    if (warp_team) __syncwarp(); else __syncthreads();
+    // the next item rewrites rowoff / slots in shared memory: everyone must be done reading them
+    if constexpr (!kRegRowoff || !kRegSlots) { if (warp_team) __syncwarp(); else __syncthreads(); }
   }
   // a CTA's shared memory may still be read by its cluster peers until they pass this point
   if (cluster > 1) cluster_sync_all();

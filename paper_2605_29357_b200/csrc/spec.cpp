@@ -101,21 +101,23 @@ bool is_unary(int op) { return op >= OP_NEG && op <= OP_I2F; }
 bool is_binary(int op) { return op >= OP_ADD && op <= OP_LSEFIN; }
 
 // One program range [pc, end) as statements.  vl/ng are the tile shape (1, 1 for scalar programs).
-bool emit_program(const KernelParams& P, int pc, int end, bool scalar, int vl, int ng, std::string& out, std::string& err) {
+bool emit_program(const KernelParams& P, int pc, int end, bool scalar, int vl, int ng, bool full, bool reg_slots,
+                  std::string& out, std::string& err) {
   const std::string V = std::to_string(vl * ng), VLNG = std::to_string(vl) + ", " + std::to_string(ng);
+  const std::string VLNGF = VLNG + (full ? ", true" : ", false");
   while (pc < end) {
     const uint32_t w = P.code[pc++];
     const int op = w & 0xFF, a = (w >> 8) & 0xFF, b = (w >> 16) & 0xFF, c = w >> 24;
     const std::string A = std::to_string(a), B = std::to_string(b), OP = std::to_string(op);
     auto dt = [&](int io) { return std::to_string((int)P.io[io].dtype); };
     std::string s;
-    if (op == OP_LDRAW) s = "op_ldraw<" + VLNG + ">(p, cx, " + A + ", " + dt(a) + ", " + regname(b) + ");";
+    if (op == OP_LDRAW) s = "op_ldraw<" + VLNGF + ">(p, cx, " + A + ", " + dt(a) + ", " + regname(b) + ");";
     else if (op == OP_WIDEN) s = "op_widen<" + VLNG + ">(" + dt(a) + ", " + regname(b) + ");";
     else if (op == OP_LDBC) s = "op_ldbc<" + V + ">(p, cx, " + A + ", " + dt(a) + ", " + regname(b) + ");";
     else if (op == OP_LD) s = "op_mov<" + V + ">(acc, " + regname(a) + ");";
     else if (op == OP_ST) s = "op_mov<" + V + ">(" + regname(a) + ", acc);";
     else if (op == OP_STOUT) s = scalar ? "op_stout_scalar(p, cx, " + A + ", " + dt(a) + ", acc[0]);"
-                                        : "op_stout<" + VLNG + ">(p, cx, " + A + ", " + dt(a) + ", acc);";
+                                        : "op_stout<" + VLNGF + ">(p, cx, " + A + ", " + dt(a) + ", acc);";
     else if (op == OP_STOUT_I) s = "op_stout_index(p, cx, " + A + ", " + dt(a) + ", acc[0]);";
     else if (is_unary(op)) s = "op_unary<" + OP + ", " + V + ">(acc);";
     else if (is_binary(op)) {
@@ -131,14 +133,14 @@ bool emit_program(const KernelParams& P, int pc, int end, bool scalar, int vl, i
       else { pre += "float yt[" + V + "]; op_splat<" + V + ">(yt, " + (ky == OPK_IMM ? fbits(P.code[pc++]) : "cx.slots[" + B + "]") + "); "; y = "yt"; }
       s = pre + "op_ternary<" + OP + ", " + V + ">(acc, " + x + ", " + y + "); }";
     }
-    else if (op == OP_RED) s = "op_red<" + VLNG + ">(cx, " + A + ", " + B + ", acc, ts);";
+    else if (op == OP_RED) s = "op_red<" + VLNGF + ">(cx, " + A + ", parts[" + B + "], acc, ts);";
     else if (op == OP_SCALE_TS) s = "op_scale_ts<" + V + ">(cx, " + A + ", " + B + ", acc, ts);";
     else if (op == OP_SPILL) s = "op_spill<" + V + ">(cx, " + B + ", " + regname(a) + ");";
     else if (op == OP_FILL) s = "op_fill<" + V + ">(cx, " + B + ", " + regname(a) + ");";
     else if (op == OP_SPILL_TS) s = "*stash_ptr<" + V + ">(cx, " + B + ") = ts;";
     else if (op == OP_FILL_TS) s = "ts = *stash_ptr<" + V + ">(cx, " + B + ");";
     else if (op == OP_SLD) s = "op_splat<" + V + ">(acc, cx.slots[" + A + "]);";
-    else if (op == OP_SST) s = "op_sst(cx, " + A + ", acc[0]);";
+    else if (op == OP_SST) s = std::string("op_sst<") + (reg_slots ? "true" : "false") + ">(cx, " + A + ", acc[0]);";
     else if (op == OP_END) continue;
     else { err = "specialiser: unknown opcode " + OP; return false; }
     out += "        " + s + "\n";
@@ -155,6 +157,19 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
   s += "\nnamespace pn {\nstruct Spec {\n";
   s += "  static constexpr int VL = " + I(lp.vl) + ", NG = " + I(lp.ng) + ", K = " + I(lp.k) + ";\n";
   s += "  static constexpr bool kStatic = true;\n  static constexpr int kStages = " + I(P.n_stages) + ";\n";
+  s += "  static constexpr int kFamily = " + I(P.family) + ", kNumIo = " + I(P.n_io) + ";\n";
+  s += "  static PN_DEV unsigned lead_dim(const KernelParams&, int i) { return i == 0 ? " + I(P.lead_dim[0]) + "u : i == 1 ? " +
+       I(P.lead_dim[1]) + "u : " + I(P.lead_dim[2]) + "u; }\n";
+  s += "  static PN_DEV long long lead_stride(const KernelParams&, int io, int i) {\n    switch (io * 3 + i) {\n";
+  for (int q = 0; q < P.n_io; ++q)
+    for (int i = 0; i < 3; ++i)
+      if (P.io[q].lead_stride[i] != 0) s += "      case " + I(q * 3 + i) + ": return " + I(P.io[q].lead_stride[i]) + "ll;\n";
+  s += "      default: return 0;\n    }\n  }\n";
+  // every group of every tile inside the row: no validity tests in the generated code
+  const int team_threads = P.family <= FAM_WARP ? 32 : lp.block;
+  const bool full = (long long)P.chunks * team_threads * lp.vl * lp.ng == P.slice_len &&
+                    (long long)P.slice_len * P.cluster == P.row_len;
+  const bool reg_slots = P.family <= FAM_WARP;
   auto konst = [&](const char* name, long long v) {
     s += std::string("  static PN_DEV int ") + name + "(const KernelParams&) { return " + I(v) + "; }\n";
   };
@@ -175,10 +190,10 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
   for (int st = 0; st < P.n_stages; ++st) s += "      case " + I(st) + ": return " + (P.stage[st].scal_begin != P.stage[st].scal_end ? "true" : "false") + ";\n";
   s += "      default: return false;\n    }\n  }\n";
   const std::string V = I(lp.vl * lp.ng);
-  s += "  static PN_DEV void tile(const KernelParams& p, int s, const TileCtx& cx, float (&acc)[" + V + "], float (&reg)[" + I(lp.k) + "][" + V + "], float& ts) {\n    switch (s) {\n";
+  s += "  static PN_DEV void tile(const KernelParams& p, int s, const TileCtx& cx, float (&acc)[" + V + "], float (&reg)[" + I(lp.k) + "][" + V + "], float& ts, Part (&parts)[" + I(kMaxRed) + "]) {\n    switch (s) {\n";
   for (int st = 0; st < P.n_stages; ++st) {
     s += "      case " + I(st) + ": {\n";
-    if (!emit_program(P, P.stage[st].elem_begin, P.stage[st].elem_end, false, lp.vl, lp.ng, s, err)) return false;
+    if (!emit_program(P, P.stage[st].elem_begin, P.stage[st].elem_end, false, lp.vl, lp.ng, full, reg_slots, s, err)) return false;
     s += "      } break;\n";
   }
   s += "      default: break;\n    }\n  }\n";
@@ -186,7 +201,7 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
        "    float acc[1] = {0.f}; float reg[4][1] = {{0.f}, {0.f}, {0.f}, {0.f}}; float ts = 0.f;\n    (void)reg; (void)ts;\n    switch (s) {\n";
   for (int st = 0; st < P.n_stages; ++st) {
     s += "      case " + I(st) + ": {\n";
-    if (!emit_program(P, P.stage[st].scal_begin, P.stage[st].scal_end, true, 1, 1, s, err)) return false;
+    if (!emit_program(P, P.stage[st].scal_begin, P.stage[st].scal_end, true, 1, 1, false, reg_slots, s, err)) return false;
     s += "      } break;\n";
   }
   s += "      default: break;\n    }\n  }\n};\n}  // namespace pn\n\n";
