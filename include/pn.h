@@ -80,9 +80,17 @@ enum {
   PN_FLAG_FORCE_CLUSTER = 1u << 6,/* row kernels: one thread-block cluster per row        */
   PN_FLAG_FORCE_SCALAR = 1u << 7, /* element-wise (unvectorised) memory accesses          */
   PN_FLAG_FORCE_MULTICHUNK = 1u << 8,/* smallest tile: rows span several chunks per thread */
-  PN_FLAG_INTERPRET = 1u << 9     /* run the bytecode on the interpreter kernels built into the
+  PN_FLAG_INTERPRET = 1u << 9,    /* run the bytecode on the interpreter kernels built into the
                                      library instead of a kernel specialised for the graph */
+  PN_FLAG_NO_HOIST = 1u << 10,    /* do not move row-invariant operand loads out of the row loop */
+  PN_FLAG_PREFETCH = 1u << 11     /* generated kernels: issue the first stage's loads one tile
+                                     ahead (costs registers; off by default)                 */
 };
+/* Tuning overrides of the lowering's own choices, for measurements and tests: OR them into
+ * `flags`.  A value of 0 leaves the choice to the lowering; an impossible one is ignored. */
+#define PN_TUNE_CLUSTER(n) (((unsigned)(n) & 15u) << 16)      /* CTAs per cluster: 2, 4, 8      */
+#define PN_TUNE_BLOCK_LOG2(n) (((unsigned)(n) & 15u) << 20)   /* threads per block = 1 << n     */
+#define PN_TUNE_GROUPS(n) (((unsigned)(n) & 31u) << 24)       /* vector groups per thread tile  */
 
 /* pn_graph_query selectors; each writes int64 values into `out` */
 enum {

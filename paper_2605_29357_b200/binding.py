@@ -23,6 +23,14 @@ FLAG_FORCE_CLUSTER = 1 << 6
 FLAG_FORCE_SCALAR = 1 << 7
 FLAG_FORCE_MULTICHUNK = 1 << 8
 FLAG_INTERPRET = 1 << 9
+FLAG_NO_HOIST = 1 << 10
+FLAG_PREFETCH = 1 << 11
+
+
+def tune(cluster: int = 0, block: int = 0, groups: int = 0) -> int:
+    """Flag bits overriding the lowering's cluster size, block size and groups per tile."""
+    lg = block.bit_length() - 1 if block else 0
+    return ((cluster & 15) << 16) | ((lg & 15) << 20) | ((groups & 31) << 24)
 
 Q_N_INPUTS, Q_N_OUTPUTS, Q_INPUT_META, Q_OUTPUT_META, Q_COMPULSORY_BYTES = 1, 2, 3, 4, 5
 Q_N_KERNELS, Q_N_NODES, Q_WORKSPACE_BYTES, Q_KERNEL_INFO = 6, 7, 8, 9

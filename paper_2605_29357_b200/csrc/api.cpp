@@ -111,6 +111,7 @@ pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsig
   h->plan_only = (flags & PN_FLAG_PLAN_ONLY) != 0;
 
   DeviceModel dev;
+  dev.specialise = !(flags & PN_FLAG_INTERPRET) && spec_available(nullptr, h->plan_only);
   if (!h->plan_only) {
     int count = 0;
     cudaError_t e = cudaGetDeviceCount(&count);
@@ -175,7 +176,7 @@ pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsig
     }
   }
   // a kernel of its own for every launch, unless the interpreter was asked for
-  if (!h->plan_only && !(flags & PN_FLAG_INTERPRET) && spec_available(nullptr)) {
+  if (!h->plan_only && dev.specialise) {
     cudaFree(0);   // makes the device's primary context current for the driver calls
     for (PlannedLaunch& pl : h->launches)
       if (!spec_compile(pl.plan, device, dev.sm_count, pl.spec, err)) {

@@ -183,6 +183,12 @@ PN_DEV void store_group(char* base, long long elem, int dt, const float* g) {
       store_words<VL>(base + elem, w);
       break;
     }
+    case kStore01: {   // int8 / bool tensor whose values are known to be exactly 0.0f or 1.0f
+      PN_UNROLL for (int i = 0; i < (VL + 3) / 4; ++i) w[i] = 0;
+      PN_UNROLL for (int i = 0; i < VL; ++i) w[i >> 2] |= (f_bits(g[i]) >> 29) << ((i & 3) * 8);   // 1.0f = 0x3F800000
+      store_words<VL>(base + elem, w);
+      break;
+    }
     default:  // i64
       PN_UNROLL for (int i = 0; i < VL; ++i)
         reinterpret_cast<long long*>(base)[elem + i] = static_cast<long long>(__float2int_rz(g[i]));
@@ -214,7 +220,13 @@ PN_DEV float f_exp_neg(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(x * 1.4426950408889634f));
   return e;
 }
-PN_DEV float f_sigmoid(float x) { return __fdividef(1.f, 1.f + f_exp(-x)); }
+// 2^t and 1/y from the special-function unit (each about 1 ulp)
+PN_DEV float f_ex2(float t) { float e; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(t)); return e; }
+PN_DEV float f_rcp(float y) { float r; asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(y)); return r; }
+// sigmoid(x) = 1 / (1 + e^-x).  The rounding of x*log2 e perturbs e^-x by |x| * 6e-8 relative,
+// and sigmoid is less sensitive to e^-x than 1:1, so the result stays within about 1e-6
+// relative over the whole range; e^-x = inf gives 0, e^-x = 0 gives 1.
+PN_DEV float f_sigmoid(float x) { return f_rcp(1.f + f_ex2(x * -1.4426950408889634f)); }
 // 0.5 x (1 + tanh u) = x / (1 + e^(-2u)),  u = sqrt(2/pi) (x + 0.044715 x^3)
 PN_DEV float f_gelu_tanh(float x) {
   const float k0 = 0.7978845608028654f, k1 = 0.044715f;
@@ -313,7 +325,7 @@ PN_DEV Part red_combine(int kind, Part x, Part y) {
     default: {  // RED_MEANVAR: pairwise update of (count, mean, M2)
       const float n = x.a + y.a;
       if (n > 0.f) {
-        const float d = y.b - x.b, r = y.a / n;
+        const float d = y.b - x.b, r = y.a * f_rcp(n);
         x.c = x.c + y.c + d * d * x.a * r;
         x.b = fmaf(d, r, x.b);
       }
@@ -324,14 +336,52 @@ PN_DEV Part red_combine(int kind, Part x, Part y) {
   return x;
 }
 
+PN_DEV float shfl_x(float v, int o) { return __shfl_xor_sync(0xFFFFFFFFu, v, o); }
+
+// Combine the partials of the 32 lanes of a warp; every lane ends with the same result.
+// The order of operations is fixed (a butterfly over lane distance 16, 8, 4, 2, 1), so
+// results repeat bit for bit from run to run.  Lanes without data pass the identity partial.
+//   sum / max / min      one value per shuffle step
+//   argmax / argmin      (value, index) pairs, lowest index on ties
+//   logsumexp / softmax  the row maximum first, then the sums rescaled to it once
+//   mean / variance      count and sum first, giving the common mean; then each lane moves its
+//                        squared deviations to that mean (M2 + n (mean_lane - mean)^2) and the
+//                        results are added: the exact decomposition of the total sum of squares
 PN_DEV Part warp_combine(int kind, Part v) {
-  PN_UNROLL for (int o = 16; o > 0; o >>= 1) {
-    Part w;
-    w.a = __shfl_xor_sync(0xFFFFFFFFu, v.a, o);
-    w.b = __shfl_xor_sync(0xFFFFFFFFu, v.b, o);
-    w.c = __shfl_xor_sync(0xFFFFFFFFu, v.c, o);
-    // fixed operand order (lower lane first): both partners compute the same value
-    v = (threadIdx.x & o) ? red_combine(kind, w, v) : red_combine(kind, v, w);
+  switch (kind) {
+    case RED_SUM:
+      PN_UNROLL for (int o = 16; o > 0; o >>= 1) v.a += shfl_x(v.a, o);
+      break;
+    case RED_MAX:
+      PN_UNROLL for (int o = 16; o > 0; o >>= 1) v.a = f_max_nan(v.a, shfl_x(v.a, o));
+      break;
+    case RED_MIN:
+      PN_UNROLL for (int o = 16; o > 0; o >>= 1) v.a = f_min_nan(v.a, shfl_x(v.a, o));
+      break;
+    case RED_ARGMAX: case RED_ARGMIN:
+      PN_UNROLL for (int o = 16; o > 0; o >>= 1) {
+        const float wa = shfl_x(v.a, o), wb = shfl_x(v.b, o);
+        if (arg_better(wa, (int)f_bits(wb), v.a, (int)f_bits(v.b), kind == RED_ARGMAX)) { v.a = wa; v.b = wb; }
+      }
+      break;
+    case RED_LSE: case RED_SOFTMAX: {
+      float m = v.a;
+      PN_UNROLL for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, shfl_x(m, o));
+      float s = (m == -PN_INF) ? 0.f : v.b * f_exp_neg(v.a - m);
+      PN_UNROLL for (int o = 16; o > 0; o >>= 1) s += shfl_x(s, o);
+      v.a = m; v.b = s;
+      break;
+    }
+    default: {  // RED_MEANVAR
+      float n = v.a, sum = v.a * v.b;
+      PN_UNROLL for (int o = 16; o > 0; o >>= 1) { n += shfl_x(n, o); sum += shfl_x(sum, o); }
+      const float mean = n > 0.f ? sum * f_rcp(n) : 0.f;
+      const float d = v.b - mean;
+      float m2 = fmaf(v.a * d, d, v.c);
+      PN_UNROLL for (int o = 16; o > 0; o >>= 1) m2 += shfl_x(m2, o);
+      v.a = n; v.b = mean; v.c = m2;
+      break;
+    }
   }
   return v;
 }
@@ -425,6 +475,17 @@ PN_DEV void op_ternary(float (&acc)[V], const float (&x)[V], const float (&y)[V]
   PN_UNROLL for (int e = 0; e < V; ++e)
     acc[e] = (OP == OP_WHERE) ? (acc[e] != 0.f ? x[e] : y[e]) : fmaf(acc[e], x[e], y[e]);
 }
+// acc = c != 0 ? acc : y, the condition given as the storage bytes of an int8 / bool tensor
+// (VL bytes per group, as loaded): no conversion of the mask to floating point
+template <int VL, int NG>
+PN_DEV void op_where_raw(float (&acc)[VL * NG], const float (&craw)[VL * NG], const float (&y)[VL * NG]) {
+  PN_UNROLL for (int j = 0; j < NG; ++j) {
+    PN_UNROLL for (int i = 0; i < VL; ++i) {
+      const uint32_t w = f_bits(craw[j * VL + (i >> 2)]);
+      acc[j * VL + i] = (w & (0xFFu << ((i & 3) * 8))) ? acc[j * VL + i] : y[j * VL + i];
+    }
+  }
+}
 template <int V>
 PN_DEV void op_splat(float (&t)[V], float v) { PN_UNROLL for (int e = 0; e < V; ++e) t[e] = v; }
 
@@ -464,11 +525,12 @@ PN_DEV void op_red(const TileCtx& cx, int kind, Part& st, float (&acc)[VL * NG],
         PN_UNROLL for (int i = 0; i < VL; ++i) m = fmaxf(m, acc[j * VL + i]);
       }
     const float ms = (m == -PN_INF) ? 0.f : m;   // keeps exp(x - ms) free of inf - inf
+    const float L2E = 1.4426950408889634f, nms = -ms * L2E;   // e^(x - ms) = 2^(x log2e - ms log2e)
     float s = 0.f;
     PN_UNROLL for (int j = 0; j < NG; ++j) {
       const bool ok = FULL || cx.col0 + j * cx.gstride < cx.col_end;
       PN_UNROLL for (int i = 0; i < VL; ++i) {
-        const float ev = ok ? f_exp_neg(acc[j * VL + i] - ms) : 0.f;
+        const float ev = ok ? f_ex2(fmaf(acc[j * VL + i], L2E, nms)) : 0.f;
         s += ev;
         if (kind == RED_SOFTMAX) acc[j * VL + i] = ev;
       }
@@ -563,7 +625,7 @@ PN_DEV void run_program(const KernelParams& p, int pc, const int pc_end, const T
       case OP_ST: PN_WITH_REG(a, op_mov<V>(r, acc);) break;
       case OP_STOUT:
         if constexpr (SCALAR) op_stout_scalar(p, cx, a, p.io[a].dtype, acc[0]);
-        else op_stout<VL, NG>(p, cx, a, p.io[a].dtype, acc);
+        else op_stout<VL, NG>(p, cx, a, b ? kStore01 : p.io[a].dtype, acc);
         break;
       case OP_STOUT_I:
         if constexpr (SCALAR) op_stout_index(p, cx, a, p.io[a].dtype, acc[0]);
@@ -583,6 +645,15 @@ PN_DEV void run_program(const KernelParams& p, int pc, const int pc_end, const T
         if (op == OP_WHERE) op_ternary<OP_WHERE, V>(acc, xt, yt); else op_ternary<OP_FMA, V>(acc, xt, yt);
         break;
       }
+      case OP_WHERE_RAW:
+        if constexpr (!SCALAR) {
+          float yt[V];
+          const int ky = c & 15;
+          if (ky == OPK_REG) { PN_WITH_REG(b, op_mov<V>(yt, r);) }
+          else op_splat<V>(yt, ky == OPK_IMM ? bits_f(p.code[pc++]) : cx.slots[b]);
+          PN_WITH_REG(a, op_where_raw<VL, NG>(acc, r, yt);)
+        }
+        break;
       case OP_RED:
         if constexpr (!SCALAR) {
           float* ps = cx.part + b * 3 * cx.part_stride;
@@ -621,7 +692,7 @@ struct Interp {
   static constexpr int VL = VL_, NG = NG_, K = K_;
   static constexpr bool kStatic = false;   // properties are launch parameters, not constants
   static constexpr int kStages = kMaxStages;
-  static constexpr int kFamily = -1, kNumIo = kMaxIo;
+  static constexpr int kFamily = -1, kNumIo = kMaxIo, kNumPrefetch = 0;
   static PN_DEV unsigned lead_dim(const KernelParams& p, int i) { return p.lead_dim[i]; }
   static PN_DEV long long lead_stride(const KernelParams& p, int io, int i) { return p.io[io].lead_stride[i]; }
   static PN_DEV int family(const KernelParams& p) { return p.family; }
@@ -637,7 +708,8 @@ struct Interp {
   static PN_DEV int red_slot(const KernelParams& p, int s, int r) { return p.stage[s].red[r].slot; }
   static PN_DEV bool has_scalar(const KernelParams& p, int s) { return p.stage[s].scal_begin != p.stage[s].scal_end; }
   static PN_DEV void tile(const KernelParams& p, int s, const TileCtx& cx, float (&acc)[VL * NG],
-                          float (&reg)[K][VL * NG], float& ts, Part (&)[kMaxRed]) {
+                          float (&reg)[K][VL * NG], float& ts, Part (&)[kMaxRed], float (&)[1][VL * NG],
+                          const TileCtx&, bool) {
     run_program<VL, NG, K, false>(p, p.stage[s].elem_begin, p.stage[s].elem_end, cx, acc, reg, ts);
   }
   static PN_DEV void scalar(const KernelParams& p, int s, const TileCtx& cx) {
@@ -667,7 +739,9 @@ PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
   const int team_in_cta = warp_team ? warp : 0;
   const int crank = (cluster > 1) ? (int)cluster_ctarank() : 0;
 
+  constexpr int kPf = Prog::kNumPrefetch;          // stage-0 loads issued one tile ahead
   long long rowoff_reg[kRegRowoff ? Prog::kNumIo : 1];
+  long long rowoff_nxt[kPf > 0 ? Prog::kNumIo : 1];
   float slots_reg[kRegSlots ? kMaxSlots : 1];
   long long* rowoff_sm = reinterpret_cast<long long*>(smem + p.sm_rowoff) + team_in_cta * kMaxIo;
   float* wpart = reinterpret_cast<float*>(smem + p.sm_wpart);
@@ -694,14 +768,47 @@ PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
   cx.col_end = min(Prog::row_len(p), slice_lo + Prog::slice_len(p));
   const int chunk_cols = team_threads * V;
   unsigned parity = 0;
+  TileCtx nx = cx;               // addressing of the tile after the current one
+  nx.rowoff = rowoff_nxt;
 
   float acc[V];
   float reg[K][V];
+  float raw[kPf > 0 ? kPf : 1][V];
   float ts = 0.f;
   Part parts[kMaxRed];
   PN_UNROLL for (int e = 0; e < V; ++e) acc[e] = 0.f;
   PN_UNROLL for (int k = 0; k < K; ++k) { PN_UNROLL for (int e = 0; e < V; ++e) reg[k][e] = 0.f; }
   PN_UNROLL for (int r = 0; r < kMaxRed; ++r) parts[r] = Part{0.f, 0.f, 0.f};
+
+  // element offset of a row in every input / output, with the leading dims as constants
+  auto row_offsets = [&](long long row, long long (&out)[kRegRowoff ? Prog::kNumIo : 1]) {
+    if constexpr (!kRegRowoff) return;
+    const unsigned long long r0 = (unsigned long long)row;
+    const unsigned d2 = Prog::lead_dim(p, 2), d1 = Prog::lead_dim(p, 1);
+    const unsigned long long q2 = r0 / d2;
+    const long long i2 = (long long)(r0 - q2 * d2);
+    const unsigned long long q1 = q2 / d1;
+    const long long i1 = (long long)(q2 - q1 * d1);
+    PN_UNROLL for (int q = 0; q < (kRegRowoff ? Prog::kNumIo : 1); ++q)
+      out[q] = (long long)q1 * Prog::lead_stride(p, q, 0) + i1 * Prog::lead_stride(p, q, 1) + i2 * Prog::lead_stride(p, q, 2);
+  };
+
+  // loads that are the same for every row: once per thread (their row offsets are all zero)
+  if constexpr (Prog::kStatic) {
+    PN_UNROLL for (int q = 0; q < Prog::kNumIo; ++q) rowoff_reg[q] = 0;
+    cx.col0 = slice_lo + team_tid * VL;
+    Prog::prologue(p, cx, acc, reg, ts);
+  }
+  // the first tile's stage-0 loads
+  if constexpr (kPf > 0) {
+    if (team_global < n_items) {
+      long long row = team_global; int c0 = 0;
+      if (split) { row = team_global / chunks; c0 = (int)(team_global - row * chunks); }
+      row_offsets(row, rowoff_nxt);
+      nx.col0 = slice_lo + c0 * chunk_cols + team_tid * VL;
+      Prog::prefetch(p, nx, raw);
+    }
+  }
 
   for (long long item = team_global; item < n_items; item += n_teams) {
     long long row = item;
@@ -710,14 +817,7 @@ PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
 
     // element offset of this row in every input / output
     if constexpr (kRegRowoff) {
-      const unsigned long long r0 = (unsigned long long)row;
-      const unsigned d2 = Prog::lead_dim(p, 2), d1 = Prog::lead_dim(p, 1);
-      const unsigned long long q2 = r0 / d2;
-      const long long i2 = (long long)(r0 - q2 * d2);
-      const unsigned long long q1 = q2 / d1;
-      const long long i1 = (long long)(q2 - q1 * d1);
-      PN_UNROLL for (int q = 0; q < Prog::kNumIo; ++q)
-        rowoff_reg[q] = (long long)q1 * Prog::lead_stride(p, q, 0) + i1 * Prog::lead_stride(p, q, 1) + i2 * Prog::lead_stride(p, q, 2);
+      row_offsets(row, rowoff_reg);
     } else {
       if (team_tid < Prog::n_io(p)) {
         const IoDesc& io = p.io[team_tid];
@@ -735,7 +835,23 @@ PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
       for (int c = c_first; c < c_first + c_count; ++c) {
         cx.chunk = split ? 0 : c;
         cx.col0 = slice_lo + c * chunk_cols + team_tid * VL;
-        Prog::tile(p, s, cx, acc, reg, ts, parts);
+        bool has_next = false;
+        if constexpr (kPf > 0) {
+          if (s == 0) {   // where the tile after this one is: next chunk of the row, or the next item
+            if (c + 1 < c_first + c_count) {
+              has_next = true;
+              PN_UNROLL for (int q = 0; q < Prog::kNumIo; ++q) rowoff_nxt[q] = rowoff_reg[q];
+              nx.col0 = cx.col0 + chunk_cols;
+            } else if (item + n_teams < n_items) {
+              has_next = true;
+              long long nrow = item + n_teams; int nc = 0;
+              if (split) { nrow = (item + n_teams) / chunks; nc = (int)(item + n_teams - nrow * chunks); }
+              row_offsets(nrow, rowoff_nxt);
+              nx.col0 = slice_lo + nc * chunk_cols + team_tid * VL;
+            }
+          }
+        }
+        Prog::tile(p, s, cx, acc, reg, ts, parts, raw, nx, has_next);
       }
       const int n_red = Prog::n_red(p, s);
       if (n_red == 0 && !Prog::has_scalar(p, s)) continue;

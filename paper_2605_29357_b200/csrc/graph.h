@@ -60,6 +60,8 @@ struct DeviceModel {      // what the lowering needs to know about the GPU
   int sm_count = 148;
   int max_smem_per_block = 227 * 1024;
   bool have_device = false;   // occupancy queries allowed
+  bool specialise = false;    // lower for a generated kernel (many tile registers, loop-invariant
+                              // operand loads hoisted, larger tiles) rather than for the interpreter
 };
 
 // Lower a whole graph into one fused launch.  Returns a pn_status value.

@@ -33,11 +33,15 @@ struct Val {
   int io = -1;          // tile value that is a graph input not loaded yet
   bool bcast = false;   // that input has col_stride 0
   bool streamed = false;// that input has one element per element of the iteration space
+  bool invariant = false;// that input is the same for every row (all leading strides 0)
+  bool pinned = false;  // loaded once before the row loop into a register of its own
   float imm = 0.f;
   int slot = -1;        // per-row scalar: its shared-memory slot
   bool int_bits = false;// slot holds int32 bits (argmax / argmin)
   bool has_ts = false;  // exp(x - m_tile) of a softmax: travels with the tile scalar
   bool integral = false;// known to hold integer / 0-1 values
+  bool boolean = false; // known to hold exactly 0.0f or 1.0f
+  bool mask8 = false;   // graph input stored as int8 / bool
   int uses = 0;
 };
 
@@ -121,14 +125,14 @@ struct Gen {
   int find_reg(int v) const { for (int k = 0; k < K; ++k) if (regv[k] == v) return k; return -1; }
   int free_reg() {
     for (int k = 0; k < K; ++k) if (regv[k] < 0) return k;
-    for (int k = 0; k < K; ++k) if (vals[regv[k]].uses <= 0) { regv[k] = -1; regraw[k] = 0; return k; }
+    for (int k = 0; k < K; ++k) if (vals[regv[k]].uses <= 0 && !vals[regv[k]].pinned) { regv[k] = -1; regraw[k] = 0; return k; }
     err = "expression needs more tile registers than the kernel instance has";
     return -1;
   }
   int n_free() const { int n = 0; for (int k = 0; k < K; ++k) n += regv[k] < 0; return n; }
   void widen_if_raw(int k) { if (regraw[k]) { emit(OP_WIDEN, vals[regv[k]].io, k); regraw[k] = 0; } }
   void drop_dead() {
-    for (int k = 0; k < K; ++k) if (regv[k] >= 0 && vals[regv[k]].uses <= 0) { regv[k] = -1; regraw[k] = 0; }
+    for (int k = 0; k < K; ++k) if (regv[k] >= 0 && vals[regv[k]].uses <= 0 && !vals[regv[k]].pinned) { regv[k] = -1; regraw[k] = 0; }
     if (accv >= 0 && vals[accv].uses <= 0) accv = -1;
   }
   bool save_acc() {   // acc is about to be overwritten
@@ -194,7 +198,7 @@ struct Gen {
       case OP_STOUT: case OP_STOUT_I: {
         if (!place_in_acc(m.in[0])) return false;
         vals[m.in[0]].uses--;
-        emit(m.op, m.aux0);
+        emit(m.op, m.aux0, m.aux1);
         drop_dead();
         return true;
       }
@@ -221,6 +225,28 @@ struct Gen {
       }
       case OP_WHERE: case OP_FMA: {
         int x = m.in[0], X = m.in[1], Y = m.in[2];
+        // a mask read straight from an int8 / bool input and used only here is tested as bytes
+        if (m.op == OP_WHERE && !scalar && vals[x].kind == VK_E && vals[x].io >= 0 && vals[x].mask8 && !vals[x].bcast &&
+            vals[x].uses == 1 && accv != x && !stash_of.count(x) && vals[X].kind == VK_E && X != x && Y != x) {
+          int k = find_reg(x);
+          if (k < 0 || regraw[k]) {
+            if (!place_in_acc(X)) return false;
+            if (k < 0) {
+              k = free_reg();
+              if (k < 0) return false;
+              emit(OP_LDRAW, vals[x].io, k);
+              regv[k] = x; regraw[k] = 1;
+            }
+            Src sy;
+            if (!src_operand(Y, sy)) return false;
+            vals[x].uses--; vals[X].uses--; vals[Y].uses--;
+            if (!keep_if_live(X)) return false;
+            emit(OP_WHERE_RAW, k, sy.idx, sy.kind);
+            if (sy.kind == OPK_IMM) emit_f(sy.imm);
+            result(m.out);
+            return true;
+          }
+        }
         if (m.op == OP_FMA && !is_tile(x) && is_tile(X)) std::swap(x, X);
         if (vals[x].kind == VK_IMM) { err = "where / fma with a constant first operand is not lowered"; return false; }
         if (!place_in_acc(x)) return false;
@@ -280,6 +306,22 @@ struct Gen {
       }
   }
 
+  // Before the row loop: load (and widen) the operands that are the same for every row, each
+  // into a register that keeps it for the whole kernel.  Leaves `reserve` registers free.
+  void pin_invariants(const std::vector<MOp>& ops, int reserve) {
+    for (const MOp& m : ops) {
+      if (m.scalar) continue;
+      for (int i = 0; i < m.nin; ++i) {
+        const int v = m.in[i];
+        if (v < 0 || vals[v].kind != VK_E || vals[v].io < 0 || !vals[v].invariant || vals[v].pinned) continue;
+        if (n_free() <= reserve) return;
+        const int k = free_reg();
+        load_input(v, k);
+        regv[k] = v; regraw[k] = 0; vals[v].pinned = true;
+      }
+    }
+  }
+
   // End of a stage: tile values still needed later stay in registers (one chunk per thread)
   // or are parked in shared memory (several chunks per thread).
   bool end_stage() {
@@ -293,6 +335,7 @@ struct Gen {
       park(accv, kAccReg);
     for (int k = 0; k < K; ++k) {
       const int v = regv[k];
+      if (v >= 0 && vals[v].pinned) continue;
       if (v >= 0 && vals[v].uses > 0 && !stash_of.count(v)) { widen_if_raw(k); park(v, k); }
       regv[k] = -1; regraw[k] = 0;
     }
@@ -309,10 +352,11 @@ void size_grid(LaunchPlan& lp, int sms, int occ) {
   if (occ <= 0) occ = std::max(1, 512 / lp.block);
   const int64_t resident = (int64_t)sms * occ;
   const int cluster = std::max(lp.p.cluster, 1);
+  const int waves = lp.persistent ? 1 : 8;   // work hoisted out of the row loop wants long-lived CTAs
   int64_t grid;
-  if (lp.family <= FAM_WARP) grid = std::min<int64_t>((lp.items + lp.teams_per_cta - 1) / lp.teams_per_cta, resident * 8);
-  else if (lp.family == FAM_BLOCK) grid = std::min<int64_t>(lp.items, resident * 8);
-  else grid = std::min<int64_t>(lp.items, std::max<int64_t>(1, resident * 8 / cluster)) * cluster;
+  if (lp.family <= FAM_WARP) grid = std::min<int64_t>((lp.items + lp.teams_per_cta - 1) / lp.teams_per_cta, resident * waves);
+  else if (lp.family == FAM_BLOCK) grid = std::min<int64_t>(lp.items, resident * waves);
+  else grid = std::min<int64_t>(lp.items, std::max<int64_t>(1, resident * waves / cluster)) * cluster;
   lp.grid = (int)std::max<int64_t>(grid, cluster);
 }
 
@@ -487,7 +531,9 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     vals[v].io = q;
     vals[v].bcast = P.io[q].col_stride == 0;
     vals[v].streamed = io_streamed[q];
+    vals[v].invariant = P.io[q].lead_stride[0] == 0 && P.io[q].lead_stride[1] == 0 && P.io[q].lead_stride[2] == 0;
     vals[v].integral = !dtype_is_float(g.tensors[t].dtype);
+    vals[v].mask8 = g.tensors[t].dtype == kI8 || g.tensors[t].dtype == kBool;
     tval[t] = v;
   }
   std::vector<char> feeds_var(nt, 0);
@@ -547,11 +593,15 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
         if (T0.dtype == kBool) res[0] = pointwise(OP_NEZ, {pointwise(OP_I2F, {in[0]}, true)}, true);
       }
       else if (dtype_is_float(T0.dtype)) res[0] = in[0];
-      else if (T0.dtype == kBool) res[0] = (src_int && g.tensors[n.in[0]].dtype == kBool) ? in[0] : pointwise(OP_NEZ, {in[0]}, true);
+      else if (T0.dtype == kBool) {
+        res[0] = (vals[in[0]].boolean || (src_int && g.tensors[n.in[0]].dtype == kBool)) ? in[0] : pointwise(OP_NEZ, {in[0]}, true);
+        vals[res[0]].boolean = true;
+      }
       else res[0] = src_int ? in[0] : pointwise(OP_TRUNC, {in[0]}, true);
     } else if (vm_binary(n.op) >= 0) {
       for (int k = 0; k < 2; ++k) if (vals[in[k]].int_bits) in[k] = pointwise(OP_I2F, {in[k]}, true);
       res[0] = pointwise(vm_binary(n.op), {in[0], in[1]}, n.op >= N_GT);
+      vals[res[0]].boolean = n.op >= N_GT;
     } else if (n.op == N_WHERE || n.op == N_FMA) {
       for (int k = 0; k < 3; ++k) if (vals[in[k]].int_bits) in[k] = pointwise(OP_I2F, {in[k]}, true);
       res[0] = pointwise(n.op == N_WHERE ? OP_WHERE : OP_FMA, {in[0], in[1], in[2]}, false);
@@ -642,7 +692,8 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
         if (vals[v].int_bits && dtype_is_float(T.dtype)) v = pointwise(OP_I2F, {v}, true);
         const bool sc = vals[v].kind == VK_S;
         if (vals[v].int_bits && T.dtype != kI64 && T.dtype != kI32) { err = where + "index results must be stored as i32 or i64"; return PN_ERR_UNSUPPORTED_OP; }
-        add_op(vals[v].int_bits ? OP_STOUT_I : OP_STOUT, sc ? vals[v].stage - 1 : vals[v].stage, sc, {v}, -1, io_of_tensor[t]);
+        const int zero_one = (!sc && vals[v].boolean && (T.dtype == kI8 || T.dtype == kBool)) ? 1 : 0;
+        add_op(vals[v].int_bits ? OP_STOUT_I : OP_STOUT, sc ? vals[v].stage - 1 : vals[v].stage, sc, {v}, -1, io_of_tensor[t], zero_one);
       }
     }
   }
@@ -667,10 +718,12 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
   }
   int VL = (min_esize <= 2 && vec8) ? 8 : (vec4 ? 4 : 1);
   if (flags & PN_FLAG_FORCE_SCALAR) VL = 1;
+  const bool spec = dev.specialise;
   std::vector<std::pair<int, int>> ng_opts;   // (NG, K): the 8-element tile first
   if (VL == 8) ng_opts = {{1, 4}, {2, 2}};
   else if (VL == 4) ng_opts = {{2, 4}, {4, 2}};
   else ng_opts = {{8, 4}};
+  if (spec) for (auto& o : ng_opts) o.second = kSpecRegs;   // a generated kernel pays only for live registers
 
   std::vector<Config> cands;
   const int sms = dev.sm_count;
@@ -682,7 +735,8 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     const bool fm = flags & PN_FLAG_FORCE_MULTICHUNK;
     const bool any_force = fw || fb || fc;
     const bool few_rows = eff_rows < 2ll * sms;
-    auto tile_ok = [&](int T, int ng) { return !(T > 256 && VL * ng > 8); };   // 16-element tiles: <= 256 threads
+    // the interpreter's 16-element-tile instances are built for at most 256 threads
+    auto tile_ok = [&](int T, int ng) { return spec || !(T > 256 && VL * ng > 8); };
     // one chunk per thread: the smallest team that holds the row
     if (!fm && !fc) {
       for (int T : {32, 64, 128, 256, 512}) {
@@ -712,9 +766,11 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
       cands.insert(cands.end(), mc.begin(), mc.end());
     }
     if ((!any_force && few_rows) || fc || cands.empty()) {
+      std::vector<std::pair<int, int>> cl_opts = ng_opts;
+      if (spec && !fm) std::reverse(cl_opts.begin(), cl_opts.end());   // more bytes in flight per thread
       for (int C : {8, 4, 2})
-        for (auto o : ng_opts) {
-          const int T = fm ? 64 : 256;
+        for (auto o : cl_opts) {
+          const int T = fm ? 64 : (spec && (eff_N + C - 1) / C >= 2ll * 512 * VL * o.first) ? 512 : 256;
           int64_t slice = (eff_N + C - 1) / C;
           slice = (slice + VL - 1) / VL * VL;
           if (slice * (C - 1) >= eff_N) continue;                              // a CTA would get no columns
@@ -729,6 +785,37 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     }
   }
 
+  // tuning overrides: keep only the candidates that match, or add the asked-for shape
+  {
+    const int t_cluster = (flags >> 16) & 15, t_block = ((flags >> 20) & 15) ? 1 << ((flags >> 20) & 15) : 0, t_ng = (flags >> 24) & 31;
+    if ((t_cluster || t_block || t_ng) && !cands.empty()) {
+      std::vector<Config> extra;
+      for (Config c : cands) {
+        if (t_ng) {
+          bool ok = spec && (t_ng & (t_ng - 1)) == 0 && VL * t_ng <= 128;   // generated kernels take any power of two
+          for (auto o : ng_opts) ok = ok || o.first == t_ng;
+          if (!ok) continue;
+          c.ng = t_ng;
+          for (auto o : ng_opts) if (o.first == t_ng) c.k = o.second;
+        }
+        if (t_block && c.family != FAM_WARP && c.family != FAM_POINTWISE) c.block = t_block;
+        if (t_cluster && c.family == FAM_CLUSTER) c.cluster = t_cluster;
+        if (t_cluster && c.family == FAM_BLOCK && has_red) { c.family = FAM_CLUSTER; c.cluster = t_cluster; }
+        if (c.block < 32 || c.block > 1024 || (c.cluster != 1 && c.cluster != 2 && c.cluster != 4 && c.cluster != 8)) continue;
+        if (!spec && c.block > 256 && c.vl * c.ng > 8) continue;
+        const int team = c.family <= FAM_WARP ? 32 : c.block;
+        int64_t slice = (eff_N + c.cluster - 1) / c.cluster;
+        slice = (slice + VL - 1) / VL * VL;
+        if (c.cluster > 1 && slice * (c.cluster - 1) >= eff_N) continue;
+        c.slice_len = (int)slice;
+        c.chunks = chunks_of(slice, team, c.ng);
+        c.multichunk = c.family != FAM_POINTWISE && c.chunks > 1;
+        extra.push_back(c);
+      }
+      if (!extra.empty()) cands = extra;
+    }
+  }
+
   // ---- (4) code generation: first candidate whose program fits -----------------------------
   std::string gen_err = "no kernel configuration fits this graph";
   for (const Config& cf : cands) {
@@ -740,6 +827,13 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     memset(stages, 0, sizeof(stages));
     bool ok = true;
     Gen ge(code, v2, false, cf.k, cf.multichunk, stash_of, n_stash);
+    // rows held in one chunk per thread: the operands that do not depend on the row are loaded
+    // once, before the row loop (generated kernels only: they have the registers for it)
+    const bool pin = spec && cf.chunks == 1 && cf.family == FAM_WARP && !(flags & PN_FLAG_NO_HOIST);
+    const uint16_t pro_begin = (uint16_t)code.size();
+    if (pin) ge.pin_invariants(ops, 4);
+    const uint16_t pro_end = (uint16_t)code.size();
+    const bool persistent = pro_end > pro_begin;
     for (int s = 0; s < n_stages && ok; ++s) {
       stages[s].elem_begin = (uint16_t)code.size();
       ge.hoist_loads(ops, s);
@@ -777,6 +871,7 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     P.sm_stash = take((int)(stash_floats * 4));
     P.stash_floats = (int32_t)stash_floats;
     P.n_stages = n_stages;
+    P.pro_begin = pro_begin; P.pro_end = pro_end;
     memcpy(P.stage, stages, sizeof(stages));
     memset(P.code, 0, sizeof(P.code));
     memcpy(P.code, code.data(), code.size() * 4);
@@ -790,7 +885,9 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     lp.items = P.split_chunks ? eff_rows * cf.chunks : eff_rows;
     lp.teams_per_cta = teams;
     lp.specialised = 0;
-    int occ = dev.have_device ? instance_occupancy(cf.vl, cf.ng, cf.k, cf.block, off) : 0;
+    lp.persistent = persistent ? 1 : 0;
+    lp.no_prefetch = (flags & PN_FLAG_PREFETCH) ? 0 : 1;
+    int occ = (dev.have_device && !spec) ? instance_occupancy(cf.vl, cf.ng, cf.k, cf.block, off) : 0;
     size_grid(lp, sms, occ);
     return PN_OK;
   }

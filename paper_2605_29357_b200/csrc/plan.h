@@ -24,10 +24,13 @@ constexpr int kMaxStages = 4;   // reduction-separated stages
 constexpr int kMaxRed = 4;      // reductions accumulated in one stage
 constexpr int kMaxSlots = 24;   // per-row scalar slots
 constexpr int kMaxStash = 6;    // tile values parked in shared memory across stages
-constexpr int kAccReg = 7;      // register operand id that names the accumulator tile
+constexpr int kAccReg = 31;     // register operand id that names the accumulator tile
+constexpr int kSpecRegs = 12;   // tile registers of a generated kernel (only live ones cost anything)
 
 // Storage types (same numbering as the descriptor).
 enum DType : uint8_t { kF32 = 0, kF16 = 1, kBF16 = 2, kI8 = 3, kBool = 4, kI32 = 5, kI64 = 6 };
+// store-only pseudo type: an int8 / bool tensor written from values known to be 0.0f or 1.0f
+constexpr int kStore01 = 16;
 
 // Tile bytecode.  One instruction acts on the whole register tile of a thread.  The
 // machine has an accumulator tile `acc`, K tile registers, a per-tile scalar `ts`, and
@@ -41,7 +44,7 @@ enum Op : uint8_t {
   OP_LDBC,    // a = io, b = reg: last-dim-broadcast operand, one element splat over the tile
   OP_LD,      // acc = reg[a]
   OP_ST,      // reg[a] = acc
-  OP_STOUT,   // a = io: narrow acc and store it
+  OP_STOUT,   // a = io: narrow acc and store it; b = 1: the values are known to be 0 or 1
   // unary on acc
   OP_NEG, OP_ABS, OP_EXP, OP_LOG, OP_SQRT, OP_RSQRT, OP_RECIP, OP_TANH, OP_SIGMOID, OP_SILU,
   OP_GELU_TANH, OP_GELU_ERF, OP_RELU, OP_SQUARE, OP_ERF,
@@ -56,6 +59,8 @@ enum Op : uint8_t {
   // ternary: X = operand(a, kind c&15), Y = operand(b, kind c>>4)
   OP_WHERE,   // acc = acc != 0 ? X : Y
   OP_FMA,     // acc = acc * X + Y
+  OP_WHERE_RAW, // acc = C != 0 ? acc : Y; C = reg a holding the unwidened bytes of an int8 / bool
+              // tensor, Y = operand(b, kind c&15)
   // reductions over the tile into the thread's partial state
   OP_RED,      // a = RedKind, b = reduction index within the stage
   OP_SCALE_TS, // acc *= exp(ts - slot[a]) * slot[b]   (softmax epilogue)
@@ -121,6 +126,8 @@ struct KernelParams {
   int32_t split_chunks;    // pointwise graphs: every (row, chunk) is its own work item
   int32_t cluster;         // CTAs per cluster (1 unless FAM_CLUSTER)
   int32_t stash_floats;    // floats of parked tile values per CTA
+  uint16_t pro_begin, pro_end;   // tile program run once per thread before the row loop: loads of
+                                 // operands that are the same for every row (generated kernels only)
   // shared-memory layout, byte offsets into dynamic shared memory
   int32_t sm_rowoff, sm_part, sm_wpart, sm_slots, sm_ctapart, sm_stash;
   StageDesc stage[kMaxStages];
@@ -137,6 +144,8 @@ struct LaunchPlan {
   int64_t items;           // rows, or rows * chunks for pointwise graphs
   int32_t teams_per_cta;
   int32_t specialised;     // 1 when the launch uses a kernel generated for this program
+  int32_t persistent;      // 1: grid = resident CTAs, each looping over many rows
+  int32_t no_prefetch;     // 1: generated kernels issue no loads ahead of the tile in hand
   int32_t io_tensor[kMaxIo];   // tensor id behind each io entry
   int32_t io_is_output[kMaxIo];
 };

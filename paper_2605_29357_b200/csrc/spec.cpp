@@ -101,10 +101,17 @@ bool is_unary(int op) { return op >= OP_NEG && op <= OP_I2F; }
 bool is_binary(int op) { return op >= OP_ADD && op <= OP_LSEFIN; }
 
 // One program range [pc, end) as statements.  vl/ng are the tile shape (1, 1 for scalar programs).
+// n_prefetch > 0: the first n_prefetch instructions are loads whose data was fetched one tile
+// ahead into raw[0..n): they become copies out of raw[], followed by the fetch for the next tile.
 bool emit_program(const KernelParams& P, int pc, int end, bool scalar, int vl, int ng, bool full, bool reg_slots,
-                  std::string& out, std::string& err) {
+                  std::string& out, std::string& err, int n_prefetch = 0) {
   const std::string V = std::to_string(vl * ng), VLNG = std::to_string(vl) + ", " + std::to_string(ng);
   const std::string VLNGF = VLNG + (full ? ", true" : ", false");
+  for (int j = 0; j < n_prefetch; ++j) {
+    const uint32_t w = P.code[pc++];
+    out += "        op_mov<" + V + ">(" + regname((w >> 16) & 0xFF) + ", raw[" + std::to_string(j) + "]);\n";
+  }
+  if (n_prefetch > 0) out += "        if (has_next) prefetch(p, nx, raw);\n";
   while (pc < end) {
     const uint32_t w = P.code[pc++];
     const int op = w & 0xFF, a = (w >> 8) & 0xFF, b = (w >> 16) & 0xFF, c = w >> 24;
@@ -117,7 +124,7 @@ bool emit_program(const KernelParams& P, int pc, int end, bool scalar, int vl, i
     else if (op == OP_LD) s = "op_mov<" + V + ">(acc, " + regname(a) + ");";
     else if (op == OP_ST) s = "op_mov<" + V + ">(" + regname(a) + ", acc);";
     else if (op == OP_STOUT) s = scalar ? "op_stout_scalar(p, cx, " + A + ", " + dt(a) + ", acc[0]);"
-                                        : "op_stout<" + VLNGF + ">(p, cx, " + A + ", " + dt(a) + ", acc);";
+                                        : "op_stout<" + VLNGF + ">(p, cx, " + A + ", " + (b ? std::to_string(kStore01) : dt(a)) + ", acc);";
     else if (op == OP_STOUT_I) s = "op_stout_index(p, cx, " + A + ", " + dt(a) + ", acc[0]);";
     else if (is_unary(op)) s = "op_unary<" + OP + ", " + V + ">(acc);";
     else if (is_binary(op)) {
@@ -132,6 +139,13 @@ bool emit_program(const KernelParams& P, int pc, int end, bool scalar, int vl, i
       if (ky == OPK_REG) y = regname(b);
       else { pre += "float yt[" + V + "]; op_splat<" + V + ">(yt, " + (ky == OPK_IMM ? fbits(P.code[pc++]) : "cx.slots[" + B + "]") + "); "; y = "yt"; }
       s = pre + "op_ternary<" + OP + ", " + V + ">(acc, " + x + ", " + y + "); }";
+    }
+    else if (op == OP_WHERE_RAW) {
+      const int ky = c & 15;
+      std::string y, pre = "{ ";
+      if (ky == OPK_REG) y = regname(b);
+      else { pre += "float yt[" + V + "]; op_splat<" + V + ">(yt, " + (ky == OPK_IMM ? fbits(P.code[pc++]) : "cx.slots[" + B + "]") + "); "; y = "yt"; }
+      s = pre + "op_where_raw<" + VLNG + ">(acc, " + regname(a) + ", " + y + "); }";
     }
     else if (op == OP_RED) s = "op_red<" + VLNGF + ">(cx, " + A + ", parts[" + B + "], acc, ts);";
     else if (op == OP_SCALE_TS) s = "op_scale_ts<" + V + ">(cx, " + A + ", " + B + ", acc, ts);";
@@ -190,10 +204,27 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
   for (int st = 0; st < P.n_stages; ++st) s += "      case " + I(st) + ": return " + (P.stage[st].scal_begin != P.stage[st].scal_end ? "true" : "false") + ";\n";
   s += "      default: return false;\n    }\n  }\n";
   const std::string V = I(lp.vl * lp.ng);
-  s += "  static PN_DEV void tile(const KernelParams& p, int s, const TileCtx& cx, float (&acc)[" + V + "], float (&reg)[" + I(lp.k) + "][" + V + "], float& ts, Part (&parts)[" + I(kMaxRed) + "]) {\n    switch (s) {\n";
+  s += "  static PN_DEV void prologue(const KernelParams& p, const TileCtx& cx, float (&acc)[" + V + "], float (&reg)[" + I(lp.k) + "][" + V + "], float& ts) {\n"
+       "    Part parts[" + I(kMaxRed) + "]; (void)parts; (void)acc; (void)ts;\n";
+  if (!emit_program(P, P.pro_begin, P.pro_end, false, lp.vl, lp.ng, full, reg_slots, s, err)) return false;
+  s += "  }\n";
+  // the loads at the head of stage 0 are issued one tile ahead of their use
+  int n_pf = 0;
+  for (int pc = P.stage[0].elem_begin; pc < P.stage[0].elem_end && (P.code[pc] & 0xFF) == OP_LDRAW; ++pc) n_pf++;
+  if (lp.no_prefetch) n_pf = 0;
+  s += "  static constexpr int kNumPrefetch = " + I(n_pf) + ";\n";
+  s += "  static PN_DEV void prefetch(const KernelParams& p, const TileCtx& cx, float (&raw)[" + I(n_pf > 0 ? n_pf : 1) + "][" + V + "]) {\n";
+  for (int j = 0; j < n_pf; ++j) {
+    const uint32_t w = P.code[P.stage[0].elem_begin + j];
+    const int io = (w >> 8) & 0xFF;
+    s += "    op_ldraw<" + I(lp.vl) + ", " + I(lp.ng) + (full ? ", true" : ", false") + ">(p, cx, " + I(io) + ", " + I(P.io[io].dtype) + ", raw[" + I(j) + "]);\n";
+  }
+  s += "  }\n";
+  s += "  static PN_DEV void tile(const KernelParams& p, int s, const TileCtx& cx, float (&acc)[" + V + "], float (&reg)[" + I(lp.k) + "][" + V + "], float& ts, Part (&parts)[" + I(kMaxRed) + "],\n"
+       "                          float (&raw)[" + I(n_pf > 0 ? n_pf : 1) + "][" + V + "], const TileCtx& nx, bool has_next) {\n    (void)raw; (void)nx; (void)has_next;\n    switch (s) {\n";
   for (int st = 0; st < P.n_stages; ++st) {
     s += "      case " + I(st) + ": {\n";
-    if (!emit_program(P, P.stage[st].elem_begin, P.stage[st].elem_end, false, lp.vl, lp.ng, full, reg_slots, s, err)) return false;
+    if (!emit_program(P, P.stage[st].elem_begin, P.stage[st].elem_end, false, lp.vl, lp.ng, full, reg_slots, s, err, st == 0 ? n_pf : 0)) return false;
     s += "      } break;\n";
   }
   s += "      default: break;\n    }\n  }\n";
@@ -217,10 +248,11 @@ std::map<std::pair<int, std::string>, Compiled> g_cache;   // (device, source) -
 
 }  // namespace
 
-bool spec_available(std::string* why) {
+bool spec_available(std::string* why, bool compile_only) {
   const Api& a = api();
-  if (!a.ok && why) *why = a.why;
-  return a.ok;
+  const bool ok = compile_only ? a.CreateProgram != nullptr : a.ok;
+  if (!ok && why) *why = a.why;
+  return ok;
 }
 
 std::string spec_source(const LaunchPlan& lp) {

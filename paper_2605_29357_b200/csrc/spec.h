@@ -11,8 +11,9 @@ struct SpecKernel {
   int occupancy = 0;      // resident CTAs per SM at the plan's block size and shared memory
 };
 
-// True when NVRTC and the driver API could be opened; otherwise *why says what is missing.
-bool spec_available(std::string* why);
+// True when NVRTC and the driver API could be opened (compile_only: NVRTC alone is enough);
+// otherwise *why says what is missing.
+bool spec_available(std::string* why, bool compile_only = false);
 
 // Translate the plan's bytecode into a kernel, compile it for sm_100a, load it on the
 // current device and re-size the plan's grid from the kernel's occupancy.
