@@ -130,6 +130,33 @@ def time_graph(torch, g, sets, steps, warmup, flush=None):
     return evs[0].elapsed_time(evs[steps]), per
 
 
+def time_graph_replay(torch, g, sets, steps, warmup):
+    """The same launches recorded once into a CUDA graph (one launch per buffer set) and
+    replayed: the device-side time per launch, free of the host's launch rate.  Used for the
+    workloads whose kernels are shorter than a host launch.  Returns ms per launch."""
+    ptrs = [([t.data_ptr() for t in a], [t.data_ptr() for t in b]) for a, b in sets]
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for i in range(max(warmup, 3)):
+            g.run(*ptrs[i % len(ptrs)], side.cuda_stream)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        for a, b in ptrs:
+            g.run(a, b, torch.cuda.current_stream().cuda_stream)
+    reps = max(1, steps // len(ptrs))
+    graph.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / (reps * len(ptrs))
+
+
 def stats(per):
     a = np.sort(np.asarray(per))
     q1, med, q3 = np.percentile(a, [25, 50, 75])
@@ -314,6 +341,11 @@ def main():
                      "iqr_ms": sti["iqr_ms"], "gbs": cb / (sti["median_ms"] * 1e-3) / 1e9,
                      "frac_of_measured_peak": cb / (sti["median_ms"] * 1e-3) / 1e9 / peak,
                      "family": pn.FAMILY_NAMES[ki["family"]], "buffer_sets": ns}
+            if ns > 1:   # kernels shorter than a host launch: also the device-side time per launch
+                ms_r = time_graph_replay(torch, gi, si, max(args.steps, 10 * ns), warmup)
+                entry["graph_replay_ms"] = ms_r
+                entry["graph_replay_gbs"] = cb / (ms_r * 1e-3) / 1e9
+                entry["graph_replay_frac_of_measured_peak"] = entry["graph_replay_gbs"] / peak
             try:
                 gui = pn.Graph(wi.desc, local_rank, pn.FLAG_UNFUSED)
                 _, pu = time_graph(torch, gui, si, max(5, args.steps // 5), 3)

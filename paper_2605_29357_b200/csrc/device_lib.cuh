@@ -234,8 +234,9 @@ PN_DEV float f_gelu_tanh(float x) {
   return x * f_sigmoid(2.f * u);
 }
 PN_DEV float f_gelu_erf(float x) { return 0.5f * x * (1.f + erff(x * 0.7071067811865476f)); }
-PN_DEV float f_max_nan(float a, float b) { return (a != a || b != b) ? PN_NAN : fmaxf(a, b); }
-PN_DEV float f_min_nan(float a, float b) { return (a != a || b != b) ? PN_NAN : fminf(a, b); }
+// maximum / minimum that return NaN when either operand is NaN (one instruction each)
+PN_DEV float f_max_nan(float a, float b) { float d; asm("max.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b)); return d; }
+PN_DEV float f_min_nan(float a, float b) { float d; asm("min.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b)); return d; }
 
 template <int OP>
 PN_DEV float un(float x) {
@@ -316,7 +317,7 @@ PN_DEV Part red_combine(int kind, Part x, Part y) {
       if (arg_better(y.a, (int)f_bits(y.b), x.a, (int)f_bits(x.b), kind == RED_ARGMAX)) x = y;
       break;
     case RED_LSE: case RED_SOFTMAX: {
-      const float m = fmaxf(x.a, y.a);
+      const float m = f_max_nan(x.a, y.a);
       if (m == -PN_INF) { x.b = 0.f; }
       else { x.b = x.b * f_exp_neg(x.a - m) + y.b * f_exp_neg(y.a - m); }
       x.a = m;
@@ -366,7 +367,7 @@ PN_DEV Part warp_combine(int kind, Part v) {
       break;
     case RED_LSE: case RED_SOFTMAX: {
       float m = v.a;
-      PN_UNROLL for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, shfl_x(m, o));
+      PN_UNROLL for (int o = 16; o > 0; o >>= 1) m = f_max_nan(m, shfl_x(m, o));
       float s = (m == -PN_INF) ? 0.f : v.b * f_exp_neg(v.a - m);
       PN_UNROLL for (int o = 16; o > 0; o >>= 1) s += shfl_x(s, o);
       v.a = m; v.b = s;
@@ -489,68 +490,84 @@ PN_DEV void op_where_raw(float (&acc)[VL * NG], const float (&craw)[VL * NG], co
 template <int V>
 PN_DEV void op_splat(float (&t)[V], float v) { PN_UNROLL for (int e = 0; e < V; ++e) t[e] = v; }
 
-// Fold the valid elements of the tile (in element order) into the thread's partial `st` of a
-// reduction; RED_SOFTMAX also turns acc into exp(x - m_tile) and leaves m_tile in ts.
+// Fold of a tile in element order (a fixed order, so results repeat exactly).  Elements of
+// groups outside the row take the identity.
+template <int VL, int NG, bool FULL, class F>
+PN_DEV float tile_fold(const TileCtx& cx, const float (&acc)[VL * NG], float identity, F f) {
+  constexpr int V = VL * NG;
+  float t[V];
+  PN_UNROLL for (int j = 0; j < NG; ++j) {
+    const bool ok = FULL || cx.col0 + j * cx.gstride < cx.col_end;
+    PN_UNROLL for (int i = 0; i < VL; ++i) t[j * VL + i] = ok ? acc[j * VL + i] : identity;
+  }
+  PN_UNROLL for (int e = 1; e < V; ++e) t[0] = f(t[0], t[e]);
+  return t[0];
+}
+struct FoldAdd { PN_DEV float operator()(float a, float b) const { return a + b; } };
+struct FoldMaxNan { PN_DEV float operator()(float a, float b) const { return f_max_nan(a, b); } };
+struct FoldMinNan { PN_DEV float operator()(float a, float b) const { return f_min_nan(a, b); } };
+
+// Fold the valid elements of the tile into the thread's partial `st` of a reduction;
+// RED_SOFTMAX also turns acc into exp(x - m_tile) and leaves m_tile in ts.
 template <int VL, int NG, bool FULL = false>
 PN_DEV void op_red(const TileCtx& cx, int kind, Part& st, float (&acc)[VL * NG], float& ts) {
-  Part t = red_identity(kind);
-  if (kind == RED_SUM) {
-    PN_UNROLL for (int j = 0; j < NG; ++j)
-      if (FULL || cx.col0 + j * cx.gstride < cx.col_end) {
-        PN_UNROLL for (int i = 0; i < VL; ++i) t.a += acc[j * VL + i];
-      }
-  } else if (kind == RED_MAX || kind == RED_MIN) {
-    PN_UNROLL for (int j = 0; j < NG; ++j)
-      if (FULL || cx.col0 + j * cx.gstride < cx.col_end) {
-        PN_UNROLL for (int i = 0; i < VL; ++i)
-          t.a = kind == RED_MAX ? f_max_nan(t.a, acc[j * VL + i]) : f_min_nan(t.a, acc[j * VL + i]);
-      }
-  } else if (kind == RED_ARGMAX || kind == RED_ARGMIN) {
-    int bi = 0x7FFFFFFF;
-    float bv = t.a;
-    PN_UNROLL for (int j = 0; j < NG; ++j) {
-      const int col = cx.col0 + j * cx.gstride;
-      if (FULL || col < cx.col_end) {
-        PN_UNROLL for (int i = 0; i < VL; ++i) {
-          const float v = acc[j * VL + i];
-          if (arg_better(v, col + i, bv, bi, kind == RED_ARGMAX)) { bv = v; bi = col + i; }
+  constexpr int V = VL * NG;
+  if (kind == RED_ARGMAX || kind == RED_ARGMIN) {
+    // the tile extreme first; the index is searched only when it beats the running extreme
+    // (ties keep the earlier, lower-index holder; a NaN beats every number)
+    const bool mx = kind == RED_ARGMAX;
+    const float m = mx ? tile_fold<VL, NG, FULL>(cx, acc, -PN_INF, FoldMaxNan()) : tile_fold<VL, NG, FULL>(cx, acc, PN_INF, FoldMinNan());
+    const bool m_nan = m != m, s_nan = st.a != st.a;
+    const bool take = cx.chunk == 0 || (m_nan ? !s_nan : (!s_nan && (mx ? m > st.a : m < st.a)));
+    if (take) {
+      int bi = 0x7FFFFFFF;
+      PN_UNROLL for (int j = NG - 1; j >= 0; --j) {
+        const int col = cx.col0 + j * cx.gstride;
+        if (FULL || col < cx.col_end) {
+          PN_UNROLL for (int i = VL - 1; i >= 0; --i) {
+            const float v = acc[j * VL + i];
+            if (m_nan ? (v != v) : (v == m)) bi = col + i;   // descending scan: the lowest column wins
+          }
         }
       }
+      st.a = m; st.b = bits_f(static_cast<uint32_t>(bi));
     }
-    t.a = bv; t.b = bits_f(static_cast<uint32_t>(bi));
+    return;
+  }
+  Part t = red_identity(kind);
+  if (kind == RED_SUM) {
+    t.a = tile_fold<VL, NG, FULL>(cx, acc, 0.f, FoldAdd());
+  } else if (kind == RED_MAX) {
+    t.a = tile_fold<VL, NG, FULL>(cx, acc, -PN_INF, FoldMaxNan());
+  } else if (kind == RED_MIN) {
+    t.a = tile_fold<VL, NG, FULL>(cx, acc, PN_INF, FoldMinNan());
   } else if (kind == RED_LSE || kind == RED_SOFTMAX) {
-    float m = -PN_INF;
-    PN_UNROLL for (int j = 0; j < NG; ++j)
-      if (FULL || cx.col0 + j * cx.gstride < cx.col_end) {
-        PN_UNROLL for (int i = 0; i < VL; ++i) m = fmaxf(m, acc[j * VL + i]);
-      }
+    // a NaN in the tile makes m, hence every exponential and the sum, NaN
+    const float m = tile_fold<VL, NG, FULL>(cx, acc, -PN_INF, FoldMaxNan());
     const float ms = (m == -PN_INF) ? 0.f : m;   // keeps exp(x - ms) free of inf - inf
     const float L2E = 1.4426950408889634f, nms = -ms * L2E;   // e^(x - ms) = 2^(x log2e - ms log2e)
-    float s = 0.f;
+    float ev[V];
     PN_UNROLL for (int j = 0; j < NG; ++j) {
       const bool ok = FULL || cx.col0 + j * cx.gstride < cx.col_end;
-      PN_UNROLL for (int i = 0; i < VL; ++i) {
-        const float ev = ok ? f_ex2(fmaf(acc[j * VL + i], L2E, nms)) : 0.f;
-        s += ev;
-        if (kind == RED_SOFTMAX) acc[j * VL + i] = ev;
-      }
+      PN_UNROLL for (int i = 0; i < VL; ++i) ev[j * VL + i] = ok ? f_ex2(fmaf(acc[j * VL + i], L2E, nms)) : 0.f;
     }
-    t.a = m; t.b = s;
+    if (kind == RED_SOFTMAX) { PN_UNROLL for (int e = 0; e < V; ++e) acc[e] = ev[e]; }
+    PN_UNROLL for (int e = 1; e < V; ++e) ev[0] += ev[e];
+    t.a = m; t.b = ev[0];
     if (kind == RED_SOFTMAX) ts = ms;
   } else {  // RED_MEANVAR
-    float n = 0.f, sum = 0.f;
+    float n = 0.f;
     PN_UNROLL for (int j = 0; j < NG; ++j)
-      if (FULL || cx.col0 + j * cx.gstride < cx.col_end) {
-        n += static_cast<float>(VL);
-        PN_UNROLL for (int i = 0; i < VL; ++i) sum += acc[j * VL + i];
-      }
+      if (FULL || cx.col0 + j * cx.gstride < cx.col_end) n += static_cast<float>(VL);
+    const float sum = tile_fold<VL, NG, FULL>(cx, acc, 0.f, FoldAdd());
     const float mean = n > 0.f ? sum / n : 0.f;
-    float m2 = 0.f;
-    PN_UNROLL for (int j = 0; j < NG; ++j)
-      if (FULL || cx.col0 + j * cx.gstride < cx.col_end) {
-        PN_UNROLL for (int i = 0; i < VL; ++i) { const float d = acc[j * VL + i] - mean; m2 = fmaf(d, d, m2); }
-      }
-    t.a = n; t.b = mean; t.c = m2;
+    float dev[V];
+    PN_UNROLL for (int j = 0; j < NG; ++j) {
+      const bool ok = FULL || cx.col0 + j * cx.gstride < cx.col_end;
+      PN_UNROLL for (int i = 0; i < VL; ++i) { const float dd = acc[j * VL + i] - mean; dev[j * VL + i] = ok ? dd * dd : 0.f; }
+    }
+    PN_UNROLL for (int e = 1; e < V; ++e) dev[0] += dev[e];
+    t.a = n; t.b = mean; t.c = dev[0];
   }
   st = (cx.chunk > 0) ? red_combine(kind, st, t) : t;
 }
@@ -724,9 +741,9 @@ struct Interp {
 template <class Prog>
 PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
   constexpr int VL = Prog::VL, NG = Prog::NG, K = Prog::K, V = VL * NG;
-  // a generated program for warp teams keeps row offsets, partials and per-row scalars in
-  // registers (every lane computes the same values); otherwise they live in shared memory
-  constexpr bool kRegSlots = Prog::kStatic && Prog::kFamily <= FAM_WARP;
+  // a generated program keeps row offsets, partials and per-row scalars in registers (every
+  // thread computes the same values); the interpreter keeps them in shared memory
+  constexpr bool kRegSlots = Prog::kStatic;
   constexpr bool kRegRowoff = Prog::kStatic;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
   const int family = Prog::family(p);
@@ -871,6 +888,49 @@ PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
         if constexpr (!kRegSlots) __syncwarp();
         Prog::scalar(p, s, cx);
         if constexpr (!kRegSlots) __syncwarp();
+      } else if constexpr (Prog::kStatic) {
+        // generated program, block / cluster team: one barrier per stage.  Each warp leaves its
+        // partial in shared memory (two alternating buffers, so that no second barrier is
+        // needed before they are reused); after the barrier every warp combines all of them in
+        // the same fixed order and runs the scalar program itself, in registers.
+        float* wp = wpart + (parity & 1u) * (32 * kMaxRed * 3);
+        PN_UNROLL for (int r = 0; r < kMaxRed; ++r) {
+          if (r < n_red) {
+            const Part v = warp_combine(Prog::red_kind(p, s, r), parts[r]);
+            if (lane == 0) { float* w = wp + (warp * kMaxRed + r) * 3; w[0] = v.a; w[1] = v.b; w[2] = v.c; }
+          }
+        }
+        __syncthreads();
+        PN_UNROLL for (int r = 0; r < kMaxRed; ++r) {
+          if (r < n_red) {
+            const int kind = Prog::red_kind(p, s, r);
+            Part v = red_identity(kind);
+            if (lane < nwarps) { const float* w = wp + (lane * kMaxRed + r) * 3; v = Part{w[0], w[1], w[2]}; }
+            v = warp_combine(kind, v);
+            if (cluster > 1) {
+              if (tid == 0) { float* d = ctapart + ((parity & 1u) * kMaxRed + r) * 3; d[0] = v.a; d[1] = v.b; d[2] = v.c; }
+            } else {
+              float* d = slots + Prog::red_slot(p, s, r); d[0] = v.a; d[1] = v.b; d[2] = v.c;
+            }
+          }
+        }
+        if (cluster > 1) {
+          cluster_sync_all();   // every CTA's partial is now in its own shared memory
+          PN_UNROLL for (int r = 0; r < kMaxRed; ++r) {
+            if (r < n_red) {
+              const int kind = Prog::red_kind(p, s, r);
+              Part v = red_identity(kind);
+              if (lane < cluster) {
+                const float* w = ctapart + ((parity & 1u) * kMaxRed + r) * 3;
+                v = Part{ld_shared_cluster(w, lane), ld_shared_cluster(w + 1, lane), ld_shared_cluster(w + 2, lane)};
+              }
+              v = warp_combine(kind, v);
+              float* d = slots + Prog::red_slot(p, s, r); d[0] = v.a; d[1] = v.b; d[2] = v.c;
+            }
+          }
+        }
+        parity ^= 1u;
+        Prog::scalar(p, s, cx);
       } else {
         PN_UNROLL for (int r = 0; r < kMaxRed; ++r) {
           if (r < n_red) {

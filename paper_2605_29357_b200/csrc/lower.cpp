@@ -768,7 +768,13 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     if ((!any_force && few_rows) || fc || cands.empty()) {
       std::vector<std::pair<int, int>> cl_opts = ng_opts;
       if (spec && !fm) std::reverse(cl_opts.begin(), cl_opts.end());   // more bytes in flight per thread
-      for (int C : {8, 4, 2})
+      // the fewest CTAs per row that still put at least one CTA on every SM
+      std::vector<int> cl_sizes = {2, 4, 8};
+      std::stable_sort(cl_sizes.begin(), cl_sizes.end(), [&](int a, int b) {
+        const bool fa = eff_rows * a >= sms, fb2 = eff_rows * b >= sms;
+        return fa != fb2 ? fa : (fa ? a < b : a > b);
+      });
+      for (int C : cl_sizes)
         for (auto o : cl_opts) {
           const int T = fm ? 64 : (spec && (eff_N + C - 1) / C >= 2ll * 512 * VL * o.first) ? 512 : 256;
           int64_t slice = (eff_N + C - 1) / C;
@@ -864,7 +870,7 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     P.sm_rowoff = take(teams * kMaxIo * 8);
     P.sm_slots = take(teams * kMaxSlots * 4);
     P.sm_part = take(has_red ? kMaxRed * 3 * cf.block * 4 : 0);
-    P.sm_wpart = take(has_red ? 32 * kMaxRed * 3 * 4 : 0);
+    P.sm_wpart = take(has_red ? 2 * 32 * kMaxRed * 3 * 4 : 0);   // two alternating buffers
     P.sm_ctapart = take(cf.cluster > 1 ? 2 * kMaxRed * 3 * 4 : 0);
     const int64_t stash_floats = (int64_t)n_stash * cf.chunks * cf.vl * cf.ng * cf.block;
     if (off + stash_floats * 4 > dev.max_smem_per_block) { gen_err = "the row does not fit in shared memory for its epilogue"; continue; }
@@ -886,7 +892,9 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     lp.teams_per_cta = teams;
     lp.specialised = 0;
     lp.persistent = persistent ? 1 : 0;
-    lp.no_prefetch = (flags & PN_FLAG_PREFETCH) ? 0 : 1;
+    // long rows split over a cluster run few, long-lived threads: there the first stage's loads
+    // are issued one tile ahead (elsewhere the extra registers cost more than they bring)
+    lp.no_prefetch = ((flags & PN_FLAG_PREFETCH) || (cf.family == FAM_CLUSTER && cf.chunks > 1 && !(flags & PN_FLAG_NO_HOIST))) ? 0 : 1;
     int occ = (dev.have_device && !spec) ? instance_occupancy(cf.vl, cf.ng, cf.k, cf.block, off) : 0;
     size_grid(lp, sms, occ);
     return PN_OK;

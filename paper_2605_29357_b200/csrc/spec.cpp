@@ -10,6 +10,7 @@
 #include <dlfcn.h>
 #include <nvrtc.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <map>
@@ -23,6 +24,20 @@
 namespace pn {
 
 namespace {
+
+// NVRTC options: the fixed ones plus, for experiments, whatever PN_NVRTC_FLAGS lists
+// (space separated, e.g. "-DPN_SOME_SWITCH=1").
+std::vector<std::string> nvrtc_options() {
+  std::vector<std::string> o = {"-arch=sm_100a", "-std=c++17", "-lineinfo"};
+  if (const char* e = getenv("PN_NVRTC_FLAGS")) {
+    std::string cur;
+    for (const char* c = e;; ++c) {
+      if (*c == ' ' || *c == '\0') { if (!cur.empty()) o.push_back(cur); cur.clear(); if (!*c) break; }
+      else cur.push_back(*c);
+    }
+  }
+  return o;
+}
 
 // plan.h followed by device_lib.cuh, as text (written by the build step)
 const char kDeviceSource[] =
@@ -183,7 +198,7 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
   const int team_threads = P.family <= FAM_WARP ? 32 : lp.block;
   const bool full = (long long)P.chunks * team_threads * lp.vl * lp.ng == P.slice_len &&
                     (long long)P.slice_len * P.cluster == P.row_len;
-  const bool reg_slots = P.family <= FAM_WARP;
+  const bool reg_slots = true;   // generated programs keep the per-row scalars in registers
   auto konst = [&](const char* name, long long v) {
     s += std::string("  static PN_DEV int ") + name + "(const KernelParams&) { return " + I(v) + "; }\n";
   };
@@ -268,8 +283,10 @@ bool spec_check(const LaunchPlan& lp, std::string& err) {
   if (!generate_source(lp, src, err)) return false;
   nvrtcProgram prog;
   if (a.CreateProgram(&prog, src.c_str(), "pn_spec.cu", 0, nullptr, nullptr) != NVRTC_SUCCESS) { err = "nvrtcCreateProgram failed"; return false; }
-  const char* opts[] = {"-arch=sm_100a", "-std=c++17", "-lineinfo"};
-  const nvrtcResult r = a.CompileProgram(prog, 3, opts);
+  const std::vector<std::string> ov = nvrtc_options();
+  std::vector<const char*> opts;
+  for (const std::string& x : ov) opts.push_back(x.c_str());
+  const nvrtcResult r = a.CompileProgram(prog, (int)opts.size(), opts.data());
   size_t n = 0; a.GetProgramLogSize(prog, &n);
   std::string log(n, '\0');
   if (n) a.GetProgramLog(prog, &log[0]);
@@ -283,6 +300,7 @@ bool spec_compile(LaunchPlan& lp, int device, int sm_count, SpecKernel& out, std
   if (!a.ok) { err = a.why; return false; }
   std::string src;
   if (!generate_source(lp, src, err)) return false;
+  { std::string key; for (const std::string& x : nvrtc_options()) key += x + " "; src += "\n// " + key + "\n"; }
   Compiled cmp;
   {
     std::lock_guard<std::mutex> lock(g_cache_mutex);
@@ -292,8 +310,10 @@ bool spec_compile(LaunchPlan& lp, int device, int sm_count, SpecKernel& out, std
   if (!cmp.fn) {
     nvrtcProgram prog;
     if (a.CreateProgram(&prog, src.c_str(), "pn_spec.cu", 0, nullptr, nullptr) != NVRTC_SUCCESS) { err = "nvrtcCreateProgram failed"; return false; }
-    const char* opts[] = {"-arch=sm_100a", "-std=c++17", "-lineinfo"};
-    const nvrtcResult r = a.CompileProgram(prog, 3, opts);
+    const std::vector<std::string> ov = nvrtc_options();
+    std::vector<const char*> opts;
+    for (const std::string& x : ov) opts.push_back(x.c_str());
+    const nvrtcResult r = a.CompileProgram(prog, (int)opts.size(), opts.data());
     if (r != NVRTC_SUCCESS) {
       size_t n = 0; a.GetProgramLogSize(prog, &n);
       std::string log(n, '\0');

@@ -119,8 +119,8 @@ def test_lowering_of_the_benchmark_graphs(cfg):
     k = g.kernel_info[0]
     assert pn.FAMILY_NAMES[k["family"]] == FAMILY[cfg]
     assert k["vl"] * (2 if cfg in ("c2", "c3", "c5") else 4) == 16         # 128-bit accesses
-    if cfg == "c4":
-        assert k["cluster"] == 8 and k["grid"] % 8 == 0
+    if cfg == "c4":   # 64 rows: split over clusters so that every SM gets work
+        assert k["cluster"] in (2, 4, 8) and k["grid"] % k["cluster"] == 0 and 64 * k["cluster"] >= 148
     if cfg in ("c2", "c3"):
         assert k["chunks"] == 1                                             # row resident in registers
     gu = pn.Graph(w.desc, 0, PLAN | pn.FLAG_UNFUSED)
