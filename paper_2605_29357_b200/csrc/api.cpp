@@ -10,6 +10,7 @@
 
 #include "../../include/pn.h"
 #include "graph.h"
+#include "handle.h"
 #include "spec.h"
 
 namespace pn {
@@ -19,33 +20,12 @@ cudaError_t launch_plan(const LaunchPlan& lp, cudaStream_t stream);   // kernels
 using namespace pn;
 
 namespace {
-
 thread_local std::string g_last_error;
-
-int fail(int status, const std::string& msg) { g_last_error = msg; return status; }
-
-// where the pointer behind one io entry of one launch comes from
-struct IoSource { int kind; int64_t index; };   // kind 0 user input, 1 user output, 2 workspace offset
-
-struct PlannedLaunch {
-  LaunchPlan plan;
-  std::vector<IoSource> src;
-  SpecKernel spec;   // fn == nullptr: run the plan on the interpreter
-};
-
 }  // namespace
 
-struct pn_graph {
-  Graph g;
-  unsigned flags = 0;
-  int device = 0;
-  bool plan_only = false;
-  std::vector<PlannedLaunch> launches;
-  void* workspace = nullptr;
-  size_t workspace_bytes = 0;
-  int64_t compulsory_bytes = 0;
-  std::vector<void*> stage_in, stage_out;   // device staging of pn_graph_run_host
-};
+namespace pn {
+int fail(int status, const std::string& msg) { g_last_error = msg; return status; }
+}  // namespace pn
 
 namespace {
 
@@ -170,7 +150,7 @@ pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsig
       h->launches.push_back(pl);
     }
     h->workspace_bytes = ws;
-    if (!h->plan_only && ws > 0) {
+    if (!h->plan_only && ws > 0 && !(flags & PN_FLAG_STATIC_SCRATCH)) {
       cudaError_t e = cudaMalloc(&h->workspace, ws);
       if (e != cudaSuccess) { delete h; return fail(PN_ERR_CUDA, std::string("workspace: ") + cudaGetErrorString(e)); }
     }
@@ -194,6 +174,8 @@ pn_status pn_graph_run(pn_graph_t* h, const void* const* inputs, int n_inputs, v
   if (st != PN_OK) return st;
   const Graph& g = h->g;
   if (any_empty(g)) return PN_OK;   // nothing to compute
+  if ((h->flags & PN_FLAG_STATIC_SCRATCH) && h->workspace_bytes > 0)
+    return fail(PN_ERR_INVALID_ARG, "this handle owns no workspace: run it with pn_graph_run_static");
   const bool scalar = (h->flags & PN_FLAG_FORCE_SCALAR) != 0;
   for (int i = 0; i < n_inputs; ++i) {
     if (!inputs[i]) return fail(PN_ERR_INVALID_ARG, "input " + std::to_string(i) + " is null");
