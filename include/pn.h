@@ -83,9 +83,13 @@ enum {
   PN_FLAG_INTERPRET = 1u << 9,    /* run the bytecode on the interpreter kernels built into the
                                      library instead of a kernel specialised for the graph */
   PN_FLAG_NO_HOIST = 1u << 10,    /* do not move row-invariant operand loads out of the row loop */
-  PN_FLAG_PREFETCH = 1u << 11     /* generated kernels: issue the first stage's loads one tile
+  PN_FLAG_PREFETCH = 1u << 11,    /* generated kernels: issue the first stage's loads one tile
                                      ahead (costs registers; off by default)                 */
+  PN_FLAG_STATIC_SCRATCH = 1u << 12 /* with PN_FLAG_UNFUSED: allocate no workspace; the handle
+                                     is run with pn_graph_run_static only                    */
 };
+/* Size of the fixed scratch array behind pn_graph_run_static. */
+#define PN_STATIC_SCRATCH_BYTES (32ll << 20)
 /* Tuning overrides of the lowering's own choices, for measurements and tests: OR them into
  * `flags`.  A value of 0 leaves the choice to the lowering; an impossible one is ignored. */
 #define PN_TUNE_CLUSTER(n) (((unsigned)(n) & 15u) << 16)      /* CTAs per cluster: 2, 4, 8      */
@@ -152,6 +156,40 @@ pn_status pn_graph_run(pn_graph_t* g, const void* const* inputs, int n_inputs,
  */
 pn_status pn_graph_run_host(pn_graph_t* g, const void* const* inputs, int n_inputs,
                             void* const* outputs, int n_outputs, void* stream);
+
+/*
+ * pn_graph_run_static -- the unfused evaluation (one kernel per node) without any allocation.
+ * The paper has no counterpart to this call; it exists for a class of callers.
+ *
+ * Who needs it: code that runs after its process has stopped allocating device memory --
+ * a serving loop whose framework took all free HBM into its own pool at start-up (a late
+ * cudaMalloc there fails, or succeeds only by stalling every stream, since it synchronises
+ * the device), or a worker that is handed a fixed memory budget and may not grow it.  Such
+ * a caller cannot create an ordinary PN_FLAG_UNFUSED handle, whose workspace for the
+ * intermediates between the per-node kernels comes from cudaMalloc.
+ *
+ * What it does instead: the intermediates go into one fixed array of
+ * PN_STATIC_SCRATCH_BYTES (32 MiB) that is part of the library's device image.  Every GPU
+ * that loads the library holds that array until the process exits, used or not.
+ *   g       : a handle created with PN_FLAG_UNFUSED | PN_FLAG_STATIC_SCRATCH (such a create
+ *             allocates no workspace; combine it with PN_FLAG_INTERPRET if the create must
+ *             not load generated kernels either).  pn_graph_run refuses such a handle.
+ *   inputs, outputs, stream : as for pn_graph_run (HOST arrays of DEVICE pointers that the
+ *             caller owns; same alignment and no-overlap rules).
+ * Errors: PN_ERR_TOO_LARGE when the graph's intermediates need more than
+ * PN_STATIC_SCRATCH_BYTES (pn_graph_query PN_Q_WORKSPACE_BYTES tells how much);
+ * PN_ERR_INVALID_ARG for a handle without the two flags; otherwise as pn_graph_run.
+ * The call itself uses no cudaMalloc, cudaFree or other allocating routine.
+ *
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress,
+ * which may make the runtime load the library's device image); make that first call before
+ * any stream capture begins.  All calls, from all handles and threads, share the one array
+ * per device and it keeps whatever the last call left: nothing has to start at zero (each
+ * intermediate is fully written before it is read), but two calls whose kernels overlap on
+ * the GPU -- different streams, no ordering between them -- race on it.  Order them.
+ */
+pn_status pn_graph_run_static(pn_graph_t* g, const void* const* inputs, int n_inputs,
+                              void* const* outputs, int n_outputs, void* stream);
 
 /* pn_graph_destroy -- release the handle and what it owns; NULL is accepted. */
 pn_status pn_graph_destroy(pn_graph_t* g);

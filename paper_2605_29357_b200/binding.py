@@ -25,6 +25,8 @@ FLAG_FORCE_MULTICHUNK = 1 << 8
 FLAG_INTERPRET = 1 << 9
 FLAG_NO_HOIST = 1 << 10
 FLAG_PREFETCH = 1 << 11
+FLAG_STATIC_SCRATCH = 1 << 12
+STATIC_SCRATCH_BYTES = 32 << 20
 
 
 def tune(cluster: int = 0, block: int = 0, groups: int = 0) -> int:
@@ -36,7 +38,7 @@ Q_N_INPUTS, Q_N_OUTPUTS, Q_INPUT_META, Q_OUTPUT_META, Q_COMPULSORY_BYTES = 1, 2,
 Q_N_KERNELS, Q_N_NODES, Q_WORKSPACE_BYTES, Q_KERNEL_INFO = 6, 7, 8, 9
 
 FAMILY_NAMES = {0: "pointwise", 1: "warp-per-row", 2: "block-per-row", 3: "cluster-per-row"}
-EXPORTS = ["pn_graph_create", "pn_graph_run", "pn_graph_run_host", "pn_graph_destroy",
+EXPORTS = ["pn_graph_create", "pn_graph_run", "pn_graph_run_host", "pn_graph_run_static", "pn_graph_destroy",
            "pn_graph_query", "pn_graph_codegen", "pn_status_string", "pn_last_error"]
 
 
@@ -65,7 +67,7 @@ def load_library() -> ctypes.CDLL:
     vp, vpp = ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p)
     lib.pn_graph_create.restype = ctypes.c_int
     lib.pn_graph_create.argtypes = [ctypes.c_char_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_uint, vpp]
-    for fn in (lib.pn_graph_run, lib.pn_graph_run_host):
+    for fn in (lib.pn_graph_run, lib.pn_graph_run_host, lib.pn_graph_run_static):
         fn.restype = ctypes.c_int
         fn.argtypes = [vp, vpp, ctypes.c_int, vpp, ctypes.c_int, vp]
     lib.pn_graph_destroy.restype = ctypes.c_int
@@ -166,6 +168,15 @@ class Graph:
         _check(self._lib.pn_graph_run_host(self._h, self._ptr_array(input_ptrs), len(input_ptrs),
                                            self._ptr_array(output_ptrs), len(output_ptrs),
                                            ctypes.c_void_p(stream)), "pn_graph_run_host")
+
+    def run_static(self, input_ptrs: Sequence[int], output_ptrs: Sequence[int], stream: int = 0) -> None:
+        """pn_graph_run_static: the unfused evaluation with its intermediates in the library's
+        fixed scratch array, for callers that may not allocate device memory.  The handle must
+        have been created with FLAG_UNFUSED | FLAG_STATIC_SCRATCH.  Calls share the array:
+        keep them stream-ordered."""
+        _check(self._lib.pn_graph_run_static(self._h, self._ptr_array(input_ptrs), len(input_ptrs),
+                                             self._ptr_array(output_ptrs), len(output_ptrs),
+                                             ctypes.c_void_p(stream)), "pn_graph_run_static")
 
     def close(self) -> None:
         if getattr(self, "_h", None) is not None and self._h:
