@@ -703,6 +703,10 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
   for (const MOp& m : ops) n_stages = std::max(n_stages, m.stage + 1);
   if (n_stages > kMaxStages) { err = "more reduction-dependent stages than the kernel takes"; return PN_ERR_TOO_LARGE; }
 
+  bool cross_stage = false;   // a tile value made in one stage and read in a later one: the row must stay resident
+  for (const MOp& m : ops) for (int i = 0; i < m.nin; ++i)
+    if (!m.scalar && vals[m.in[i]].kind == VK_E && vals[m.in[i]].stage < m.stage) cross_stage = true;
+
   // ---- (3) family and tile shape ---------------------------------------------------------
   int min_esize = 8;
   bool vec8 = true, vec4 = true;
@@ -737,7 +741,20 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     const bool few_rows = eff_rows < 2ll * sms;
     // the interpreter's 16-element-tile instances are built for at most 256 threads
     auto tile_ok = [&](int T, int ng) { return spec || !(T > 256 && VL * ng > 8); };
-    // one chunk per thread: the smallest team that holds the row
+    // one chunk per thread.  Generated kernels (measured on B200 over row lengths 256..8192,
+    // LayerNorm and softmax graphs): a warp per row while the row fits in 64 two-byte (32
+    // four-byte) elements per lane -- no block barrier at all -- and beyond that a block of
+    // N / 32 threads holding 32 (16) elements each, when the epilogue needs the row again.
+    if (spec && !fm && !fc && VL > 1) {
+      const int v_warp = min_esize <= 2 ? 64 : 32, v_block = min_esize <= 2 ? 32 : 16;
+      if (!fb)
+        for (int ng = 1; VL * ng <= v_warp; ng *= 2)
+          if (32ll * VL * ng >= eff_N) { cands.push_back(Config{FAM_WARP, VL, ng, kSpecRegs, 256, 1, 1, (int)eff_N, false}); break; }
+      if (!fw && cands.empty() && cross_stage)   // rows that need no residency stream in chunks instead
+        for (int T : {64, 128, 256, 512})
+          if ((int64_t)T * v_block >= eff_N) { cands.push_back(Config{FAM_BLOCK, VL, v_block / VL, kSpecRegs, T, 1, 1, (int)eff_N, false}); break; }
+    }
+    // the smallest team that holds the row in one of the interpreter's tile shapes
     if (!fm && !fc) {
       for (int T : {32, 64, 128, 256, 512}) {
         if ((fw && T != 32) || (fb && T == 32)) continue;
