@@ -40,6 +40,31 @@ WORKLOAD = "c2 masked scaled softmax: bf16 scores [512,512,512], int8 causal mas
 FALLBACK_HBM_GBS = 6650.0
 
 
+def kernel_identity(g):
+    """Name of the generated kernel of a fused handle (it carries a hash of the program) and a
+    hash of the device library it is compiled against."""
+    import hashlib
+    import re
+    m = re.search(r"__launch_bounds__\(\d+\)\s+(\w+)\(", g.codegen(0))
+    name = m.group(1) if m else "interpreter"
+    lib = os.path.join(ROOT, "paper_2605_29357_b200", "csrc", "device_lib.cuh")
+    with open(lib, "rb") as f:
+        return name, hashlib.sha256(f.read()).hexdigest()[:16]
+
+
+def recorded_traffic(name, lib_hash):
+    """DRAM bytes (read + write) per launch of that kernel from the ncu capture summarised in
+    profiles/; None when the kernel or the device library has changed since."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.json")) as f:
+            rec = json.load(f).get(name)
+        if rec and rec.get("device_lib_sha256_16") == lib_hash:
+            return rec["dram_bytes_read"] + rec["dram_bytes_write"]
+    except Exception:
+        pass
+    return None
+
+
 def measured_peak():
     try:
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
@@ -256,6 +281,12 @@ def main():
         sampler.start()
     total_ms, per = time_graph(torch, g, sets, args.steps, 0)
     barrier()
+    # K steps of this workload last only milliseconds, less than one nvidia-smi sample: keep
+    # the same step running (untimed) until the sampler has seen the GPU under this load
+    if rank == 0:
+        t_end = time.perf_counter() + 1.0
+        while time.perf_counter() < t_end:
+            time_graph(torch, g, sets, 50, 0)
     clocks = sampler.stop() if rank == 0 else None
     t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
     if world > 1:
@@ -290,6 +321,7 @@ def main():
         return
 
     peak, peak_src = measured_peak()
+    kname, lib_hash = kernel_identity(g)
     st = stats(per)
     achieved = cbytes / (np.mean(per) * 1e-3) / 1e9
     line = {
@@ -306,7 +338,8 @@ def main():
         "e2e": {"value": world * cbytes / e2e_s / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s * 1e3, "steps": e2e_steps},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": None, "peak_source": peak_src, "kernel": f"fused_kernel<{info['vl']},{info['ng']}>",
+                     "traffic": recorded_traffic(kname, lib_hash), "peak_source": peak_src, "kernel": kname,
+                     "device_lib_sha256_16": lib_hash, "specialised": bool(info["specialised"]),
                      "algorithmic_bytes_per_launch": cbytes},
     }
 

@@ -177,6 +177,20 @@ bool emit_program(const KernelParams& P, int pc, int end, bool scalar, int vl, i
   return true;
 }
 
+// Name of the kernel generated for a plan: family, tile shape and a hash of the program and
+// its shape constants, so that profiler listings tell the kernels of different graphs apart.
+std::string kernel_name(const LaunchPlan& lp) {
+  static const char* fam[] = {"pointwise", "warp_row", "block_row", "cluster_row"};
+  uint64_t h = 1469598103934665603ull;
+  auto mix = [&](uint64_t v) { for (int i = 0; i < 8; ++i) { h ^= (v >> (8 * i)) & 0xFF; h *= 1099511628211ull; } };
+  for (int i = 0; i < lp.code_words; ++i) mix(lp.p.code[i]);
+  mix((uint64_t)lp.p.row_len); mix((uint64_t)lp.p.rows); mix((uint64_t)lp.block); mix((uint64_t)lp.p.cluster);
+  for (int q = 0; q < lp.p.n_io; ++q) { mix(lp.p.io[q].dtype); mix((uint64_t)lp.p.io[q].col_stride); }
+  char b[96];
+  snprintf(b, sizeof(b), "pn_spec_%s_v%dx%d_%08x", fam[lp.family & 3], lp.vl, lp.ng, (unsigned)(h ^ (h >> 32)));
+  return b;
+}
+
 bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
   const KernelParams& P = lp.p;
   auto I = [](long long v) { return std::to_string(v); };
@@ -251,7 +265,7 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
     s += "      } break;\n";
   }
   s += "      default: break;\n    }\n  }\n};\n}  // namespace pn\n\n";
-  s += "extern \"C\" __global__ void __launch_bounds__(" + I(lp.block) + ") pn_spec_kernel(const __grid_constant__ pn::KernelParams p) {\n"
+  s += "extern \"C\" __global__ void __launch_bounds__(" + I(lp.block) + ") " + kernel_name(lp) + "(const __grid_constant__ pn::KernelParams p) {\n"
        "  extern __shared__ __align__(16) unsigned char smem[];\n  pn::fused_body<pn::Spec>(p, smem);\n}\n";
   src.swap(s);
   return true;
@@ -329,7 +343,7 @@ bool spec_compile(LaunchPlan& lp, int device, int sm_count, SpecKernel& out, std
     a.DestroyProgram(&prog);
     CUresult cr = a.ModuleLoadData(&cmp.mod, cubin.data());
     if (cr != CUDA_SUCCESS) { err = "cuModuleLoadData: " + cu_err(cr); return false; }
-    cr = a.ModuleGetFunction(&cmp.fn, cmp.mod, "pn_spec_kernel");
+    cr = a.ModuleGetFunction(&cmp.fn, cmp.mod, kernel_name(lp).c_str());
     if (cr != CUDA_SUCCESS) { err = "cuModuleGetFunction: " + cu_err(cr); return false; }
     std::lock_guard<std::mutex> lock(g_cache_mutex);
     g_cache[std::make_pair(device, src)] = cmp;
