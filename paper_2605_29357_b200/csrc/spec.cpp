@@ -13,6 +13,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <algorithm>
 #include <map>
 #include <mutex>
 #include <string>
@@ -265,7 +266,15 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
     s += "      } break;\n";
   }
   s += "      default: break;\n    }\n  }\n};\n}  // namespace pn\n\n";
-  s += "extern \"C\" __global__ void __launch_bounds__(" + I(lp.block) + ") " + kernel_name(lp) + "(const __grid_constant__ pn::KernelParams p) {\n"
+  // Blocks that hold a whole row in registers: ask the compiler to keep registers low enough
+  // for 1024 resident threads per SM, since resident warps are what hides the HBM latency
+  // (measured: +5 % on the LayerNorm workload).  Streaming kernels need no hint: they are
+  // small already, and a bound would only license more registers.
+  const int min_blocks = (P.family == FAM_BLOCK && P.chunks == 1) ? std::max(1, 1024 / lp.block) : 1;
+  s += "#ifndef PN_MIN_BLOCKS\n#define PN_MIN_BLOCKS " + I(min_blocks) + "\n#endif\n";
+  s += "#if PN_MIN_BLOCKS > 1\n#define PN_BOUNDS __launch_bounds__(" + I(lp.block) + ", PN_MIN_BLOCKS)\n#else\n"
+       "#define PN_BOUNDS __launch_bounds__(" + I(lp.block) + ")\n#endif\n";
+  s += "extern \"C\" __global__ void PN_BOUNDS " + kernel_name(lp) + "(const __grid_constant__ pn::KernelParams p) {\n"
        "  extern __shared__ __align__(16) unsigned char smem[];\n  pn::fused_body<pn::Spec>(p, smem);\n}\n";
   src.swap(s);
   return true;
