@@ -516,6 +516,14 @@ TOLERANCES = {
 }
 
 
+# smallest magnitude that rounds to infinity (largest finite value plus half a unit in the last place)
+_OVERFLOW_AT = {
+    _DT_F32: (2.0 - 2.0 ** -24) * 2.0 ** 127,
+    _DT_BF16: (2.0 - 2.0 ** -8) * 2.0 ** 127,
+    _DT_F16: 65520.0,
+}
+
+
 def compare(got: np.ndarray, ref: np.ndarray, dtype: int) -> dict:
     """err(f_G(x), f_pi(G)(x)) <= t, elementwise: |got - ref| <= atol + rtol*|ref| for
     float outputs; infinities must agree exactly and NaN must sit where NaN sits;
@@ -530,6 +538,11 @@ def compare(got: np.ndarray, ref: np.ndarray, dtype: int) -> dict:
     rtol, atol = TOLERANCES[dtype]
     g = got.astype(np.float64)
     r = ref.astype(np.float64)
+    # The reference is unrounded; the output is stored in `dtype`.  A value at or beyond the
+    # point where round-to-nearest overflows that type is, correctly stored, an infinity.
+    lim = _OVERFLOW_AT[dtype]
+    with np.errstate(invalid="ignore"):
+        r = np.where(np.abs(r) >= lim, np.sign(r) * np.inf, r)
     fin = np.isfinite(r)
     with np.errstate(invalid="ignore"):
         bad_special = (~fin) & ~((np.isnan(r) & np.isnan(g)) | (g == r))

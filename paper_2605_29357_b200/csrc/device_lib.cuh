@@ -323,12 +323,14 @@ PN_DEV Part red_combine(int kind, Part x, Part y) {
       x.a = m;
       break;
     }
-    default: {  // RED_MEANVAR: pairwise update of (count, mean, M2)
+    default: {  // RED_MEANVAR: merge of (count, mean, M2)
       const float n = x.a + y.a;
       if (n > 0.f) {
-        const float d = y.b - x.b, r = y.a * f_rcp(n);
-        x.c = x.c + y.c + d * d * x.a * r;
-        x.b = fmaf(d, r, x.b);
+        const float rn = f_rcp(n), d = y.b - x.b;
+        x.c = x.c + y.c + d * d * x.a * (y.a * rn);
+        // the mean from the two sums, not from the difference of the means: rows holding an
+        // infinity then give that infinity (inf - inf would give NaN)
+        x.b = (x.a * x.b + y.a * y.b) * rn;
       }
       x.a = n;
       break;

@@ -455,5 +455,10 @@ def test_tolerance_rule_matches_the_papers_ladder():
     assert not E.compare(np.array([1.0, np.nan, 0.0, np.inf, np.nan]), ref, D.F32)["ok"]
     assert E.compare(np.array([1.015]), np.array([1.0]), D.BF16)["ok"]
     assert not E.compare(np.array([1.02]), np.array([1.0]), D.BF16)["ok"]
+    # a reference beyond the output type's range is an infinity once stored (IEEE overflow)
+    assert E.compare(np.array([np.inf, -np.inf]), np.array([2.7e43, -1e39]), D.F32)["ok"]
+    assert not E.compare(np.array([3.0e38]), np.array([2.7e43]), D.F32)["ok"]
+    assert E.compare(np.array([np.inf]), np.array([70000.0]), D.F16)["ok"]
+    assert not E.compare(np.array([np.inf]), np.array([3.0e38]), D.F32)["ok"]
     assert not E.compare(np.array([1, 2, 4]), np.array([1, 2, 3]), D.I64)["ok"]
     assert E.compare(np.array([1, 2, 3], np.int8), np.array([1, 2, 3]), D.I8)["ok"]
