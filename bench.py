@@ -182,6 +182,28 @@ def time_graph_replay(torch, g, sets, steps, warmup):
     return e0.elapsed_time(e1) / (reps * len(ptrs))
 
 
+def rank_workload(name, rank, **size):
+    """The batch rank `rank` works on: the same graph and shapes on every rank, inputs drawn
+    from the rank's own seed.  Rows are independent, so sharding a larger job by rows needs no
+    exchange between ranks at all."""
+    return C.CONFIGS[name](seed=rank, **size)
+
+
+def max_over_ranks(x, world, device):
+    """The slowest rank's time: what a whole-job throughput has to be divided by."""
+    import torch
+    t = torch.tensor([float(x)], device=device, dtype=torch.float64)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(world, bytes_per_rank, seconds_per_step):
+    """Whole-job GB/s: the bytes all ranks moved in a step over the slowest rank's step time."""
+    return world * bytes_per_rank / seconds_per_step / 1e9
+
+
 def stats(per):
     a = np.sort(np.asarray(per))
     q1, med, q3 = np.percentile(a, [25, 50, 75])
@@ -261,7 +283,7 @@ def main():
     warmup = max(args.warmup, 3)
 
     # ---- the benchmark workload: one batch per rank, seed = rank ---------------------------
-    w = C.CONFIGS[args.workload](seed=rank)
+    w = rank_workload(args.workload, rank)
     g = pn.Graph(w.desc, local_rank, 0)
     info = g.kernel_info[0]
     cbytes = g.compulsory_bytes
@@ -288,12 +310,9 @@ def main():
         while time.perf_counter() < t_end:
             time_graph(torch, g, sets, 50, 0)
     clocks = sampler.stop() if rank == 0 else None
-    t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, world, "cuda")
     ms_per_step = total_ms / args.steps
-    value = world * cbytes / (ms_per_step * 1e-3) / 1e9
+    value = job_value(world, cbytes, ms_per_step * 1e-3)
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region -----
     pin_in = [torch.from_numpy(np.ascontiguousarray(a).reshape(-1).view(np.uint8)).pin_memory() for a in w.inputs]
@@ -308,10 +327,7 @@ def main():
         g.run_host([t_.data_ptr() for t_ in pin_in], [t_.data_ptr() for t_ in pin_out], stream)
     torch.cuda.synchronize()
     e2e_s = (time.perf_counter() - t0) / e2e_steps
-    t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_s = float(t.item())
+    e2e_s = max_over_ranks(e2e_s, world, "cuda")
     h2d = int(sum(a.nbytes for a in w.inputs))
     d2h = int(sum(nbytes_of(w.output_meta)))
 
@@ -335,7 +351,7 @@ def main():
                    "nodes": g.n_nodes, "per_step": st, "pct_of_8000": 100 * value / world / 8000.0},
         "clocks": clocks,
         "gpu_launches": args.steps * g.n_kernels,
-        "e2e": {"value": world * cbytes / e2e_s / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
+        "e2e": {"value": job_value(world, cbytes, e2e_s), "unit": "GB/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s * 1e3, "steps": e2e_steps},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": recorded_traffic(kname, lib_hash), "peak_source": peak_src, "kernel": kname,
