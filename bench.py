@@ -56,7 +56,7 @@ def recorded_traffic(name, lib_hash):
     """DRAM bytes (read + write) per launch of that kernel from the ncu capture summarised in
     profiles/; None when the kernel or the device library has changed since."""
     try:
-        with open(os.path.join(ROOT, "profiles", "dram_traffic.json")) as f:
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.txt")) as f:
             rec = json.load(f).get(name)
         if rec and rec.get("device_lib_sha256_16") == lib_hash:
             return rec["dram_bytes_read"] + rec["dram_bytes_write"]
