@@ -59,6 +59,7 @@ _OP_NAMES = {
     96: "sum", 97: "mean", 98: "var", 99: "amax", 100: "amin", 101: "argmax", 102: "argmin",
     103: "logsumexp",
     128: "softmax", 129: "log_softmax", 130: "layer_norm", 131: "rms_norm",
+    160: "roll", 161: "slice", 162: "view",
 }
 
 
@@ -361,6 +362,30 @@ def comp_rms_norm(x, gamma, eps: float):
     return y
 
 
+def op_roll(x, dim: int, shift: int):
+    """y[..., i, ...] = x[..., (i - shift) mod D, ...] along `dim`: the circular shift that the
+    paper's fused kernel replaces by index arithmetic, idx = (S + i - shift) mod S (Section 4.4)."""
+    x = np.asarray(x)
+    d = x.shape[dim]
+    idx = (np.arange(d) - shift) % d
+    return np.take(x, idx, axis=dim)
+
+
+def op_slice(x, dim: int, start: int, length: int):
+    """y[..., i, ...] = x[..., start + i, ...] for i < length along `dim`."""
+    x = np.asarray(x)
+    if start < 0 or start + length > x.shape[dim]:
+        raise ValueError("slice outside the tensor")
+    sl = [slice(None)] * x.ndim
+    sl[dim] = slice(start, start + length)
+    return x[tuple(sl)]
+
+
+def op_view(x, dims):
+    """Same elements in the same row-major order under another shape."""
+    return np.ascontiguousarray(x).reshape(dims)
+
+
 def op_cast(x, dst_dtype: int):
     """Value conversion.  Float -> integer truncates toward zero; anything -> bool
     tests for non-zero; to a float type the value is kept (narrow-float rounding is
@@ -437,6 +462,12 @@ def evaluate(desc: bytes, inputs: Sequence[np.ndarray],
                 res = [np.minimum(np.maximum(a[0], a[1]), a[2])]
             elif n.op == "fma":
                 res = [a[0] * a[1] + a[2]]
+            elif n.op == "roll":
+                res = [op_roll(a[0], int(n.attr[0]), int(n.attr[1]))]
+            elif n.op == "slice":
+                res = [op_slice(a[0], int(n.attr[0]), int(n.attr[1]), int(out_t[0].dims[int(n.attr[0])]))]
+            elif n.op == "view":
+                res = [op_view(a[0], tuple(out_t[0].dims))]
             elif n.op == "sum":
                 res = [red_sum(a[0])]
             elif n.op == "mean":

@@ -234,6 +234,39 @@ def c5(M: int = 8192, N: int = 14336, seed: int = 0, dtype: int = D.BF16) -> Wor
                    ["h", "mask", "mean", "var"], [av, gv, cv, rv])
 
 
+# ---------------------------------------------------------------------------
+# N1: roll + slice + add + LayerNorm with two outputs (the operator sequence of the paper's
+# first case study: contiguous, view, roll, slice, contiguous, view, add, layer_norm)
+# ---------------------------------------------------------------------------
+def n1(S: int = 133, SC: int = 128, Cc: int = 96, shift: int = 3, seed: int = 0, dtype: int = D.BF16,
+       eps: float = 1e-5) -> Workload:
+    g = GraphBuilder()
+    x = g.input(dtype, (1, S * S, Cc))           # the window-partitioned feature map, flat
+    res = g.input(dtype, (1, SC * SC, Cc))
+    gamma = g.input(dtype, (Cc,))
+    beta = g.input(dtype, (Cc,))
+    v = g.op("view", [x], dtype, (S, S, Cc))
+    r0 = g.op("roll", [v], dtype, (S, S, Cc), attr=[0, shift])
+    r1 = g.op("roll", [r0], dtype, (S, S, Cc), attr=[1, shift])
+    s0 = g.op("slice", [r1], dtype, (SC, S, Cc), attr=[0, 0])
+    s1 = g.op("slice", [s0], dtype, (SC, SC, Cc), attr=[1, 0])
+    w = g.op("view", [s1], dtype, (1, SC * SC, Cc))
+    cast = (lambda t, dm: g.op("cast", [t], D.F32, dm)) if dtype != D.F32 else (lambda t, dm: t)
+    h = g.op("add", [cast(res, (1, SC * SC, Cc)), cast(w, (1, SC * SC, Cc))], D.F32, (1, SC * SC, Cc))
+    y = g.node("layer_norm", [h, cast(gamma, (Cc,)), cast(beta, (Cc,))], [D.F32], [(1, SC * SC, Cc)], extra_imm=[eps])[0]
+    out_add = g.op("cast", [h], dtype, (1, SC * SC, Cc)) if dtype != D.F32 else h
+    out_ln = g.op("cast", [y], dtype, (1, SC * SC, Cc)) if dtype != D.F32 else y
+    names = {out_add: "add", out_ln: "layer_norm"}
+    for t in names:
+        g.mark_output(t)
+    xs = _store(_draw(_rng(seed, 6, 0), "normal", (1, S * S, Cc), 0.0, 1.0), dtype)
+    rs = _store(_draw(_rng(seed, 6, 1), "normal", (1, SC * SC, Cc), 0.0, 1.0), dtype)
+    ga = _store(_draw(_rng(seed, 6, 2), "uniform", (Cc,), 0.5, 1.5), dtype)
+    be = _store(_draw(_rng(seed, 6, 3), "normal", (Cc,), 0.0, 0.1), dtype)
+    return _finish("n1_roll_slice_add_layernorm", g, ["x", "residual", "gamma", "beta"],
+                   [names[i] for i in g.output_ids()], [xs, rs, ga, be], {"eps": eps, "shift": shift})
+
+
 CONFIGS = {"c1": c1, "c2": c2, "c3": c3, "c4": c4, "c5": c5}
 
 # Reduced sizes of the same graphs: several tiles plus a ragged tail each, small enough

@@ -60,6 +60,10 @@ OPCODES = {
     "argmax": 101, "argmin": 102, "logsumexp": 103,
     # composites over the last dim
     "softmax": 128, "log_softmax": 129, "layer_norm": 130, "rms_norm": 131,
+    # index operators on leading dimensions (they move data, they compute nothing):
+    # roll: attr = (dim, shift); slice: attr = (dim, start), length from the output shape;
+    # view: regroups leading dimensions, the last one and the element order unchanged
+    "roll": 160, "slice": 161, "view": 162,
 }
 
 

@@ -462,3 +462,49 @@ def test_tolerance_rule_matches_the_papers_ladder():
     assert not E.compare(np.array([np.inf]), np.array([3.0e38]), D.F32)["ok"]
     assert not E.compare(np.array([1, 2, 4]), np.array([1, 2, 3]), D.I64)["ok"]
     assert E.compare(np.array([1, 2, 3], np.int8), np.array([1, 2, 3]), D.I8)["ok"]
+
+
+# ---------------------------------------------------------------------------
+# index operators: roll + slice as the paper's index arithmetic
+# ---------------------------------------------------------------------------
+def test_roll_slice_view_match_the_papers_index_formula():
+    """Section 4.4 / Appendix G, case 1: roll(shift) followed by slice[:SC] on an [S, S, C] tensor
+    equals reading row (S + i - shift) mod S, column (S + j - shift) mod S."""
+    S, SC, Cc, shift = 7, 5, 4, 3
+    rng = np.random.default_rng(9)
+    x = rng.standard_normal((1, S * S, Cc)).astype(np.float32)
+    g = GraphBuilder()
+    xi = g.input(D.F32, x.shape)
+    v = g.op("view", [xi], D.F32, (S, S, Cc))
+    r = g.op("roll", [g.op("roll", [v], D.F32, (S, S, Cc), attr=[0, shift])], D.F32, (S, S, Cc), attr=[1, shift])
+    s = g.op("slice", [g.op("slice", [r], D.F32, (SC, S, Cc), attr=[0, 0])], D.F32, (SC, SC, Cc), attr=[1, 0])
+    g.mark_output(g.op("view", [s], D.F32, (1, SC * SC, Cc)))
+    got = E.evaluate(g.build(), [x])[0]
+    x3 = x.reshape(S, S, Cc)
+    for i in range(SC):
+        for j in range(SC):
+            src = x3[(S + i - shift) % S, (S + j - shift) % S]
+            assert np.array_equal(got[0, i * SC + j], src.astype(np.float64))
+    # negative and oversized shifts wrap; a slice that starts inside the tensor
+    a = np.arange(10, dtype=np.float32).reshape(5, 2)
+    for sh in (-1, 7):
+        out = run1("roll", [a], [D.F32], D.F32, (5, 2), attr=(0, sh))
+        assert out[:, 0].tolist() == [float(a[(i - sh) % 5, 0]) for i in range(5)]
+    out = run1("slice", [a], [D.F32], D.F32, (2, 2), attr=(0, 2))
+    assert out.tolist() == [[4.0, 5.0], [6.0, 7.0]]
+
+
+def test_n1_restated():
+    w = C.n1(S=6, SC=4, Cc=8, shift=2)
+    x, res, ga, be = [_bf(t) for t in w.inputs]
+    out = dict(zip(w.output_names, E.evaluate(w.desc, w.inputs)))
+    x3 = x.reshape(6, 6, 8)
+    for i in range(4):
+        for j in range(4):
+            h = [res[0, i * 4 + j, c] + x3[(6 + i - 2) % 6, (6 + j - 2) % 6, c] for c in range(8)]
+            mu = math.fsum(h) / 8
+            var = math.fsum((t - mu) ** 2 for t in h) / 8
+            for c in range(8):
+                assert out["add"][0, i * 4 + j, c] == h[c]
+                ref = (h[c] - mu) / math.sqrt(var + 1e-5) * ga[c] + be[c]
+                assert abs(out["layer_norm"][0, i * 4 + j, c] - ref) < 1e-12
