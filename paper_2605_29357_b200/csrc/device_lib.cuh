@@ -406,6 +406,24 @@ PN_DEV float ld_shared_cluster(const float* local_smem_ptr, uint32_t rank) {
 }
 
 // ---------------------------------------------------------------------------------------
+// inputs read through roll / slice / view: the data is never moved, the row's start is
+// computed instead (the index arithmetic idx = (S + i - shift) mod S of the paper's first case
+// study, Section 4.4, for any chain of rolls and slices on leading dimensions)
+// ---------------------------------------------------------------------------------------
+struct IoMap { int d0, d1, d2, a0, a1, a2, m0, m1, m2; long long s0, s1, s2; };
+PN_DEV long long mapped_row_offset(unsigned long long row, const IoMap m) {
+  const unsigned long long q2 = row / (unsigned)m.d2;
+  int c2 = (int)(row - q2 * (unsigned)m.d2) + m.a2;
+  const unsigned long long q1 = q2 / (unsigned)m.d1;
+  int c1 = (int)(q2 - q1 * (unsigned)m.d1) + m.a1;
+  int c0 = (int)q1 + m.a0;
+  if (m.m2) c2 %= m.m2;
+  if (m.m1) c1 %= m.m1;
+  if (m.m0) c0 %= m.m0;
+  return c0 * m.s0 + c1 * m.s1 + c2 * m.s2;
+}
+
+// ---------------------------------------------------------------------------------------
 // tile operations: one function per bytecode instruction
 // ---------------------------------------------------------------------------------------
 struct TileCtx {
@@ -714,6 +732,12 @@ struct Interp {
   static constexpr int kFamily = -1, kNumIo = kMaxIo, kNumPrefetch = 0;
   static PN_DEV unsigned lead_dim(const KernelParams& p, int i) { return p.lead_dim[i]; }
   static PN_DEV long long lead_stride(const KernelParams& p, int io, int i) { return p.io[io].lead_stride[i]; }
+  static PN_DEV bool io_mapped(const KernelParams& p, int io) { return p.io[io].mapped != 0; }
+  static PN_DEV IoMap io_map(const KernelParams& p, int q) {
+    const IoDesc& io = p.io[q];
+    return IoMap{io.map_dim[0], io.map_dim[1], io.map_dim[2], io.map_add[0], io.map_add[1], io.map_add[2],
+                 io.map_mod[0], io.map_mod[1], io.map_mod[2], io.lead_stride[0], io.lead_stride[1], io.lead_stride[2]};
+  }
   static PN_DEV int family(const KernelParams& p) { return p.family; }
   static PN_DEV int cluster(const KernelParams& p) { return p.cluster; }
   static PN_DEV int chunks(const KernelParams& p) { return p.chunks; }
@@ -808,8 +832,10 @@ PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
     const long long i2 = (long long)(r0 - q2 * d2);
     const unsigned long long q1 = q2 / d1;
     const long long i1 = (long long)(q2 - q1 * d1);
-    PN_UNROLL for (int q = 0; q < (kRegRowoff ? Prog::kNumIo : 1); ++q)
-      out[q] = (long long)q1 * Prog::lead_stride(p, q, 0) + i1 * Prog::lead_stride(p, q, 1) + i2 * Prog::lead_stride(p, q, 2);
+    PN_UNROLL for (int q = 0; q < (kRegRowoff ? Prog::kNumIo : 1); ++q) {
+      if (Prog::io_mapped(p, q)) out[q] = mapped_row_offset(r0, Prog::io_map(p, q));
+      else out[q] = (long long)q1 * Prog::lead_stride(p, q, 0) + i1 * Prog::lead_stride(p, q, 1) + i2 * Prog::lead_stride(p, q, 2);
+    }
   };
 
   // loads that are the same for every row: once per thread (their row offsets are all zero)
@@ -843,7 +869,8 @@ PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
         long long r = row;
         const long long i2 = r % p.lead_dim[2]; r /= p.lead_dim[2];
         const long long i1 = r % p.lead_dim[1]; r /= p.lead_dim[1];
-        rowoff_sm[team_tid] = r * io.lead_stride[0] + i1 * io.lead_stride[1] + i2 * io.lead_stride[2];
+        rowoff_sm[team_tid] = io.mapped ? mapped_row_offset((unsigned long long)row, IoMap{io.map_dim[0], io.map_dim[1], io.map_dim[2], io.map_add[0], io.map_add[1], io.map_add[2], io.map_mod[0], io.map_mod[1], io.map_mod[2], io.lead_stride[0], io.lead_stride[1], io.lead_stride[2]})
+                                        : r * io.lead_stride[0] + i1 * io.lead_stride[1] + i2 * io.lead_stride[2];
       }
       if (warp_team) __syncwarp(); else __syncthreads();
     }

@@ -17,7 +17,8 @@ enum NodeOp : uint16_t {
   N_ADD = 32, N_SUB, N_MUL, N_DIV, N_MAX, N_MIN, N_GT, N_GE, N_LT, N_LE, N_EQ, N_NE,
   N_WHERE = 64, N_CLAMP, N_FMA,
   N_SUM = 96, N_MEAN, N_VAR, N_AMAX, N_AMIN, N_ARGMAX, N_ARGMIN, N_LOGSUMEXP,
-  N_SOFTMAX = 128, N_LOG_SOFTMAX, N_LAYER_NORM, N_RMS_NORM
+  N_SOFTMAX = 128, N_LOG_SOFTMAX, N_LAYER_NORM, N_RMS_NORM,
+  N_ROLL = 160, N_SLICE, N_VIEW   // index operators on leading dimensions
 };
 
 constexpr uint32_t kImm0 = 0xFFFFFFFFu, kImm1 = 0xFFFFFFFEu;
@@ -52,6 +53,7 @@ inline int dtype_bytes(int dt) {
 inline bool dtype_is_float(int dt) { return dt == kF32 || dt == kF16 || dt == kBF16; }
 inline bool is_reduction(uint16_t op) { return op >= N_SUM && op <= N_LOGSUMEXP; }
 inline bool is_composite(uint16_t op) { return op >= N_SOFTMAX && op <= N_RMS_NORM; }
+inline bool is_index_op(uint16_t op) { return op >= N_ROLL && op <= N_VIEW; }
 
 // Returns a pn_status value (see pn.h).
 int parse_descriptor(const void* desc, size_t bytes, Graph& g, std::string& err);

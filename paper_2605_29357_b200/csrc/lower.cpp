@@ -378,7 +378,69 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     if (is_reduction(n.op) || is_composite(n.op)) has_red = true;
     for (int k = 0; k < n.n_in; ++k) if (n.in[k] < (uint32_t)nt) n_consumers[n.in[k]]++;
   }
+  // ---- index operators: roll / slice / view chains that start at a graph input are folded into
+  // the addressing of that input (no data is moved) --------------------------------------
+  struct IdxMap {
+    int root = -1;                       // the graph input the chain starts at
+    int64_t ext[3] = {1, 1, 1}, add[3] = {0, 0, 0}, mod[3] = {0, 0, 0}, stride[3] = {0, 0, 0};
+    bool sliced[3] = {false, false, false};
+    bool plain = true;                   // still the dense tensor itself (views only)
+    bool frozen = false;                 // regrouped by a view after rolls / slices: no further index ops
+  };
+  std::vector<IdxMap> imap(nt);
+  auto plain_map = [&](int root, const Tensor& T) {
+    IdxMap m; m.root = root;
+    const Shape4 s = align4(T);
+    int64_t st = s.d[3];
+    for (int i = 2; i >= 0; --i) { m.ext[i] = s.d[i]; m.stride[i] = st; st *= s.d[i]; }
+    return m;
+  };
+  for (int t : g.inputs) imap[t] = plain_map(t, g.tensors[t]);
+  std::vector<char> by_compute(nt, 0);   // read by an arithmetic node, or a graph output
+  for (const Node& n : g.nodes)
+    if (!is_index_op(n.op)) for (int k = 0; k < n.n_in; ++k) if (n.in[k] < (uint32_t)nt) by_compute[n.in[k]] = 1;
+  for (int o : g.outputs) by_compute[o] = 1;
+  for (size_t ni = 0; ni < g.nodes.size(); ++ni) {
+    const Node& n = g.nodes[ni];
+    if (!is_index_op(n.op)) continue;
+    const std::string where = "node " + std::to_string(ni) + ": ";
+    const Tensor& X = g.tensors[n.in[0]]; const Tensor& Y = g.tensors[n.out[0]];
+    IdxMap m = imap[n.in[0]];
+    if (m.root < 0) { err = where + "roll / slice / view apply to graph inputs (or chains of them) only"; return PN_ERR_UNSUPPORTED_OP; }
+    if (Y.dtype != X.dtype) { err = where + "an index operator keeps the dtype"; return PN_ERR_UNSUPPORTED_OP; }
+    if (X.rank < 1 || Y.rank < 1 || X.dims[X.rank - 1] != Y.dims[Y.rank - 1]) { err = where + "index operators act on leading dimensions; the last one must be unchanged"; return PN_ERR_SHAPE; }
+    if (n.op == N_VIEW) {
+      if (X.numel() != Y.numel()) { err = where + "a view keeps the number of elements"; return PN_ERR_SHAPE; }
+      if (m.plain) m = plain_map(m.root, Y); else m.frozen = true;
+    } else {
+      if (m.frozen) { err = where + "roll / slice after a view of a rolled or sliced tensor is not lowered"; return PN_ERR_UNSUPPORTED_OP; }
+      const int64_t k = n.attr[0];
+      if (k < 0 || k >= X.rank - 1 || X.rank > 4) { err = where + "roll / slice dimension must be a leading one"; return PN_ERR_SHAPE; }
+      const int kk = 3 - (X.rank - 1) + (int)k;
+      for (int d = 0; d < X.rank; ++d)
+        if (d != k && X.dims[d] != Y.dims[d]) { err = where + "only the rolled / sliced dimension may change"; return PN_ERR_SHAPE; }
+      if (X.rank != Y.rank) { err = where + "rank must be kept"; return PN_ERR_SHAPE; }
+      const int64_t Dk = X.dims[k];
+      if (n.op == N_ROLL) {
+        if (Y.dims[k] != Dk) { err = where + "a roll keeps the shape"; return PN_ERR_SHAPE; }
+        if (m.sliced[kk]) { err = where + "roll after slice on the same dimension is not lowered"; return PN_ERR_UNSUPPORTED_OP; }
+        if (Dk > 0) { m.add[kk] = ((m.add[kk] - n.attr[1]) % Dk + Dk) % Dk; m.mod[kk] = Dk; }
+      } else {
+        const int64_t a = n.attr[1], L = Y.dims[k];
+        if (a < 0 || a + L > Dk) { err = where + "slice outside the tensor"; return PN_ERR_SHAPE; }
+        m.add[kk] += a; m.ext[kk] = L; m.sliced[kk] = true;
+        if (m.mod[kk]) m.add[kk] %= m.mod[kk];
+      }
+      m.plain = false;
+    }
+    imap[n.out[0]] = m;
+  }
+  // tensors that exist only to be re-indexed take no part in the iteration space
+  std::vector<char> index_only(nt, 0);
+  for (int t = 0; t < nt; ++t) index_only[t] = imap[t].root >= 0 && !by_compute[t];
+
   for (const Node& n : g.nodes) {   // per-row scalars
+    if (is_index_op(n.op)) continue;
     if (is_reduction(n.op)) is_s[n.out[0]] = 1;
     else if (n.op == N_LAYER_NORM) { for (int k = 1; k < n.n_out; ++k) is_s[n.out[k]] = 1; }
     else if (!is_composite(n.op)) {
@@ -402,7 +464,7 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     }
   }
   for (int t = 0; t < nt; ++t) {
-    if (is_s[t]) continue;
+    if (is_s[t] || index_only[t]) continue;
     const Shape4 s = align4(g.tensors[t]);
     if (has_red) {
       for (int i = 0; i < 4; ++i)
@@ -415,6 +477,7 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
   if (N >= (int64_t(1) << 30)) { err = "last dimension too long"; return PN_ERR_TOO_LARGE; }
   for (size_t ni = 0; ni < g.nodes.size(); ++ni) {   // per-node shape rules
     const Node& n = g.nodes[ni];
+    if (is_index_op(n.op)) continue;   // checked with the chains above
     const std::string where = "node " + std::to_string(ni) + ": ";
     auto row_shaped = [&](const Tensor& t, const Tensor& src) {
       if (t.rank == src.rank - 1) { for (int i = 0; i < t.rank; ++i) if (t.dims[i] != src.dims[i]) return false; return true; }
@@ -453,14 +516,19 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
   // ---- io table ------------------------------------------------------------------------
   memset(&lp, 0, sizeof(lp));
   KernelParams& P = lp.p;
-  const int n_io = (int)(g.inputs.size() + g.outputs.size());
+  // input-like entries: graph inputs read directly, and re-indexed views of graph inputs
+  std::vector<int> in_like;
+  for (int t = 0; t < nt; ++t)
+    if (imap[t].root >= 0 && by_compute[t] && ((g.tensors[t].role & 1) || g.tensors[t].producer >= 0)) in_like.push_back(t);
+  const int n_io = (int)(in_like.size() + g.outputs.size());
   if (n_io > kMaxIo) { err = "more graph inputs + outputs than one kernel takes (" + std::to_string(kMaxIo) + ")"; return PN_ERR_TOO_LARGE; }
   P.n_io = n_io;
-  std::vector<int> io_of_tensor(nt, -1);
+  std::vector<int> io_of_tensor(nt, -1), in_io_of_tensor(nt, -1);
   std::vector<char> io_streamed(n_io, 0);
+  bool any_mapped = false;
   {
     int idx = 0;
-    auto add_io = [&](int t, bool is_out) {
+    auto add_io = [&](int t, bool is_out) -> bool {
       IoDesc& io = P.io[idx];
       const Tensor& T = g.tensors[t];
       io.dtype = T.dtype;
@@ -476,10 +544,23 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
         io.col_stride = (s.d[3] == 1 && N != 1) ? 0 : 1;
         io_streamed[idx] = full;
       }
-      lp.io_tensor[idx] = t; lp.io_is_output[idx] = is_out;
-      io_of_tensor[t] = idx++;
+      if (!is_out && !imap[t].plain) {   // read through rolls / slices: own coordinates, source strides
+        const IdxMap& m = imap[t];
+        const Shape4 s = align4(T);
+        if (m.ext[0] * m.ext[1] * m.ext[2] != rows || s.d[3] != N) return false;
+        io.mapped = 1; io.col_stride = 1; io_streamed[idx] = 1; any_mapped = true;
+        for (int i = 0; i < 3; ++i) {
+          io.lead_stride[i] = m.stride[i];
+          io.map_dim[i] = (int32_t)std::max<int64_t>(m.ext[i], 1); io.map_add[i] = (int32_t)m.add[i]; io.map_mod[i] = (int32_t)m.mod[i];
+        }
+      }
+      lp.io_tensor[idx] = is_out ? t : imap[t].root; lp.io_is_output[idx] = is_out;
+      if (is_out) io_of_tensor[t] = idx; else in_io_of_tensor[t] = idx;
+      ++idx;
+      return true;
     };
-    for (int t : g.inputs) add_io(t, false);
+    for (int t : in_like)
+      if (!add_io(t, false)) { err = "tensor " + std::to_string(t) + ": a rolled / sliced input must cover the whole iteration space"; return PN_ERR_UNSUPPORTED_OP; }
     for (int t : g.outputs) add_io(t, true);
   }
   // collapse leading dims that every io walks contiguously (or broadcasts) together
@@ -489,10 +570,11 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
       if (lead_dim[i] == 1) continue;
       bool ok = true;
       if (lead_dim[i + 1] != 1)
-        for (int q = 0; q < n_io && ok; ++q) ok = P.io[q].lead_stride[i] == P.io[q].lead_stride[i + 1] * lead_dim[i + 1];
+        for (int q = 0; q < n_io && ok; ++q) ok = P.io[q].mapped || P.io[q].lead_stride[i] == P.io[q].lead_stride[i + 1] * lead_dim[i + 1];
       if (!ok) continue;
       for (int q = 0; q < n_io; ++q) {
         IoDesc& io = P.io[q];
+        if (io.mapped) continue;   // splits the row index by its own extents
         if (lead_dim[i + 1] == 1) io.lead_stride[i + 1] = io.lead_stride[i];
         io.lead_stride[i] = 0;
       }
@@ -502,7 +584,7 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
   for (int i = 0; i < 3; ++i) if (lead_dim[i] > 0xFFFFFFFFll) { err = "leading dimension too large"; return PN_ERR_TOO_LARGE; }
   int64_t eff_rows = rows, eff_N = N;
   // a purely pointwise graph whose tensors all have the full shape is one long row
-  if (!has_red && rows > 1 && rows * N < (int64_t(1) << 30) && lead_dim[0] == 1 && lead_dim[1] == 1) {
+  if (!has_red && !any_mapped && rows > 1 && rows * N < (int64_t(1) << 30) && lead_dim[0] == 1 && lead_dim[1] == 1) {
     bool flat = true;
     for (int q = 0; q < n_io; ++q) flat = flat && P.io[q].col_stride == 1 && P.io[q].lead_stride[2] == N;
     if (flat) { eff_N = rows * N; eff_rows = 1; lead_dim[2] = 1; for (int q = 0; q < n_io; ++q) P.io[q].lead_stride[2] = 0; }
@@ -525,13 +607,13 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     for (int v : in) m.in[m.nin++] = v;
     m.out = out; m.aux0 = a0; m.aux1 = a1; ops.push_back(m);
   };
-  for (int t : g.inputs) {
+  for (int t : in_like) {
     const int v = new_val(VK_E, 0);
-    const int q = io_of_tensor[t];
+    const int q = in_io_of_tensor[t];
     vals[v].io = q;
     vals[v].bcast = P.io[q].col_stride == 0;
     vals[v].streamed = io_streamed[q];
-    vals[v].invariant = P.io[q].lead_stride[0] == 0 && P.io[q].lead_stride[1] == 0 && P.io[q].lead_stride[2] == 0;
+    vals[v].invariant = !P.io[q].mapped && P.io[q].lead_stride[0] == 0 && P.io[q].lead_stride[1] == 0 && P.io[q].lead_stride[2] == 0;
     vals[v].integral = !dtype_is_float(g.tensors[t].dtype);
     vals[v].mask8 = g.tensors[t].dtype == kI8 || g.tensors[t].dtype == kBool;
     tval[t] = v;
@@ -579,6 +661,14 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
       if (n.in[k] == kImm0) in[k] = imm_val(n.imm[0]);
       else if (n.in[k] == kImm1) in[k] = imm_val(n.imm[1]);
       else in[k] = tval[n.in[k]];
+    }
+    if (is_index_op(n.op)) {
+      const int t = n.out[0];
+      if (g.tensors[t].role & 2) {
+        if (tval[t] < 0) { err = where + "internal: re-indexed output without a value"; return PN_ERR_UNSUPPORTED_OP; }
+        add_op(OP_STOUT, 0, false, {tval[t]}, -1, io_of_tensor[t], 0);
+      }
+      continue;
     }
     int res[3] = {-1, -1, -1};
     const Tensor& T0 = g.tensors[n.out[0]];

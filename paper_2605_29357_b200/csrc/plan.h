@@ -96,7 +96,13 @@ struct IoDesc {
   int32_t col_stride;      // 1, or 0 when the last dim is broadcast
   uint8_t dtype;
   uint8_t is_row_scalar;   // per-row result tensor (one element per row)
-  uint8_t pad[2];
+  uint8_t mapped;          // an input read through roll / slice / view: the row index is split by
+                           // map_dim (row-major) into coordinates c_d, and the row starts at
+                           // sum_d ((c_d + map_add[d]) mod map_mod[d]) * lead_stride[d]  (mod 0 = none)
+  uint8_t pad[1];
+  int32_t map_dim[3];
+  int32_t map_add[3];
+  int32_t map_mod[3];
 };
 
 struct RedDesc {

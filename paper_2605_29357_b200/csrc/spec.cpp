@@ -186,7 +186,11 @@ std::string kernel_name(const LaunchPlan& lp) {
   auto mix = [&](uint64_t v) { for (int i = 0; i < 8; ++i) { h ^= (v >> (8 * i)) & 0xFF; h *= 1099511628211ull; } };
   for (int i = 0; i < lp.code_words; ++i) mix(lp.p.code[i]);
   mix((uint64_t)lp.p.row_len); mix((uint64_t)lp.p.rows); mix((uint64_t)lp.block); mix((uint64_t)lp.p.cluster);
-  for (int q = 0; q < lp.p.n_io; ++q) { mix(lp.p.io[q].dtype); mix((uint64_t)lp.p.io[q].col_stride); }
+  for (int q = 0; q < lp.p.n_io; ++q) {
+    const IoDesc& io = lp.p.io[q];
+    mix(io.dtype); mix((uint64_t)io.col_stride); mix(io.mapped);
+    for (int i = 0; i < 3; ++i) { mix((uint64_t)io.lead_stride[i]); mix((uint64_t)io.map_dim[i]); mix((uint64_t)io.map_add[i]); mix((uint64_t)io.map_mod[i]); }
+  }
   char b[96];
   snprintf(b, sizeof(b), "pn_spec_%s_v%dx%d_%08x", fam[lp.family & 3], lp.vl, lp.ng, (unsigned)(h ^ (h >> 32)));
   return b;
@@ -209,6 +213,18 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
     for (int i = 0; i < 3; ++i)
       if (P.io[q].lead_stride[i] != 0) s += "      case " + I(q * 3 + i) + ": return " + I(P.io[q].lead_stride[i]) + "ll;\n";
   s += "      default: return 0;\n    }\n  }\n";
+  s += "  static PN_DEV bool io_mapped(const KernelParams&, int io) {\n    switch (io) {\n";
+  for (int q = 0; q < P.n_io; ++q) if (P.io[q].mapped) s += "      case " + I(q) + ": return true;\n";
+  s += "      default: return false;\n    }\n  }\n";
+  s += "  static PN_DEV IoMap io_map(const KernelParams&, int io) {\n    switch (io) {\n";
+  for (int q = 0; q < P.n_io; ++q)
+    if (P.io[q].mapped) {
+      const IoDesc& io = P.io[q];
+      s += "      case " + I(q) + ": return IoMap{" + I(io.map_dim[0]) + ", " + I(io.map_dim[1]) + ", " + I(io.map_dim[2]) + ", " +
+           I(io.map_add[0]) + ", " + I(io.map_add[1]) + ", " + I(io.map_add[2]) + ", " + I(io.map_mod[0]) + ", " + I(io.map_mod[1]) + ", " +
+           I(io.map_mod[2]) + ", " + I(io.lead_stride[0]) + "ll, " + I(io.lead_stride[1]) + "ll, " + I(io.lead_stride[2]) + "ll};\n";
+    }
+  s += "      default: return IoMap{1, 1, 1, 0, 0, 0, 0, 0, 0, 0, 0, 0};\n    }\n  }\n";
   // every group of every tile inside the row: no validity tests in the generated code
   const int team_threads = P.family <= FAM_WARP ? 32 : lp.block;
   const bool full = (long long)P.chunks * team_threads * lp.vl * lp.ng == P.slice_len &&

@@ -160,3 +160,59 @@ def test_forced_families():
     # a row length that is not a multiple of the vector width falls back to element accesses
     k = pn.Graph(C.c3(M=4, N=1001).desc, 0, PLAN).kernel_info[0]
     assert k["vl"] == 1
+
+
+# ---- index operators (Section 3.2: index-remapped loads) --------------------------------
+def test_index_chain_becomes_addressing_of_one_kernel():
+    w = _descriptor_only_n1()
+    g = pn.Graph(w.desc, 0, PLAN)
+    assert g.n_kernels == 1
+    k = g.kernel_info[0]
+    assert k["rows"] == 128 * 128 and k["row_len"] == 96 and k["stages"] == 2
+    src = g.codegen(0, compile=True)
+    m = re.search(r"static PN_DEV bool io_mapped\(.*?\n((?:.*\n)*?)\s*default: return false;", src)
+    assert m and m.group(1).count("return true") == 1          # exactly the rolled input
+    # rolls by +3 over 133 read from (i + 130) mod 133; source strides are those of the 133 x 133 map
+    assert "IoMap{1, 128, 128, 0, 130, 130, 0, 133, 133," in src and "12768ll, 96ll}" in src
+    gu = pn.Graph(w.desc, 0, PLAN | pn.FLAG_UNFUSED)
+    assert gu.n_kernels > 8                                    # every index op is a copy kernel there
+    for i in range(gu.n_kernels):
+        gu.codegen(i, compile=True)
+
+
+def _descriptor_only_n1():
+    import numpy as np
+    real_draw = C._draw
+    C._draw = lambda rng, kind, shape, a, b, chunk=0: np.zeros(shape, dtype=np.float32)
+    try:
+        return C.n1()
+    finally:
+        C._draw = real_draw
+
+
+def test_index_operator_errors():
+    def one(op, in_shape, out_shape, attr, dtype_out=D.F32):
+        g = GraphBuilder(); x = g.input(D.F32, in_shape)
+        g.mark_output(g.op(op, [x], dtype_out, out_shape, attr=attr))
+        return _status(g.build())
+    assert one("roll", (4, 8), (4, 8), [0, 1]) == 0
+    assert one("roll", (4, 8), (4, 8), [1, 1]) == -4            # the last dimension is not a leading one
+    assert one("roll", (4, 8), (5, 8), [0, 1]) == -4            # a roll keeps the shape
+    assert one("roll", (4, 8), (4, 8), [0, 1], D.BF16) == -3    # and the dtype
+    assert one("slice", (4, 8), (3, 8), [0, 1]) == 0
+    assert one("slice", (4, 8), (3, 8), [0, 2]) == -4           # 2 + 3 > 4
+    assert one("slice", (4, 8), (3, 4), [0, 0]) == -4           # last dimension must be whole
+    assert one("view", (4, 6, 8), (3, 8, 8), [0, 0]) == 0
+    assert one("view", (4, 6, 8), (3, 8, 4), [0, 0]) == -4
+    # index operators read graph inputs (or chains of them), not computed values
+    g = GraphBuilder(); x = g.input(D.F32, (4, 8))
+    y = g.op("neg", [x], D.F32, (4, 8))
+    g.mark_output(g.op("roll", [y], D.F32, (4, 8), attr=[0, 1]))
+    assert _status(g.build()) == -3
+    assert _status(g.build(), PLAN | pn.FLAG_UNFUSED) == 0      # one node at a time it is a plain copy
+    # roll after slice on the same dimension would need a second modulus
+    g = GraphBuilder(); x = g.input(D.F32, (6, 8))
+    s = g.op("slice", [x], D.F32, (4, 8), attr=[0, 1])
+    g.mark_output(g.op("roll", [s], D.F32, (4, 8), attr=[0, 1]))
+    assert _status(g.build()) == -3
+    assert _status(g.build(), PLAN | pn.FLAG_UNFUSED) == 0
