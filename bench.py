@@ -375,12 +375,12 @@ def main():
     # ---- the other benchmark subgraphs (N = 1 only) ------------------------------------------
     if world == 1 and not args.no_sweep:
         sweep = {}
-        for name in C.CONFIGS:
+        for name, make in {**C.CONFIGS, **C.EXTENDED}.items():
             if name == args.workload:
                 continue
-            wi = C.CONFIGS[name]()
+            wi = make()
             gi = pn.Graph(wi.desc, local_rank, 0)
-            cb = gi.compulsory_bytes
+            cb = int(wi.notes.get("touched_bytes", gi.compulsory_bytes))
             ns = 1 if cb > 2 * l2 else int(2 * l2 // cb) + 2
             si = device_sets(torch, wi, ns)
             _, pi = time_graph(torch, gi, si, args.steps, warmup)

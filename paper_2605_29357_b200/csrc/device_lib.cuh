@@ -533,25 +533,29 @@ template <int VL, int NG, bool FULL = false>
 PN_DEV void op_red(const TileCtx& cx, int kind, Part& st, float (&acc)[VL * NG], float& ts) {
   constexpr int V = VL * NG;
   if (kind == RED_ARGMAX || kind == RED_ARGMIN) {
-    // the tile extreme first; the index is searched only when it beats the running extreme
-    // (ties keep the earlier, lower-index holder; a NaN beats every number)
+    // Branch-free: the tile extreme by a fold, then its first holder by a descending scan of
+    // equality tests (the lowest slot is written last), then one predicated update of the
+    // running (extreme, column).  Ties keep the earlier, lower-index holder; a NaN beats every
+    // number, which only the rarely taken branch below has to know about.
     const bool mx = kind == RED_ARGMAX;
     const float m = mx ? tile_fold<VL, NG, FULL>(cx, acc, -PN_INF, FoldMaxNan()) : tile_fold<VL, NG, FULL>(cx, acc, PN_INF, FoldMinNan());
-    const bool m_nan = m != m, s_nan = st.a != st.a;
-    const bool take = cx.chunk == 0 || (m_nan ? !s_nan : (!s_nan && (mx ? m > st.a : m < st.a)));
-    if (take) {
-      int bi = 0x7FFFFFFF;
-      PN_UNROLL for (int j = NG - 1; j >= 0; --j) {
-        const int col = cx.col0 + j * cx.gstride;
-        if (FULL || col < cx.col_end) {
-          PN_UNROLL for (int i = VL - 1; i >= 0; --i) {
-            const float v = acc[j * VL + i];
-            if (m_nan ? (v != v) : (v == m)) bi = col + i;   // descending scan: the lowest column wins
-          }
-        }
-      }
-      st.a = m; st.b = bits_f(static_cast<uint32_t>(bi));
+    int slot = 0;
+    PN_UNROLL for (int j = NG - 1; j >= 0; --j) {
+      const bool ok = FULL || cx.col0 + j * cx.gstride < cx.col_end;
+      PN_UNROLL for (int i = VL - 1; i >= 0; --i) slot = (ok && acc[j * VL + i] == m) ? j * VL + i : slot;
     }
+    const bool m_nan = m != m, s_nan = st.a != st.a;
+    if (m_nan) {   // the fold returns NaN when the tile holds one: find the first
+      PN_UNROLL for (int j = NG - 1; j >= 0; --j) {
+        const bool ok = FULL || cx.col0 + j * cx.gstride < cx.col_end;
+        PN_UNROLL for (int i = VL - 1; i >= 0; --i) slot = (ok && acc[j * VL + i] != acc[j * VL + i]) ? j * VL + i : slot;
+      }
+    }
+    const bool take = cx.chunk == 0 || (m_nan ? !s_nan : (!s_nan && (mx ? m > st.a : m < st.a)));
+    // a thread whose tile lies wholly outside the row keeps the sentinel column, which loses every tie
+    const int bi = (FULL || cx.col0 < cx.col_end) ? cx.col0 + (slot / VL) * cx.gstride + (slot % VL) : 0x7FFFFFFF;
+    st.a = take ? m : st.a;
+    st.b = take ? bits_f(static_cast<uint32_t>(bi)) : st.b;
     return;
   }
   Part t = red_identity(kind);

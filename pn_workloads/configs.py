@@ -264,10 +264,15 @@ def n1(S: int = 133, SC: int = 128, Cc: int = 96, shift: int = 3, seed: int = 0,
     ga = _store(_draw(_rng(seed, 6, 2), "uniform", (Cc,), 0.5, 1.5), dtype)
     be = _store(_draw(_rng(seed, 6, 3), "normal", (Cc,), 0.0, 0.1), dtype)
     return _finish("n1_roll_slice_add_layernorm", g, ["x", "residual", "gamma", "beta"],
-                   [names[i] for i in g.output_ids()], [xs, rs, ga, be], {"eps": eps, "shift": shift})
+                   [names[i] for i in g.output_ids()], [xs, rs, ga, be],
+                   {"eps": eps, "shift": shift,
+                    # only the SC x SC window of x is ever read
+                    "touched_bytes": D.DTYPE_BYTES[dtype] * (4 * SC * SC * Cc + 2 * Cc)})
 
 
 CONFIGS = {"c1": c1, "c2": c2, "c3": c3, "c4": c4, "c5": c5}
+# subgraphs beyond the five benchmark ones (index-remapped loads)
+EXTENDED = {"n1": n1}
 
 # Reduced sizes of the same graphs: several tiles plus a ragged tail each, small enough
 # for the CPU oracle to finish in well under a second.
