@@ -24,9 +24,10 @@ final rounding is judged against the exact value.
 
 Operator definitions follow the usual closed forms; the LayerNorm form (biased
 variance, 1/sqrt(var + eps), (x - mean) * rstd * gamma + beta) is the one the
-paper's fused add+LayerNorm kernel computes (Appendix G, case 1); the clamped
-division of its masked-mean-pooling kernel (Appendix G, case 2) is expressible
-with clamp and div.
+paper's fused add+LayerNorm kernel computes (Appendix G, case 1); its
+masked-mean-pooling pattern (Appendix G, case 2: cast, mul, two sums over the
+sequence dimension, clamp, div, a one-operand cat) is evaluated operator by
+operator with the reductions over a leading dimension below.
 
 Every function is pinned by tests/test_oracle_pins.py against closed forms,
 invariants, brute force on tiny inputs and a third restatement; nothing here is
@@ -57,9 +58,9 @@ _OP_NAMES = {
     38: "gt", 39: "ge", 40: "lt", 41: "le", 42: "eq", 43: "ne",
     64: "where", 65: "clamp", 66: "fma",
     96: "sum", 97: "mean", 98: "var", 99: "amax", 100: "amin", 101: "argmax", 102: "argmin",
-    103: "logsumexp",
+    103: "logsumexp", 104: "sum_dim", 105: "mean_dim", 106: "amax_dim", 107: "amin_dim",
     128: "softmax", 129: "log_softmax", 130: "layer_norm", 131: "rms_norm",
-    160: "roll", 161: "slice", 162: "view",
+    160: "roll", 161: "slice", 162: "view", 163: "cat",
 }
 
 
@@ -318,6 +319,31 @@ def red_logsumexp(x):
     return out[..., 0]
 
 
+def red_over_dim(kind: str, x, dim: int):
+    """Reduction over one dimension `dim` of x, that dimension dropped from the result:
+    sum_k x[.., k, ..]; mean = that sum / D; amax / amin = the extreme (a NaN along the
+    dimension makes the result NaN).  This is what the paper's masked-mean-pooling pattern
+    uses twice (Appendix G, case 2: sum(hidden * mask, 1) and sum(mask, 1) over the sequence
+    dimension of [B, S, D] tensors)."""
+    x = _f(x)
+    if not 0 <= dim < x.ndim:
+        raise ValueError("reduced dimension outside the tensor")
+    if kind == "sum_dim":
+        return x.sum(axis=dim)
+    if kind == "mean_dim":
+        return x.sum(axis=dim) / x.shape[dim]
+    if kind == "amax_dim":
+        return np.max(x, axis=dim)
+    if kind == "amin_dim":
+        return np.min(x, axis=dim)
+    raise ValueError(kind)
+
+
+def op_cat(parts, dim: int):
+    """Concatenation of the operands along `dim` (one operand: the operand itself)."""
+    return np.concatenate([np.asarray(p) for p in parts], axis=dim)
+
+
 def comp_softmax(x):
     """softmax(x)_j = e^(x_j - m) / sum_k e^(x_k - m), m the row maximum.
     A row that is -inf throughout yields NaN (inf - inf), as IEEE arithmetic does."""
@@ -468,6 +494,10 @@ def evaluate(desc: bytes, inputs: Sequence[np.ndarray],
                 res = [op_slice(a[0], int(n.attr[0]), int(n.attr[1]), int(out_t[0].dims[int(n.attr[0])]))]
             elif n.op == "view":
                 res = [op_view(a[0], tuple(out_t[0].dims))]
+            elif n.op in ("sum_dim", "mean_dim", "amax_dim", "amin_dim"):
+                res = [red_over_dim(n.op, a[0], int(n.attr[0]))]
+            elif n.op == "cat":
+                res = [op_cat(a, int(n.attr[0]))]
             elif n.op == "sum":
                 res = [red_sum(a[0])]
             elif n.op == "mean":

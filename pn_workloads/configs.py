@@ -270,9 +270,41 @@ def n1(S: int = 133, SC: int = 128, Cc: int = 96, shift: int = 3, seed: int = 0,
                     "touched_bytes": D.DTYPE_BYTES[dtype] * (4 * SC * SC * Cc + 2 * Cc)})
 
 
+# ---------------------------------------------------------------------------
+# N2: masked mean pooling (the operator sequence of the paper's second case study: cast, mul,
+# sum, sum, clamp, div, cat): both sums run over the sequence dimension S of [B, S, D]
+# ---------------------------------------------------------------------------
+def n2(B: int = 256, S: int = 512, Dh: int = 1024, seed: int = 0, dtype: int = D.BF16,
+       mask_dtype: int = D.I64, dense_mask: bool = False, floor: float = 1e-9) -> Workload:
+    g = GraphBuilder()
+    mshape = (B, S, Dh) if dense_mask else (B, S, 1)     # an expanded mask is a stride-0 view
+    cshape = (B, Dh) if dense_mask else (B, 1)
+    mask = g.input(mask_dtype, mshape)
+    hidden = g.input(dtype, (B, S, Dh))
+    m = g.op("cast", [mask], D.F32, mshape)
+    prod = g.op("mul", [hidden, m], D.F32, (B, S, Dh))
+    num = g.op("sum_dim", [prod], D.F32, (B, Dh), attr=[1, 0])
+    cnt = g.op("sum_dim", [m], D.F32, cshape, attr=[1, 0])
+    den = g.op("clamp", [cnt, Imm(floor), Imm(math.inf)], D.F32, cshape)
+    q = g.op("div", [num, den], D.F32, (B, Dh))
+    out = g.op("cat", [q], D.F32, (B, Dh), attr=[1, 0])
+    g.mark_output(out)
+    hs = _store(_draw(_rng(seed, 7, 0), "normal", (B, S, Dh), 0.0, 1.0), dtype)
+    # a padded batch: sequence b keeps its first L_b positions, L_b uniform on [S/4, S]
+    lens = _rng(seed, 7, 1).integers(max(1, S // 4), S + 1, size=B)
+    keep = (np.arange(S)[None, :] < lens[:, None])
+    mv = np.broadcast_to(keep[:, :, None], mshape)
+    if mask_dtype in (D.F32, D.BF16, D.F16):
+        ms = _store(np.ascontiguousarray(mv, dtype=np.float32), mask_dtype)
+    else:
+        ms = np.ascontiguousarray(mv).astype(NP_STORAGE[mask_dtype])
+    return _finish("n2_masked_mean_pooling", g, ["mask", "hidden"], ["pooled"], [ms, hs],
+                   {"floor": floor, "lengths_min": int(lens.min()), "lengths_max": int(lens.max())})
+
+
 CONFIGS = {"c1": c1, "c2": c2, "c3": c3, "c4": c4, "c5": c5}
-# subgraphs beyond the five benchmark ones (index-remapped loads)
-EXTENDED = {"n1": n1}
+# subgraphs beyond the five benchmark ones (index-remapped loads; a reduction over a leading dimension)
+EXTENDED = {"n1": n1, "n2": n2}
 
 # Reduced sizes of the same graphs: several tiles plus a ragged tail each, small enough
 # for the CPU oracle to finish in well under a second.
@@ -282,4 +314,6 @@ SMALL = {
     "c3": dict(M=33, N=1000),
     "c4": dict(M=5, N=10007),
     "c5": dict(M=19, N=1432),
+    "n1": dict(S=21, SC=16, Cc=96),
+    "n2": dict(B=3, S=37, Dh=200),
 }

@@ -58,12 +58,18 @@ OPCODES = {
     # last-dim reductions
     "sum": 96, "mean": 97, "var": 98, "amax": 99, "amin": 100,
     "argmax": 101, "argmin": 102, "logsumexp": 103,
+    # reductions over one leading dimension: attr = (dim, 0); the result has the input's shape
+    # with that dimension dropped or kept as 1
+    "sum_dim": 104, "mean_dim": 105, "amax_dim": 106, "amin_dim": 107,
     # composites over the last dim
     "softmax": 128, "log_softmax": 129, "layer_norm": 130, "rms_norm": 131,
     # index operators on leading dimensions (they move data, they compute nothing):
     # roll: attr = (dim, shift); slice: attr = (dim, start), length from the output shape;
     # view: regroups leading dimensions, the last one and the element order unchanged
     "roll": 160, "slice": 161, "view": 162,
+    # cat: attr = (dim, 0); the concatenation of its operands along dim.  With one operand it is
+    # the identity (graph traces keep such nodes)
+    "cat": 163,
 }
 
 

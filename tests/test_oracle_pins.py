@@ -508,3 +508,83 @@ def test_n1_restated():
                 assert out["add"][0, i * 4 + j, c] == h[c]
                 ref = (h[c] - mu) / math.sqrt(var + 1e-5) * ga[c] + be[c]
                 assert abs(out["layer_norm"][0, i * 4 + j, c] - ref) < 1e-12
+
+
+# ---------------------------------------------------------------------------
+# reductions over a leading dimension, cat, and masked mean pooling
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("shape,dim", [((5, 3), 0), ((4, 6, 5), 1), ((4, 6, 5), 0), ((2, 3, 4, 5), 2), ((2, 3, 4, 5), 1)])
+def test_reductions_over_a_leading_dimension_brute_force(shape, dim):
+    x = np.random.default_rng(21).standard_normal(shape).astype(np.float32)
+    out_shape = shape[:dim] + shape[dim + 1:]
+    got = {op: run1(op, [x], [D.F32], D.F32, out_shape, attr=(dim, 0)) for op in ("sum_dim", "mean_dim", "amax_dim", "amin_dim")}
+    for idx in np.ndindex(*out_shape):
+        line = [float(x[idx[:dim] + (k,) + idx[dim:]]) for k in range(shape[dim])]
+        assert abs(got["sum_dim"][idx] - math.fsum(line)) < 1e-13
+        assert abs(got["mean_dim"][idx] - math.fsum(line) / len(line)) < 1e-14
+        assert got["amax_dim"][idx] == max(line) and got["amin_dim"][idx] == min(line)
+    # the reduced dimension kept as 1 is the same values under the other shape
+    kept = shape[:dim] + (1,) + shape[dim + 1:]
+    assert np.array_equal(run1("sum_dim", [x], [D.F32], D.F32, kept, attr=(dim, 0)).reshape(out_shape), got["sum_dim"])
+
+
+def test_reductions_over_a_leading_dimension_closed_forms_and_nan():
+    # x[b, s, d] = b + 10 s + 100 d:  sum over s = S b + 10 S (S - 1) / 2 + 100 S d
+    B, S, Dh = 3, 7, 4
+    b, s, d = np.meshgrid(np.arange(B), np.arange(S), np.arange(Dh), indexing="ij")
+    x = (b + 10 * s + 100 * d).astype(np.float32)
+    tot = run1("sum_dim", [x], [D.F32], D.F32, (B, Dh), attr=(1, 0))
+    for bb in range(B):
+        for dd in range(Dh):
+            assert tot[bb, dd] == S * bb + 10 * S * (S - 1) // 2 + 100 * S * dd
+    assert np.array_equal(run1("amax_dim", [x], [D.F32], D.F32, (B, Dh), attr=(1, 0)), x[:, S - 1, :])
+    assert np.array_equal(run1("amin_dim", [x], [D.F32], D.F32, (B, Dh), attr=(1, 0)), x[:, 0, :])
+    x[1, 3, 2] = np.nan
+    mx = run1("amax_dim", [x], [D.F32], D.F32, (B, Dh), attr=(1, 0))
+    assert np.isnan(mx[1, 2]) and np.isnan(mx).sum() == 1
+    assert np.isnan(run1("sum_dim", [x], [D.F32], D.F32, (B, Dh), attr=(1, 0))[1, 2])
+    # integer tensors are summed exactly
+    m = np.arange(24, dtype=np.int64).reshape(2, 3, 4) % 2
+    cnt = run1("sum_dim", [m], [D.I64], D.F32, (2, 4), attr=(1, 0))
+    assert cnt.tolist() == [[0.0, 3.0, 0.0, 3.0], [0.0, 3.0, 0.0, 3.0]]
+
+
+def test_cat_of_one_operand_is_the_identity_and_of_two_is_stacking():
+    a = np.arange(6, dtype=np.float32).reshape(2, 3); b = -a
+    assert np.array_equal(run1("cat", [a], [D.F32], D.F32, (2, 3), attr=(1, 0)), a)
+    out = run1("cat", [a, b], [D.F32, D.F32], D.F32, (2, 6), attr=(1, 0))
+    assert out.tolist() == [[0, 1, 2, -0.0, -1, -2], [3, 4, 5, -3, -4, -5]]
+    out = run1("cat", [a, b], [D.F32, D.F32], D.F32, (4, 3), attr=(0, 0))
+    assert out[2:].tolist() == b.tolist() and out[:2].tolist() == a.tolist()
+
+
+@pytest.mark.parametrize("dense_mask,mask_dtype", [(False, D.I64), (True, D.F32), (True, D.I8)])
+def test_n2_masked_mean_pooling_restated(dense_mask, mask_dtype):
+    """Appendix G, case 2: out[b, d] = sum_s(hidden * mask) / max(sum_s(mask), 1e-9)."""
+    w = C.n2(B=3, S=9, Dh=5, dense_mask=dense_mask, mask_dtype=mask_dtype)
+    mask, hidden = w.inputs
+    h = _bf(hidden)
+    m = np.broadcast_to(np.asarray(mask, dtype=np.float64), h.shape)
+    out = E.evaluate(w.desc, w.inputs)[0]
+    assert out.shape == (3, 5)
+    for b in range(3):
+        for d in range(5):
+            num = math.fsum(h[b, s, d] * m[b, s, d] for s in range(9))
+            cnt = math.fsum(m[b, s, d] for s in range(9))
+            assert abs(out[b, d] - num / max(cnt, 1e-9)) < 1e-14
+    assert 1 <= w.notes["lengths_min"] <= w.notes["lengths_max"] <= 9
+
+
+def test_masked_mean_pooling_special_cases():
+    rows = dict((r[0], r) for r in _gold("sparkle_max_diff.txt"))
+    assert float(rows["masked_mean_pooling"][1]) == 0.0      # Table 2: the fused kernel is bitwise identical
+    w = C.n2(B=4, S=6, Dh=8)
+    mask, hidden = [a.copy() for a in w.inputs]
+    h = _bf(hidden)
+    mask[0, :, 0] = 1                     # nothing masked: the plain mean over S
+    mask[1, :, 0] = 0                     # everything masked: 0 / 1e-9 = 0
+    mask[2, :, 0] = 0; mask[2, 4, 0] = 1  # one position kept: that row of hidden, exactly
+    out = E.evaluate(w.desc, [mask, hidden])[0]
+    assert np.allclose(out[0], h[0].sum(axis=0) / 6, rtol=0, atol=1e-15)
+    assert np.array_equal(out[1], np.zeros(8))
+    assert np.array_equal(out[2], h[2, 4])
