@@ -186,7 +186,7 @@ def rank_workload(name, rank, **size):
     """The batch rank `rank` works on: the same graph and shapes on every rank, inputs drawn
     from the rank's own seed.  Rows are independent, so sharding a larger job by rows needs no
     exchange between ranks at all."""
-    return C.CONFIGS[name](seed=rank, **size)
+    return {**C.CONFIGS, **C.EXTENDED}[name](seed=rank, **size)
 
 
 def max_over_ranks(x, world, device):
@@ -260,7 +260,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-sweep", action="store_true")
-    ap.add_argument("--workload", default="c2", choices=list(C.CONFIGS))
+    ap.add_argument("--workload", default="c2", choices=list(C.CONFIGS) + list(C.EXTENDED))
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

@@ -37,7 +37,7 @@ def tune(cluster: int = 0, block: int = 0, groups: int = 0) -> int:
 Q_N_INPUTS, Q_N_OUTPUTS, Q_INPUT_META, Q_OUTPUT_META, Q_COMPULSORY_BYTES = 1, 2, 3, 4, 5
 Q_N_KERNELS, Q_N_NODES, Q_WORKSPACE_BYTES, Q_KERNEL_INFO = 6, 7, 8, 9
 
-FAMILY_NAMES = {0: "pointwise", 1: "warp-per-row", 2: "block-per-row", 3: "cluster-per-row"}
+FAMILY_NAMES = {0: "pointwise", 1: "warp-per-row", 2: "block-per-row", 3: "cluster-per-row", 4: "column-reduce"}
 EXPORTS = ["pn_graph_create", "pn_graph_run", "pn_graph_run_host", "pn_graph_run_static", "pn_graph_destroy",
            "pn_graph_query", "pn_graph_codegen", "pn_status_string", "pn_last_error"]
 

@@ -19,6 +19,8 @@ bool arity_of(uint16_t op, Arity& a) {
   if (op >= N_ADD && op <= N_NE) { a = {2, 2, 1, 1}; return true; }
   if (op == N_WHERE || op == N_CLAMP || op == N_FMA) { a = {3, 3, 1, 1}; return true; }
   if (op >= N_SUM && op <= N_LOGSUMEXP) { a = {1, 1, 1, 1}; return true; }
+  if (op >= N_SUM_DIM && op <= N_AMIN_DIM) { a = {1, 1, 1, 1}; return true; }
+  if (op == N_CAT) { a = {1, 4, 1, 1}; return true; }
   if (op == N_SOFTMAX || op == N_LOG_SOFTMAX) { a = {1, 1, 1, 1}; return true; }
   if (op == N_LAYER_NORM) { a = {1, 3, 1, 3}; return true; }
   if (op == N_RMS_NORM) { a = {1, 2, 1, 1}; return true; }

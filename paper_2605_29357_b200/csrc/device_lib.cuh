@@ -510,6 +510,16 @@ PN_DEV void op_where_raw(float (&acc)[VL * NG], const float (&craw)[VL * NG], co
 template <int V>
 PN_DEV void op_splat(float (&t)[V], float v) { PN_UNROLL for (int e = 0; e < V; ++e) t[e] = v; }
 
+// column kernels: reg = reg (op) acc element by element, the running reduction over the walked
+// dimension (sum, or NaN-propagating max / min)
+PN_DEV float accum_combine(int kind, float a, float b) {
+  return kind == RED_SUM ? a + b : (kind == RED_MAX ? f_max_nan(a, b) : f_min_nan(a, b));
+}
+template <int V>
+PN_DEV void op_accum(int kind, float (&r)[V], const float (&acc)[V]) {
+  PN_UNROLL for (int e = 0; e < V; ++e) r[e] = accum_combine(kind, r[e], acc[e]);
+}
+
 // Fold of a tile in element order (a fixed order, so results repeat exactly).  Elements of
 // groups outside the row take the identity.
 template <int VL, int NG, bool FULL, class F>
@@ -716,6 +726,9 @@ PN_DEV void run_program(const KernelParams& p, int pc, const int pc_end, const T
       case OP_FILL_TS:
         if constexpr (!SCALAR) ts = *stash_ptr<V>(cx, b);
         break;
+      case OP_ACCUM:
+        if constexpr (!SCALAR) { PN_WITH_REG(b, op_accum<V>(a, r, acc);) }
+        break;
       case OP_SLD: op_splat<V>(acc, cx.slots[a]); break;
       case OP_SST:
         if constexpr (SCALAR) op_sst<false>(cx, a, acc[0]);
@@ -742,6 +755,10 @@ struct Interp {
     return IoMap{io.map_dim[0], io.map_dim[1], io.map_dim[2], io.map_add[0], io.map_add[1], io.map_add[2],
                  io.map_mod[0], io.map_mod[1], io.map_mod[2], io.lead_stride[0], io.lead_stride[1], io.lead_stride[2]};
   }
+  static constexpr int kWalkUnroll = 1;
+  static PN_DEV long long red_stride(const KernelParams& p, int io) { return p.io[io].red_stride; }
+  static PN_DEV int col_tx(const KernelParams& p) { return p.col_tx; }
+  static PN_DEV int red_len(const KernelParams& p) { return p.red_len; }
   static PN_DEV int family(const KernelParams& p) { return p.family; }
   static PN_DEV int cluster(const KernelParams& p) { return p.cluster; }
   static PN_DEV int chunks(const KernelParams& p) { return p.chunks; }
@@ -1016,6 +1033,95 @@ PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
   }
   // a CTA's shared memory may still be read by its cluster peers until they pass this point
   if (cluster > 1) cluster_sync_all();
+}
+
+// ---------------------------------------------------------------------------------------
+// the kernel body of the column family: reductions over a leading dimension
+// ---------------------------------------------------------------------------------------
+// Iteration space [rows, R, C], reduced over R.  A CTA is TX threads along the columns by
+// TY = blockDim.x / TX along R and owns one (row, column tile) item at a time; a column tile is
+// NG groups of VL columns per thread, group j of thread tx at column tile_base + j * TX * VL +
+// tx * VL, so that the threads of a warp read whole 128-bit words of one contiguous run per
+// step.  Thread (tx, ty) walks the steps ty, ty + TY, ...: the stage-0 tile program loads and
+// evaluates one step and folds it into the accumulators (tile registers 0 .. n_red-1).  The
+// accumulators of the TY walkers of a column are then combined through shared memory by the
+// ty = 0 thread, in the fixed order ty = 0, 1, ..., so results repeat bit for bit; that thread
+// runs the stage-1 program (the epilogue on the reduced values) and stores.  Every input element
+// is read once.  Hand-offs are __syncthreads only.
+template <class Prog>
+PN_DEV void column_body(const KernelParams& p, unsigned char* smem) {
+  constexpr int VL = Prog::VL, NG = Prog::NG, K = Prog::K, V = VL * NG;
+  constexpr int kAcc = K < kMaxRed ? K : kMaxRed;
+  const int tid = threadIdx.x, nthreads = blockDim.x;
+  const int TX = Prog::col_tx(p), TY = nthreads / TX;
+  const int tx = tid % TX, ty = tid / TX;
+  const int R = Prog::red_len(p);
+  const int n_ctiles = Prog::chunks(p);
+  const int n_red = Prog::n_red(p, 0);
+
+  long long rowoff[Prog::kNumIo];
+  float no_slots[1] = {0.f};
+  TileCtx cx;
+  cx.rowoff = rowoff;
+  cx.part = nullptr; cx.stash = nullptr;
+  cx.slots = no_slots;
+  cx.part_stride = nthreads;
+  cx.gstride = TX * VL;
+  cx.col_end = Prog::row_len(p);
+  cx.chunk = 0; cx.chunks = 1;
+  cx.leader = false;
+  float* stage = reinterpret_cast<float*>(smem + p.sm_part);
+
+  float acc[V];
+  float reg[K][V];
+  float raw[1][V];
+  float ts = 0.f;
+  Part parts[kMaxRed];
+  PN_UNROLL for (int e = 0; e < V; ++e) { acc[e] = 0.f; raw[0][e] = 0.f; }
+  PN_UNROLL for (int k = 0; k < K; ++k) { PN_UNROLL for (int e = 0; e < V; ++e) reg[k][e] = 0.f; }
+  PN_UNROLL for (int r = 0; r < kMaxRed; ++r) parts[r] = Part{0.f, 0.f, 0.f};
+
+  const long long n_items = p.rows * n_ctiles;
+  for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
+    const long long o = item / n_ctiles;
+    const int ct = (int)(item - o * n_ctiles);
+    cx.col0 = ct * (TX * V) + tx * VL;
+    PN_UNROLL for (int r = 0; r < kAcc; ++r) {
+      if (r < n_red) {
+        const float ident = red_identity(Prog::red_kind(p, 0, r)).a;
+        PN_UNROLL for (int e = 0; e < V; ++e) reg[r][e] = ident;
+      }
+    }
+#pragma unroll(Prog::kWalkUnroll)
+    for (int s = ty; s < R; s += TY) {
+      PN_UNROLL for (int q = 0; q < Prog::kNumIo; ++q) rowoff[q] = o * Prog::lead_stride(p, q, 2) + s * Prog::red_stride(p, q);
+      Prog::tile(p, 0, cx, acc, reg, ts, parts, raw, cx, false);
+    }
+    if (TY > 1) {
+      PN_UNROLL for (int r = 0; r < kAcc; ++r) {
+        if (r < n_red) { PN_UNROLL for (int e = 0; e < V; ++e) stage[(r * V + e) * nthreads + tid] = reg[r][e]; }
+      }
+      __syncthreads();
+      if (ty == 0) {
+        PN_UNROLL for (int r = 0; r < kAcc; ++r) {
+          if (r < n_red) {
+            const int kind = Prog::red_kind(p, 0, r);
+            PN_UNROLL for (int e = 0; e < V; ++e) {
+              const float* col = stage + (r * V + e) * nthreads + tx;
+              float v = col[0];
+              for (int y = 1; y < TY; ++y) v = accum_combine(kind, v, col[y * TX]);
+              reg[r][e] = v;
+            }
+          }
+        }
+      }
+    }
+    if (ty == 0) {
+      PN_UNROLL for (int q = 0; q < Prog::kNumIo; ++q) rowoff[q] = o * Prog::lead_stride(p, q, 2);
+      Prog::tile(p, 1, cx, acc, reg, ts, parts, raw, cx, false);
+    }
+    if (TY > 1) __syncthreads();   // the next item rewrites the staging area
+  }
 }
 
 }  // namespace pn

@@ -17,8 +17,10 @@ enum NodeOp : uint16_t {
   N_ADD = 32, N_SUB, N_MUL, N_DIV, N_MAX, N_MIN, N_GT, N_GE, N_LT, N_LE, N_EQ, N_NE,
   N_WHERE = 64, N_CLAMP, N_FMA,
   N_SUM = 96, N_MEAN, N_VAR, N_AMAX, N_AMIN, N_ARGMAX, N_ARGMIN, N_LOGSUMEXP,
+  N_SUM_DIM = 104, N_MEAN_DIM, N_AMAX_DIM, N_AMIN_DIM,   // over one leading dimension, attr[0] = dim
   N_SOFTMAX = 128, N_LOG_SOFTMAX, N_LAYER_NORM, N_RMS_NORM,
-  N_ROLL = 160, N_SLICE, N_VIEW   // index operators on leading dimensions
+  N_ROLL = 160, N_SLICE, N_VIEW,   // index operators on leading dimensions
+  N_CAT = 163                      // concatenation along attr[0]
 };
 
 constexpr uint32_t kImm0 = 0xFFFFFFFFu, kImm1 = 0xFFFFFFFEu;
@@ -52,6 +54,7 @@ inline int dtype_bytes(int dt) {
 }
 inline bool dtype_is_float(int dt) { return dt == kF32 || dt == kF16 || dt == kBF16; }
 inline bool is_reduction(uint16_t op) { return op >= N_SUM && op <= N_LOGSUMEXP; }
+inline bool is_dim_reduction(uint16_t op) { return op >= N_SUM_DIM && op <= N_AMIN_DIM; }
 inline bool is_composite(uint16_t op) { return op >= N_SOFTMAX && op <= N_RMS_NORM; }
 inline bool is_index_op(uint16_t op) { return op >= N_ROLL && op <= N_VIEW; }
 
@@ -68,6 +71,9 @@ struct DeviceModel {      // what the lowering needs to know about the GPU
 
 // Lower a whole graph into one fused launch.  Returns a pn_status value.
 int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPlan& out, std::string& err);
+
+// The same for a graph whose reductions run over a leading dimension (lower_col.cpp).
+int lower_column_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPlan& out, std::string& err);
 
 // Grid size of a planned launch given the SM count and its kernel's resident CTAs per SM.
 void size_grid(LaunchPlan& lp, int sms, int occ);

@@ -12,7 +12,8 @@ template <int VL, int NG, int K>
 __global__ void __launch_bounds__(VL * NG > 8 ? 256 : 512)
 fused_kernel(const __grid_constant__ KernelParams p) {
   extern __shared__ __align__(16) unsigned char smem[];
-  fused_body<Interp<VL, NG, K>>(p, smem);
+  if (p.family == FAM_COLUMN) column_body<Interp<VL, NG, K>>(p, smem);
+  else fused_body<Interp<VL, NG, K>>(p, smem);
 }
 
 template <int VL, int NG, int K>

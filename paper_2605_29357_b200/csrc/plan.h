@@ -71,6 +71,8 @@ enum Op : uint8_t {
   OP_SLD,     // acc = slot[a]
   OP_SST,     // slot[a] = acc
   OP_STOUT_I, // a = io: store the int32 bits held in acc as an integer (argmax / argmin)
+  // column kernels (reductions over a leading dimension)
+  OP_ACCUM,   // a = RedKind (sum / max / min), b = reg: reg = reg (op) acc, element by element
   OP_COUNT_
 };
 
@@ -88,7 +90,7 @@ enum RedKind : uint8_t {
   RED_MEANVAR      // a = count, b = mean, c = sum of squared deviations
 };
 
-enum Family : int32_t { FAM_POINTWISE = 0, FAM_WARP = 1, FAM_BLOCK = 2, FAM_CLUSTER = 3 };
+enum Family : int32_t { FAM_POINTWISE = 0, FAM_WARP = 1, FAM_BLOCK = 2, FAM_CLUSTER = 3, FAM_COLUMN = 4 };
 
 struct IoDesc {
   void* base;              // device pointer; filled in per run
@@ -103,6 +105,7 @@ struct IoDesc {
   int32_t map_dim[3];
   int32_t map_add[3];
   int32_t map_mod[3];
+  int64_t red_stride;      // column kernels: elements per step of the reduced dimension; 0 = broadcast
 };
 
 struct RedDesc {
@@ -132,6 +135,12 @@ struct KernelParams {
   int32_t split_chunks;    // pointwise graphs: every (row, chunk) is its own work item
   int32_t cluster;         // CTAs per cluster (1 unless FAM_CLUSTER)
   int32_t stash_floats;    // floats of parked tile values per CTA
+  // column kernels: the iteration space is [rows, red_len, row_len], reduced over the middle
+  // dimension.  A CTA is col_tx threads along the columns by blockDim.x / col_tx along the reduced
+  // dimension; stage 0 runs per (row, step, column tile) and ends in OP_ACCUM into tile registers
+  // 0 .. n_red-1, stage 1 runs once per (row, column tile) on the combined registers.
+  int32_t red_len;
+  int32_t col_tx;
   uint16_t pro_begin, pro_end;   // tile program run once per thread before the row loop: loads of
                                  // operands that are the same for every row (generated kernels only)
   // shared-memory layout, byte offsets into dynamic shared memory

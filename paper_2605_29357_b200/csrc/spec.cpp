@@ -169,6 +169,7 @@ bool emit_program(const KernelParams& P, int pc, int end, bool scalar, int vl, i
     else if (op == OP_FILL) s = "op_fill<" + V + ">(cx, " + B + ", " + regname(a) + ");";
     else if (op == OP_SPILL_TS) s = "*stash_ptr<" + V + ">(cx, " + B + ") = ts;";
     else if (op == OP_FILL_TS) s = "ts = *stash_ptr<" + V + ">(cx, " + B + ");";
+    else if (op == OP_ACCUM) s = "op_accum<" + V + ">(" + A + ", " + regname(b) + ", acc);";
     else if (op == OP_SLD) s = "op_splat<" + V + ">(acc, cx.slots[" + A + "]);";
     else if (op == OP_SST) s = std::string("op_sst<") + (reg_slots ? "true" : "false") + ">(cx, " + A + ", acc[0]);";
     else if (op == OP_END) continue;
@@ -181,18 +182,20 @@ bool emit_program(const KernelParams& P, int pc, int end, bool scalar, int vl, i
 // Name of the kernel generated for a plan: family, tile shape and a hash of the program and
 // its shape constants, so that profiler listings tell the kernels of different graphs apart.
 std::string kernel_name(const LaunchPlan& lp) {
-  static const char* fam[] = {"pointwise", "warp_row", "block_row", "cluster_row"};
+  static const char* fam[] = {"pointwise", "warp_row", "block_row", "cluster_row", "column_red"};
   uint64_t h = 1469598103934665603ull;
   auto mix = [&](uint64_t v) { for (int i = 0; i < 8; ++i) { h ^= (v >> (8 * i)) & 0xFF; h *= 1099511628211ull; } };
   for (int i = 0; i < lp.code_words; ++i) mix(lp.p.code[i]);
   mix((uint64_t)lp.p.row_len); mix((uint64_t)lp.p.rows); mix((uint64_t)lp.block); mix((uint64_t)lp.p.cluster);
+  mix((uint64_t)lp.p.red_len); mix((uint64_t)lp.p.col_tx);
   for (int q = 0; q < lp.p.n_io; ++q) {
     const IoDesc& io = lp.p.io[q];
-    mix(io.dtype); mix((uint64_t)io.col_stride); mix(io.mapped);
+    mix(io.dtype); mix((uint64_t)io.col_stride); mix(io.mapped); mix((uint64_t)io.red_stride);
     for (int i = 0; i < 3; ++i) { mix((uint64_t)io.lead_stride[i]); mix((uint64_t)io.map_dim[i]); mix((uint64_t)io.map_add[i]); mix((uint64_t)io.map_mod[i]); }
   }
   char b[96];
-  snprintf(b, sizeof(b), "pn_spec_%s_v%dx%d_%08x", fam[lp.family & 3], lp.vl, lp.ng, (unsigned)(h ^ (h >> 32)));
+  snprintf(b, sizeof(b), "pn_spec_%s_v%dx%d_%08x", fam[lp.family >= 0 && lp.family <= FAM_COLUMN ? lp.family : 0], lp.vl, lp.ng, (unsigned)(h ^ (h >> 32)));
+  static_assert(FAM_COLUMN == 4, "family names");
   return b;
 }
 
@@ -213,6 +216,10 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
     for (int i = 0; i < 3; ++i)
       if (P.io[q].lead_stride[i] != 0) s += "      case " + I(q * 3 + i) + ": return " + I(P.io[q].lead_stride[i]) + "ll;\n";
   s += "      default: return 0;\n    }\n  }\n";
+  s += "  static PN_DEV long long red_stride(const KernelParams&, int io) {\n    switch (io) {\n";
+  for (int q = 0; q < P.n_io; ++q) if (P.io[q].red_stride != 0) s += "      case " + I(q) + ": return " + I(P.io[q].red_stride) + "ll;\n";
+  s += "      default: return 0;\n    }\n  }\n";
+  s += "  static constexpr int kWalkUnroll = " + I(P.family == FAM_COLUMN ? 4 : 1) + ";\n";
   s += "  static PN_DEV bool io_mapped(const KernelParams&, int io) {\n    switch (io) {\n";
   for (int q = 0; q < P.n_io; ++q) if (P.io[q].mapped) s += "      case " + I(q) + ": return true;\n";
   s += "      default: return false;\n    }\n  }\n";
@@ -226,7 +233,7 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
     }
   s += "      default: return IoMap{1, 1, 1, 0, 0, 0, 0, 0, 0, 0, 0, 0};\n    }\n  }\n";
   // every group of every tile inside the row: no validity tests in the generated code
-  const int team_threads = P.family <= FAM_WARP ? 32 : lp.block;
+  const int team_threads = P.family == FAM_COLUMN ? P.col_tx : P.family <= FAM_WARP ? 32 : lp.block;
   const bool full = (long long)P.chunks * team_threads * lp.vl * lp.ng == P.slice_len &&
                     (long long)P.slice_len * P.cluster == P.row_len;
   const bool reg_slots = true;   // generated programs keep the per-row scalars in registers
@@ -235,6 +242,7 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
   };
   konst("family", P.family); konst("cluster", P.cluster); konst("chunks", P.chunks); konst("split_chunks", P.split_chunks);
   konst("row_len", P.row_len); konst("slice_len", P.slice_len); konst("n_stages", P.n_stages); konst("n_io", P.n_io);
+  konst("col_tx", P.col_tx); konst("red_len", P.red_len);
   auto table = [&](const char* name, const char* type, auto get) {
     s += std::string("  static PN_DEV ") + type + " " + name + "(const KernelParams&, int s, int r) {\n    switch (s * " + I(kMaxRed) + " + r) {\n";
     for (int st = 0; st < P.n_stages; ++st)
@@ -291,7 +299,7 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
   s += "#if PN_MIN_BLOCKS > 1\n#define PN_BOUNDS __launch_bounds__(" + I(lp.block) + ", PN_MIN_BLOCKS)\n#else\n"
        "#define PN_BOUNDS __launch_bounds__(" + I(lp.block) + ")\n#endif\n";
   s += "extern \"C\" __global__ void PN_BOUNDS " + kernel_name(lp) + "(const __grid_constant__ pn::KernelParams p) {\n"
-       "  extern __shared__ __align__(16) unsigned char smem[];\n  pn::fused_body<pn::Spec>(p, smem);\n}\n";
+       "  extern __shared__ __align__(16) unsigned char smem[];\n  pn::" + std::string(P.family == FAM_COLUMN ? "column_body" : "fused_body") + "<pn::Spec>(p, smem);\n}\n";
   src.swap(s);
   return true;
 }

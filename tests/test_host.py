@@ -216,3 +216,59 @@ def test_index_operator_errors():
     g.mark_output(g.op("roll", [s], D.F32, (4, 8), attr=[0, 1]))
     assert _status(g.build()) == -3
     assert _status(g.build(), PLAN | pn.FLAG_UNFUSED) == 0
+
+
+# ---- reductions over a leading dimension (the column-reduce family) ----------------------
+def _descriptor_only_n2(**kw):
+    import numpy as np
+    real_draw = C._draw
+    C._draw = lambda rng, kind, shape, a, b, chunk=0: np.zeros(shape, dtype=np.float32)
+    try:
+        return C.n2(**kw)
+    finally:
+        C._draw = real_draw
+
+
+def test_masked_mean_pooling_lowers_to_one_column_kernel():
+    w = _descriptor_only_n2()
+    g = pn.Graph(w.desc, 0, PLAN)
+    assert g.n_kernels == 1 and g.n_nodes == 7
+    k = g.kernel_info[0]
+    assert pn.FAMILY_NAMES[k["family"]] == "column-reduce" and k["stages"] == 2
+    assert k["rows"] == 256 and k["row_len"] == 1024 and k["vl"] == 8      # 128-bit loads of the bf16 hidden states
+    assert g.compulsory_bytes == 256 * 512 * 1024 * 2 + 256 * 512 * 8 + 256 * 1024 * 4
+    src = g.codegen(0, compile=True)
+    assert "pn::column_body<pn::Spec>" in src and src.count("op_accum<8>") == 2   # both sums in one walk
+    gu = pn.Graph(w.desc, 0, PLAN | pn.FLAG_UNFUSED)
+    assert gu.n_kernels == 7
+    for i in range(gu.n_kernels):
+        gu.codegen(i, compile=True)
+    # ragged and scalar-access shapes compile too
+    for kw in (dict(B=3, S=37, Dh=203), dict(B=2, S=9, Dh=64, dense_mask=True, mask_dtype=D.I8)):
+        pn.Graph(_descriptor_only_n2(**kw).desc, 0, PLAN).codegen(0, compile=True)
+
+
+def test_unsupported_column_forms_are_refused():
+    def status(g):
+        try:
+            pn.Graph(g.build(), 0, PLAN).close()
+            return 0
+        except pn.PnError as e:
+            return e.status
+    g = GraphBuilder(); x = g.input(D.F32, (4, 6, 8))
+    s = g.op("sum_dim", [x], D.F32, (4, 1, 8), attr=[1, 0])
+    g.mark_output(g.op("sub", [x, s], D.F32, (4, 6, 8)))             # needs a second pass over the dimension
+    assert status(g) == -3
+    g = GraphBuilder(); x = g.input(D.F32, (4, 6, 8))
+    g.mark_output(g.op("sum_dim", [x], D.F32, (4, 6), attr=[2, 0]))  # the last dimension has its own opcodes
+    assert status(g) == -3
+    g = GraphBuilder(); x = g.input(D.F32, (4, 6, 8))
+    g.mark_output(g.op("sum_dim", [x], D.F32, (4, 7), attr=[1, 0]))
+    assert status(g) == -4
+    g = GraphBuilder(); x = g.input(D.F32, (4, 6, 8))
+    g.mark_output(g.op("sum_dim", [x], D.F32, (4, 8), attr=[1, 0]))
+    g.mark_output(g.op("sum_dim", [x], D.F32, (6, 8), attr=[0, 0]))  # two different dimensions in one graph
+    assert status(g) == -3
+    g = GraphBuilder(); x = g.input(D.F32, (4, 6, 8)); y = g.input(D.F32, (4, 6, 8))
+    g.mark_output(g.op("cat", [x, y], D.F32, (4, 12, 8), attr=[1, 0]))   # a real concatenation is not lowered
+    assert status(g) == -3
