@@ -457,9 +457,50 @@ template <int VL, int NG>
 PN_DEV void op_widen(int dt, float (&r)[VL * NG]) {
   if (dt != kF32 && dt != kI64) { PN_UNROLL for (int j = 0; j < NG; ++j) widen_group<VL>(&r[j * VL], dt); }
 }
+PN_DEV float op_ldbc_scalar(const KernelParams& p, const TileCtx& cx, int io, int dt) {
+  return widen_scalar(static_cast<const char*>(p.io[io].base) + cx.rowoff[io] * dtype_size(dt), dt);
+}
+// The same load split in two, so that loads issued ahead of their use do not wait for their own
+// conversion: the storage bits of the element (two words for i64) ...
+template <int V>
+PN_DEV void op_ldbc_raw(const KernelParams& p, const TileCtx& cx, int io, int dt, float (&r)[V]) {
+  const char* a = static_cast<const char*>(p.io[io].base) + cx.rowoff[io] * dtype_size(dt);
+  uint32_t w0 = 0, w1 = 0;
+  switch (dt) {
+    case kF32: case kI32: w0 = __ldg(reinterpret_cast<const unsigned int*>(a)); break;
+    case kF16: case kBF16: w0 = __ldg(reinterpret_cast<const unsigned short*>(a)); break;
+    case kI8: case kBool: w0 = __ldg(reinterpret_cast<const unsigned char*>(a)); break;
+    default: { const uint2 v = __ldg(reinterpret_cast<const uint2*>(a)); w0 = v.x; w1 = v.y; break; }
+  }
+  r[0] = bits_f(w0);
+  if constexpr (V > 1) r[1] = bits_f(w1);
+}
+// ... and their conversion, splat over the tile
+template <int V>
+PN_DEV void op_ldbc_widen(int dt, float (&d)[V], const float (&r)[V]) {
+  const uint32_t w0 = f_bits(r[0]);
+  float v;
+  switch (dt) {
+    case kF32: v = bits_f(w0); break;
+    case kF16: v = half_to_float(w0); break;
+    case kBF16: v = bits_f(w0 << 16); break;
+    case kI8: v = static_cast<float>(static_cast<signed char>(w0)); break;
+    case kBool: v = w0 ? 1.f : 0.f; break;
+    case kI32: v = static_cast<float>(static_cast<int>(w0)); break;
+    default: {
+      uint32_t w1 = 0;
+      if constexpr (V > 1) w1 = f_bits(r[1]);
+      // values that fit 32 bits (masks, counts, indices: nearly always) convert in one instruction
+      if (static_cast<int>(w1) == (static_cast<int>(w0) >> 31)) v = static_cast<float>(static_cast<int>(w0));
+      else v = static_cast<float>(static_cast<long long>((static_cast<unsigned long long>(w1) << 32) | w0));
+      break;
+    }
+  }
+  PN_UNROLL for (int e = 0; e < V; ++e) d[e] = v;
+}
 template <int V>
 PN_DEV void op_ldbc(const KernelParams& p, const TileCtx& cx, int io, int dt, float (&r)[V]) {
-  const float v = widen_scalar(static_cast<const char*>(p.io[io].base) + cx.rowoff[io] * dtype_size(dt), dt);
+  const float v = op_ldbc_scalar(p, cx, io, dt);
   PN_UNROLL for (int e = 0; e < V; ++e) r[e] = v;
 }
 template <int V>
@@ -1072,13 +1113,16 @@ PN_DEV void column_body(const KernelParams& p, unsigned char* smem) {
   cx.leader = false;
   float* stage = reinterpret_cast<float*>(smem + p.sm_part);
 
+  constexpr int kPf = Prog::kNumPrefetch;            // loads at the head of the stage-0 program
+  constexpr int U = kPf > 0 ? Prog::kWalkUnroll : 1; // steps whose loads are in flight together
   float acc[V];
   float reg[K][V];
-  float raw[1][V];
+  float raw[U][kPf > 0 ? kPf : 1][V];
   float ts = 0.f;
   Part parts[kMaxRed];
-  PN_UNROLL for (int e = 0; e < V; ++e) { acc[e] = 0.f; raw[0][e] = 0.f; }
+  PN_UNROLL for (int e = 0; e < V; ++e) acc[e] = 0.f;
   PN_UNROLL for (int k = 0; k < K; ++k) { PN_UNROLL for (int e = 0; e < V; ++e) reg[k][e] = 0.f; }
+  PN_UNROLL for (int u = 0; u < U; ++u) { PN_UNROLL for (int j = 0; j < (kPf > 0 ? kPf : 1); ++j) { PN_UNROLL for (int e = 0; e < V; ++e) raw[u][j][e] = 0.f; } }
   PN_UNROLL for (int r = 0; r < kMaxRed; ++r) parts[r] = Part{0.f, 0.f, 0.f};
 
   const long long n_items = p.rows * n_ctiles;
@@ -1092,10 +1136,28 @@ PN_DEV void column_body(const KernelParams& p, unsigned char* smem) {
         PN_UNROLL for (int e = 0; e < V; ++e) reg[r][e] = ident;
       }
     }
-#pragma unroll(Prog::kWalkUnroll)
-    for (int s = ty; s < R; s += TY) {
+    auto at_step = [&](int s) {
       PN_UNROLL for (int q = 0; q < Prog::kNumIo; ++q) rowoff[q] = o * Prog::lead_stride(p, q, 2) + s * Prog::red_stride(p, q);
-      Prog::tile(p, 0, cx, acc, reg, ts, parts, raw, cx, false);
+    };
+    if constexpr (kPf > 0) {
+      // U steps at a time: all their loads are issued, then their arithmetic runs in step order.
+      // (Measured on B200: issuing the next batch before the arithmetic of the current one costs
+      // more in registers, hence resident warps, than it gains.)
+      for (int s0 = ty; s0 < R; s0 += U * TY) {
+        PN_UNROLL for (int u = 0; u < U; ++u) {
+          const int s = s0 + u * TY;
+          if (s < R) { at_step(s); Prog::prefetch(p, cx, raw[u]); }
+        }
+        PN_UNROLL for (int u = 0; u < U; ++u) {
+          const int s = s0 + u * TY;
+          if (s < R) { at_step(s); Prog::tile(p, 0, cx, acc, reg, ts, parts, raw[u], cx, false); }
+        }
+      }
+    } else {
+      for (int s = ty; s < R; s += TY) {
+        at_step(s);
+        Prog::tile(p, 0, cx, acc, reg, ts, parts, raw[0], cx, false);
+      }
     }
     if (TY > 1) {
       PN_UNROLL for (int r = 0; r < kAcc; ++r) {
@@ -1118,7 +1180,7 @@ PN_DEV void column_body(const KernelParams& p, unsigned char* smem) {
     }
     if (ty == 0) {
       PN_UNROLL for (int q = 0; q < Prog::kNumIo; ++q) rowoff[q] = o * Prog::lead_stride(p, q, 2);
-      Prog::tile(p, 1, cx, acc, reg, ts, parts, raw, cx, false);
+      Prog::tile(p, 1, cx, acc, reg, ts, parts, raw[0], cx, false);
     }
     if (TY > 1) __syncthreads();   // the next item rewrites the staging area
   }

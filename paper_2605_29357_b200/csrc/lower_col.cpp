@@ -298,9 +298,11 @@ int lower_column_graph(const Graph& g, unsigned flags, const DeviceModel& dev, L
   int NG = VL == 8 ? 1 : (VL == 4 ? 2 : 8), K = 4;
   if (spec) { NG = VL == 1 ? 4 : 1; K = kSpecRegs; }
   const int t_ng = (flags >> 24) & 31;
-  if (spec && t_ng && (t_ng & (t_ng - 1)) == 0 && VL * t_ng <= 32) NG = t_ng;
+  if (spec && t_ng && (t_ng & (t_ng - 1)) == 0 && VL * t_ng <= 32 && VL * t_ng >= 2) NG = t_ng;   // (an i64 element in flight takes two tile slots)
   if ((int)reds.size() > K - 2) { err = "more reductions than the kernel has tile registers for"; return PN_ERR_TOO_LARGE; }
-  int block = 256;
+  // generated kernels: 128 threads (4 walkers of a warp-wide column tile each), measured best on
+  // B200 with the register bound that keeps 1024 threads resident per SM
+  int block = spec ? 128 : 256;
   const int t_block = ((flags >> 20) & 15) ? 1 << ((flags >> 20) & 15) : 0;
   if (t_block >= 32 && t_block <= (spec ? 1024 : 256)) block = t_block;
   // threads along the columns: enough to cover C, at most a warp (a warp then reads 32 x 16
@@ -320,7 +322,7 @@ int lower_column_graph(const Graph& g, unsigned flags, const DeviceModel& dev, L
   memset(stages, 0, sizeof(stages));
   for (int s = 0; s < 2; ++s) {
     stages[s].elem_begin = (uint16_t)code.size();
-    ge.hoist_loads(ex.ops, s);
+    ge.hoist_loads(ex.ops, s, true);
     for (const MOp& m : ex.ops) {
       if (m.stage != s) continue;
       if (m.scalar) { err = "internal: scalar operation in a column kernel"; return PN_ERR_UNSUPPORTED_OP; }
@@ -353,7 +355,8 @@ int lower_column_graph(const Graph& g, unsigned flags, const DeviceModel& dev, L
   lp.block = block; lp.smem_bytes = off; lp.code_words = (int)code.size();
   lp.items = O * n_ctiles;
   lp.teams_per_cta = 1;
-  lp.specialised = 0; lp.persistent = 0; lp.no_prefetch = 1;
+  // generated kernels issue the loads of several steps of the walk before the arithmetic of the first
+  lp.specialised = 0; lp.persistent = 0; lp.no_prefetch = (flags & PN_FLAG_NO_HOIST) ? 1 : 0;
   const int occ = (dev.have_device && !spec) ? instance_occupancy(VL, NG, K, block, off) : 0;
   size_grid(lp, dev.sm_count, occ);
   return PN_OK;

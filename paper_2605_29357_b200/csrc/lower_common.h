@@ -286,20 +286,22 @@ struct Gen {
 
   // Issue the loads of this stage's inputs before any arithmetic, so that they are all in
   // flight together; the large (streamed) operands first.
-  void hoist_loads(const std::vector<MOp>& ops, int stage) {
+  // also_bcast: the one-element loads of last-dim-broadcast operands are issued there too.
+  void hoist_loads(const std::vector<MOp>& ops, int stage, bool also_bcast = false) {
     if (scalar) return;
-    for (int pass = 0; pass < 2; ++pass)
+    for (int pass = 0; pass < (also_bcast ? 3 : 2); ++pass)
       for (const MOp& m : ops) {
         if (m.stage != stage || m.scalar) continue;
         for (int i = 0; i < m.nin; ++i) {
           const int v = m.in[i];
-          if (v < 0 || vals[v].kind != VK_E || vals[v].io < 0 || vals[v].bcast) continue;
-          if (vals[v].streamed != (pass == 0)) continue;
+          if (v < 0 || vals[v].kind != VK_E || vals[v].io < 0) continue;
+          if (vals[v].bcast != (pass == 2)) continue;
+          if (pass < 2 && vals[v].streamed != (pass == 0)) continue;
           if (find_reg(v) >= 0 || accv == v || stash_of.count(v)) continue;
           if (n_free() <= 1) return;
           const int k = free_reg();
-          emit(OP_LDRAW, vals[v].io, k);
-          regv[k] = v; regraw[k] = 1;
+          if (pass == 2) { emit(OP_LDBC, vals[v].io, k); regv[k] = v; regraw[k] = 0; }
+          else { emit(OP_LDRAW, vals[v].io, k); regv[k] = v; regraw[k] = 1; }
         }
       }
   }

@@ -125,9 +125,11 @@ bool emit_program(const KernelParams& P, int pc, int end, bool scalar, int vl, i
   const std::string VLNGF = VLNG + (full ? ", true" : ", false");
   for (int j = 0; j < n_prefetch; ++j) {
     const uint32_t w = P.code[pc++];
-    out += "        op_mov<" + V + ">(" + regname((w >> 16) & 0xFF) + ", raw[" + std::to_string(j) + "]);\n";
+    if ((w & 0xFF) == OP_LDBC) out += "        op_ldbc_widen<" + V + ">(" + std::to_string((int)P.io[(w >> 8) & 0xFF].dtype) + ", " + regname((w >> 16) & 0xFF) + ", raw[" + std::to_string(j) + "]);\n";
+    else out += "        op_mov<" + V + ">(" + regname((w >> 16) & 0xFF) + ", raw[" + std::to_string(j) + "]);\n";
   }
-  if (n_prefetch > 0) out += "        if (has_next) prefetch(p, nx, raw);\n";
+  // row kernels fetch the next tile here; column kernels batch the loads of several steps themselves
+  if (n_prefetch > 0 && P.family != FAM_COLUMN) out += "        if (has_next) prefetch(p, nx, raw);\n";
   while (pc < end) {
     const uint32_t w = P.code[pc++];
     const int op = w & 0xFF, a = (w >> 8) & 0xFF, b = (w >> 16) & 0xFF, c = w >> 24;
@@ -219,7 +221,7 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
   s += "  static PN_DEV long long red_stride(const KernelParams&, int io) {\n    switch (io) {\n";
   for (int q = 0; q < P.n_io; ++q) if (P.io[q].red_stride != 0) s += "      case " + I(q) + ": return " + I(P.io[q].red_stride) + "ll;\n";
   s += "      default: return 0;\n    }\n  }\n";
-  s += "  static constexpr int kWalkUnroll = " + I(P.family == FAM_COLUMN ? 4 : 1) + ";\n";
+  s += "#ifndef PN_WALK_UNROLL\n#define PN_WALK_UNROLL " + I(P.family == FAM_COLUMN ? 4 : 1) + "\n#endif\n  static constexpr int kWalkUnroll = PN_WALK_UNROLL;\n";
   s += "  static PN_DEV bool io_mapped(const KernelParams&, int io) {\n    switch (io) {\n";
   for (int q = 0; q < P.n_io; ++q) if (P.io[q].mapped) s += "      case " + I(q) + ": return true;\n";
   s += "      default: return false;\n    }\n  }\n";
@@ -264,14 +266,18 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
   s += "  }\n";
   // the loads at the head of stage 0 are issued one tile ahead of their use
   int n_pf = 0;
-  for (int pc = P.stage[0].elem_begin; pc < P.stage[0].elem_end && (P.code[pc] & 0xFF) == OP_LDRAW; ++pc) n_pf++;
+  for (int pc = P.stage[0].elem_begin; pc < P.stage[0].elem_end; ++pc) {
+    const int op = P.code[pc] & 0xFF;
+    if (op == OP_LDRAW || (op == OP_LDBC && P.family == FAM_COLUMN)) n_pf++; else break;
+  }
   if (lp.no_prefetch) n_pf = 0;
   s += "  static constexpr int kNumPrefetch = " + I(n_pf) + ";\n";
   s += "  static PN_DEV void prefetch(const KernelParams& p, const TileCtx& cx, float (&raw)[" + I(n_pf > 0 ? n_pf : 1) + "][" + V + "]) {\n";
   for (int j = 0; j < n_pf; ++j) {
     const uint32_t w = P.code[P.stage[0].elem_begin + j];
     const int io = (w >> 8) & 0xFF;
-    s += "    op_ldraw<" + I(lp.vl) + ", " + I(lp.ng) + (full ? ", true" : ", false") + ">(p, cx, " + I(io) + ", " + I(P.io[io].dtype) + ", raw[" + I(j) + "]);\n";
+    if ((w & 0xFF) == OP_LDBC) s += "    op_ldbc_raw<" + V + ">(p, cx, " + I(io) + ", " + I(P.io[io].dtype) + ", raw[" + I(j) + "]);\n";
+    else s += "    op_ldraw<" + I(lp.vl) + ", " + I(lp.ng) + (full ? ", true" : ", false") + ">(p, cx, " + I(io) + ", " + I(P.io[io].dtype) + ", raw[" + I(j) + "]);\n";
   }
   s += "  }\n";
   s += "  static PN_DEV void tile(const KernelParams& p, int s, const TileCtx& cx, float (&acc)[" + V + "], float (&reg)[" + I(lp.k) + "][" + V + "], float& ts, Part (&parts)[" + I(kMaxRed) + "],\n"
@@ -294,7 +300,10 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
   // for 1024 resident threads per SM, since resident warps are what hides the HBM latency
   // (measured: +5 % on the LayerNorm workload).  Streaming kernels need no hint: they are
   // small already, and a bound would only license more registers.
-  const int min_blocks = (P.family == FAM_BLOCK && P.chunks == 1) ? std::max(1, 1024 / lp.block) : 1;
+  // Column kernels likewise: their walk keeps several steps of loads in flight per thread, and the
+  // bound keeps that from eating the resident warps (measured: 64 registers with 4 steps in flight
+  // beats every larger budget on the pooling workload).
+  const int min_blocks = ((P.family == FAM_BLOCK && P.chunks == 1) || P.family == FAM_COLUMN) ? std::max(1, 1024 / lp.block) : 1;
   s += "#ifndef PN_MIN_BLOCKS\n#define PN_MIN_BLOCKS " + I(min_blocks) + "\n#endif\n";
   s += "#if PN_MIN_BLOCKS > 1\n#define PN_BOUNDS __launch_bounds__(" + I(lp.block) + ", PN_MIN_BLOCKS)\n#else\n"
        "#define PN_BOUNDS __launch_bounds__(" + I(lp.block) + ")\n#endif\n";
