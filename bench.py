@@ -182,6 +182,52 @@ def time_graph_replay(torch, g, sets, steps, warmup):
     return e0.elapsed_time(e1) / (reps * len(ptrs))
 
 
+def tiny_graph_latency(torch, pn, device, passes, repeats=8):
+    """Latency of many small subgraphs run back to back (the regime where the paper finds fixed
+    per-call overhead decisive): the reduced-size graphs of every workload, `repeats` instances
+    each on their own buffers, (a) launched one by one from the host with pn_graph_run,
+    (b) recorded once as a sequence and replayed in order, (c) the same as independent items.
+    Returns microseconds per subgraph for each; the inputs are L2-resident, so this is launch
+    and latency, not bandwidth."""
+    makers = {**C.CONFIGS, **C.EXTENDED}
+    graphs, items, keep = {}, [], []
+    for rep in range(repeats):
+        for name, make in makers.items():
+            w = make(seed=rep, **C.SMALL[name])
+            if name not in graphs:
+                graphs[name] = pn.Graph(w.desc, device, 0)
+            (d_in, d_out), = device_sets(torch, w, 1)
+            keep.append((d_in, d_out))
+            items.append((graphs[name], [t.data_ptr() for t in d_in], [t.data_ptr() for t in d_out]))
+    stream = torch.cuda.current_stream()
+
+    def timed(run_pass):
+        for _ in range(3):
+            run_pass()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(passes):
+            run_pass()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / (passes * len(items))
+
+    def host_pass():
+        for g, i, o in items:
+            g.run(i, o, stream.cuda_stream)
+
+    out = {"subgraphs": len(items), "distinct_graphs": len(graphs), "kernels_per_pass": sum(g.n_kernels for g, _, _ in items),
+           "host_launched_us_per_subgraph": timed(host_pass)}
+    for key, indep in (("sequence_us_per_subgraph", False), ("sequence_independent_us_per_subgraph", True)):
+        seq = pn.Sequence(items, independent=indep)
+        out[key] = timed(lambda: seq.run(stream.cuda_stream))
+        seq.close()
+    for g in graphs.values():
+        g.close()
+    return out
+
+
 def rank_workload(name, rank, **size):
     """The batch rank `rank` works on: the same graph and shapes on every rank, inputs drawn
     from the rank's own seed.  Rows are independent, so sharding a larger job by rows needs no
@@ -409,6 +455,7 @@ def main():
             del si
             torch.cuda.empty_cache()
         line["sweep"] = sweep
+        line["tiny_graphs"] = tiny_graph_latency(torch, pn, local_rank, max(10, args.steps // 2))
 
     # ---- the CPU oracle on a bounded sample of the same workload ------------------------------
     sample = oracle_sample(32)

@@ -2,9 +2,9 @@
  * pn.h -- C ABI of the fused-subgraph executor for NVIDIA B200 (sm_100a).
  *
  * The library runs a "long-tail fusible subgraph" -- a DAG of pointwise operators
- * with broadcasting, optional reductions over the last dimension, and a
- * normalisation / scaling epilogue -- as ONE pass over HBM instead of one kernel
- * per operator.  The input is the paper's computational graph G = (V, E, tau, sigma)
+ * with broadcasting, optional reductions (over the last dimension, or over one leading
+ * dimension), and a normalisation / scaling epilogue -- as ONE pass over HBM instead of
+ * one kernel per operator.  The input is the paper's computational graph G = (V, E, tau, sigma)
  * (Definition 3.1: operator nodes, data dependencies, an operator type per node and a
  * static output shape per node), serialised as a descriptor.  What a handle computes
  * is f_G; a fused execution is acceptable when it equals the per-operator evaluation
@@ -38,6 +38,18 @@
  * 102 argmin (lowest index on ties; i32 / i64 result), 103 logsumexp; 128 softmax,
  * 129 log_softmax, 130 layer_norm(x[, gamma[, beta]]) -> y[, mean, rstd] with
  * imm[0] = eps, 131 rms_norm(x[, gamma]) with imm[0] = eps.
+ * Reductions over ONE LEADING dimension (the masked-mean-pooling shape of the paper's second
+ * case study, Section 4.4): 104 sum_dim, 105 mean_dim, 106 amax_dim, 107 amin_dim with
+ * attr[0] = the reduced dimension (not the last one); the result has the operand's shape with
+ * that dimension dropped or kept as 1.  A graph may hold several of them over the same
+ * dimension, a pointwise chain before them and one after them on the reduced values; a reduced
+ * value cannot flow back into a tensor that still has the reduced dimension.
+ * Index operators (the index-remapped loads of the paper's first case study, Section 4.4): 160
+ * roll (attr = dim, shift), 161 slice (attr = dim, start; length from the output shape), 162 view
+ * (regroups leading dimensions).  They act on leading dimensions of graph inputs, or of chains of
+ * index operators that start at one, and cost no data movement: the fused kernel computes the
+ * source row instead (idx = (S + i - shift) mod S).  163 cat (attr[0] = dim): with one operand it
+ * is the identity, as graph traces contain it; several operands are not lowered.
  * Arithmetic is fp32 in registers whatever the storage types; integer and boolean
  * tensors take part as exact small integers / predicates; a node whose declared
  * output dtype is bf16 / f16 is rounded to it (nearest even) for its consumers.
@@ -107,7 +119,9 @@ enum {
   PN_Q_N_NODES = 7,         /* 1 value: operator nodes in the descriptor                 */
   PN_Q_WORKSPACE_BYTES = 8, /* 1 value: device memory owned by the handle                */
   PN_Q_KERNEL_INFO = 9      /* per kernel 13 values: family (0 pointwise, 1 warp-per-row,
-                               2 block-per-row, 3 cluster-per-row), grid, block, cluster,
+                               2 block-per-row, 3 cluster-per-row, 4 column-reduce: rows =
+                               the dimensions before the reduced one, row length = those after
+                               it), grid, block, cluster,
                                dynamic smem bytes, vector length, groups per tile, chunks
                                per row slice, bytecode words, stages, rows, row length,
                                specialised (1) or interpreted (0)                        */
@@ -190,6 +204,52 @@ pn_status pn_graph_run_host(pn_graph_t* g, const void* const* inputs, int n_inpu
  */
 pn_status pn_graph_run_static(pn_graph_t* g, const void* const* inputs, int n_inputs,
                               void* const* outputs, int n_outputs, void* stream);
+
+/*
+ * Sequences: many small evaluations replayed with one call.
+ *
+ * The paper traces 61.5 % of the end-to-end slowdowns it measures under a graph compiler to
+ * fixed per-call overhead on graphs of fewer than 15 nodes: about 0.14 ms of dispatch per call
+ * while the kernels themselves got faster (Table 6, root-cause decomposition).  A fused kernel
+ * of a few microseconds meets the same kind of cost in the host's launch path.  A sequence
+ * pays it once: pn_sequence_create runs the pointer checks and records the launches of all its
+ * items into a CUDA graph; pn_sequence_run replays them with a single launch call, the kernels
+ * running back to back on the GPU.
+ *
+ * pn_sequence_create
+ *   n                : number of items (> 0).
+ *   graphs           : HOST array of n handles, all bound to one device; a handle may appear
+ *                      several times.  The handles must outlive the sequence.
+ *   inputs, outputs  : HOST arrays of n pointers to HOST arrays of DEVICE pointers, per item
+ *                      as for pn_graph_run; n_inputs / n_outputs give their lengths.  The
+ *                      device pointers are recorded: the sequence reads and writes exactly
+ *                      those buffers at every run; the caller keeps them alive.
+ *   flags            : 0: the items run in order, each after the one before (outputs of one
+ *                      may be inputs of the next).  PN_SEQ_INDEPENDENT: the caller states that
+ *                      no item reads or writes what another writes; items are then recorded on
+ *                      parallel branches and small kernels may overlap on the GPU.
+ *   out              : receives the sequence; NULL on failure.
+ * Creates streams and events for the recording and releases them before it returns; allocates
+ * no device memory of its own.  Errors: those of pn_graph_run for any item (the message names
+ * the item); PN_ERR_DEVICE for handles of different devices; PN_ERR_INVALID_ARG for a
+ * PN_FLAG_STATIC_SCRATCH handle, or for an unfused handle that appears twice in an
+ * independent sequence (its runs share one workspace).
+ *
+ * pn_sequence_run -- enqueue one replay on `stream` (a cudaStream_t); asynchronous.  Replays of
+ * one sequence, and a replay and a direct run of an unfused handle it contains, must be
+ * stream-ordered by the caller.
+ * pn_sequence_query -- PN_SQ_N_ITEMS / PN_SQ_N_KERNELS: one int64 into `out` (HOST memory).
+ * pn_sequence_destroy -- release the sequence (not its handles); NULL is accepted.
+ */
+typedef struct pn_sequence pn_sequence_t;
+enum { PN_SEQ_INDEPENDENT = 1u << 0 };
+enum { PN_SQ_N_ITEMS = 1, PN_SQ_N_KERNELS = 2 };
+pn_status pn_sequence_create(int n, pn_graph_t* const* graphs, const void* const* const* inputs,
+                             const int* n_inputs, void* const* const* outputs, const int* n_outputs,
+                             unsigned flags, pn_sequence_t** out);
+pn_status pn_sequence_run(pn_sequence_t* s, void* stream);
+pn_status pn_sequence_query(const pn_sequence_t* s, int what, void* out, size_t out_bytes);
+pn_status pn_sequence_destroy(pn_sequence_t* s);
 
 /* pn_graph_destroy -- release the handle and what it owns; NULL is accepted. */
 pn_status pn_graph_destroy(pn_graph_t* g);

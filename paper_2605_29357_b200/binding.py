@@ -39,7 +39,9 @@ Q_N_KERNELS, Q_N_NODES, Q_WORKSPACE_BYTES, Q_KERNEL_INFO = 6, 7, 8, 9
 
 FAMILY_NAMES = {0: "pointwise", 1: "warp-per-row", 2: "block-per-row", 3: "cluster-per-row", 4: "column-reduce"}
 EXPORTS = ["pn_graph_create", "pn_graph_run", "pn_graph_run_host", "pn_graph_run_static", "pn_graph_destroy",
-           "pn_graph_query", "pn_graph_codegen", "pn_status_string", "pn_last_error"]
+           "pn_graph_query", "pn_graph_codegen", "pn_status_string", "pn_last_error",
+           "pn_sequence_create", "pn_sequence_run", "pn_sequence_query", "pn_sequence_destroy"]
+SEQ_INDEPENDENT = 1 << 0
 
 
 class PnError(RuntimeError):
@@ -77,6 +79,15 @@ def load_library() -> ctypes.CDLL:
     lib.pn_graph_codegen.restype = ctypes.c_int
     lib.pn_graph_codegen.argtypes = [vp, ctypes.c_int, ctypes.c_int, ctypes.c_char_p, ctypes.c_size_t,
                                      ctypes.POINTER(ctypes.c_size_t)]
+    lib.pn_sequence_create.restype = ctypes.c_int
+    lib.pn_sequence_create.argtypes = [ctypes.c_int, vpp, ctypes.POINTER(vpp), ctypes.POINTER(ctypes.c_int),
+                                       ctypes.POINTER(vpp), ctypes.POINTER(ctypes.c_int), ctypes.c_uint, vpp]
+    lib.pn_sequence_run.restype = ctypes.c_int
+    lib.pn_sequence_run.argtypes = [vp, vp]
+    lib.pn_sequence_query.restype = ctypes.c_int
+    lib.pn_sequence_query.argtypes = [vp, ctypes.c_int, vp, ctypes.c_size_t]
+    lib.pn_sequence_destroy.restype = ctypes.c_int
+    lib.pn_sequence_destroy.argtypes = [vp]
     lib.pn_status_string.restype = ctypes.c_char_p
     lib.pn_status_string.argtypes = [ctypes.c_int]
     lib.pn_last_error.restype = ctypes.c_char_p
@@ -181,6 +192,57 @@ class Graph:
     def close(self) -> None:
         if getattr(self, "_h", None) is not None and self._h:
             self._lib.pn_graph_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class Sequence:
+    """pn_sequence_t: n (graph, input pointers, output pointers) items recorded once and replayed
+    with one call.  ``items`` is a list of (Graph, [input device pointers], [output device
+    pointers]); with ``independent=True`` the caller states that no item touches what another
+    writes, and the items may overlap on the GPU."""
+
+    def __init__(self, items, independent: bool = False):
+        self._lib = load_library()
+        self._h = ctypes.c_void_p()
+        self._graphs = [g for g, _, _ in items]          # the handles must outlive the sequence
+        n = len(items)
+        vpp = ctypes.POINTER(ctypes.c_void_p)
+        gh = (ctypes.c_void_p * max(n, 1))(*[g._h for g, _, _ in items])
+        ins = [Graph._ptr_array(i) for _, i, _ in items]
+        outs = [Graph._ptr_array(o) for _, _, o in items]
+        in_pp = (vpp * max(n, 1))(*[ctypes.cast(a, vpp) for a in ins])
+        out_pp = (vpp * max(n, 1))(*[ctypes.cast(a, vpp) for a in outs])
+        n_in = (ctypes.c_int * max(n, 1))(*[len(i) for _, i, _ in items])
+        n_out = (ctypes.c_int * max(n, 1))(*[len(o) for _, _, o in items])
+        _check(self._lib.pn_sequence_create(n, gh, in_pp, n_in, out_pp, n_out,
+                                            SEQ_INDEPENDENT if independent else 0, ctypes.byref(self._h)),
+               "pn_sequence_create")
+
+    def _query(self, what: int) -> int:
+        v = ctypes.c_int64()
+        _check(self._lib.pn_sequence_query(self._h, what, ctypes.byref(v), 8), "pn_sequence_query")
+        return int(v.value)
+
+    @property
+    def n_items(self) -> int:
+        return self._query(1)
+
+    @property
+    def n_kernels(self) -> int:
+        return self._query(2)
+
+    def run(self, stream: int = 0) -> None:
+        _check(self._lib.pn_sequence_run(self._h, ctypes.c_void_p(stream)), "pn_sequence_run")
+
+    def close(self) -> None:
+        if getattr(self, "_h", None) is not None and self._h:
+            self._lib.pn_sequence_destroy(self._h)
             self._h = ctypes.c_void_p()
 
     def __del__(self):

@@ -16,11 +16,11 @@ cudaError_t launch_plan(const LaunchPlan& lp, cudaStream_t stream);   // kernels
 
 using namespace pn;
 
-namespace {
+// The scratch itself, at file scope.  Every GPU that loads the library holds these bytes until
+// the process exits, whether or not the entry point is ever called.
+static __device__ __align__(256) unsigned char g_static_scratch[PN_STATIC_SCRATCH_BYTES];
 
-// The scratch itself.  Every GPU that loads the library holds these bytes until the process
-// exits, whether or not the entry point is ever called.
-__device__ __align__(256) unsigned char g_static_scratch[PN_STATIC_SCRATCH_BYTES];
+namespace {
 
 // In host code the name above is only a stand-in for the symbol: its address as a device
 // pointer has to be asked for, once per device, with that device current.
