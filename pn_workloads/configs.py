@@ -188,17 +188,19 @@ def c3(M: int = 16384, N: int = 4096, seed: int = 0, dtype: int = D.BF16, eps: f
 # C4: long-row reduction: logsumexp (f32) and argmax (i64)
 # ---------------------------------------------------------------------------
 def c4(M: int = 64, N: int = 262144, seed: int = 0, spike_p: float = 0.01,
-       spike: float = 30.0) -> Workload:
+       spike: float = 30.0, dtype: int = D.F32) -> Workload:
     g = GraphBuilder()
-    x = g.input(D.F32, (M, N))
-    lse = g.op("logsumexp", [x], D.F32, (M,))
-    idx = g.op("argmax", [x], D.I64, (M,))
+    x = g.input(dtype, (M, N))
+    xf = g.op("cast", [x], D.F32, (M, N)) if dtype != D.F32 else x
+    lse = g.op("logsumexp", [xf], D.F32, (M,))
+    idx = g.op("argmax", [xf], D.I64, (M,))
     g.mark_output(lse); g.mark_output(idx)
     rng = _rng(seed, 4, 0)
     xs = _draw(rng, "normal", (M, N), 0.0, 2.0)          # variance 4
     hit = _draw(rng, "uniform", (M, N), 0.0, 1.0) < spike_p
     xs[hit] = np.float32(spike)
     per_row = hit.sum(axis=1)
+    xs = _store(xs, dtype)
     return _finish("c4_long_row_reduction", g, ["x"], ["logsumexp", "argmax"], [xs],
                    {"spikes_per_row_min": int(per_row.min()), "spike": spike})
 
