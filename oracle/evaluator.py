@@ -24,8 +24,8 @@ final rounding is judged against the exact value.
 
 Operator definitions follow the usual closed forms; the LayerNorm form (biased
 variance, 1/sqrt(var + eps), (x - mean) * rstd * gamma + beta) is the one the
-paper's fused add+LayerNorm kernel computes (Appendix G, case 1); its
-masked-mean-pooling pattern (Appendix G, case 2: cast, mul, two sums over the
+paper's fused add+LayerNorm kernel computes (Appendix H, case 1); its
+masked-mean-pooling pattern (Appendix H, case 2: cast, mul, two sums over the
 sequence dimension, clamp, div, a one-operand cat) is evaluated operator by
 operator with the reductions over a leading dimension below.
 
@@ -323,7 +323,7 @@ def red_over_dim(kind: str, x, dim: int):
     """Reduction over one dimension `dim` of x, that dimension dropped from the result:
     sum_k x[.., k, ..]; mean = that sum / D; amax / amin = the extreme (a NaN along the
     dimension makes the result NaN).  This is what the paper's masked-mean-pooling pattern
-    uses twice (Appendix G, case 2: sum(hidden * mask, 1) and sum(mask, 1) over the sequence
+    uses twice (Appendix H, case 2: sum(hidden * mask, 1) and sum(mask, 1) over the sequence
     dimension of [B, S, D] tensors)."""
     x = _f(x)
     if not 0 <= dim < x.ndim:

@@ -1,5 +1,5 @@
 // lower_col.cpp -- host lowering of graphs whose reductions run over a leading dimension
-// (the masked-mean-pooling shape of the paper's second case study, Section 4.4 and Appendix G:
+// (the masked-mean-pooling shape of the paper's second case study, Section 4.4 and Appendix H:
 // two sums over the sequence dimension of [B, S, D] tensors, then a clamped division on
 // [B, D]).
 //

@@ -1,5 +1,5 @@
 """GPU parity of the reductions over a leading dimension (the masked-mean-pooling shape of the
-paper's second case study, Section 4.4 / Appendix G case 2) against the CPU oracle, through the
+paper's second case study, Section 4.4 / Appendix H case 2) against the CPU oracle, through the
 C ABI: each reduction alone over ranks, dimensions and ragged sizes; graphs with values before
 and after the reduction; the pooling subgraph at reduced and full size, fused and unfused, on
 generated kernels and on the interpreter."""

@@ -189,7 +189,7 @@ def test_composites(n, dtype, mode):
 def test_user_written_two_stage_softmax_and_scalar_arithmetic(mode):
     """Reductions feeding later stages by hand: m = amax(x); e = exp(x - m); y = e / sum(e),
     with per-row scalar arithmetic in between, and the clamped divide of the paper's masked
-    mean pooling kernel (Appendix G, case 2) on per-row values."""
+    mean pooling kernel (Appendix H, case 2) on per-row values."""
     rows, n = 9, 1536
     x = rnd((rows, n), 17, 2.0); msk = (np.random.default_rng(18).random((rows, n)) < 0.3).astype(np.float32)
     msk[4, :] = 0                                        # empty mask row: the clamp decides

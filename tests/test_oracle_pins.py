@@ -468,7 +468,7 @@ def test_tolerance_rule_matches_the_papers_ladder():
 # index operators: roll + slice as the paper's index arithmetic
 # ---------------------------------------------------------------------------
 def test_roll_slice_view_match_the_papers_index_formula():
-    """Section 4.4 / Appendix G, case 1: roll(shift) followed by slice[:SC] on an [S, S, C] tensor
+    """Section 4.4 / Appendix H, case 1: roll(shift) followed by slice[:SC] on an [S, S, C] tensor
     equals reading row (S + i - shift) mod S, column (S + j - shift) mod S."""
     S, SC, Cc, shift = 7, 5, 4, 3
     rng = np.random.default_rng(9)
@@ -560,7 +560,7 @@ def test_cat_of_one_operand_is_the_identity_and_of_two_is_stacking():
 
 @pytest.mark.parametrize("dense_mask,mask_dtype", [(False, D.I64), (True, D.F32), (True, D.I8)])
 def test_n2_masked_mean_pooling_restated(dense_mask, mask_dtype):
-    """Appendix G, case 2: out[b, d] = sum_s(hidden * mask) / max(sum_s(mask), 1e-9)."""
+    """Appendix H, case 2: out[b, d] = sum_s(hidden * mask) / max(sum_s(mask), 1e-9)."""
     w = C.n2(B=3, S=9, Dh=5, dense_mask=dense_mask, mask_dtype=mask_dtype)
     mask, hidden = w.inputs
     h = _bf(hidden)
