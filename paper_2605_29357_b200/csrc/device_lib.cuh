@@ -561,6 +561,10 @@ PN_DEV void op_accum(int kind, float (&r)[V], const float (&acc)[V]) {
   PN_UNROLL for (int e = 0; e < V; ++e) r[e] = accum_combine(kind, r[e], acc[e]);
 }
 
+// the same for a value held identically in every element: one element carries the reduction
+template <int V>
+PN_DEV void op_accum_u(int kind, float (&r)[V], const float (&acc)[V]) { r[0] = accum_combine(kind, r[0], acc[0]); }
+
 // Fold of a tile in element order (a fixed order, so results repeat exactly).  Elements of
 // groups outside the row take the identity.
 template <int VL, int NG, bool FULL, class F>
@@ -768,7 +772,10 @@ PN_DEV void run_program(const KernelParams& p, int pc, const int pc_end, const T
         if constexpr (!SCALAR) ts = *stash_ptr<V>(cx, b);
         break;
       case OP_ACCUM:
-        if constexpr (!SCALAR) { PN_WITH_REG(b, op_accum<V>(a, r, acc);) }
+        if constexpr (!SCALAR) {
+          if (a & 0x80) { PN_WITH_REG(b, op_accum_u<V>(a & 0x7F, r, acc);) }
+          else { PN_WITH_REG(b, op_accum<V>(a, r, acc);) }
+        }
         break;
       case OP_SLD: op_splat<V>(acc, cx.slots[a]); break;
       case OP_SST:
@@ -811,6 +818,7 @@ struct Interp {
   static PN_DEV int n_red(const KernelParams& p, int s) { return p.stage[s].n_red; }
   static PN_DEV int red_kind(const KernelParams& p, int s, int r) { return p.stage[s].red[r].kind; }
   static PN_DEV int red_slot(const KernelParams& p, int s, int r) { return p.stage[s].red[r].slot; }
+  static PN_DEV bool red_uniform(const KernelParams& p, int s, int r) { return p.stage[s].red[r].uniform != 0; }
   static PN_DEV bool has_scalar(const KernelParams& p, int s) { return p.stage[s].scal_begin != p.stage[s].scal_end; }
   static PN_DEV void tile(const KernelParams& p, int s, const TileCtx& cx, float (&acc)[VL * NG],
                           float (&reg)[K][VL * NG], float& ts, Part (&)[kMaxRed], float (&)[1][VL * NG],
@@ -1158,6 +1166,9 @@ PN_DEV void column_body(const KernelParams& p, unsigned char* smem) {
         at_step(s);
         Prog::tile(p, 0, cx, acc, reg, ts, parts, raw[0], cx, false);
       }
+    }
+    PN_UNROLL for (int r = 0; r < kAcc; ++r) {   // reductions carried by one element: now in all of them
+      if (r < n_red && Prog::red_uniform(p, 0, r)) { PN_UNROLL for (int e = 1; e < V; ++e) reg[r][e] = reg[r][0]; }
     }
     if (TY > 1) {
       PN_UNROLL for (int r = 0; r < kAcc; ++r) {

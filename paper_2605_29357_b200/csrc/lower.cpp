@@ -315,7 +315,7 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     if (s >= kMaxStages - 1) return -1;
     if ((int)stage_reds[s].size() >= kMaxRed) return -2;
     const int base = new_slot(3);
-    RedDesc rd; rd.kind = (uint8_t)kind; rd.slot = (uint8_t)base;
+    RedDesc rd; rd.kind = (uint8_t)kind; rd.slot = (uint8_t)base; rd.uniform = 0;
     const int ridx = (int)stage_reds[s].size();
     stage_reds[s].push_back(rd);
     int e = -1;

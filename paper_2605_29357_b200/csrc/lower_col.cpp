@@ -227,6 +227,7 @@ int lower_column_graph(const Graph& g, unsigned flags, const DeviceModel& dev, L
     const int q = io_of_tensor[t];
     ex.vals[v].io = q;
     ex.vals[v].bcast = P.io[q].col_stride == 0;
+    ex.vals[v].uniform = P.io[q].col_stride == 0 && C != 1;
     ex.vals[v].streamed = io_streamed[q];
     ex.vals[v].integral = !dtype_is_float(g.tensors[t].dtype);
     ex.vals[v].mask8 = g.tensors[t].dtype == kI8 || g.tensors[t].dtype == kBool;
@@ -253,13 +254,15 @@ int lower_column_graph(const Graph& g, unsigned flags, const DeviceModel& dev, L
       else {
         if ((int)reds.size() >= kMaxRed) { err = where + "more reductions than the kernel takes"; return PN_ERR_TOO_LARGE; }
         a = (int)reds.size();
-        RedDesc rd; rd.kind = (uint8_t)kind; rd.slot = (uint8_t)a;   // accumulator a is tile register a
+        const bool uni = ex.vals[in[0]].uniform;
+        RedDesc rd; rd.kind = (uint8_t)kind; rd.slot = (uint8_t)a; rd.uniform = uni ? 1 : 0;   // accumulator a is tile register a
         reds.push_back(rd);
         const int v = ex.new_val(VK_E, 1);
         ex.vals[v].pinned = true;
         ex.vals[v].integral = ex.vals[in[0]].integral;
         red_val.push_back(v);
-        ex.add_op(OP_ACCUM, 0, false, {in[0]}, -1, kind, a);
+        ex.vals[v].uniform = uni;
+        ex.add_op(OP_ACCUM, 0, false, {in[0]}, -1, kind | (uni ? 0x80 : 0), a);
         red_cache[key] = a;
       }
       res[0] = red_val[a];

@@ -33,6 +33,7 @@ struct Val {
   bool integral = false;// known to hold integer / 0-1 values
   bool boolean = false; // known to hold exactly 0.0f or 1.0f
   bool mask8 = false;   // graph input stored as int8 / bool
+  bool uniform = false; // column kernels: the same value in every column of a tile
   int uses = 0;
 };
 
@@ -362,11 +363,12 @@ struct Expander {
   // a pointwise micro-operation: a tile operation in the latest stage of its operands, or a
   // per-row scalar operation when no operand is a tile value
   int pointwise(int vmop, std::initializer_list<int> in, bool integral) {
-    bool any_e = false; int stage = 0;
-    for (int v : in) { any_e |= vals[v].kind == VK_E; stage = std::max(stage, vals[v].stage); }
+    bool any_e = false, uni = true; int stage = 0;
+    for (int v : in) { any_e |= vals[v].kind == VK_E; stage = std::max(stage, vals[v].stage); uni = uni && (vals[v].uniform || vals[v].kind == VK_IMM); }
     const bool sc = !any_e;
     const int r = new_val(sc ? VK_S : VK_E, stage);
     vals[r].integral = integral;
+    vals[r].uniform = uni;
     if (sc) vals[r].slot = new_slot(1);
     add_op(vmop, sc ? stage - 1 : stage, sc, in, r);
     return r;

@@ -72,7 +72,8 @@ enum Op : uint8_t {
   OP_SST,     // slot[a] = acc
   OP_STOUT_I, // a = io: store the int32 bits held in acc as an integer (argmax / argmin)
   // column kernels (reductions over a leading dimension)
-  OP_ACCUM,   // a = RedKind (sum / max / min), b = reg: reg = reg (op) acc, element by element
+  OP_ACCUM,   // a = RedKind (sum / max / min), b = reg: reg = reg (op) acc, element by element;
+              // a | 0x80: acc holds one value in all its elements, only element 0 is accumulated
   OP_COUNT_
 };
 
@@ -111,6 +112,8 @@ struct IoDesc {
 struct RedDesc {
   uint8_t kind;
   uint8_t slot;   // first of the 3 slots receiving the combined (a, b, c)
+  uint8_t uniform;// column kernels: the reduced value is the same in every column of a tile (it comes
+                  // from operands broadcast over the columns): one element is accumulated, then copied
 };
 
 struct StageDesc {

@@ -171,7 +171,7 @@ bool emit_program(const KernelParams& P, int pc, int end, bool scalar, int vl, i
     else if (op == OP_FILL) s = "op_fill<" + V + ">(cx, " + B + ", " + regname(a) + ");";
     else if (op == OP_SPILL_TS) s = "*stash_ptr<" + V + ">(cx, " + B + ") = ts;";
     else if (op == OP_FILL_TS) s = "ts = *stash_ptr<" + V + ">(cx, " + B + ");";
-    else if (op == OP_ACCUM) s = "op_accum<" + V + ">(" + A + ", " + regname(b) + ", acc);";
+    else if (op == OP_ACCUM) s = std::string(a & 0x80 ? "op_accum_u<" : "op_accum<") + V + ">(" + std::to_string(a & 0x7F) + ", " + regname(b) + ", acc);";
     else if (op == OP_SLD) s = "op_splat<" + V + ">(acc, cx.slots[" + A + "]);";
     else if (op == OP_SST) s = std::string("op_sst<") + (reg_slots ? "true" : "false") + ">(cx, " + A + ", acc[0]);";
     else if (op == OP_END) continue;
@@ -253,6 +253,7 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
   };
   table("red_kind", "int", [&](int st, int r) { return (long long)P.stage[st].red[r].kind; });
   table("red_slot", "int", [&](int st, int r) { return (long long)P.stage[st].red[r].slot; });
+  table("red_uniform", "bool", [&](int st, int r) { return (long long)P.stage[st].red[r].uniform; });
   s += "  static PN_DEV int n_red(const KernelParams&, int s) {\n    switch (s) {\n";
   for (int st = 0; st < P.n_stages; ++st) s += "      case " + I(st) + ": return " + I(P.stage[st].n_red) + ";\n";
   s += "      default: return 0;\n    }\n  }\n";

@@ -238,7 +238,7 @@ def test_masked_mean_pooling_lowers_to_one_column_kernel():
     assert k["rows"] == 256 and k["row_len"] == 1024 and k["vl"] == 8      # 128-bit loads of the bf16 hidden states
     assert g.compulsory_bytes == 256 * 512 * 1024 * 2 + 256 * 512 * 8 + 256 * 1024 * 4
     src = g.codegen(0, compile=True)
-    assert "pn::column_body<pn::Spec>" in src and src.count("op_accum<8>") == 2   # both sums in one walk
+    assert "pn::column_body<pn::Spec>" in src and src.count("op_accum<8>") + src.count("op_accum_u<8>") == 2   # both sums in one walk
     gu = pn.Graph(w.desc, 0, PLAN | pn.FLAG_UNFUSED)
     assert gu.n_kernels == 7
     for i in range(gu.n_kernels):
