@@ -341,7 +341,8 @@ PN_DEV Part red_combine(int kind, Part x, Part y) {
 
 PN_DEV float shfl_x(float v, int o) { return __shfl_xor_sync(0xFFFFFFFFu, v, o); }
 
-// Combine the partials of the 32 lanes of a warp; every lane ends with the same result.
+// Combine the partials of the 32 lanes of a warp (or of each aligned group of `lanes` = 16 or 8
+// lanes, for rows short enough that several share a warp); every lane ends with the same result.
 // The order of operations is fixed (a butterfly over lane distance 16, 8, 4, 2, 1), so
 // results repeat bit for bit from run to run.  Lanes without data pass the identity partial.
 //   sum / max / min      one value per shuffle step
@@ -350,38 +351,39 @@ PN_DEV float shfl_x(float v, int o) { return __shfl_xor_sync(0xFFFFFFFFu, v, o);
 //   mean / variance      count and sum first, giving the common mean; then each lane moves its
 //                        squared deviations to that mean (M2 + n (mean_lane - mean)^2) and the
 //                        results are added: the exact decomposition of the total sum of squares
-PN_DEV Part warp_combine(int kind, Part v) {
+PN_DEV Part warp_combine(int kind, Part v, int lanes = 32) {
   switch (kind) {
     case RED_SUM:
-      PN_UNROLL for (int o = 16; o > 0; o >>= 1) v.a += shfl_x(v.a, o);
+      PN_UNROLL for (int o = 16; o > 0; o >>= 1) if (o < lanes) v.a += shfl_x(v.a, o);
       break;
     case RED_MAX:
-      PN_UNROLL for (int o = 16; o > 0; o >>= 1) v.a = f_max_nan(v.a, shfl_x(v.a, o));
+      PN_UNROLL for (int o = 16; o > 0; o >>= 1) if (o < lanes) v.a = f_max_nan(v.a, shfl_x(v.a, o));
       break;
     case RED_MIN:
-      PN_UNROLL for (int o = 16; o > 0; o >>= 1) v.a = f_min_nan(v.a, shfl_x(v.a, o));
+      PN_UNROLL for (int o = 16; o > 0; o >>= 1) if (o < lanes) v.a = f_min_nan(v.a, shfl_x(v.a, o));
       break;
     case RED_ARGMAX: case RED_ARGMIN:
       PN_UNROLL for (int o = 16; o > 0; o >>= 1) {
+        if (o >= lanes) continue;
         const float wa = shfl_x(v.a, o), wb = shfl_x(v.b, o);
         if (arg_better(wa, (int)f_bits(wb), v.a, (int)f_bits(v.b), kind == RED_ARGMAX)) { v.a = wa; v.b = wb; }
       }
       break;
     case RED_LSE: case RED_SOFTMAX: {
       float m = v.a;
-      PN_UNROLL for (int o = 16; o > 0; o >>= 1) m = f_max_nan(m, shfl_x(m, o));
+      PN_UNROLL for (int o = 16; o > 0; o >>= 1) if (o < lanes) m = f_max_nan(m, shfl_x(m, o));
       float s = (m == -PN_INF) ? 0.f : v.b * f_exp_neg(v.a - m);
-      PN_UNROLL for (int o = 16; o > 0; o >>= 1) s += shfl_x(s, o);
+      PN_UNROLL for (int o = 16; o > 0; o >>= 1) if (o < lanes) s += shfl_x(s, o);
       v.a = m; v.b = s;
       break;
     }
     default: {  // RED_MEANVAR
       float n = v.a, sum = v.a * v.b;
-      PN_UNROLL for (int o = 16; o > 0; o >>= 1) { n += shfl_x(n, o); sum += shfl_x(sum, o); }
+      PN_UNROLL for (int o = 16; o > 0; o >>= 1) if (o < lanes) { n += shfl_x(n, o); sum += shfl_x(sum, o); }
       const float mean = n > 0.f ? sum * f_rcp(n) : 0.f;
       const float d = v.b - mean;
       float m2 = fmaf(v.a * d, d, v.c);
-      PN_UNROLL for (int o = 16; o > 0; o >>= 1) m2 += shfl_x(m2, o);
+      PN_UNROLL for (int o = 16; o > 0; o >>= 1) if (o < lanes) m2 += shfl_x(m2, o);
       v.a = n; v.b = mean; v.c = m2;
       break;
     }
@@ -812,6 +814,7 @@ struct Interp {
   static PN_DEV int chunks(const KernelParams& p) { return p.chunks; }
   static PN_DEV int split_chunks(const KernelParams& p) { return p.split_chunks; }
   static PN_DEV int row_len(const KernelParams& p) { return p.row_len; }
+  static PN_DEV int team_lanes(const KernelParams&) { return 32; }   // short rows sharing a warp: generated kernels only
   static PN_DEV int slice_len(const KernelParams& p) { return p.slice_len; }
   static PN_DEV int n_stages(const KernelParams& p) { return p.n_stages; }
   static PN_DEV int n_io(const KernelParams& p) { return p.n_io; }
@@ -847,8 +850,12 @@ PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
   const int chunks = Prog::chunks(p);
   const bool split = Prog::split_chunks(p) != 0;
   const bool warp_team = family <= FAM_WARP;
-  const int team_threads = warp_team ? 32 : (int)blockDim.x;
-  const int team_tid = warp_team ? lane : tid;
+  // Rows of at most 16 (8) groups: two (four) rows share a warp, each owned by an aligned group
+  // of TL lanes; the shuffles of a combine then stop at lane distance TL / 2.
+  const int TL = warp_team ? Prog::team_lanes(p) : 32;
+  const int sub = TL < 32 ? lane / TL : 0;              // which of the warp's teams this lane is in
+  const int team_threads = warp_team ? TL : (int)blockDim.x;
+  const int team_tid = warp_team ? (TL < 32 ? lane % TL : lane) : tid;
   const int team_in_cta = warp_team ? warp : 0;
   const int crank = (cluster > 1) ? (int)cluster_ctarank() : 0;
 
@@ -874,7 +881,10 @@ PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
 
   const long long n_items = split ? p.rows * chunks : p.rows;
   long long team_global, n_teams;
-  if (warp_team) { team_global = (long long)blockIdx.x * nwarps + warp; n_teams = (long long)gridDim.x * nwarps; }
+  if (warp_team) {
+    const int per_warp = 32 / TL;
+    team_global = ((long long)blockIdx.x * nwarps + warp) * per_warp + sub; n_teams = (long long)gridDim.x * nwarps * per_warp;
+  }
   else { team_global = blockIdx.x / cluster; n_teams = gridDim.x / cluster; }
 
   const int slice_lo = crank * Prog::slice_len(p);
@@ -925,8 +935,18 @@ PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
     }
   }
 
-  for (long long item = team_global; item < n_items; item += n_teams) {
+  const int col_end_all = cx.col_end;
+  const bool leader_all = cx.leader;
+  // the teams of a warp stay together: the loop runs while the warp's first team has an item; a
+  // team without one goes through the motions on the last row with every access switched off
+  for (long long item = team_global; item - sub < n_items; item += n_teams) {
     long long row = item;
+    if (TL < 32) {
+      const bool active = item < n_items;
+      if (!active) row = n_items - 1;
+      cx.col_end = active ? col_end_all : 0;
+      cx.leader = active && leader_all;
+    }
     int c_first = 0, c_count = chunks;
     if (split) { row = item / chunks; c_first = (int)(item - row * chunks); c_count = 1; }
 
@@ -980,7 +1000,7 @@ PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
             Part v = Prog::kStatic ? parts[r]
                                    : Part{cx.part[(r * 3) * cx.part_stride], cx.part[(r * 3 + 1) * cx.part_stride],
                                           cx.part[(r * 3 + 2) * cx.part_stride]};
-            v = warp_combine(kind, v);
+            v = warp_combine(kind, v, TL);
             if (kRegSlots || lane == 0) { float* d = slots + Prog::red_slot(p, s, r); d[0] = v.a; d[1] = v.b; d[2] = v.c; }
           }
         }

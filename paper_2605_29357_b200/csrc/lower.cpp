@@ -43,7 +43,7 @@ void size_grid(LaunchPlan& lp, int sms, int occ) {
 
 namespace {
 
-struct Config { int family, vl, ng, k, block, cluster, chunks, slice_len; bool multichunk; };
+struct Config { int family, vl, ng, k, block, cluster, chunks, slice_len; bool multichunk; int lanes; };
 
 }  // namespace
 
@@ -472,7 +472,12 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
       const int v_warp = min_esize <= 2 ? 64 : 32, v_block = min_esize <= 2 ? 32 : 16;
       if (!fb)
         for (int ng = 1; VL * ng <= v_warp; ng *= 2)
-          if (32ll * VL * ng >= eff_N) { cands.push_back(Config{FAM_WARP, VL, ng, kSpecRegs, 256, 1, 1, (int)eff_N, false}); break; }
+          if (32ll * VL * ng >= eff_N) {
+            // rows of at most 16 (8) groups: two (four) of them share a warp, so that most lanes work
+            const int lanes = ng > 1 ? 32 : (8ll * VL >= eff_N ? 8 : (16ll * VL >= eff_N ? 16 : 32));
+            cands.push_back(Config{FAM_WARP, VL, ng, kSpecRegs, 256, 1, 1, (int)eff_N, false, lanes});
+            break;
+          }
       if (!fw && cands.empty() && cross_stage)   // rows that need no residency stream in chunks instead
         for (int T : {64, 128, 256, 512})
           if ((int64_t)T * v_block >= eff_N) { cands.push_back(Config{FAM_BLOCK, VL, v_block / VL, kSpecRegs, T, 1, 1, (int)eff_N, false}); break; }
@@ -604,7 +609,8 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     if (n_stash > kMaxStash) { gen_err = "too many tile values cross a reduction"; continue; }
 
     // ---- (5) shared memory and grid ------------------------------------------------------
-    const int teams = cf.family <= FAM_WARP ? cf.block / 32 : 1;
+    const int lanes = (cf.family == FAM_WARP && (cf.lanes == 16 || cf.lanes == 8)) ? cf.lanes : 32;
+    const int teams = cf.family <= FAM_WARP ? cf.block / lanes : 1;
     int off = 0;
     auto take = [&](int bytes) { const int o = off; off += (bytes + 15) / 16 * 16; return o; };
     P.sm_rowoff = take(teams * kMaxIo * 8);
@@ -625,6 +631,7 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     P.chunks = cf.chunks;
     P.split_chunks = cf.family == FAM_POINTWISE;
     P.cluster = cf.cluster;
+    P.team_lanes = lanes;
     lp.family = cf.family; lp.vl = cf.vl; lp.ng = cf.ng; lp.k = cf.k;
     lp.block = cf.block; lp.smem_bytes = off; lp.code_words = (int)code.size();
     P.family = cf.family;

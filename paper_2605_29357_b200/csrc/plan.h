@@ -144,6 +144,8 @@ struct KernelParams {
   // 0 .. n_red-1, stage 1 runs once per (row, column tile) on the combined registers.
   int32_t red_len;
   int32_t col_tx;
+  int32_t team_lanes;      // warp-per-row kernels: lanes per row (32, or 16 / 8 when short rows share a warp)
+  int32_t pad1;
   uint16_t pro_begin, pro_end;   // tile program run once per thread before the row loop: loads of
                                  // operands that are the same for every row (generated kernels only)
   // shared-memory layout, byte offsets into dynamic shared memory

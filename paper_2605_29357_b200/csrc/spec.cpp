@@ -189,7 +189,7 @@ std::string kernel_name(const LaunchPlan& lp) {
   auto mix = [&](uint64_t v) { for (int i = 0; i < 8; ++i) { h ^= (v >> (8 * i)) & 0xFF; h *= 1099511628211ull; } };
   for (int i = 0; i < lp.code_words; ++i) mix(lp.p.code[i]);
   mix((uint64_t)lp.p.row_len); mix((uint64_t)lp.p.rows); mix((uint64_t)lp.block); mix((uint64_t)lp.p.cluster);
-  mix((uint64_t)lp.p.red_len); mix((uint64_t)lp.p.col_tx);
+  mix((uint64_t)lp.p.red_len); mix((uint64_t)lp.p.col_tx); mix((uint64_t)lp.p.team_lanes);
   for (int q = 0; q < lp.p.n_io; ++q) {
     const IoDesc& io = lp.p.io[q];
     mix(io.dtype); mix((uint64_t)io.col_stride); mix(io.mapped); mix((uint64_t)io.red_stride);
@@ -236,7 +236,9 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
   s += "      default: return IoMap{1, 1, 1, 0, 0, 0, 0, 0, 0, 0, 0, 0};\n    }\n  }\n";
   // every group of every tile inside the row: no validity tests in the generated code
   const int team_threads = P.family == FAM_COLUMN ? P.col_tx : P.family <= FAM_WARP ? 32 : lp.block;
-  const bool full = (long long)P.chunks * team_threads * lp.vl * lp.ng == P.slice_len &&
+  const int team_lanes = (P.family == FAM_WARP && (P.team_lanes == 16 || P.team_lanes == 8)) ? P.team_lanes : 32;
+  // (teams that share a warp may be switched off for a row: their accesses keep their validity tests)
+  const bool full = team_lanes == 32 && (long long)P.chunks * team_threads * lp.vl * lp.ng == P.slice_len &&
                     (long long)P.slice_len * P.cluster == P.row_len;
   const bool reg_slots = true;   // generated programs keep the per-row scalars in registers
   auto konst = [&](const char* name, long long v) {
@@ -244,7 +246,7 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
   };
   konst("family", P.family); konst("cluster", P.cluster); konst("chunks", P.chunks); konst("split_chunks", P.split_chunks);
   konst("row_len", P.row_len); konst("slice_len", P.slice_len); konst("n_stages", P.n_stages); konst("n_io", P.n_io);
-  konst("col_tx", P.col_tx); konst("red_len", P.red_len);
+  konst("col_tx", P.col_tx); konst("red_len", P.red_len); konst("team_lanes", team_lanes);
   auto table = [&](const char* name, const char* type, auto get) {
     s += std::string("  static PN_DEV ") + type + " " + name + "(const KernelParams&, int s, int r) {\n    switch (s * " + I(kMaxRed) + " + r) {\n";
     for (int st = 0; st < P.n_stages; ++st)

@@ -265,3 +265,35 @@ def test_results_repeat_bit_for_bit():
     h = pn.Graph(w.desc, 0, 0)
     a = run_graph(h, w.inputs); b = run_graph(h, w.inputs)
     assert all(np.array_equal(x, y) for x, y in zip(a, b))
+
+
+@pytest.mark.parametrize("dtype", [D.F32, D.BF16])
+@pytest.mark.parametrize("rows,n", [(1, 8), (5, 16), (37, 24), (64, 40), (3, 64), (1001, 96), (130, 128), (7, 32)])
+def test_short_rows_that_share_a_warp(rows, n, dtype):
+    """Rows of at most 16 (8) vector groups are owned by half (quarter) warps; row counts that leave
+    some of a warp's teams without a row in the last round; every kind of reduction, an index
+    result, a composite with a full-shape output."""
+    x = np.round(rnd((rows, n), 40 + rows + n, 2.0) * 4) / 4
+    x = x.astype(np.float32)
+    xs = x if dtype == D.F32 else C.to_bf16_bits(x)
+    gamma = rnd((n,), 41); beta = rnd((n,), 42)
+    g = GraphBuilder(); xi = g.input(dtype, (rows, n)); gi = g.input(D.F32, (n,)); bi = g.input(D.F32, (n,))
+    xf = g.op("cast", [xi], D.F32, (rows, n)) if dtype != D.F32 else xi
+    y, mean, rstd = g.node("layer_norm", [xf, gi, bi], [D.F32, D.F32, D.F32], [(rows, n), (rows,), (rows,)], extra_imm=[1e-5])
+    g.mark_output(g.op("cast", [y], dtype, (rows, n)) if dtype != D.F32 else y)
+    g.mark_output(mean); g.mark_output(rstd)
+    g.mark_output(g.op("argmax", [xf], D.I64, (rows,)))
+    g.mark_output(g.op("sum", [xf], D.F32, (rows, 1)))
+    h = pn.Graph(g.build(), 0, 0)
+    k = h.kernel_info[0]
+    assert pn.FAMILY_NAMES[k["family"]] == "warp-per-row"
+    outs = run_graph(h, [xs, gamma, beta])
+    check_against_oracle(g.build(), [xs, gamma, beta], outs, [g.tensor_meta(t) for t in g.output_ids()])
+    again = run_graph(h, [xs, gamma, beta])
+    assert all(np.array_equal(a, b, equal_nan=True) for a, b in zip(outs, again))
+    g = GraphBuilder(); xi = g.input(dtype, (rows, n))
+    xf = g.op("cast", [xi], D.F32, (rows, n)) if dtype != D.F32 else xi
+    sm = g.op("softmax", [xf], D.F32, (rows, n))
+    g.mark_output(g.op("cast", [sm], dtype, (rows, n)) if dtype != D.F32 else sm)
+    g.mark_output(g.op("logsumexp", [xf], D.F32, (rows,)))
+    check(g, [xs])
