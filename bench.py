@@ -120,6 +120,14 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def driver_version():
+    try:
+        out = subprocess.run(["nvidia-smi", "--query-gpu=driver_version", "--format=csv,noheader"], capture_output=True, text=True, timeout=20)
+        return out.stdout.strip().splitlines()[0]
+    except Exception:
+        return None
+
+
 def nbytes_of(meta):
     return [D.DTYPE_BYTES[dt] * int(np.prod(dims, dtype=np.int64)) for dt, dims in meta]
 
@@ -372,7 +380,15 @@ def main():
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-    total_ms, per = time_graph(torch, g, sets, args.steps, 0)
+    # the paper's protocol: the median of the timed runs, measured again (up to three times in all)
+    # while the interquartile range exceeds 20 % of the median
+    reruns = 0
+    while True:
+        total_ms, per = time_graph(torch, g, sets, args.steps, 0)
+        st_try = stats(per)
+        if st_try["iqr_ms"] <= 0.2 * st_try["median_ms"] or reruns >= 2:
+            break
+        reruns += 1
     barrier()
     # K steps of this workload last only milliseconds, less than one nvidia-smi sample: keep
     # the same step running (untimed) until the sampler has seen the GPU under this load
@@ -419,7 +435,8 @@ def main():
                    "l2": "inputs larger than L2" if n_sets == 1 else f"{n_sets} rotating buffer sets larger than 2x L2",
                    "family": pn.FAMILY_NAMES[info["family"]], "grid": info["grid"], "block": info["block"],
                    "cluster": info["cluster"], "tile": [info["vl"], info["ng"]], "kernels": g.n_kernels,
-                   "nodes": g.n_nodes, "per_step": st, "pct_of_8000": 100 * value / world / 8000.0},
+                   "nodes": g.n_nodes, "per_step": st, "reruns_for_iqr": reruns, "pct_of_8000": 100 * value / world / 8000.0,
+                   "gpu": torch.cuda.get_device_name(local_rank), "driver": driver_version(), "cuda": torch.version.cuda},
         "clocks": clocks,
         "gpu_launches": args.steps * g.n_kernels,
         "e2e": {"value": job_value(world, cbytes, e2e_s), "unit": "GB/s", "h2d_bytes_per_step": h2d,
@@ -478,6 +495,22 @@ def main():
             sweep[name] = entry
             gi.close()
             del si
+            torch.cuda.empty_cache()
+        # supplementary: the two small graphs scaled up until their inputs exceed the L2, to show their
+        # kernels' bandwidth once launch, ramp and tail no longer dominate (not benchmark configs)
+        for name, make in (("c1_scaled_8192x8192", lambda: C.c1(M=8192, N=8192)), ("c4_scaled_256x262144", lambda: C.c4(M=256))):
+            wi = make()
+            gi = pn.Graph(wi.desc, local_rank, 0)
+            si = device_sets(torch, wi, 1)
+            _, pi = time_graph(torch, gi, si, args.steps, warmup)
+            sti = stats(pi)
+            ki = gi.kernel_info[0]
+            sweep[name] = {"supplementary": True, "compulsory_bytes": gi.compulsory_bytes, "median_ms": sti["median_ms"], "min_ms": sti["min_ms"],
+                           "iqr_ms": sti["iqr_ms"], "gbs": gi.compulsory_bytes / (sti["median_ms"] * 1e-3) / 1e9,
+                           "frac_of_measured_peak": gi.compulsory_bytes / (sti["median_ms"] * 1e-3) / 1e9 / peak,
+                           "family": pn.FAMILY_NAMES[ki["family"]], "buffer_sets": 1}
+            gi.close()
+            del si, wi
             torch.cuda.empty_cache()
         line["sweep"] = sweep
         line["tiny_graphs"] = tiny_graph_latency(torch, pn, local_rank, max(10, args.steps // 2))

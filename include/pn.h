@@ -97,8 +97,13 @@ enum {
   PN_FLAG_NO_HOIST = 1u << 10,    /* do not move row-invariant operand loads out of the row loop */
   PN_FLAG_PREFETCH = 1u << 11,    /* generated kernels: issue the first stage's loads one tile
                                      ahead (costs registers; off by default)                 */
-  PN_FLAG_STATIC_SCRATCH = 1u << 12 /* with PN_FLAG_UNFUSED: allocate no workspace; the handle
+  PN_FLAG_STATIC_SCRATCH = 1u << 12,/* with PN_FLAG_UNFUSED: allocate no workspace; the handle
                                      is run with pn_graph_run_static only                    */
+  PN_FLAG_BOUNDS = 1u << 13       /* checked accessors: every global access of the kernels is tested
+                                     against the extent of its tensor; one that falls outside is
+                                     skipped and recorded in a status word on the device (4 bytes
+                                     owned by the handle), read with PN_Q_BOUNDS_STATUS.  A debugging
+                                     aid at some cost in speed; a correct build always reads 0   */
 };
 /* Size of the fixed scratch array behind pn_graph_run_static. */
 #define PN_STATIC_SCRATCH_BYTES (32ll << 20)
@@ -118,6 +123,9 @@ enum {
   PN_Q_N_KERNELS = 6,       /* 1 value: launches per pn_graph_run (1 when fused)         */
   PN_Q_N_NODES = 7,         /* 1 value: operator nodes in the descriptor                 */
   PN_Q_WORKSPACE_BYTES = 8, /* 1 value: device memory owned by the handle                */
+  PN_Q_BOUNDS_STATUS = 10,  /* 1 value, PN_FLAG_BOUNDS handles only: bit q set when an access to the
+                               q-th input / output entry of a launch fell outside its tensor;
+                               waits for the device                                        */
   PN_Q_KERNEL_INFO = 9      /* per kernel 13 values: family (0 pointwise, 1 warp-per-row,
                                2 block-per-row, 3 cluster-per-row, 4 column-reduce: rows =
                                the dimensions before the reduced one, row length = those after

@@ -26,6 +26,7 @@ FLAG_INTERPRET = 1 << 9
 FLAG_NO_HOIST = 1 << 10
 FLAG_PREFETCH = 1 << 11
 FLAG_STATIC_SCRATCH = 1 << 12
+FLAG_BOUNDS = 1 << 13
 STATIC_SCRATCH_BYTES = 32 << 20
 
 
@@ -141,6 +142,11 @@ class Graph:
     @property
     def n_nodes(self) -> int:
         return self._query(Q_N_NODES, 1)[0]
+
+    @property
+    def bounds_status(self) -> int:
+        """Status word of a FLAG_BOUNDS handle: 0 unless an access fell outside its tensor."""
+        return self._query(10, 1)[0]
 
     @property
     def workspace_bytes(self) -> int:

@@ -86,6 +86,7 @@ pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsig
   std::string err;
   int st = parse_descriptor(desc, desc_bytes, h->g, err);
   if (st != PN_OK) { delete h; return fail(st, err); }
+  if ((flags & PN_FLAG_BOUNDS) && (flags & PN_FLAG_STATIC_SCRATCH)) { delete h; return fail(PN_ERR_INVALID_ARG, "PN_FLAG_BOUNDS allocates a status word: it cannot be combined with PN_FLAG_STATIC_SCRATCH"); }
   h->flags = flags;
   h->device = device;
   h->plan_only = (flags & PN_FLAG_PLAN_ONLY) != 0;
@@ -118,6 +119,7 @@ pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsig
     if (st != PN_OK) { delete h; return fail(st, err); }
     for (int q = 0; q < pl.plan.p.n_io; ++q) {
       const int t = pl.plan.io_tensor[q];
+      pl.plan.p.io[q].numel = g.tensors[t].numel();
       IoSource s{pl.plan.io_is_output[q] ? 1 : 0, 0};
       const std::vector<int>& list = pl.plan.io_is_output[q] ? g.outputs : g.inputs;
       for (size_t i = 0; i < list.size(); ++i) if (list[i] == t) s.index = (int64_t)i;
@@ -142,6 +144,7 @@ pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsig
       if (st != PN_OK) { delete h; return fail(st, "node " + std::to_string(ni) + " (unfused): " + err); }
       for (int q = 0; q < pl.plan.p.n_io; ++q) {
         const int t = orig[pl.plan.io_tensor[q]];
+        pl.plan.p.io[q].numel = g.tensors[t].numel();
         IoSource s{2, ws_off[t]};
         for (size_t i = 0; i < g.inputs.size(); ++i) if (g.inputs[i] == t) s = IoSource{0, (int64_t)i};
         for (size_t i = 0; i < g.outputs.size(); ++i) if (g.outputs[i] == t) s = IoSource{1, (int64_t)i};
@@ -153,6 +156,16 @@ pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsig
     if (!h->plan_only && ws > 0 && !(flags & PN_FLAG_STATIC_SCRATCH)) {
       cudaError_t e = cudaMalloc(&h->workspace, ws);
       if (e != cudaSuccess) { delete h; return fail(PN_ERR_CUDA, std::string("workspace: ") + cudaGetErrorString(e)); }
+    }
+  }
+  // checked accessors: one status word on the device, shared by the launches of the handle
+  if (flags & PN_FLAG_BOUNDS) {
+    for (PlannedLaunch& pl : h->launches) pl.plan.bounds = 1;
+    if (!h->plan_only) {
+      cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&h->status), sizeof(uint32_t));
+      if (e == cudaSuccess) e = cudaMemset(h->status, 0, sizeof(uint32_t));
+      if (e != cudaSuccess) { pn_graph_destroy(h); return fail(PN_ERR_CUDA, std::string("status word: ") + cudaGetErrorString(e)); }
+      for (PlannedLaunch& pl : h->launches) pl.plan.p.status = h->status;
     }
   }
   // a kernel of its own for every launch, unless the interpreter was asked for
@@ -259,6 +272,7 @@ pn_status pn_graph_destroy(pn_graph_t* h) {
   if (!h) return PN_OK;
   if (!h->plan_only) {
     if (h->workspace) cudaFree(h->workspace);
+    if (h->status) cudaFree(h->status);
     for (void* p : h->stage_in) cudaFree(p);
     for (void* p : h->stage_out) cudaFree(p);
   }
@@ -294,6 +308,14 @@ pn_status pn_graph_query(const pn_graph_t* h, int what, void* out, size_t out_by
         v.insert(v.end(), row, row + 13);
       }
       break;
+    case PN_Q_BOUNDS_STATUS: {
+      if (!(h->flags & PN_FLAG_BOUNDS) || !h->status) return fail(PN_ERR_INVALID_ARG, "the handle was not created with PN_FLAG_BOUNDS on a device");
+      uint32_t w = 0;
+      const cudaError_t e = cudaMemcpy(&w, h->status, sizeof(w), cudaMemcpyDeviceToHost);   // waits for the device
+      if (e != cudaSuccess) return fail(PN_ERR_CUDA, std::string("status word: ") + cudaGetErrorString(e));
+      v.push_back((int64_t)w);
+      break;
+    }
     default: return fail(PN_ERR_INVALID_ARG, "unknown query");
   }
   if (out_bytes < v.size() * sizeof(int64_t)) return fail(PN_ERR_INVALID_ARG, "query buffer too small");

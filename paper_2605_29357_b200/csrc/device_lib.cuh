@@ -426,6 +426,26 @@ PN_DEV long long mapped_row_offset(unsigned long long row, const IoMap m) {
 }
 
 // ---------------------------------------------------------------------------------------
+// checked accessors (PN_FLAG_BOUNDS): every global access is tested against the extent of its
+// tensor; one that falls outside is skipped (a load delivers zeros) and its io entry is marked
+// in the status word, which the host reads back.  Nothing traps.  Generated kernels compile the
+// tests in only when asked (PN_BOUNDS); the interpreter kernels test a launch parameter.
+// ---------------------------------------------------------------------------------------
+#if defined(PN_BOUNDS)
+#define PN_CHECKING(p) true
+#elif defined(PN_BOUNDS_RUNTIME)
+#define PN_CHECKING(p) ((p).status != nullptr)
+#else
+#define PN_CHECKING(p) false
+#endif
+PN_DEV bool in_bounds(const KernelParams& p, int io, long long elem, int n) {
+  if (!PN_CHECKING(p)) return true;
+  if (elem >= 0 && elem + n <= p.io[io].numel) return true;
+  atomicOr(p.status, 1u << io);
+  return false;
+}
+
+// ---------------------------------------------------------------------------------------
 // tile operations: one function per bytecode instruction
 // ---------------------------------------------------------------------------------------
 struct TileCtx {
@@ -448,7 +468,7 @@ PN_DEV void op_ldraw(const KernelParams& p, const TileCtx& cx, int io, int dt, f
   const long long off = cx.rowoff[io];
   PN_UNROLL for (int j = 0; j < NG; ++j) {
     const int col = cx.col0 + j * cx.gstride;
-    if (FULL || col < cx.col_end) {
+    if ((FULL || col < cx.col_end) && in_bounds(p, io, off + col, VL)) {
       load_group_raw<VL>(base, off + col, dt, &r[j * VL]);
     } else {
       PN_UNROLL for (int i = 0; i < VL; ++i) r[j * VL + i] = 0.f;
@@ -460,6 +480,7 @@ PN_DEV void op_widen(int dt, float (&r)[VL * NG]) {
   if (dt != kF32 && dt != kI64) { PN_UNROLL for (int j = 0; j < NG; ++j) widen_group<VL>(&r[j * VL], dt); }
 }
 PN_DEV float op_ldbc_scalar(const KernelParams& p, const TileCtx& cx, int io, int dt) {
+  if (!in_bounds(p, io, cx.rowoff[io], 1)) return 0.f;
   return widen_scalar(static_cast<const char*>(p.io[io].base) + cx.rowoff[io] * dtype_size(dt), dt);
 }
 // The same load split in two, so that loads issued ahead of their use do not wait for their own
@@ -468,7 +489,8 @@ template <int V>
 PN_DEV void op_ldbc_raw(const KernelParams& p, const TileCtx& cx, int io, int dt, float (&r)[V]) {
   const char* a = static_cast<const char*>(p.io[io].base) + cx.rowoff[io] * dtype_size(dt);
   uint32_t w0 = 0, w1 = 0;
-  switch (dt) {
+  switch (in_bounds(p, io, cx.rowoff[io], 1) ? dt : -1) {
+    case -1: break;
     case kF32: case kI32: w0 = __ldg(reinterpret_cast<const unsigned int*>(a)); break;
     case kF16: case kBF16: w0 = __ldg(reinterpret_cast<const unsigned short*>(a)); break;
     case kI8: case kBool: w0 = __ldg(reinterpret_cast<const unsigned char*>(a)); break;
@@ -513,15 +535,15 @@ PN_DEV void op_stout(const KernelParams& p, const TileCtx& cx, int io, int dt, c
   const long long off = cx.rowoff[io];
   PN_UNROLL for (int j = 0; j < NG; ++j) {
     const int col = cx.col0 + j * cx.gstride;
-    if (FULL || col < cx.col_end) store_group<VL>(base, off + col, dt, &acc[j * VL]);
+    if ((FULL || col < cx.col_end) && in_bounds(p, io, off + col, VL)) store_group<VL>(base, off + col, dt, &acc[j * VL]);
   }
 }
 // per-row scalar stores (leader thread only)
 PN_DEV void op_stout_scalar(const KernelParams& p, const TileCtx& cx, int io, int dt, float v) {
-  if (cx.leader) store_group<1>(static_cast<char*>(p.io[io].base), cx.rowoff[io], dt, &v);
+  if (cx.leader && in_bounds(p, io, cx.rowoff[io], 1)) store_group<1>(static_cast<char*>(p.io[io].base), cx.rowoff[io], dt, &v);
 }
 PN_DEV void op_stout_index(const KernelParams& p, const TileCtx& cx, int io, int dt, float v) {
-  if (cx.leader) {
+  if (cx.leader && in_bounds(p, io, cx.rowoff[io], 1)) {
     const int i = static_cast<int>(f_bits(v));
     if (dt == kI64) static_cast<long long*>(p.io[io].base)[cx.rowoff[io]] = i;
     else static_cast<int*>(p.io[io].base)[cx.rowoff[io]] = i;

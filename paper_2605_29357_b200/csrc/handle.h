@@ -34,4 +34,5 @@ struct pn_graph {
   size_t workspace_bytes = 0;
   int64_t compulsory_bytes = 0;
   std::vector<void*> stage_in, stage_out;   // device staging of pn_graph_run_host
+  uint32_t* status = nullptr;               // device word of the checked accessors (PN_FLAG_BOUNDS)
 };

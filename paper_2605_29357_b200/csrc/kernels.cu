@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 
 #include "plan.h"
+#define PN_BOUNDS_RUNTIME 1   // the interpreter kernels check when the launch carries a status word
 #include "device_lib.cuh"
 
 namespace pn {

@@ -107,6 +107,7 @@ struct IoDesc {
   int32_t map_add[3];
   int32_t map_mod[3];
   int64_t red_stride;      // column kernels: elements per step of the reduced dimension; 0 = broadcast
+  int64_t numel;           // elements of the tensor behind this entry (checked accessors)
 };
 
 struct RedDesc {
@@ -144,6 +145,8 @@ struct KernelParams {
   // 0 .. n_red-1, stage 1 runs once per (row, column tile) on the combined registers.
   int32_t red_len;
   int32_t col_tx;
+  uint32_t* status;        // checked accessors (PN_FLAG_BOUNDS): bit q is set when an access to io entry q
+                           // fell outside its tensor; null when checking is off
   int32_t team_lanes;      // warp-per-row kernels: lanes per row (32, or 16 / 8 when short rows share a warp)
   int32_t pad1;
   uint16_t pro_begin, pro_end;   // tile program run once per thread before the row loop: loads of
@@ -166,6 +169,7 @@ struct LaunchPlan {
   int32_t specialised;     // 1 when the launch uses a kernel generated for this program
   int32_t persistent;      // 1: grid = resident CTAs, each looping over many rows
   int32_t no_prefetch;     // 1: generated kernels issue no loads ahead of the tile in hand
+  int32_t bounds;          // 1: the generated kernel is compiled with checked accessors
   int32_t io_tensor[kMaxIo];   // tensor id behind each io entry
   int32_t io_is_output[kMaxIo];
 };

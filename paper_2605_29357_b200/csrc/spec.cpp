@@ -206,6 +206,7 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
   auto I = [](long long v) { return std::to_string(v); };
   std::string s;
   s.reserve(sizeof(kDeviceSource) + 8192);
+  if (lp.bounds) s += "#define PN_BOUNDS 1\n";
   s += kDeviceSource;
   s += "\nnamespace pn {\nstruct Spec {\n";
   s += "  static constexpr int VL = " + I(lp.vl) + ", NG = " + I(lp.ng) + ", K = " + I(lp.k) + ";\n";
@@ -332,7 +333,7 @@ bool spec_available(std::string* why, bool compile_only) {
 std::string spec_source(const LaunchPlan& lp) {
   std::string src, err;
   if (!generate_source(lp, src, err)) return "// " + err;
-  return src.substr(sizeof(kDeviceSource) - 1);   // the generated part only
+  return src.substr(sizeof(kDeviceSource) - 1 + (lp.bounds ? sizeof("#define PN_BOUNDS 1\n") - 1 : 0));   // the generated part only
 }
 
 bool spec_check(const LaunchPlan& lp, std::string& err) {

@@ -272,3 +272,11 @@ def test_unsupported_column_forms_are_refused():
     g = GraphBuilder(); x = g.input(D.F32, (4, 6, 8)); y = g.input(D.F32, (4, 6, 8))
     g.mark_output(g.op("cat", [x, y], D.F32, (4, 12, 8), attr=[1, 0]))   # a real concatenation is not lowered
     assert status(g) == -3
+
+
+def test_checked_accessors_are_compiled_in_only_on_request():
+    w = C.c3(**C.SMALL["c3"])
+    plain = pn.Graph(w.desc, 0, PLAN)
+    checked = pn.Graph(w.desc, 0, PLAN | pn.FLAG_BOUNDS)
+    assert plain.codegen(0, compile=True) == checked.codegen(0, compile=True)   # same program; the switch is a macro
+    assert _status(w.desc, PLAN | pn.FLAG_BOUNDS | pn.FLAG_UNFUSED | pn.FLAG_STATIC_SCRATCH) == -1
