@@ -828,6 +828,7 @@ struct Interp {
                  io.map_mod[0], io.map_mod[1], io.map_mod[2], io.lead_stride[0], io.lead_stride[1], io.lead_stride[2]};
   }
   static constexpr int kWalkUnroll = 1;
+  static PN_DEV int block_threads() { return (int)blockDim.x; }
   static PN_DEV long long red_stride(const KernelParams& p, int io) { return p.io[io].red_stride; }
   static PN_DEV int col_tx(const KernelParams& p) { return p.col_tx; }
   static PN_DEV int red_len(const KernelParams& p) { return p.red_len; }
@@ -866,7 +867,8 @@ PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
   // thread computes the same values); the interpreter keeps them in shared memory
   constexpr bool kRegSlots = Prog::kStatic;
   constexpr bool kRegRowoff = Prog::kStatic;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+  const int bdim = Prog::block_threads();   // a constant in generated kernels
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = bdim >> 5;
   const int family = Prog::family(p);
   const int cluster = Prog::cluster(p);
   const int chunks = Prog::chunks(p);
@@ -876,7 +878,7 @@ PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
   // of TL lanes; the shuffles of a combine then stop at lane distance TL / 2.
   const int TL = warp_team ? Prog::team_lanes(p) : 32;
   const int sub = TL < 32 ? lane / TL : 0;              // which of the warp's teams this lane is in
-  const int team_threads = warp_team ? TL : (int)blockDim.x;
+  const int team_threads = warp_team ? TL : bdim;
   const int team_tid = warp_team ? (TL < 32 ? lane % TL : lane) : tid;
   const int team_in_cta = warp_team ? warp : 0;
   const int crank = (cluster > 1) ? (int)cluster_ctarank() : 0;
@@ -893,7 +895,7 @@ PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
   TileCtx cx;
   cx.rowoff = kRegRowoff ? rowoff_reg : rowoff_sm;
   cx.part = reinterpret_cast<float*>(smem + p.sm_part) + tid;
-  cx.part_stride = blockDim.x;
+  cx.part_stride = bdim;
   cx.slots = slots;
   cx.stash = reinterpret_cast<float*>(smem + p.sm_stash) + tid;
   cx.gstride = team_threads * VL;
@@ -1143,7 +1145,7 @@ template <class Prog>
 PN_DEV void column_body(const KernelParams& p, unsigned char* smem) {
   constexpr int VL = Prog::VL, NG = Prog::NG, K = Prog::K, V = VL * NG;
   constexpr int kAcc = K < kMaxRed ? K : kMaxRed;
-  const int tid = threadIdx.x, nthreads = blockDim.x;
+  const int tid = threadIdx.x, nthreads = Prog::block_threads();   // a constant in generated kernels
   const int TX = Prog::col_tx(p), TY = nthreads / TX;
   const int tx = tid % TX, ty = tid / TX;
   const int R = Prog::red_len(p);
@@ -1186,8 +1188,10 @@ PN_DEV void column_body(const KernelParams& p, unsigned char* smem) {
         PN_UNROLL for (int e = 0; e < V; ++e) reg[r][e] = ident;
       }
     }
+    long long item_off[Prog::kNumIo];   // offset of this item's first step in every input / output
+    PN_UNROLL for (int q = 0; q < Prog::kNumIo; ++q) item_off[q] = o * Prog::lead_stride(p, q, 2);
     auto at_step = [&](int s) {
-      PN_UNROLL for (int q = 0; q < Prog::kNumIo; ++q) rowoff[q] = o * Prog::lead_stride(p, q, 2) + s * Prog::red_stride(p, q);
+      PN_UNROLL for (int q = 0; q < Prog::kNumIo; ++q) rowoff[q] = item_off[q] + s * Prog::red_stride(p, q);
     };
     if constexpr (kPf > 0) {
       // U steps at a time: all their loads are issued, then their arithmetic runs in step order.
@@ -1232,7 +1236,7 @@ PN_DEV void column_body(const KernelParams& p, unsigned char* smem) {
       }
     }
     if (ty == 0) {
-      PN_UNROLL for (int q = 0; q < Prog::kNumIo; ++q) rowoff[q] = o * Prog::lead_stride(p, q, 2);
+      PN_UNROLL for (int q = 0; q < Prog::kNumIo; ++q) rowoff[q] = item_off[q];
       Prog::tile(p, 1, cx, acc, reg, ts, parts, raw[0], cx, false);
     }
     if (TY > 1) __syncthreads();   // the next item rewrites the staging area

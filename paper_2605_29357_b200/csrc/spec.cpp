@@ -210,6 +210,11 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
   s += kDeviceSource;
   s += "\nnamespace pn {\nstruct Spec {\n";
   s += "  static constexpr int VL = " + I(lp.vl) + ", NG = " + I(lp.ng) + ", K = " + I(lp.k) + ";\n";
+  // The block size as a constant folds the address arithmetic of a tile into the loads' immediate
+  // offsets.  Not for rows streamed in several chunks by a block or cluster: there the constant
+  // costs registers (47 against 32 on the gated multi-output workload), hence resident warps.
+  const bool const_block = !((P.family == FAM_BLOCK || P.family == FAM_CLUSTER) && P.chunks > 1);
+  s += "  static PN_DEV int block_threads() { return " + (const_block ? I(lp.block) : std::string("(int)blockDim.x")) + "; }\n";
   s += "  static constexpr bool kStatic = true;\n  static constexpr int kStages = " + I(P.n_stages) + ";\n";
   s += "  static constexpr int kFamily = " + I(P.family) + ", kNumIo = " + I(P.n_io) + ";\n";
   s += "  static PN_DEV unsigned lead_dim(const KernelParams&, int i) { return i == 0 ? " + I(P.lead_dim[0]) + "u : i == 1 ? " +
