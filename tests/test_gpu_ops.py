@@ -284,6 +284,11 @@ def test_short_rows_that_share_a_warp(rows, n, dtype):
     g.mark_output(mean); g.mark_output(rstd)
     g.mark_output(g.op("argmax", [xf], D.I64, (rows,)))
     g.mark_output(g.op("sum", [xf], D.F32, (rows, 1)))
+    for flags in (pn.FLAG_PREFETCH, pn.FLAG_NO_HOIST, pn.FLAG_BOUNDS):     # loads issued a tile ahead, nothing hoisted, checked
+        hf = pn.Graph(g.build(), 0, flags)
+        check_against_oracle(g.build(), [xs, gamma, beta], run_graph(hf, [xs, gamma, beta]), [g.tensor_meta(t) for t in g.output_ids()])
+        if flags == pn.FLAG_BOUNDS:
+            assert hf.bounds_status == 0
     h = pn.Graph(g.build(), 0, 0)
     k = h.kernel_info[0]
     assert pn.FAMILY_NAMES[k["family"]] == "warp-per-row"
