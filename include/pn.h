@@ -174,7 +174,13 @@ pn_status pn_graph_run(pn_graph_t* g, const void* const* inputs, int n_inputs,
  * tensors live in HOST memory: copies each input to the device, runs, copies each output
  * back and waits.  `inputs` / `outputs` are HOST arrays of HOST pointers to dense buffers
  * of the sizes the descriptor states (pinned memory lets the copies run at full speed).
- * Staging buffers are allocated on first use and owned by the handle.
+ * Staging buffers are allocated on first use and owned by the handle.  When the inputs are
+ * large (tens of MB) and the work of a fused handle can be cut along its outermost dimension,
+ * the call works in pieces: the copy in of one piece, the kernel on the piece before and the
+ * copy out of the one before that run at the same time, on two copy streams of the handle's
+ * own beside `stream`, so that both directions of the host link are busy; tensors without the
+ * outermost dimension (broadcast operands) are copied whole first.  The results are the same
+ * bits as in one piece.  The call returns when everything has arrived.
  */
 pn_status pn_graph_run_host(pn_graph_t* g, const void* const* inputs, int n_inputs,
                             void* const* outputs, int n_outputs, void* stream);

@@ -251,20 +251,120 @@ pn_status pn_graph_run_host(pn_graph_t* h, const void* const* inputs, int n_inpu
         (pass == 0 ? h->stage_in : h->stage_out).push_back(p);
       }
   }
-  for (int i = 0; i < n_inputs; ++i) {
-    if (!inputs[i]) return fail(PN_ERR_INVALID_ARG, "input " + std::to_string(i) + " is null");
-    e = cudaMemcpyAsync(h->stage_in[i], inputs[i], (size_t)tensor_bytes(g.tensors[g.inputs[i]]), cudaMemcpyHostToDevice, s);
-    if (e != cudaSuccess) return fail(PN_ERR_CUDA, std::string("copy in: ") + cudaGetErrorString(e));
+  for (int i = 0; i < n_inputs; ++i) if (!inputs[i]) return fail(PN_ERR_INVALID_ARG, "input " + std::to_string(i) + " is null");
+  for (int i = 0; i < n_outputs; ++i) if (!outputs[i]) return fail(PN_ERR_INVALID_ARG, "output " + std::to_string(i) + " is null");
+
+  // ---- can the work be cut into pieces along its outermost dimension? ----------------------
+  // A fused launch walks its work items in order of the outermost leading dimension, and every
+  // dense tensor that has that dimension holds one contiguous slab per index of it.  Then the copy
+  // in of piece k + 1, the kernel on piece k and the copy out of piece k - 1 run at the same time
+  // (the two copy directions use the link in both directions at once).
+  struct Cut { int64_t outer = 0, items_per_outer = 0; std::vector<int64_t> stride; } cut;   // stride in elements per outer index; 0 = whole tensor
+  int64_t in_bytes = 0;
+  for (int t : g.inputs) in_bytes += tensor_bytes(g.tensors[t]);
+  if (h->launches.size() == 1 && in_bytes >= (8ll << 20)) {
+    const LaunchPlan& lp = h->launches[0].plan;
+    const KernelParams& P = lp.p;
+    bool ok = P.cluster >= 1;
+    for (int q = 0; q < P.n_io; ++q) ok = ok && !P.io[q].mapped;
+    cut.stride.assign(P.n_io, 0);
+    if (ok && P.family == FAM_COLUMN) {
+      cut.outer = P.rows; cut.items_per_outer = P.chunks;
+      for (int q = 0; q < P.n_io; ++q) cut.stride[q] = P.io[q].lead_stride[2];
+    } else if (ok && P.split_chunks && P.rows == 1) {
+      const int64_t chunk_cols = 32ll * lp.vl * lp.ng;
+      cut.outer = P.chunks; cut.items_per_outer = 1;
+      for (int q = 0; q < P.n_io; ++q) cut.stride[q] = P.io[q].col_stride ? chunk_cols : 0;
+    } else if (ok) {
+      int d0 = -1;
+      for (int i = 0; i < 3 && d0 < 0; ++i) if (P.lead_dim[i] > 1) d0 = i;
+      if (d0 >= 0) {
+        cut.outer = P.lead_dim[d0];
+        cut.items_per_outer = P.rows / cut.outer * (P.split_chunks ? P.chunks : 1);
+        for (int q = 0; q < P.n_io; ++q) cut.stride[q] = P.io[q].lead_stride[d0];
+      }
+    }
+    for (int q = 0; q < P.n_io && cut.outer > 0; ++q)
+      if (h->launches[0].src[q].kind == 1 && cut.stride[q] == 0) cut.outer = 0;   // an output without the outer dimension
   }
-  st = pn_graph_run(h, (const void* const*)h->stage_in.data(), n_inputs, h->stage_out.data(), n_outputs, stream);
-  if (st != PN_OK) return st;
-  for (int i = 0; i < n_outputs; ++i) {
-    if (!outputs[i]) return fail(PN_ERR_INVALID_ARG, "output " + std::to_string(i) + " is null");
-    e = cudaMemcpyAsync(outputs[i], h->stage_out[i], (size_t)tensor_bytes(g.tensors[g.outputs[i]]), cudaMemcpyDeviceToHost, s);
-    if (e != cudaSuccess) return fail(PN_ERR_CUDA, std::string("copy out: ") + cudaGetErrorString(e));
+  const int pieces = (int)std::min<int64_t>(std::min<int64_t>(cut.outer, 16), std::max<int64_t>(1, in_bytes / (24ll << 20)));
+  if (pieces < 2) {   // plain: copy in, run, copy out
+    for (int i = 0; i < n_inputs; ++i) {
+      e = cudaMemcpyAsync(h->stage_in[i], inputs[i], (size_t)tensor_bytes(g.tensors[g.inputs[i]]), cudaMemcpyHostToDevice, s);
+      if (e != cudaSuccess) return fail(PN_ERR_CUDA, std::string("copy in: ") + cudaGetErrorString(e));
+    }
+    st = pn_graph_run(h, (const void* const*)h->stage_in.data(), n_inputs, h->stage_out.data(), n_outputs, stream);
+    if (st != PN_OK) return st;
+    for (int i = 0; i < n_outputs; ++i) {
+      e = cudaMemcpyAsync(outputs[i], h->stage_out[i], (size_t)tensor_bytes(g.tensors[g.outputs[i]]), cudaMemcpyDeviceToHost, s);
+      if (e != cudaSuccess) return fail(PN_ERR_CUDA, std::string("copy out: ") + cudaGetErrorString(e));
+    }
+    e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return fail(PN_ERR_CUDA, std::string("sync: ") + cudaGetErrorString(e));
+    return PN_OK;
   }
+
+  // ---- pipelined: copy-in stream, the caller's stream for the kernels, copy-out stream -----------
+  if (!h->copy_in) {
+    cudaStream_t a = nullptr, b = nullptr;
+    e = cudaStreamCreateWithFlags(&a, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&b, cudaStreamNonBlocking);
+    if (e != cudaSuccess) { if (a) cudaStreamDestroy(a); return fail(PN_ERR_CUDA, std::string("copy streams: ") + cudaGetErrorString(e)); }
+    h->copy_in = a; h->copy_out = b;
+  }
+  while ((int)h->pipe_events.size() < 2 * pieces + 1) {
+    cudaEvent_t ev = nullptr;
+    e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+    if (e != cudaSuccess) return fail(PN_ERR_CUDA, std::string("events: ") + cudaGetErrorString(e));
+    h->pipe_events.push_back(ev);
+  }
+  cudaStream_t s_in = (cudaStream_t)h->copy_in, s_out = (cudaStream_t)h->copy_out;
+  PlannedLaunch& pl = h->launches[0];
+  auto ev = [&](int i) { return (cudaEvent_t)h->pipe_events[i]; };
+  auto check = [&](cudaError_t err, const char* what) { return err == cudaSuccess ? PN_OK : fail(PN_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(err)); };
+  // what the caller queued on its stream comes first
+  if ((st = check(cudaEventRecord(ev(2 * pieces), s), "event")) != PN_OK) return st;
+  if ((st = check(cudaStreamWaitEvent(s_in, ev(2 * pieces), 0), "wait")) != PN_OK) return st;
+  // tensors without the outer dimension: whole, before the first piece
+  for (int q = 0; q < pl.plan.p.n_io; ++q) {
+    const IoSource& src = pl.src[q];
+    if (src.kind != 0 || cut.stride[q] != 0) continue;
+    e = cudaMemcpyAsync(h->stage_in[src.index], inputs[src.index], (size_t)tensor_bytes(g.tensors[g.inputs[src.index]]), cudaMemcpyHostToDevice, s_in);
+    if ((st = check(e, "copy in")) != PN_OK) return st;
+  }
+  pn_status result = PN_OK;
+  for (int k = 0; k < pieces && result == PN_OK; ++k) {
+    const int64_t a = cut.outer * k / pieces, b = cut.outer * (k + 1) / pieces;
+    for (int q = 0; q < pl.plan.p.n_io && result == PN_OK; ++q) {
+      const IoSource& src = pl.src[q];
+      if (src.kind != 0 || cut.stride[q] == 0) continue;
+      const Tensor& T = g.tensors[g.inputs[src.index]];
+      const int64_t es = dtype_bytes(T.dtype), lo = a * cut.stride[q], hi = std::min<int64_t>(b * cut.stride[q], T.numel());
+      if (hi > lo) result = check(cudaMemcpyAsync((char*)h->stage_in[src.index] + lo * es, (const char*)inputs[src.index] + lo * es, (size_t)((hi - lo) * es), cudaMemcpyHostToDevice, s_in), "copy in");
+    }
+    if (result == PN_OK) result = check(cudaEventRecord(ev(2 * k), s_in), "event");
+    if (result == PN_OK) result = check(cudaStreamWaitEvent(s, ev(2 * k), 0), "wait");
+    if (result != PN_OK) break;
+    pl.plan.p.item_begin = a * cut.items_per_outer;
+    pl.plan.p.item_end = b * cut.items_per_outer;
+    result = pn_graph_run(h, (const void* const*)h->stage_in.data(), n_inputs, h->stage_out.data(), n_outputs, stream);
+    pl.plan.p.item_begin = pl.plan.p.item_end = 0;
+    if (result == PN_OK) result = check(cudaEventRecord(ev(2 * k + 1), s), "event");
+    if (result == PN_OK) result = check(cudaStreamWaitEvent(s_out, ev(2 * k + 1), 0), "wait");
+    for (int q = 0; q < pl.plan.p.n_io && result == PN_OK; ++q) {
+      const IoSource& src = pl.src[q];
+      if (src.kind != 1) continue;
+      const Tensor& T = g.tensors[g.outputs[src.index]];
+      const int64_t es = dtype_bytes(T.dtype), lo = a * cut.stride[q], hi = std::min<int64_t>(b * cut.stride[q], T.numel());
+      if (hi > lo) result = check(cudaMemcpyAsync((char*)outputs[src.index] + lo * es, (const char*)h->stage_out[src.index] + lo * es, (size_t)((hi - lo) * es), cudaMemcpyDeviceToHost, s_out), "copy out");
+    }
+  }
+  // wait for everything that was queued, also after a failure
+  cudaStreamSynchronize(s_in);
   e = cudaStreamSynchronize(s);
-  if (e != cudaSuccess) return fail(PN_ERR_CUDA, std::string("sync: ") + cudaGetErrorString(e));
+  const cudaError_t e2 = cudaStreamSynchronize(s_out);
+  if (result != PN_OK) return result;
+  if (e != cudaSuccess || e2 != cudaSuccess) return fail(PN_ERR_CUDA, std::string("sync: ") + cudaGetErrorString(e != cudaSuccess ? e : e2));
   return PN_OK;
 }
 
@@ -273,6 +373,9 @@ pn_status pn_graph_destroy(pn_graph_t* h) {
   if (!h->plan_only) {
     if (h->workspace) cudaFree(h->workspace);
     if (h->status) cudaFree(h->status);
+    if (h->copy_in) cudaStreamDestroy((cudaStream_t)h->copy_in);
+    if (h->copy_out) cudaStreamDestroy((cudaStream_t)h->copy_out);
+    for (void* ev : h->pipe_events) cudaEventDestroy((cudaEvent_t)ev);
     for (void* p : h->stage_in) cudaFree(p);
     for (void* p : h->stage_out) cudaFree(p);
   }

@@ -903,7 +903,7 @@ PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
   cx.chunk = 0;
   cx.leader = (team_tid == 0) && (crank == 0);
 
-  const long long n_items = split ? p.rows * chunks : p.rows;
+  const long long n_items = p.item_end > 0 ? p.item_end : (split ? p.rows * chunks : p.rows);
   long long team_global, n_teams;
   if (warp_team) {
     const int per_warp = 32 / TL;
@@ -911,6 +911,7 @@ PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
   }
   else { team_global = blockIdx.x / cluster; n_teams = gridDim.x / cluster; }
 
+  if (p.item_end > 0) team_global += p.item_begin;   // a launch over part of the work
   const int slice_lo = crank * Prog::slice_len(p);
   cx.col_end = min(Prog::row_len(p), slice_lo + Prog::slice_len(p));
   const int chunk_cols = team_threads * V;
@@ -1177,8 +1178,8 @@ PN_DEV void column_body(const KernelParams& p, unsigned char* smem) {
   PN_UNROLL for (int u = 0; u < U; ++u) { PN_UNROLL for (int j = 0; j < (kPf > 0 ? kPf : 1); ++j) { PN_UNROLL for (int e = 0; e < V; ++e) raw[u][j][e] = 0.f; } }
   PN_UNROLL for (int r = 0; r < kMaxRed; ++r) parts[r] = Part{0.f, 0.f, 0.f};
 
-  const long long n_items = p.rows * n_ctiles;
-  for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
+  const long long n_items = p.item_end > 0 ? p.item_end : p.rows * n_ctiles;
+  for (long long item = (p.item_end > 0 ? p.item_begin : 0) + blockIdx.x; item < n_items; item += gridDim.x) {
     const long long o = item / n_ctiles;
     const int ct = (int)(item - o * n_ctiles);
     cx.col0 = ct * (TX * V) + tx * VL;

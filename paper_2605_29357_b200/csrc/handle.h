@@ -34,5 +34,8 @@ struct pn_graph {
   size_t workspace_bytes = 0;
   int64_t compulsory_bytes = 0;
   std::vector<void*> stage_in, stage_out;   // device staging of pn_graph_run_host
+  void* copy_in = nullptr;                  // streams and events of the pipelined pn_graph_run_host
+  void* copy_out = nullptr;                 // (cudaStream_t / cudaEvent_t, created on first use)
+  std::vector<void*> pipe_events;
   uint32_t* status = nullptr;               // device word of the checked accessors (PN_FLAG_BOUNDS)
 };

@@ -145,6 +145,8 @@ struct KernelParams {
   // 0 .. n_red-1, stage 1 runs once per (row, column tile) on the combined registers.
   int32_t red_len;
   int32_t col_tx;
+  int64_t item_begin, item_end;   // item_end > 0: this launch does the work items [item_begin, item_end) only
+                                  // (rows, or (row, chunk) / (row, column tile) pairs in launch order)
   uint32_t* status;        // checked accessors (PN_FLAG_BOUNDS): bit q is set when an access to io entry q
                            // fell outside its tensor; null when checking is off
   int32_t team_lanes;      // warp-per-row kernels: lanes per row (32, or 16 / 8 when short rows share a warp)
