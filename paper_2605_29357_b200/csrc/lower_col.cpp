@@ -312,6 +312,18 @@ int lower_column_graph(const Graph& g, unsigned flags, const DeviceModel& dev, L
   // contiguous bytes per step); the rest of the block splits R
   int TX = 1;
   while (TX < 32 && (int64_t)TX * VL * NG < C) TX *= 2;
+  // Few (row, column tile) items for the size of the GPU: more walkers per item first (blocks of up
+  // to 512 threads, while every walker keeps a batch of steps), then narrower column tiles (down to
+  // 8 threads: 128 contiguous bytes per step and item), then blocks of 1024.  This is what keeps a
+  // small batch of long sequences from running on a handful of SMs.
+  if (spec && !t_block) {
+    const int64_t want = (int64_t)dev.sm_count * 512;   // threads for a quarter of the resident capacity
+    auto threads = [&](int tx, int blk) { return O * ((C + (int64_t)tx * VL * NG - 1) / ((int64_t)tx * VL * NG)) * blk; };
+    auto steps_ok = [&](int tx, int blk) { return R / (blk / tx) >= 8; };
+    while (threads(TX, block) < want && block < 512 && steps_ok(TX, block * 2)) block *= 2;
+    while (threads(TX, block) < want && TX > 8 && (int64_t)(TX / 2) * VL * NG * 2 <= C * 2 && steps_ok(TX / 2, block)) TX /= 2;
+    while (threads(TX, block) < want && block < 1024 && steps_ok(TX, block * 2)) block *= 2;
+  }
   const int64_t ctile = (int64_t)TX * VL * NG;
   const int64_t n_ctiles = (C + ctile - 1) / ctile;
 
