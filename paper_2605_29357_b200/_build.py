@@ -17,6 +17,7 @@ LIB = os.path.join(HERE, "libpn.so")
 SOURCES = ["kernels.cu", "no_alloc.cu", "lower.cpp", "lower_col.cpp", "descriptor.cpp", "spec.cpp", "api.cpp", "sequence.cpp"]
 HEADERS = [os.path.join(CSRC, "plan.h"), os.path.join(CSRC, "graph.h"), os.path.join(CSRC, "spec.h"), os.path.join(CSRC, "handle.h"), os.path.join(CSRC, "lower_common.h"),
            os.path.join(CSRC, "device_lib.cuh"), os.path.join(INCLUDE, "pn.h")]
+INSTANCES = [(1, 8, 4), (4, 2, 4), (4, 4, 2), (8, 1, 4), (8, 2, 2)]   # (VL, NG, K), as listed in kernels.cu
 FLAGS = ["-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
          "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
 
@@ -49,16 +50,28 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     nvcc = _nvcc()
     newest_header = max(os.path.getmtime(h) for h in HEADERS)
     objs, relink = [], force or not os.path.exists(LIB)
-    for src in SOURCES:
+    jobs = []
+    units = [(src, src + ".o", []) for src in SOURCES]
+    # the interpreter kernels: one translation unit per tile shape, so that they build side by side
+    units += [("kernels.cu", "kernels_%d_%d_%d.o" % inst, ["-DPN_VL=%d" % inst[0], "-DPN_NG=%d" % inst[1], "-DPN_K=%d" % inst[2]])
+              for inst in INSTANCES]
+    for src, obj, defs in units:
         s = os.path.join(CSRC, src)
-        o = os.path.join(OBJ, src + ".o")
+        o = os.path.join(OBJ, obj)
         objs.append(o)
         if force or not os.path.exists(o) or os.path.getmtime(o) < max(os.path.getmtime(s), newest_header):
-            cmd = [nvcc, "-c", *FLAGS, "-o", o, s]
+            jobs.append([nvcc, "-c", *FLAGS, *defs, "-o", o, s])
+    if jobs:   # the translation units are independent: compile them side by side
+        from concurrent.futures import ThreadPoolExecutor
+
+        def run(cmd):
             if verbose:
                 print(" ".join(cmd), file=sys.stderr)
             subprocess.run(cmd, check=True)
-            relink = True
+
+        with ThreadPoolExecutor(max_workers=min(len(jobs), os.cpu_count() or 1)) as pool:
+            list(pool.map(run, jobs))
+        relink = True
     if relink or any(os.path.getmtime(o) > os.path.getmtime(LIB) for o in objs):
         subprocess.run([nvcc, "-shared", "-o", LIB, *objs], check=True)
     return LIB
