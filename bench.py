@@ -76,7 +76,7 @@ def measured_peak():
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap,clocks.mem")
 
     def __init__(self, index):
         self.index, self.proc, self.lines = index, None, []
@@ -103,7 +103,7 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             pass
-        sm, mx, reasons = [], [], set()
+        sm, mx, mem, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for ln in self.lines:
             f = [x.strip() for x in ln.split(",")]
@@ -116,8 +116,12 @@ class ClockSampler:
             for n, v in zip(names, f[2:6]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
+            try:
+                mem.append(float(f[6]))
+            except (IndexError, ValueError):
+                pass
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "mem_mhz": float(np.median(mem)) if mem else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
 def driver_version():
@@ -303,6 +307,17 @@ def _c2_descriptor(b, q, k):
         finally:
             C._draw = real
     return _C2_DESC[key]
+
+
+def cpu_model():
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.startswith("model name"):
+                    return line.split(":", 1)[1].strip()
+    except Exception:
+        pass
+    return None
 
 
 def oracle_threads():
@@ -522,7 +537,7 @@ def main():
     t_or = time_oracle(sample, 2, block=32)
     line["cpu_baseline"] = {"value": sample.compulsory_bytes / t_or / 1e9, "unit": "GB/s", "cores": oracle_threads(),
                             "kind": "oracle", "sample": "all 512 batches of the c2 workload (134 M elements), evaluated 32 batches at a time, best of 2",
-                            "seconds": t_or}
+                            "seconds": t_or, "cpu_model": cpu_model(), "host_cores": os.cpu_count()}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
