@@ -444,8 +444,27 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     }
   }
   int VL = (min_esize <= 2 && vec8) ? 8 : (vec4 ? 4 : 1);
-  if (flags & PN_FLAG_FORCE_SCALAR) VL = 1;
   const bool spec = dev.specialise;
+  // A group of 8 elements of a 4-byte operand is two 128-bit accesses 32 bytes apart from lane to
+  // lane: each touches every 128-byte line of the warp's span and uses half of it, so the operand
+  // costs twice the L1 wavefronts.  Measured on the residual + LayerNorm workload (bf16 rows, fp32
+  // gamma and beta re-read by every row): the L1 data pipe at 74 % with groups of 8, and 73.7 ->
+  // 66.4 us with groups of 4 (the 2-byte rows then move in 64-bit accesses, which stay whole).
+  // Groups of 8 are kept where such operands are loaded once per thread, not per row: the
+  // warp-per-row kernels, which pin row-invariant operands in registers.
+  if (VL == 8 && vec4) {
+    bool wide_per_row = false, wide_varying = false;
+    for (int q = 0; q < n_io; ++q) {
+      const IoDesc& io = P.io[q];
+      if (io.is_row_scalar || io.col_stride == 0 || dtype_bytes(io.dtype) < 4) continue;
+      wide_per_row = true;
+      if (io.mapped || io.lead_stride[0] != 0 || io.lead_stride[1] != 0 || io.lead_stride[2] != 0 || lp.io_is_output[q]) wide_varying = true;
+    }
+    const bool pinned_in_warp = has_red && spec && !wide_varying && eff_N <= 32 * 64 &&
+                                !(flags & (PN_FLAG_FORCE_BLOCK | PN_FLAG_FORCE_CLUSTER | PN_FLAG_FORCE_MULTICHUNK | PN_FLAG_NO_HOIST));
+    if (wide_per_row && !pinned_in_warp) VL = 4;
+  }
+  if (flags & PN_FLAG_FORCE_SCALAR) VL = 1;
   std::vector<std::pair<int, int>> ng_opts;   // (NG, K): the 8-element tile first
   if (VL == 8) ng_opts = {{1, 4}, {2, 2}};
   else if (VL == 4) ng_opts = {{2, 4}, {4, 2}};

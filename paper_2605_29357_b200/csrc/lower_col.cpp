@@ -294,6 +294,11 @@ int lower_column_graph(const Graph& g, unsigned flags, const DeviceModel& dev, L
     }
   }
   int VL = (min_esize <= 2 && vec8) ? 8 : (vec4 ? 4 : 1);
+  // groups of 8 elements of a 4-byte operand read at every step are two half-used 128-bit accesses
+  // (see lower.cpp): such graphs take groups of 4
+  if (VL == 8 && vec4)
+    for (int q = 0; q < n_io; ++q)
+      if (P.io[q].col_stride != 0 && io_streamed[q] && dtype_bytes(P.io[q].dtype) >= 4) VL = 4;
   if (flags & PN_FLAG_FORCE_SCALAR) VL = 1;
   const bool spec = dev.specialise;
   // (NG, K): the interpreter's instances with four tile registers; generated kernels take one
