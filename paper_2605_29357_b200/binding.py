@@ -180,6 +180,19 @@ class Graph:
                                       self._ptr_array(output_ptrs), len(output_ptrs),
                                       ctypes.c_void_p(stream)), "pn_graph_run")
 
+    def bind(self, input_ptrs: Sequence[int], output_ptrs: Sequence[int]):
+        """A callable `f(stream=0)` that enqueues one evaluation on these device pointers.  The
+        pointer arrays are marshalled once, so that a caller who launches the same buffers many
+        times pays only the call itself."""
+        ins, outs = self._ptr_array(input_ptrs), self._ptr_array(output_ptrs)
+        n_in, n_out, fn, h = len(input_ptrs), len(output_ptrs), self._lib.pn_graph_run, self._h
+
+        def launch(stream: int = 0, _vp=ctypes.c_void_p) -> None:
+            st = fn(h, ins, n_in, outs, n_out, _vp(stream))
+            if st != PN_OK:
+                _check(st, "pn_graph_run")
+        return launch
+
     def run_host(self, input_ptrs: Sequence[int], output_ptrs: Sequence[int], stream: int = 0) -> None:
         """Evaluate on HOST buffers (addresses): copy in, run, copy out, wait."""
         _check(self._lib.pn_graph_run_host(self._h, self._ptr_array(input_ptrs), len(input_ptrs),
