@@ -56,3 +56,23 @@ def test_unfused_handle_through_host_memory():
     g = pn.Graph(w.desc, 0, pn.FLAG_UNFUSED)
     got = _run_host(g, w, True)
     check_against_oracle(w.desc, w.inputs, got, w.output_meta, w.output_names)
+
+
+def test_bound_launch_equals_plain_run():
+    """Graph.bind marshals the pointer arrays once; launching through it gives the same bits."""
+    import torch
+    from gpu_util import device_bytes, poisoned
+    w = C.c5(**C.SMALL["c5"])
+    g = pn.Graph(w.desc, 0, 0)
+    ref = run_graph(g, w.inputs)
+    d_in = [device_bytes(a) for a in w.inputs]
+    sizes = [D.DTYPE_BYTES[dt] * int(np.prod(dims, dtype=np.int64)) for dt, dims in w.output_meta]
+    d_out = [poisoned(s) for s in sizes]
+    launch = g.bind([t.data_ptr() for t in d_in], [t.data_ptr() for t in d_out])
+    for _ in range(2):
+        launch(torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    for t, (dt, dims), s, r in zip(d_out, w.output_meta, sizes, ref):
+        assert np.array_equal(t.cpu().numpy()[:s].view(C.NP_STORAGE[dt]).reshape(dims), r, equal_nan=True)
+    with pytest.raises(pn.PnError):
+        g.bind([t.data_ptr() for t in d_in][:-1], [t.data_ptr() for t in d_out])(0)
