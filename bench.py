@@ -45,7 +45,7 @@ def kernel_identity(g):
     hash of the device library it is compiled against."""
     import hashlib
     import re
-    m = re.search(r"__global__ void PN_BOUNDS (\w+)\(", g.codegen(0))
+    m = re.search(r"__global__ void PN_LAUNCH_BOUNDS (\w+)\(", g.codegen(0))
     name = m.group(1) if m else "interpreter"
     lib = os.path.join(ROOT, "paper_2605_29357_b200", "csrc", "device_lib.cuh")
     with open(lib, "rb") as f:

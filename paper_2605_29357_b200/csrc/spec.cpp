@@ -314,9 +314,9 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
   // beats every larger budget on the pooling workload).
   const int min_blocks = ((P.family == FAM_BLOCK && P.chunks == 1) || P.family == FAM_COLUMN) ? std::max(1, 1024 / lp.block) : 1;
   s += "#ifndef PN_MIN_BLOCKS\n#define PN_MIN_BLOCKS " + I(min_blocks) + "\n#endif\n";
-  s += "#if PN_MIN_BLOCKS > 1\n#define PN_BOUNDS __launch_bounds__(" + I(lp.block) + ", PN_MIN_BLOCKS)\n#else\n"
-       "#define PN_BOUNDS __launch_bounds__(" + I(lp.block) + ")\n#endif\n";
-  s += "extern \"C\" __global__ void PN_BOUNDS " + kernel_name(lp) + "(const __grid_constant__ pn::KernelParams p) {\n"
+  s += "#if PN_MIN_BLOCKS > 1\n#define PN_LAUNCH_BOUNDS __launch_bounds__(" + I(lp.block) + ", PN_MIN_BLOCKS)\n#else\n"
+       "#define PN_LAUNCH_BOUNDS __launch_bounds__(" + I(lp.block) + ")\n#endif\n";
+  s += "extern \"C\" __global__ void PN_LAUNCH_BOUNDS " + kernel_name(lp) + "(const __grid_constant__ pn::KernelParams p) {\n"
        "  extern __shared__ __align__(16) unsigned char smem[];\n  pn::" + std::string(P.family == FAM_COLUMN ? "column_body" : "fused_body") + "<pn::Spec>(p, smem);\n}\n";
   src.swap(s);
   return true;

@@ -147,7 +147,7 @@ def test_generated_kernels_compile(cfg, flags):
     w = C.CONFIGS[cfg](**C.SMALL[cfg])
     g = pn.Graph(w.desc, 0, PLAN | flags)
     src = g.codegen(0, compile=True)
-    assert "__global__ void PN_BOUNDS pn_spec_" in src and "struct Spec" in src
+    assert "__global__ void PN_LAUNCH_BOUNDS pn_spec_" in src and "struct Spec" in src
 
 
 def test_forced_families():
