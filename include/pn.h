@@ -112,6 +112,7 @@ enum {
 #define PN_TUNE_CLUSTER(n) (((unsigned)(n) & 15u) << 16)      /* CTAs per cluster: 2, 4, 8      */
 #define PN_TUNE_BLOCK_LOG2(n) (((unsigned)(n) & 15u) << 20)   /* threads per block = 1 << n     */
 #define PN_TUNE_GROUPS(n) (((unsigned)(n) & 31u) << 24)       /* vector groups per thread tile  */
+#define PN_TUNE_WAVES(n) (((unsigned)(n) & 7u) << 29)         /* grid <= 2^(n-1) x the resident CTAs; 7: one CTA per work item */
 
 /* pn_graph_query selectors; each writes int64 values into `out` */
 enum {
@@ -287,6 +288,47 @@ pn_status pn_graph_query(const pn_graph_t* g, int what, void* out, size_t out_by
  */
 pn_status pn_graph_codegen(const pn_graph_t* g, int kernel, int compile, char* out, size_t out_bytes,
                            size_t* needed);
+
+/*
+ * pn_stream_probe -- a streaming kernel that only moves bytes, for the roofline: the rate it
+ * reaches in a given read : write mix is the ceiling that a fused kernel of the same mix can be
+ * judged against (the paper times whole subgraphs, Appendix C's protocol, and has no counterpart
+ * to a bandwidth ceiling; this call is a measuring aid, not part of evaluating f_G).
+ *   mix    : PN_MIX_READ   read a                      (a long-row reduction)
+ *            PN_MIX_WRITE  write c
+ *            PN_MIX_1_1    read a, write c             (softmax, a plain copy)
+ *            PN_MIX_2_1    read a and b, write c       (residual + LayerNorm)
+ *            PN_MIX_4_3    read a and b, write c and d (two 2-byte inputs, a 2-byte and a 1-byte output)
+ *   cfg    : HOST pointer; how to move them (see the struct).
+ *   a, b, c: DEVICE buffers of units * 16 bytes each; d of units * 8 bytes; those the mix does not
+ *            use may be NULL.  All aligned to 16 bytes; owned by the caller; a, b are only read.
+ *   units  : 16-byte units per array.
+ *   status_word : DEVICE pointer to 4 zeroed bytes (aligned to 16): bit 0 / 1 set when a bounded
+ *            wait of the bulk loader's producer / consumers ran out (the kernel then stops early,
+ *            after its copies in flight have landed); always 0 for the other loaders.
+ *   stream : a cudaStream_t.  Asynchronous; allocates nothing.
+ * Errors: PN_ERR_INVALID_ARG / PN_ERR_ALIGNMENT / PN_ERR_TOO_LARGE for a bad configuration,
+ * PN_ERR_CUDA for a failed launch.
+ */
+enum { PN_MIX_READ = 0, PN_MIX_WRITE = 1, PN_MIX_1_1 = 2, PN_MIX_2_1 = 3, PN_MIX_4_3 = 4 };
+enum {
+  PN_PROBE_LDG = 0,         /* 128-bit loads through the read-only path                      */
+  PN_PROBE_LDG_NOALLOC = 1, /* the same, not allocating in L1                                */
+  PN_PROBE_BULK = 2         /* 1-D bulk copies into a shared-memory ring (mbarrier completion;
+                               one extra producer warp per block; this GPU's memory only)    */
+};
+typedef struct pn_probe_config {
+  int loader;           /* PN_PROBE_*                                                         */
+  int streaming_stores; /* 1: stores carry the evict-first hint                               */
+  int layout;           /* direct loaders: 0 grid-stride over units, 1 a contiguous range per block */
+  int block;            /* threads that load / store per block (multiple of 32, <= 992)       */
+  int unroll;           /* direct loaders: units in flight per thread (1, 2, 4, 8)            */
+  int grid;             /* blocks                                                             */
+  int stages;           /* bulk loader: ring depth (2..16)                                    */
+  int tile_units;       /* bulk loader: units per array per stage (32..4096)                  */
+} pn_probe_config;
+pn_status pn_stream_probe(int mix, const pn_probe_config* cfg, const void* a, const void* b, void* c, void* d,
+                          size_t units, void* status_word, void* stream);
 
 /* Static text for a status code. */
 const char* pn_status_string(pn_status s);

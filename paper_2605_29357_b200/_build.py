@@ -14,7 +14,7 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 OBJ = os.path.join(CSRC, "_build")
 LIB = os.path.join(HERE, "libpn.so")
-SOURCES = ["kernels.cu", "no_alloc.cu", "lower.cpp", "lower_col.cpp", "descriptor.cpp", "spec.cpp", "api.cpp", "sequence.cpp"]
+SOURCES = ["kernels.cu", "no_alloc.cu", "probe.cu", "lower.cpp", "lower_col.cpp", "descriptor.cpp", "spec.cpp", "api.cpp", "sequence.cpp"]
 HEADERS = [os.path.join(CSRC, "plan.h"), os.path.join(CSRC, "graph.h"), os.path.join(CSRC, "spec.h"), os.path.join(CSRC, "handle.h"), os.path.join(CSRC, "lower_common.h"),
            os.path.join(CSRC, "device_lib.cuh"), os.path.join(INCLUDE, "pn.h")]
 INSTANCES = [(1, 8, 4), (4, 2, 4), (4, 4, 2), (8, 1, 4), (8, 2, 2)]   # (VL, NG, K), as listed in kernels.cu

@@ -30,10 +30,11 @@ FLAG_BOUNDS = 1 << 13
 STATIC_SCRATCH_BYTES = 32 << 20
 
 
-def tune(cluster: int = 0, block: int = 0, groups: int = 0) -> int:
-    """Flag bits overriding the lowering's cluster size, block size and groups per tile."""
+def tune(cluster: int = 0, block: int = 0, groups: int = 0, waves: int = 0) -> int:
+    """Flag bits overriding the lowering's cluster size, block size, groups per tile and grid size
+    (waves n: at most 2^(n-1) times the resident CTAs; 7: one CTA per work item)."""
     lg = block.bit_length() - 1 if block else 0
-    return ((cluster & 15) << 16) | ((lg & 15) << 20) | ((groups & 31) << 24)
+    return ((cluster & 15) << 16) | ((lg & 15) << 20) | ((groups & 31) << 24) | ((waves & 7) << 29)
 
 Q_N_INPUTS, Q_N_OUTPUTS, Q_INPUT_META, Q_OUTPUT_META, Q_COMPULSORY_BYTES = 1, 2, 3, 4, 5
 Q_N_KERNELS, Q_N_NODES, Q_WORKSPACE_BYTES, Q_KERNEL_INFO = 6, 7, 8, 9
@@ -41,8 +42,18 @@ Q_N_KERNELS, Q_N_NODES, Q_WORKSPACE_BYTES, Q_KERNEL_INFO = 6, 7, 8, 9
 FAMILY_NAMES = {0: "pointwise", 1: "warp-per-row", 2: "block-per-row", 3: "cluster-per-row", 4: "column-reduce"}
 EXPORTS = ["pn_graph_create", "pn_graph_run", "pn_graph_run_host", "pn_graph_run_static", "pn_graph_destroy",
            "pn_graph_query", "pn_graph_codegen", "pn_status_string", "pn_last_error",
-           "pn_sequence_create", "pn_sequence_run", "pn_sequence_query", "pn_sequence_destroy"]
+           "pn_sequence_create", "pn_sequence_run", "pn_sequence_query", "pn_sequence_destroy",
+           "pn_stream_probe"]
 SEQ_INDEPENDENT = 1 << 0
+MIX_READ, MIX_WRITE, MIX_1_1, MIX_2_1, MIX_4_3 = range(5)
+PROBE_LDG, PROBE_LDG_NOALLOC, PROBE_BULK = range(3)
+
+
+class ProbeConfig(ctypes.Structure):
+    """pn_probe_config: how pn_stream_probe moves its bytes."""
+    _fields_ = [("loader", ctypes.c_int), ("streaming_stores", ctypes.c_int), ("layout", ctypes.c_int),
+                ("block", ctypes.c_int), ("unroll", ctypes.c_int), ("grid", ctypes.c_int),
+                ("stages", ctypes.c_int), ("tile_units", ctypes.c_int)]
 
 
 class PnError(RuntimeError):
@@ -89,6 +100,8 @@ def load_library() -> ctypes.CDLL:
     lib.pn_sequence_query.argtypes = [vp, ctypes.c_int, vp, ctypes.c_size_t]
     lib.pn_sequence_destroy.restype = ctypes.c_int
     lib.pn_sequence_destroy.argtypes = [vp]
+    lib.pn_stream_probe.restype = ctypes.c_int
+    lib.pn_stream_probe.argtypes = [ctypes.c_int, ctypes.POINTER(ProbeConfig), vp, vp, vp, vp, ctypes.c_size_t, vp, vp]
     lib.pn_status_string.restype = ctypes.c_char_p
     lib.pn_status_string.argtypes = [ctypes.c_int]
     lib.pn_last_error.restype = ctypes.c_char_p
@@ -101,6 +114,14 @@ def _check(status: int, what: str) -> None:
     if status != PN_OK:
         lib = load_library()
         raise PnError(status, what + ": " + lib.pn_status_string(status).decode(), lib.pn_last_error().decode())
+
+
+def stream_probe(mix: int, cfg: ProbeConfig, a: int, b: int, c: int, d: int, units: int, status_word: int,
+                 stream: int = 0) -> None:
+    """pn_stream_probe on device pointers (integers; 0 for the buffers the mix does not use)."""
+    vp = ctypes.c_void_p
+    _check(load_library().pn_stream_probe(mix, ctypes.byref(cfg), vp(a), vp(b), vp(c), vp(d), units, vp(status_word),
+                                          vp(stream)), "pn_stream_probe")
 
 
 class Graph:

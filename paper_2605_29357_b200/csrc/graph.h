@@ -77,5 +77,6 @@ int lower_column_graph(const Graph& g, unsigned flags, const DeviceModel& dev, L
 
 // Grid size of a planned launch given the SM count and its kernel's resident CTAs per SM.
 void size_grid(LaunchPlan& lp, int sms, int occ);
+int tune_waves(unsigned flags);   // the PN_TUNE_WAVES field of the create flags as LaunchPlan::grid_waves
 
 }  // namespace pn

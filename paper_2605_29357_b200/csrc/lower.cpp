@@ -35,13 +35,18 @@ void size_grid(LaunchPlan& lp, int sms, int occ) {
   if (occ <= 0) occ = std::max(1, 512 / lp.block);
   const int64_t resident = (int64_t)sms * occ;
   const int cluster = std::max(lp.p.cluster, 1);
-  const int waves = lp.persistent ? 1 : 8;   // work hoisted out of the row loop wants long-lived CTAs
+  int64_t waves = lp.persistent ? 1 : 8;   // work hoisted out of the row loop wants long-lived CTAs
+  if (lp.grid_waves > 0) waves = lp.grid_waves;
+  if (lp.grid_waves < 0) waves = int64_t(1) << 40;
   int64_t grid;
   if (lp.family <= FAM_WARP) grid = std::min<int64_t>((lp.items + lp.teams_per_cta - 1) / lp.teams_per_cta, resident * waves);
   else if (lp.family == FAM_BLOCK) grid = std::min<int64_t>(lp.items, resident * waves);
   else grid = std::min<int64_t>(lp.items, std::max<int64_t>(1, resident * waves / cluster)) * cluster;
   lp.grid = (int)std::max<int64_t>(grid, cluster);
 }
+
+// PN_TUNE_WAVES: 0 default, 7 one CTA per item, n: 2^(n-1) waves
+int tune_waves(unsigned flags) { const int w = (flags >> 29) & 7; return w == 0 ? 0 : (w == 7 ? -1 : 1 << (w - 1)); }
 
 namespace {
 
@@ -667,6 +672,7 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     lp.teams_per_cta = teams;
     lp.specialised = 0;
     lp.persistent = persistent ? 1 : 0;
+    lp.grid_waves = tune_waves(flags);
     // long rows split over a cluster run few, long-lived threads: there the first stage's loads
     // are issued one tile ahead (elsewhere the extra registers cost more than they bring)
     lp.no_prefetch = ((flags & PN_FLAG_PREFETCH) || (cf.family == FAM_CLUSTER && cf.chunks > 1 && !(flags & PN_FLAG_NO_HOIST))) ? 0 : 1;

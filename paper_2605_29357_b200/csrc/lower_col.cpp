@@ -376,7 +376,7 @@ int lower_column_graph(const Graph& g, unsigned flags, const DeviceModel& dev, L
   lp.items = O * n_ctiles;
   lp.teams_per_cta = 1;
   // generated kernels issue the loads of several steps of the walk before the arithmetic of the first
-  lp.specialised = 0; lp.persistent = 0; lp.no_prefetch = (flags & PN_FLAG_NO_HOIST) ? 1 : 0;
+  lp.specialised = 0; lp.persistent = 0; lp.grid_waves = tune_waves(flags); lp.no_prefetch = (flags & PN_FLAG_NO_HOIST) ? 1 : 0;
   const int occ = (dev.have_device && !spec) ? instance_occupancy(VL, NG, K, block, off) : 0;
   size_grid(lp, dev.sm_count, occ);
   return PN_OK;

@@ -170,6 +170,8 @@ struct LaunchPlan {
   int32_t teams_per_cta;
   int32_t specialised;     // 1 when the launch uses a kernel generated for this program
   int32_t persistent;      // 1: grid = resident CTAs, each looping over many rows
+  int32_t grid_waves;      // tuning override: the grid is at most this many times the resident CTAs (0 = the default rule,
+                           // -1 = one CTA per work item whatever their number)
   int32_t no_prefetch;     // 1: generated kernels issue no loads ahead of the tile in hand
   int32_t bounds;          // 1: the generated kernel is compiled with checked accessors
   int32_t io_tensor[kMaxIo];   // tensor id behind each io entry

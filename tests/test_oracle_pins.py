@@ -588,3 +588,91 @@ def test_masked_mean_pooling_special_cases():
     assert np.allclose(out[0], h[0].sum(axis=0) / 6, rtol=0, atol=1e-15)
     assert np.array_equal(out[1], np.zeros(8))
     assert np.array_equal(out[2], h[2, 4])
+
+
+# ---------------------------------------------------------------------------
+# conventions at the edges: NaN operands, casts to bool / integer, gamma of rms_norm, fp16 rounding.
+# Each expected value below is written out by hand or comes from the struct module's IEEE half
+# conversion, never from the function under test.
+# ---------------------------------------------------------------------------
+def test_binary_max_min_propagate_nan_from_either_operand():
+    """Pins `max` / `min`: the elementwise maximum of array libraries returns NaN when either
+    operand is NaN (an `fmax`-style "ignore the NaN" would return the number instead)."""
+    nan = float("nan")
+    a, b = f32(nan, 1.0, nan, -2.0, 3.0), f32(1.0, nan, nan, 5.0, -7.0)
+    mx = run1("max", [a, b], [D.F32, D.F32], D.F32, (5,))
+    mn = run1("min", [a, b], [D.F32, D.F32], D.F32, (5,))
+    assert np.isnan(mx[:3]).all() and mx[3:].tolist() == [5.0, 3.0]
+    assert np.isnan(mn[:3]).all() and mn[3:].tolist() == [-2.0, -7.0]
+    # the same through an immediate operand, and through clamp (max then min)
+    assert np.isnan(run1("max", [f32(nan)], [D.F32], D.F32, (1,), imms=[0.0])[0])
+    cl = run1("clamp", [f32(nan, -9.0, 9.0)], [D.F32], D.F32, (3,), imms=[-1.0, 1.0])
+    assert np.isnan(cl[0]) and cl[1:].tolist() == [-1.0, 1.0]
+
+
+def test_relu_keeps_nan_and_maps_the_rest_of_the_extended_line():
+    """Pins `relu`: NaN stays NaN (a `where(x > 0, x, 0)` would give 0), -inf -> 0, +inf stays."""
+    got = run1("relu", [f32(float("nan"), -np.inf, np.inf, -0.0, -1e-30, 2.5)], [D.F32], D.F32, (6,))
+    assert np.isnan(got[0]) and got[1:].tolist() == [0.0, np.inf, 0.0, 0.0, 2.5]
+
+
+def test_logsumexp_of_rows_holding_nan_or_infinities():
+    """Pins the special rows of `logsumexp`: a NaN anywhere gives NaN (also beside an infinity),
+    a +inf gives +inf, a row of -inf gives -inf, and -inf entries add nothing."""
+    nan, inf = float("nan"), np.inf
+    x = np.array([[0.0, nan, 1.0], [nan, inf, 0.0], [inf, 0.0, -inf], [-inf, -inf, -inf], [-inf, 0.0, 0.0]], dtype=np.float32)
+    got = run1("logsumexp", [x], [D.F32], D.F32, (5,))
+    assert np.isnan(got[0]) and np.isnan(got[1]) and got[2] == inf and got[3] == -inf
+    assert got[4] == math.log(2.0)
+    # log_softmax of the NaN row is NaN throughout; softmax likewise
+    assert np.isnan(run1("log_softmax", [x[:1]], [D.F32], D.F32, (1, 3))).all()
+    assert np.isnan(run1("softmax", [x[:1]], [D.F32], D.F32, (1, 3))).all()
+
+
+def test_cast_to_bool_and_to_integers():
+    """Pins `cast`: to bool is "non-zero" (so -0.0 is false, NaN and fractions are true); float to
+    integer truncates toward zero; integer to float keeps the value."""
+    src = f32(0.0, -0.0, 0.5, float("nan"), -3.0, 1e-40)
+    assert run1("cast", [src], [D.F32], D.BOOL, (6,)).tolist() == [0, 0, 1, 1, 1, 1]
+    assert run1("cast", [f32(-1.7, 1.7, -0.5, 0.99, 126.5)], [D.F32], D.I8, (5,)).tolist() == [-1, 1, 0, 0, 126]
+    assert run1("cast", [f32(-1.7, 70000.9)], [D.F32], D.I32, (2,)).tolist() == [-1, 70000]
+    assert run1("cast", [np.array([-128, 0, 127], np.int8)], [D.I8], D.BOOL, (3,)).tolist() == [1, 0, 1]
+    back = run1("cast", [np.array([-5, 0, 2**40], np.int64)], [D.I64], D.F32, (3,))
+    assert back.dtype == np.float64 and back.tolist() == [-5.0, 0.0, float(2**40)]
+
+
+def test_rms_norm_with_gamma_against_plain_python():
+    """Pins `rms_norm`'s gamma: y_j = x_j / sqrt(sum(x^2)/N + eps) * gamma_j, restated with
+    Python floats (a dropped or transposed gamma, or eps outside the root, fails)."""
+    x = [[3.0, -4.0, 12.0, 0.5], [1.0, 1.0, -1.0, 2.0]]
+    gamma = [2.0, -0.5, 0.25, 3.0]
+    eps = 0.125
+    want = []
+    for row in x:
+        ms = sum(v * v for v in row) / len(row)
+        want.append([v / math.sqrt(ms + eps) * g for v, g in zip(row, gamma)])
+    got = run1("rms_norm", [np.array(x, np.float32), np.array(gamma, np.float32)], [D.F32, D.F32], D.F32, (2, 4), extra_imm=[eps])
+    np.testing.assert_allclose(got, want, rtol=1e-15)
+    # 3-4-12 with eps = 0: the root mean square is 13/2 exactly
+    g0 = run1("rms_norm", [f32(3.0, 4.0, 12.0, 0.0)[None, :]], [D.F32], D.F32, (1, 4), extra_imm=[0.0])
+    np.testing.assert_allclose(g0[0], [6.0 / 13.0, 8.0 / 13.0, 24.0 / 13.0, 0.0], rtol=1e-15)
+
+
+def test_round_to_f16_against_the_ieee_half_type_everywhere():
+    """Pins `round_to_f16` against the struct module's binary16 conversion: every finite half
+    value is a fixed point, every midpoint of two neighbouring halves goes to the one with the
+    even mantissa, points a little to either side of a midpoint go to their nearer neighbour,
+    and the overflow threshold is 65520."""
+    bits = np.arange(0x7C00, dtype=np.uint16)                      # all non-negative finite halves
+    vals = np.array([struct.unpack("<e", struct.pack("<H", int(b)))[0] for b in bits])
+    assert np.array_equal(E.round_to_f16(vals), vals) and np.array_equal(E.round_to_f16(-vals), -vals)
+    mids = (vals[:-1] + vals[1:]) / 2
+    want_mid = np.where(bits[:-1] % 2 == 0, vals[:-1], vals[1:])
+    assert np.array_equal(E.round_to_f16(mids), want_mid)
+    gap = vals[1:] - vals[:-1]
+    assert np.array_equal(E.round_to_f16(mids - gap / 8), vals[:-1]) and np.array_equal(E.round_to_f16(mids + gap / 8), vals[1:])
+    # the struct module agrees on the same points (it rounds a double to half, nearest even)
+    probe = np.concatenate([mids[::97], mids[::89] + gap[::89] / 8, vals[::101] * (1 + 2.0 ** -30)])
+    ref = np.array([struct.unpack("<e", struct.pack("<e", float(v)))[0] for v in probe])
+    assert np.array_equal(E.round_to_f16(probe), ref)
+    assert E.round_to_f16(np.array([65519.9, 65520.0, -65520.0, 2.0 ** -25, 2.0 ** -25 * 1.01])).tolist() == [65504.0, np.inf, -np.inf, 0.0, 2.0 ** -24]
