@@ -67,6 +67,14 @@ extern "C" {
 typedef struct pn_graph pn_graph_t; /* opaque handle */
 typedef int pn_status;
 
+/*
+ * Status codes.  The paper sorts the ways a rewritten graph can fail into three categories
+ * (Section 3.5: accuracy, compilation, runtime).  Here a "compilation" failure is any negative
+ * status of pn_graph_create (the graph could not be parsed, lowered or compiled: codes -2 .. -5,
+ * -8, and -9 with the compiler's log), a "runtime" failure any negative status of a run call
+ * (codes -1, -6, -7, -9), and an "accuracy" failure is not a status at all: it is what the
+ * tolerance rule of Eq. 1 detects when outputs are compared (the tests, and the report module).
+ */
 enum {
   PN_OK = 0,
   PN_ERR_INVALID_ARG = -1,    /* null pointer, bad enum, bad size                       */
@@ -99,6 +107,9 @@ enum {
                                      ahead (costs registers; off by default)                 */
   PN_FLAG_STATIC_SCRATCH = 1u << 12,/* with PN_FLAG_UNFUSED: allocate no workspace; the handle
                                      is run with pn_graph_run_static only                    */
+  PN_FLAG_ALLOW_INTERPRET = 1u << 14,/* a create that cannot specialise kernels (NVRTC or the driver
+                                     library cannot be opened) normally fails with PN_ERR_DEVICE;
+                                     with this flag it runs on the interpreter kernels instead  */
   PN_FLAG_BOUNDS = 1u << 13       /* checked accessors: every global access of the kernels is tested
                                      against the extent of its tensor; one that falls outside is
                                      skipped and recorded in a status word on the device (4 bytes
@@ -127,6 +138,8 @@ enum {
   PN_Q_BOUNDS_STATUS = 10,  /* 1 value, PN_FLAG_BOUNDS handles only: bit q set when an access to the
                                q-th input / output entry of a launch fell outside its tensor;
                                waits for the device                                        */
+  PN_Q_KERNEL_CACHE = 11,   /* 2 values, process-wide: generated kernels now loaded, and how many of
+                               them a live handle uses                                      */
   PN_Q_KERNEL_INFO = 9      /* per kernel 13 values: family (0 pointwise, 1 warp-per-row,
                                2 block-per-row, 3 cluster-per-row, 4 column-reduce: rows =
                                the dimensions before the reduced one, row length = those after
@@ -138,8 +151,9 @@ enum {
 
 /*
  * pn_graph_create -- parse, validate and lower a graph (the host side of running G of
- * Definition 3.1; the lowering picks a kernel family per shape, which is the hardware
- * cost model whose absence the paper lists as a failure mode, Section 4.4).
+ * Definition 3.1; the lowering picks a kernel family and tile per shape: the hardware
+ * cost model whose absence -- one tile shape kept whatever the tensor shape -- the paper counts
+ * among the failure modes of generated passes, Section 4.4).
  *   desc, desc_bytes : HOST pointer to the descriptor; copied, caller may free it.
  *   device           : CUDA device ordinal the handle is bound to.
  *   flags            : PN_FLAG_* bits.
@@ -148,8 +162,15 @@ enum {
  * handle and released by pn_graph_destroy.  Launches no kernel.
  * Unless PN_FLAG_INTERPRET is given, the bytecode of each launch is also translated into a
  * kernel of its own and compiled for sm_100a with NVRTC (a few hundred ms per distinct
- * kernel; loaded kernels are cached for the life of the process).  If NVRTC or the driver
- * library cannot be opened the handle runs on the interpreter; PN_Q_KERNEL_INFO tells which.
+ * kernel).  Loaded kernels are shared through a process-wide cache, reference-counted by the
+ * handles that use them; unused ones are unloaded, least recently used first, beyond 256.  With
+ * the environment variable PN_CACHE_DIR set, compiled kernels are also kept in that directory
+ * (keyed by a hash of the source, the NVRTC version and sm_100a) and a later process loads them
+ * without compiling.  NVRTC is looked for at PN_NVRTC_PATH, else under CUDA_HOME / CUDA_PATH /
+ * /usr/local/cuda, else by soname.  If NVRTC or the driver library cannot be opened the create
+ * FAILS with PN_ERR_DEVICE and the reason, unless PN_FLAG_INTERPRET or PN_FLAG_ALLOW_INTERPRET
+ * was given (the interpreter kernels are more than ten times slower); PN_Q_KERNEL_INFO tells
+ * which kind a handle runs.  The calling thread's current device is left as it was.
  */
 pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsigned flags,
                           pn_graph_t** out);
@@ -163,12 +184,40 @@ pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsig
  * Asynchronous: returns after the launch(es).  No allocation, no host synchronisation.
  * Pointers must be aligned to 16 bytes unless the handle was created with
  * PN_FLAG_FORCE_SCALAR (then to the element size); otherwise PN_ERR_ALIGNMENT.  Inputs
- * and outputs must not overlap.  The library never retains or frees user memory.  Runs on
- * one PN_FLAG_UNFUSED handle share its workspace and must be stream-ordered by the caller.
- * A graph any of whose inputs or outputs has zero elements runs as a no-op.
+ * and outputs must not overlap, not even exactly: the kernels read inputs through the
+ * read-only data path, which does not see a kernel's own writes.  The library never retains or
+ * frees user memory.  The handle itself is only read, so runs of one fused handle may be issued
+ * from several threads and streams at once; runs of a handle that has a workspace
+ * (PN_Q_WORKSPACE_BYTES > 0: unfused handles, graphs cut into several launches, rows split over
+ * independent blocks) share that workspace and must be stream-ordered by the caller.  The launch
+ * goes to the handle's device whatever device the calling thread has current, and that choice
+ * is left as it was.  A graph any of whose inputs or outputs has zero elements runs as a no-op.
  */
 pn_status pn_graph_run(pn_graph_t* g, const void* const* inputs, int n_inputs,
                        void* const* outputs, int n_outputs, void* stream);
+
+/*
+ * pn_graph_bind / pn_bound_run / pn_bound_destroy -- the same evaluation of f_G (Definition 3.1)
+ * with the per-call work done once.  The paper finds fixed per-call overhead to be what sinks
+ * small graphs (Table 6); for a fused kernel of a few microseconds the argument checks and the
+ * marshalling of a 4 KB parameter block are that kind of cost.  pn_graph_bind runs the checks of
+ * pn_graph_run on one set of pointers and stores the filled-in launch parameters in a bound
+ * object; pn_bound_run(b, stream) is then one launch call per kernel and nothing else.
+ *   g, inputs, outputs : as for pn_graph_run; the DEVICE pointers are recorded, the caller keeps
+ *                        the buffers alive and unmoved while the bound object is used.
+ *   out                : receives the bound object (HOST memory owned by the library); NULL on
+ *                        failure.  It must be destroyed before its handle.
+ * Errors of pn_graph_bind: those of pn_graph_run; PN_ERR_INVALID_ARG for a PN_FLAG_STATIC_SCRATCH
+ * handle.  pn_bound_run: PN_ERR_INVALID_ARG for NULL, PN_ERR_CUDA for a failed launch.  A bound
+ * object is immutable: pn_bound_run may be called from several threads at once (the workspace
+ * rule of pn_graph_run applies).  Asynchronous, no allocation at run time, capturable in a CUDA
+ * graph like pn_graph_run.
+ */
+typedef struct pn_bound pn_bound_t;
+pn_status pn_graph_bind(pn_graph_t* g, const void* const* inputs, int n_inputs, void* const* outputs,
+                        int n_outputs, pn_bound_t** out);
+pn_status pn_bound_run(pn_bound_t* b, void* stream);
+pn_status pn_bound_destroy(pn_bound_t* b);
 
 /*
  * pn_graph_run_host -- the same evaluation of f_G (Definition 3.1) for callers whose
@@ -198,24 +247,30 @@ pn_status pn_graph_run_host(pn_graph_t* g, const void* const* inputs, int n_inpu
  * intermediates between the per-node kernels comes from cudaMalloc.
  *
  * What it does instead: the intermediates go into one fixed array of
- * PN_STATIC_SCRATCH_BYTES (32 MiB) that is part of the library's device image.  Every GPU
- * that loads the library holds that array until the process exits, used or not.
- *   g       : a handle created with PN_FLAG_UNFUSED | PN_FLAG_STATIC_SCRATCH (such a create
- *             allocates no workspace; combine it with PN_FLAG_INTERPRET if the create must
- *             not load generated kernels either).  pn_graph_run refuses such a handle.
+ * PN_STATIC_SCRATCH_BYTES (32 MiB) that is part of the library's device image.  A GPU starts
+ * holding that array when the library's device code for it is first loaded there -- which
+ * pn_graph_create does for a handle with PN_FLAG_STATIC_SCRATCH -- and holds it until the
+ * process exits.
+ *   g       : a handle created with PN_FLAG_UNFUSED | PN_FLAG_STATIC_SCRATCH.  That create is
+ *             the set-up step and the one place that may fail for lack of memory: it allocates
+ *             no workspace, but it looks up the array's device address (cudaGetSymbolAddress,
+ *             once per device, with that device current), and under the CUDA runtime's lazy
+ *             loading that lookup is what reserves the 32 MiB on the device.  Do it while the
+ *             process may still allocate, and before any stream capture begins.  Combine the
+ *             flags with PN_FLAG_INTERPRET if the create must not load generated kernels
+ *             either.  pn_graph_run, pn_graph_run_host and pn_graph_bind refuse such a handle.
  *   inputs, outputs, stream : as for pn_graph_run (HOST arrays of DEVICE pointers that the
- *             caller owns; same alignment and no-overlap rules).
+ *             caller owns; the same alignment and no-overlap rules, checked by the same code).
  * Errors: PN_ERR_TOO_LARGE when the graph's intermediates need more than
  * PN_STATIC_SCRATCH_BYTES (pn_graph_query PN_Q_WORKSPACE_BYTES tells how much);
  * PN_ERR_INVALID_ARG for a handle without the two flags; otherwise as pn_graph_run.
- * The call itself uses no cudaMalloc, cudaFree or other allocating routine.
+ * The call itself uses no cudaMalloc, cudaFree or other allocating routine, looks nothing up,
+ * and leaves the free device memory exactly as it found it.
  *
- * The first call on a device looks up the array's device address (cudaGetSymbolAddress,
- * which may make the runtime load the library's device image); make that first call before
- * any stream capture begins.  All calls, from all handles and threads, share the one array
- * per device and it keeps whatever the last call left: nothing has to start at zero (each
- * intermediate is fully written before it is read), but two calls whose kernels overlap on
- * the GPU -- different streams, no ordering between them -- race on it.  Order them.
+ * All calls, from all handles and threads, share the one array per device and it keeps
+ * whatever the last call left: nothing has to start at zero (each intermediate is fully
+ * written before it is read), but two calls whose kernels overlap on the GPU -- different
+ * streams, no ordering between them -- race on it.  Order them.
  */
 pn_status pn_graph_run_static(pn_graph_t* g, const void* const* inputs, int n_inputs,
                               void* const* outputs, int n_outputs, void* stream);
@@ -266,7 +321,10 @@ pn_status pn_sequence_run(pn_sequence_t* s, void* stream);
 pn_status pn_sequence_query(const pn_sequence_t* s, int what, void* out, size_t out_bytes);
 pn_status pn_sequence_destroy(pn_sequence_t* s);
 
-/* pn_graph_destroy -- release the handle and what it owns; NULL is accepted. */
+/* pn_graph_destroy -- end of the life of one instance of G (Definition 3.1; Section 3.1: one handle
+ * per shape / dtype instance): releases the handle, its workspace, staging buffers and status word,
+ * and gives its kernels back to the process-wide cache.  Bound launches and sequences made from
+ * the handle must be destroyed first.  NULL is accepted. */
 pn_status pn_graph_destroy(pn_graph_t* g);
 
 /*
@@ -330,10 +388,14 @@ typedef struct pn_probe_config {
 pn_status pn_stream_probe(int mix, const pn_probe_config* cfg, const void* a, const void* b, void* c, void* d,
                           size_t units, void* status_word, void* stream);
 
-/* Static text for a status code. */
+/* pn_status_string -- static text for a status code (the failure classes of Section 3.5 as mapped
+ * beside the status enum above); never NULL. */
 const char* pn_status_string(pn_status s);
 
-/* Detail of the calling thread's most recent failure ("" if none). */
+/* pn_last_error -- detail of the calling thread's most recent failure ("" if none): for a
+ * "compilation" failure (Section 3.5) the node and the rule it broke, or the run-time compiler's
+ * log; for a "runtime" failure the argument or the CUDA error.  The pointer stays valid until the
+ * same thread's next failing call. */
 const char* pn_last_error(void);
 
 #ifdef __cplusplus

@@ -27,6 +27,7 @@ FLAG_NO_HOIST = 1 << 10
 FLAG_PREFETCH = 1 << 11
 FLAG_STATIC_SCRATCH = 1 << 12
 FLAG_BOUNDS = 1 << 13
+FLAG_ALLOW_INTERPRET = 1 << 14
 STATIC_SCRATCH_BYTES = 32 << 20
 
 
@@ -41,6 +42,7 @@ Q_N_KERNELS, Q_N_NODES, Q_WORKSPACE_BYTES, Q_KERNEL_INFO = 6, 7, 8, 9
 
 FAMILY_NAMES = {0: "pointwise", 1: "warp-per-row", 2: "block-per-row", 3: "cluster-per-row", 4: "column-reduce"}
 EXPORTS = ["pn_graph_create", "pn_graph_run", "pn_graph_run_host", "pn_graph_run_static", "pn_graph_destroy",
+           "pn_graph_bind", "pn_bound_run", "pn_bound_destroy",
            "pn_graph_query", "pn_graph_codegen", "pn_status_string", "pn_last_error",
            "pn_sequence_create", "pn_sequence_run", "pn_sequence_query", "pn_sequence_destroy",
            "pn_stream_probe"]
@@ -86,6 +88,12 @@ def load_library() -> ctypes.CDLL:
         fn.argtypes = [vp, vpp, ctypes.c_int, vpp, ctypes.c_int, vp]
     lib.pn_graph_destroy.restype = ctypes.c_int
     lib.pn_graph_destroy.argtypes = [vp]
+    lib.pn_graph_bind.restype = ctypes.c_int
+    lib.pn_graph_bind.argtypes = [vp, vpp, ctypes.c_int, vpp, ctypes.c_int, vpp]
+    lib.pn_bound_run.restype = ctypes.c_int
+    lib.pn_bound_run.argtypes = [vp, vp]
+    lib.pn_bound_destroy.restype = ctypes.c_int
+    lib.pn_bound_destroy.argtypes = [vp]
     lib.pn_graph_query.restype = ctypes.c_int
     lib.pn_graph_query.argtypes = [vp, ctypes.c_int, vp, ctypes.c_size_t]
     lib.pn_graph_codegen.restype = ctypes.c_int
@@ -170,6 +178,12 @@ class Graph:
         return self._query(10, 1)[0]
 
     @property
+    def kernel_cache(self) -> Tuple[int, int]:
+        """(generated kernels loaded in this process, how many of them a live handle uses)."""
+        v = self._query(11, 2)
+        return v[0], v[1]
+
+    @property
     def workspace_bytes(self) -> int:
         return self._query(Q_WORKSPACE_BYTES, 1)[0]
 
@@ -201,18 +215,11 @@ class Graph:
                                       self._ptr_array(output_ptrs), len(output_ptrs),
                                       ctypes.c_void_p(stream)), "pn_graph_run")
 
-    def bind(self, input_ptrs: Sequence[int], output_ptrs: Sequence[int]):
-        """A callable `f(stream=0)` that enqueues one evaluation on these device pointers.  The
-        pointer arrays are marshalled once, so that a caller who launches the same buffers many
-        times pays only the call itself."""
-        ins, outs = self._ptr_array(input_ptrs), self._ptr_array(output_ptrs)
-        n_in, n_out, fn, h = len(input_ptrs), len(output_ptrs), self._lib.pn_graph_run, self._h
-
-        def launch(stream: int = 0, _vp=ctypes.c_void_p) -> None:
-            st = fn(h, ins, n_in, outs, n_out, _vp(stream))
-            if st != PN_OK:
-                _check(st, "pn_graph_run")
-        return launch
+    def bind(self, input_ptrs: Sequence[int], output_ptrs: Sequence[int]) -> "Bound":
+        """pn_graph_bind: a callable `f(stream=0)` that enqueues one evaluation on these device
+        pointers.  The argument checks run once, here; each call is pn_bound_run, one launch
+        call per kernel."""
+        return Bound(self, input_ptrs, output_ptrs)
 
     def run_host(self, input_ptrs: Sequence[int], output_ptrs: Sequence[int], stream: int = 0) -> None:
         """Evaluate on HOST buffers (addresses): copy in, run, copy out, wait."""
@@ -232,6 +239,35 @@ class Graph:
     def close(self) -> None:
         if getattr(self, "_h", None) is not None and self._h:
             self._lib.pn_graph_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class Bound:
+    """pn_bound_t: the launches of a Graph with one set of device pointers filled in."""
+
+    def __init__(self, graph: Graph, input_ptrs: Sequence[int], output_ptrs: Sequence[int]):
+        self._lib = graph._lib
+        self._graph = graph                      # the handle must outlive its bound launches
+        self._h = ctypes.c_void_p()
+        _check(self._lib.pn_graph_bind(graph._h, Graph._ptr_array(input_ptrs), len(input_ptrs),
+                                       Graph._ptr_array(output_ptrs), len(output_ptrs), ctypes.byref(self._h)),
+               "pn_graph_bind")
+        self._run = self._lib.pn_bound_run
+
+    def __call__(self, stream: int = 0, _vp=ctypes.c_void_p) -> None:
+        st = self._run(self._h, _vp(stream))
+        if st != PN_OK:
+            _check(st, "pn_bound_run")
+
+    def close(self) -> None:
+        if getattr(self, "_h", None) is not None and self._h:
+            self._lib.pn_bound_destroy(self._h)
             self._h = ctypes.c_void_p()
 
     def __del__(self):

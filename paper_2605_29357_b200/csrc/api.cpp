@@ -36,28 +36,41 @@ bool any_empty(const Graph& g) {
   return false;
 }
 
-// The single-node graph executed by one launch of the unfused path.
-void node_subgraph(const Graph& g, const Node& n, Graph& sub, std::vector<int>& orig_of_sub) {
+// The graph executed by one launch: the nodes `members` of g (ascending, hence topological).  Its
+// inputs are the tensors the members read that no member produces; its outputs are the tensors a
+// member produces that a node outside the group reads or that are outputs of g.
+void group_subgraph(const Graph& g, const std::vector<int>& members, Graph& sub, std::vector<int>& orig_of_sub) {
   sub = Graph();
   orig_of_sub.clear();
-  Node m = n;
-  auto add = [&](int orig, uint8_t role) {
+  std::vector<char> inside(g.nodes.size(), 0), made_here(g.tensors.size(), 0), read_outside(g.tensors.size(), 0);
+  for (int ni : members) inside[ni] = 1;
+  for (int ni : members) for (int k = 0; k < g.nodes[ni].n_out; ++k) made_here[g.nodes[ni].out[k]] = 1;
+  for (size_t ni = 0; ni < g.nodes.size(); ++ni)
+    if (!inside[ni])
+      for (int k = 0; k < g.nodes[ni].n_in; ++k)
+        if (g.nodes[ni].in[k] < g.tensors.size()) read_outside[g.nodes[ni].in[k]] = 1;
+  auto add = [&](int orig) {
     for (size_t i = 0; i < orig_of_sub.size(); ++i) if (orig_of_sub[i] == orig) return (int)i;
     Tensor t = g.tensors[orig];
-    t.role = role; t.producer = -1;
+    t.role = made_here[orig] ? (uint8_t)(((g.tensors[orig].role & 2) || read_outside[orig]) ? 2 : 0) : (uint8_t)1;
+    t.producer = -1;
     sub.tensors.push_back(t);
     orig_of_sub.push_back(orig);
     return (int)sub.tensors.size() - 1;
   };
-  for (int k = 0; k < n.n_in; ++k) {
-    if (n.in[k] == kImm0 || n.in[k] == kImm1) continue;
-    m.in[k] = (uint32_t)add((int)n.in[k], 1);
+  for (int ni : members) {
+    const Node& n = g.nodes[ni];
+    Node m = n;
+    for (int k = 0; k < n.n_in; ++k) {
+      if (n.in[k] == kImm0 || n.in[k] == kImm1) continue;
+      m.in[k] = (uint32_t)add((int)n.in[k]);
+    }
+    for (int k = 0; k < n.n_out; ++k) {
+      m.out[k] = (uint32_t)add((int)n.out[k]);
+      sub.tensors[m.out[k]].producer = (int)sub.nodes.size();
+    }
+    sub.nodes.push_back(m);
   }
-  for (int k = 0; k < n.n_out; ++k) {
-    m.out[k] = (uint32_t)add((int)n.out[k], 2);
-    sub.tensors[m.out[k]].producer = 0;
-  }
-  sub.nodes.push_back(m);
   for (size_t i = 0; i < sub.tensors.size(); ++i) {
     if (sub.tensors[i].role & 1) sub.inputs.push_back((int)i);
     if (sub.tensors[i].role & 2) sub.outputs.push_back((int)i);
@@ -73,7 +86,80 @@ pn_status check_counts(const pn_graph* h, const void* const* inputs, int n_input
   return PN_OK;
 }
 
+void fill_pointers(const pn_graph* h, const PlannedLaunch& pl, const void* const* inputs, void* const* outputs, void* workspace, LaunchPlan& lp) {
+  for (int q = 0; q < lp.p.n_io; ++q) {
+    const IoSource& s = pl.src[q];
+    lp.p.io[q].base = s.kind == 0 ? const_cast<void*>(inputs[s.index])
+                    : s.kind == 1 ? outputs[s.index]
+                                  : (void*)((char*)workspace + s.index);
+  }
+  (void)h;
+}
+
+pn_status launch_filled(const PlannedLaunch& pl, const LaunchPlan& lp, void* stream) {
+  if (pl.spec.fn) {
+    std::string err;
+    if (!spec_launch(pl.spec, lp, stream, err)) return fail(PN_ERR_CUDA, err);
+  } else {
+    const cudaError_t e = launch_plan(lp, (cudaStream_t)stream);
+    if (e != cudaSuccess) return fail(PN_ERR_CUDA, std::string("launch: ") + cudaGetErrorString(e));
+  }
+  return PN_OK;
+}
+
 }  // namespace
+
+namespace pn {
+
+int check_run_arguments(const pn_graph* h, const void* const* inputs, int n_inputs, void* const* outputs, int n_outputs) {
+  const pn_status st = check_counts(h, inputs, n_inputs, outputs, n_outputs);
+  if (st != PN_OK) return st;
+  const Graph& g = h->g;
+  const bool scalar = (h->flags & PN_FLAG_FORCE_SCALAR) != 0;
+  for (int i = 0; i < n_inputs; ++i) {
+    if (!inputs[i]) return fail(PN_ERR_INVALID_ARG, "input " + std::to_string(i) + " is null");
+    const uintptr_t m = scalar ? (uintptr_t)(dtype_bytes(g.tensors[g.inputs[i]].dtype) - 1) : 15;
+    if ((uintptr_t)inputs[i] & m) return fail(PN_ERR_ALIGNMENT, "input " + std::to_string(i) + " is not aligned");
+  }
+  for (int i = 0; i < n_outputs; ++i) {
+    if (!outputs[i]) return fail(PN_ERR_INVALID_ARG, "output " + std::to_string(i) + " is null");
+    const uintptr_t m = scalar ? (uintptr_t)(dtype_bytes(g.tensors[g.outputs[i]].dtype) - 1) : 15;
+    if ((uintptr_t)outputs[i] & m) return fail(PN_ERR_ALIGNMENT, "output " + std::to_string(i) + " is not aligned");
+  }
+  // inputs go through the read-only data path: none may overlap an output; outputs are
+  // written independently: none may overlap another
+  for (int o = 0; o < n_outputs; ++o) {
+    const char* b0 = (const char*)outputs[o];
+    const char* b1 = b0 + tensor_bytes(g.tensors[g.outputs[o]]);
+    for (int i = 0; i < n_inputs; ++i) {
+      const char* a0 = (const char*)inputs[i];
+      const char* a1 = a0 + tensor_bytes(g.tensors[g.inputs[i]]);
+      if (a0 < b1 && b0 < a1) return fail(PN_ERR_INVALID_ARG, "input " + std::to_string(i) + " overlaps output " + std::to_string(o));
+    }
+    for (int i = 0; i < o; ++i) {
+      const char* a0 = (const char*)outputs[i];
+      const char* a1 = a0 + tensor_bytes(g.tensors[g.outputs[i]]);
+      if (a0 < b1 && b0 < a1) return fail(PN_ERR_INVALID_ARG, "outputs " + std::to_string(i) + " and " + std::to_string(o) + " overlap");
+    }
+  }
+  return PN_OK;
+}
+
+int enqueue_launches(const pn_graph* h, const void* const* inputs, void* const* outputs, void* workspace,
+                     void* stream, int64_t item_begin, int64_t item_end) {
+  DeviceScope dev(h->device);
+  if (dev.err != cudaSuccess) return fail(PN_ERR_CUDA, std::string("cudaSetDevice: ") + cudaGetErrorString(dev.err));
+  for (const PlannedLaunch& pl : h->launches) {
+    LaunchPlan lp = pl.plan;   // the pointers go into a copy: the handle itself is only read
+    fill_pointers(h, pl, inputs, outputs, workspace, lp);
+    if (item_end > 0) { lp.p.item_begin = item_begin; lp.p.item_end = item_end; }
+    const pn_status st = launch_filled(pl, lp, stream);
+    if (st != PN_OK) return st;
+  }
+  return PN_OK;
+}
+
+}  // namespace pn
 
 extern "C" {
 #pragma GCC visibility push(default)
@@ -91,8 +177,17 @@ pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsig
   h->device = device;
   h->plan_only = (flags & PN_FLAG_PLAN_ONLY) != 0;
 
+  // The kernels specialised per graph need NVRTC (and, to be loaded, the driver library).  A create
+  // that cannot have them fails rather than fall back silently to the interpreter, which is an
+  // order of magnitude slower: the caller has to ask for the interpreter by name.
   DeviceModel dev;
-  dev.specialise = !(flags & PN_FLAG_INTERPRET) && spec_available(nullptr, h->plan_only);
+  std::string why;
+  dev.specialise = !(flags & PN_FLAG_INTERPRET) && spec_available(&why, h->plan_only);
+  if (!dev.specialise && !(flags & (PN_FLAG_INTERPRET | PN_FLAG_ALLOW_INTERPRET))) {
+    delete h;
+    return fail(PN_ERR_DEVICE, "kernels cannot be specialised for this graph: " + why +
+                                   " (PN_FLAG_ALLOW_INTERPRET accepts the much slower built-in interpreter kernels instead)");
+  }
   if (!h->plan_only) {
     int count = 0;
     cudaError_t e = cudaGetDeviceCount(&count);
@@ -101,62 +196,80 @@ pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsig
     e = cudaGetDeviceProperties(&prop, device);
     if (e != cudaSuccess) { delete h; return fail(PN_ERR_CUDA, cudaGetErrorString(e)); }
     if (prop.major != 10) { delete h; return fail(PN_ERR_DEVICE, "the kernels are built for sm_100a only"); }
-    e = cudaSetDevice(device);
-    if (e != cudaSuccess) { delete h; return fail(PN_ERR_CUDA, cudaGetErrorString(e)); }
     dev.sm_count = prop.multiProcessorCount;
     dev.max_smem_per_block = (int)prop.sharedMemPerBlockOptin;
     dev.have_device = true;
   }
+  // everything below that touches the device does so with it current; the caller's own current
+  // device is put back when this function returns
+  DeviceScope scope(h->plan_only ? -1 : device);
+  if (!h->plan_only && scope.err != cudaSuccess) { delete h; return fail(PN_ERR_CUDA, std::string("cudaSetDevice: ") + cudaGetErrorString(scope.err)); }
 
   const Graph& g = h->g;
   for (int t : g.inputs) h->compulsory_bytes += tensor_bytes(g.tensors[t]);
   for (int t : g.outputs) h->compulsory_bytes += tensor_bytes(g.tensors[t]);
   if (any_empty(g)) { *out = h; return PN_OK; }   // nothing to compute: runs are no-ops
 
-  if (!(flags & PN_FLAG_UNFUSED)) {
-    PlannedLaunch pl;
-    st = lower_graph(g, flags, dev, pl.plan, err);
-    if (st != PN_OK) { delete h; return fail(st, err); }
-    for (int q = 0; q < pl.plan.p.n_io; ++q) {
-      const int t = pl.plan.io_tensor[q];
-      pl.plan.p.io[q].numel = g.tensors[t].numel();
-      IoSource s{pl.plan.io_is_output[q] ? 1 : 0, 0};
-      const std::vector<int>& list = pl.plan.io_is_output[q] ? g.outputs : g.inputs;
-      for (size_t i = 0; i < list.size(); ++i) if (list[i] == t) s.index = (int64_t)i;
-      pl.src.push_back(s);
-    }
-    h->launches.push_back(pl);
+  // ---- which nodes run in which launch -----------------------------------------------------------
+  std::vector<std::vector<int>> groups;
+  if (flags & PN_FLAG_UNFUSED) {
+    for (size_t ni = 0; ni < g.nodes.size(); ++ni) groups.push_back({(int)ni});   // one launch per node
   } else {
-    // one launch per node; intermediates live in a workspace in their declared dtype
-    std::vector<int64_t> ws_off(g.tensors.size(), -1);
-    size_t ws = 0;
+    groups.emplace_back();
+    for (size_t ni = 0; ni < g.nodes.size(); ++ni) groups[0].push_back((int)ni);
+  }
+  // tensors that cross from one launch to a later one live in a workspace, in their declared dtype
+  std::vector<int> group_of_node(g.nodes.size(), 0);
+  for (size_t gi = 0; gi < groups.size(); ++gi) for (int ni : groups[gi]) group_of_node[ni] = (int)gi;
+  std::vector<int64_t> ws_off(g.tensors.size(), -1);
+  size_t ws = 0;
+  if (groups.size() > 1)
     for (size_t t = 0; t < g.tensors.size(); ++t) {
       if (g.tensors[t].role != 0 || g.tensors[t].producer < 0) continue;
+      bool crosses = false;
+      for (size_t ni = 0; ni < g.nodes.size() && !crosses; ++ni)
+        for (int k = 0; k < g.nodes[ni].n_in; ++k)
+          if (g.nodes[ni].in[k] == t && group_of_node[ni] != group_of_node[g.tensors[t].producer]) crosses = true;
+      if (!crosses) continue;
       ws_off[t] = (int64_t)ws;
       ws += ((size_t)tensor_bytes(g.tensors[t]) + 255) / 256 * 256;
     }
-    for (size_t ni = 0; ni < g.nodes.size(); ++ni) {
+  for (size_t gi = 0; gi < groups.size(); ++gi) {
+    PlannedLaunch pl;
+    std::vector<int> orig;
+    if (groups.size() == 1) {
+      st = lower_graph(g, flags, dev, pl.plan, err);
+      for (size_t t = 0; t < g.tensors.size(); ++t) orig.push_back((int)t);
+    } else {
       Graph sub;
-      std::vector<int> orig;
-      node_subgraph(g, g.nodes[ni], sub, orig);
-      PlannedLaunch pl;
+      group_subgraph(g, groups[gi], sub, orig);
       st = lower_graph(sub, flags, dev, pl.plan, err);
-      if (st != PN_OK) { delete h; return fail(st, "node " + std::to_string(ni) + " (unfused): " + err); }
-      for (int q = 0; q < pl.plan.p.n_io; ++q) {
-        const int t = orig[pl.plan.io_tensor[q]];
-        pl.plan.p.io[q].numel = g.tensors[t].numel();
-        IoSource s{2, ws_off[t]};
-        for (size_t i = 0; i < g.inputs.size(); ++i) if (g.inputs[i] == t) s = IoSource{0, (int64_t)i};
-        for (size_t i = 0; i < g.outputs.size(); ++i) if (g.outputs[i] == t) s = IoSource{1, (int64_t)i};
-        pl.src.push_back(s);
-      }
-      h->launches.push_back(pl);
+      if (st != PN_OK) err = (groups[gi].size() == 1 ? "node " + std::to_string(groups[gi][0]) + " (unfused): " : "launch " + std::to_string(gi) + ": ") + err;
     }
-    h->workspace_bytes = ws;
-    if (!h->plan_only && ws > 0 && !(flags & PN_FLAG_STATIC_SCRATCH)) {
-      cudaError_t e = cudaMalloc(&h->workspace, ws);
-      if (e != cudaSuccess) { delete h; return fail(PN_ERR_CUDA, std::string("workspace: ") + cudaGetErrorString(e)); }
+    if (st != PN_OK) { delete h; return fail(st, err); }
+    for (int q = 0; q < pl.plan.p.n_io; ++q) {
+      const int t = orig[pl.plan.io_tensor[q]];
+      pl.plan.p.io[q].numel = g.tensors[t].numel();
+      IoSource s{2, ws_off[t]};
+      // a tensor that is both read and written by the graph's caller (an input passed through) is
+      // looked up on the side this launch uses it on
+      if (!pl.plan.io_is_output[q]) for (size_t i = 0; i < g.inputs.size(); ++i) if (g.inputs[i] == t) s = IoSource{0, (int64_t)i};
+      if (pl.plan.io_is_output[q] || s.kind == 2) for (size_t i = 0; i < g.outputs.size(); ++i) if (g.outputs[i] == t) s = IoSource{1, (int64_t)i};
+      if (s.kind == 2 && s.index < 0) { delete h; return fail(PN_ERR_INVALID_ARG, "internal: a tensor between two launches has no storage"); }
+      pl.src.push_back(s);
     }
+    h->launches.push_back(pl);
+  }
+  h->workspace_bytes = ws;
+  if (!h->plan_only && ws > 0 && !(flags & PN_FLAG_STATIC_SCRATCH)) {
+    cudaError_t e = cudaMalloc(&h->workspace, ws);
+    if (e != cudaSuccess) { delete h; return fail(PN_ERR_CUDA, std::string("workspace: ") + cudaGetErrorString(e)); }
+  }
+  // a handle that will run from the fixed scratch array: its address on this device is looked up
+  // now, at set-up, so that the runs themselves only read it
+  if (!h->plan_only && (flags & PN_FLAG_STATIC_SCRATCH)) {
+    st = static_scratch_address(device, &h->static_scratch);
+    if (st != PN_OK) { delete h; return st; }
   }
   // checked accessors: one status word on the device, shared by the launches of the handle
   if (flags & PN_FLAG_BOUNDS) {
@@ -185,52 +298,51 @@ pn_status pn_graph_run(pn_graph_t* h, const void* const* inputs, int n_inputs, v
                        int n_outputs, void* stream) {
   pn_status st = check_counts(h, inputs, n_inputs, outputs, n_outputs);
   if (st != PN_OK) return st;
-  const Graph& g = h->g;
-  if (any_empty(g)) return PN_OK;   // nothing to compute
-  if ((h->flags & PN_FLAG_STATIC_SCRATCH) && h->workspace_bytes > 0)
+  if (h->flags & PN_FLAG_STATIC_SCRATCH)
     return fail(PN_ERR_INVALID_ARG, "this handle owns no workspace: run it with pn_graph_run_static");
-  const bool scalar = (h->flags & PN_FLAG_FORCE_SCALAR) != 0;
-  for (int i = 0; i < n_inputs; ++i) {
-    if (!inputs[i]) return fail(PN_ERR_INVALID_ARG, "input " + std::to_string(i) + " is null");
-    const uintptr_t m = scalar ? (uintptr_t)(dtype_bytes(g.tensors[g.inputs[i]].dtype) - 1) : 15;
-    if ((uintptr_t)inputs[i] & m) return fail(PN_ERR_ALIGNMENT, "input " + std::to_string(i) + " is not aligned");
+  if (any_empty(h->g)) return PN_OK;   // nothing to compute
+  st = check_run_arguments(h, inputs, n_inputs, outputs, n_outputs);
+  if (st != PN_OK) return st;
+  return enqueue_launches(h, inputs, outputs, h->workspace, stream, 0, 0);
+}
+
+pn_status pn_graph_bind(pn_graph_t* h, const void* const* inputs, int n_inputs, void* const* outputs, int n_outputs,
+                        pn_bound_t** out) {
+  if (out) *out = nullptr;
+  if (!out) return fail(PN_ERR_INVALID_ARG, "null argument");
+  pn_status st = check_counts(h, inputs, n_inputs, outputs, n_outputs);
+  if (st != PN_OK) return st;
+  if (h->flags & PN_FLAG_STATIC_SCRATCH) return fail(PN_ERR_INVALID_ARG, "static-scratch handles are run with pn_graph_run_static");
+  if (!any_empty(h->g)) {
+    st = check_run_arguments(h, inputs, n_inputs, outputs, n_outputs);
+    if (st != PN_OK) return st;
   }
-  for (int i = 0; i < n_outputs; ++i) {
-    if (!outputs[i]) return fail(PN_ERR_INVALID_ARG, "output " + std::to_string(i) + " is null");
-    const uintptr_t m = scalar ? (uintptr_t)(dtype_bytes(g.tensors[g.outputs[i]].dtype) - 1) : 15;
-    if ((uintptr_t)outputs[i] & m) return fail(PN_ERR_ALIGNMENT, "output " + std::to_string(i) + " is not aligned");
+  pn_bound* b = new (std::nothrow) pn_bound();
+  if (!b) return fail(PN_ERR_INVALID_ARG, "out of host memory");
+  b->g = h;
+  if (!any_empty(h->g))
+    for (const PlannedLaunch& pl : h->launches) {
+      b->plans.push_back(pl.plan);
+      fill_pointers(h, pl, inputs, outputs, h->workspace, b->plans.back());
+    }
+  *out = b;
+  return PN_OK;
+}
+
+pn_status pn_bound_run(pn_bound_t* b, void* stream) {
+  if (!b || !b->g) return fail(PN_ERR_INVALID_ARG, "null argument");
+  const pn_graph* h = b->g;
+  DeviceScope dev(h->device);
+  if (dev.err != cudaSuccess) return fail(PN_ERR_CUDA, std::string("cudaSetDevice: ") + cudaGetErrorString(dev.err));
+  for (size_t i = 0; i < b->plans.size(); ++i) {
+    const pn_status st = launch_filled(h->launches[i], b->plans[i], stream);
+    if (st != PN_OK) return st;
   }
-  // inputs go through the read-only data path: none may overlap an output; outputs are
-  // written independently: none may overlap another
-  for (int o = 0; o < n_outputs; ++o) {
-    const char* b0 = (const char*)outputs[o];
-    const char* b1 = b0 + tensor_bytes(g.tensors[g.outputs[o]]);
-    for (int i = 0; i < n_inputs; ++i) {
-      const char* a0 = (const char*)inputs[i];
-      const char* a1 = a0 + tensor_bytes(g.tensors[g.inputs[i]]);
-      if (a0 < b1 && b0 < a1) return fail(PN_ERR_INVALID_ARG, "input " + std::to_string(i) + " overlaps output " + std::to_string(o));
-    }
-    for (int i = 0; i < o; ++i) {
-      const char* a0 = (const char*)outputs[i];
-      const char* a1 = a0 + tensor_bytes(g.tensors[g.outputs[i]]);
-      if (a0 < b1 && b0 < a1) return fail(PN_ERR_INVALID_ARG, "outputs " + std::to_string(i) + " and " + std::to_string(o) + " overlap");
-    }
-  }
-  for (PlannedLaunch& pl : h->launches) {
-    for (int q = 0; q < pl.plan.p.n_io; ++q) {
-      const IoSource& s = pl.src[q];
-      pl.plan.p.io[q].base = s.kind == 0 ? const_cast<void*>(inputs[s.index])
-                           : s.kind == 1 ? outputs[s.index]
-                                         : (void*)((char*)h->workspace + s.index);
-    }
-    if (pl.spec.fn) {
-      std::string err;
-      if (!spec_launch(pl.spec, pl.plan, stream, err)) return fail(PN_ERR_CUDA, err);
-    } else {
-      cudaError_t e = launch_plan(pl.plan, (cudaStream_t)stream);
-      if (e != cudaSuccess) return fail(PN_ERR_CUDA, std::string("launch: ") + cudaGetErrorString(e));
-    }
-  }
+  return PN_OK;
+}
+
+pn_status pn_bound_destroy(pn_bound_t* b) {
+  delete b;
   return PN_OK;
 }
 
@@ -238,8 +350,12 @@ pn_status pn_graph_run_host(pn_graph_t* h, const void* const* inputs, int n_inpu
                             int n_outputs, void* stream) {
   pn_status st = check_counts(h, inputs, n_inputs, outputs, n_outputs);
   if (st != PN_OK) return st;
+  if (h->flags & PN_FLAG_STATIC_SCRATCH)   // before anything is allocated for it
+    return fail(PN_ERR_INVALID_ARG, "this handle owns no workspace and may not allocate: run it with pn_graph_run_static on device buffers");
   const Graph& g = h->g;
   if (any_empty(g)) return PN_OK;
+  DeviceScope dev(h->device);
+  if (dev.err != cudaSuccess) return fail(PN_ERR_CUDA, std::string("cudaSetDevice: ") + cudaGetErrorString(dev.err));
   cudaStream_t s = (cudaStream_t)stream;
   cudaError_t e;
   if (h->stage_in.empty() && h->stage_out.empty()) {
@@ -319,7 +435,7 @@ pn_status pn_graph_run_host(pn_graph_t* h, const void* const* inputs, int n_inpu
     h->pipe_events.push_back(ev);
   }
   cudaStream_t s_in = (cudaStream_t)h->copy_in, s_out = (cudaStream_t)h->copy_out;
-  PlannedLaunch& pl = h->launches[0];
+  const PlannedLaunch& pl = h->launches[0];
   auto ev = [&](int i) { return (cudaEvent_t)h->pipe_events[i]; };
   auto check = [&](cudaError_t err, const char* what) { return err == cudaSuccess ? PN_OK : fail(PN_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(err)); };
   // what the caller queued on its stream comes first
@@ -345,10 +461,8 @@ pn_status pn_graph_run_host(pn_graph_t* h, const void* const* inputs, int n_inpu
     if (result == PN_OK) result = check(cudaEventRecord(ev(2 * k), s_in), "event");
     if (result == PN_OK) result = check(cudaStreamWaitEvent(s, ev(2 * k), 0), "wait");
     if (result != PN_OK) break;
-    pl.plan.p.item_begin = a * cut.items_per_outer;
-    pl.plan.p.item_end = b * cut.items_per_outer;
-    result = pn_graph_run(h, (const void* const*)h->stage_in.data(), n_inputs, h->stage_out.data(), n_outputs, stream);
-    pl.plan.p.item_begin = pl.plan.p.item_end = 0;
+    result = enqueue_launches(h, (const void* const*)h->stage_in.data(), h->stage_out.data(), h->workspace, stream,
+                              a * cut.items_per_outer, b * cut.items_per_outer);
     if (result == PN_OK) result = check(cudaEventRecord(ev(2 * k + 1), s), "event");
     if (result == PN_OK) result = check(cudaStreamWaitEvent(s_out, ev(2 * k + 1), 0), "wait");
     for (int q = 0; q < pl.plan.p.n_io && result == PN_OK; ++q) {
@@ -371,6 +485,8 @@ pn_status pn_graph_run_host(pn_graph_t* h, const void* const* inputs, int n_inpu
 pn_status pn_graph_destroy(pn_graph_t* h) {
   if (!h) return PN_OK;
   if (!h->plan_only) {
+    DeviceScope scope(h->device);
+    for (PlannedLaunch& pl : h->launches) spec_release(pl.spec.fn);   // the kernel cache may unload what nobody uses
     if (h->workspace) cudaFree(h->workspace);
     if (h->status) cudaFree(h->status);
     if (h->copy_in) cudaStreamDestroy((cudaStream_t)h->copy_in);
@@ -417,6 +533,12 @@ pn_status pn_graph_query(const pn_graph_t* h, int what, void* out, size_t out_by
       const cudaError_t e = cudaMemcpy(&w, h->status, sizeof(w), cudaMemcpyDeviceToHost);   // waits for the device
       if (e != cudaSuccess) return fail(PN_ERR_CUDA, std::string("status word: ") + cudaGetErrorString(e));
       v.push_back((int64_t)w);
+      break;
+    }
+    case PN_Q_KERNEL_CACHE: {
+      int64_t modules = 0, in_use = 0;
+      spec_cache_stats(&modules, &in_use);
+      v.push_back(modules); v.push_back(in_use);
       break;
     }
     default: return fail(PN_ERR_INVALID_ARG, "unknown query");

@@ -5,8 +5,8 @@
 // last-dim reductions); (2) expansion of every node into tile / reduction / scalar
 // micro-operations, split into stages at reduction boundaries; (3) choice of the kernel
 // family and tile shape from (rows, N, dtypes, SM count) -- the per-shape cost model whose
-// absence the paper names as a failure mode ("static tiling across varying shapes",
-// Section 4.4); (4) accumulator-machine code generation with register allocation;
+// absence (tile shapes fixed whatever the tensor shape) the paper counts among the failure
+// modes of generated passes, Section 4.4; (4) accumulator-machine code generation with register allocation;
 // (5) shared-memory layout and grid.  Graphs whose reductions run over a leading dimension are
 // lowered by lower_col.cpp (the column-reduce family); roll / slice / view chains on graph inputs
 // become the addressing of the kernel's loads here.

@@ -10,14 +10,11 @@
 #include "../../include/pn.h"
 #include "handle.h"
 
-namespace pn {
-cudaError_t launch_plan(const LaunchPlan& lp, cudaStream_t stream);   // kernels.cu
-}
-
 using namespace pn;
 
-// The scratch itself, at file scope.  Every GPU that loads the library holds these bytes until
-// the process exits, whether or not the entry point is ever called.
+// The scratch itself, at file scope.  A GPU starts holding these bytes when this file's device
+// code is first loaded onto it (the set-up below, at the create of a static-scratch handle) and
+// holds them until the process exits.
 static __device__ __align__(256) unsigned char g_static_scratch[PN_STATIC_SCRATCH_BYTES];
 
 namespace {
@@ -28,14 +25,22 @@ constexpr int kMaxDevices = 64;
 void* g_scratch_ptr[kMaxDevices] = {};
 std::mutex g_setup_mutex;
 
-pn_status scratch_for_device(int device, void** out) {
+}  // namespace
+
+namespace pn {
+
+// Set-up, called by pn_graph_create for PN_FLAG_STATIC_SCRATCH handles: the lookup may make the
+// runtime load this file's device code onto the device, which is when the array's memory is
+// reserved there -- so it happens at create time, where a failure can be reported, and never in
+// a run.  The caller's current device is left as it was.
+int static_scratch_address(int device, void** out) {
   if (device < 0 || device >= kMaxDevices) return fail(PN_ERR_DEVICE, "device ordinal out of range");
   std::lock_guard<std::mutex> lock(g_setup_mutex);
   if (!g_scratch_ptr[device]) {
-    cudaError_t e = cudaSetDevice(device);
-    if (e != cudaSuccess) return fail(PN_ERR_CUDA, std::string("cudaSetDevice: ") + cudaGetErrorString(e));
+    DeviceScope scope(device);
+    if (scope.err != cudaSuccess) return fail(PN_ERR_CUDA, std::string("cudaSetDevice: ") + cudaGetErrorString(scope.err));
     void* ptr = nullptr;
-    e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+    const cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
     if (e != cudaSuccess || !ptr) return fail(PN_ERR_CUDA, std::string("cudaGetSymbolAddress: ") + cudaGetErrorString(e));
     g_scratch_ptr[device] = ptr;
   }
@@ -43,9 +48,7 @@ pn_status scratch_for_device(int device, void** out) {
   return PN_OK;
 }
 
-int64_t bytes_of(const Tensor& t) { return t.numel() * dtype_bytes(t.dtype); }
-
-}  // namespace
+}  // namespace pn
 
 extern "C" {
 #pragma GCC visibility push(default)
@@ -64,46 +67,14 @@ pn_status pn_graph_run_static(pn_graph_t* h, const void* const* inputs, int n_in
     return fail(PN_ERR_TOO_LARGE, "the graph's intermediates need " + std::to_string(h->workspace_bytes) +
                                       " bytes; the static scratch holds " + std::to_string((long long)PN_STATIC_SCRATCH_BYTES));
   for (const Tensor& t : g.tensors) if (t.numel() == 0) return PN_OK;   // nothing to compute
-  const bool scalar = (h->flags & PN_FLAG_FORCE_SCALAR) != 0;
-  for (int i = 0; i < n_inputs; ++i) {
-    if (!inputs[i]) return fail(PN_ERR_INVALID_ARG, "input " + std::to_string(i) + " is null");
-    const uintptr_t m = scalar ? (uintptr_t)(dtype_bytes(g.tensors[g.inputs[i]].dtype) - 1) : 15;
-    if ((uintptr_t)inputs[i] & m) return fail(PN_ERR_ALIGNMENT, "input " + std::to_string(i) + " is not aligned");
-  }
-  for (int o = 0; o < n_outputs; ++o) {
-    if (!outputs[o]) return fail(PN_ERR_INVALID_ARG, "output " + std::to_string(o) + " is null");
-    const uintptr_t m = scalar ? (uintptr_t)(dtype_bytes(g.tensors[g.outputs[o]].dtype) - 1) : 15;
-    if ((uintptr_t)outputs[o] & m) return fail(PN_ERR_ALIGNMENT, "output " + std::to_string(o) + " is not aligned");
-    const char* b0 = (const char*)outputs[o];
-    const char* b1 = b0 + bytes_of(g.tensors[g.outputs[o]]);
-    for (int i = 0; i < n_inputs; ++i) {
-      const char* a0 = (const char*)inputs[i];
-      if (a0 < b1 && b0 < a0 + bytes_of(g.tensors[g.inputs[i]]))
-        return fail(PN_ERR_INVALID_ARG, "input " + std::to_string(i) + " overlaps output " + std::to_string(o));
-    }
-  }
-  void* scratch = nullptr;
-  pn_status st = scratch_for_device(h->device, &scratch);
+  // the same pointer rules as pn_graph_run: alignment, no output over an input or another output
+  const pn_status st = check_run_arguments(h, inputs, n_inputs, outputs, n_outputs);
   if (st != PN_OK) return st;
+  if (!h->static_scratch) return fail(PN_ERR_CUDA, "the static scratch was not set up when the handle was created");
   // Every intermediate is fully written by the kernel that produces it before any kernel
   // reads it (the launches are stream-ordered), so nothing left by an earlier call is ever
   // read and nothing needs clearing.
-  for (PlannedLaunch& pl : h->launches) {
-    for (int q = 0; q < pl.plan.p.n_io; ++q) {
-      const IoSource& s = pl.src[q];
-      pl.plan.p.io[q].base = s.kind == 0 ? const_cast<void*>(inputs[s.index])
-                           : s.kind == 1 ? outputs[s.index]
-                                         : (void*)((char*)scratch + s.index);
-    }
-    if (pl.spec.fn) {
-      std::string err;
-      if (!spec_launch(pl.spec, pl.plan, stream, err)) return fail(PN_ERR_CUDA, err);
-    } else {
-      const cudaError_t e = launch_plan(pl.plan, (cudaStream_t)stream);
-      if (e != cudaSuccess) return fail(PN_ERR_CUDA, std::string("launch: ") + cudaGetErrorString(e));
-    }
-  }
-  return PN_OK;
+  return enqueue_launches(h, inputs, outputs, h->static_scratch, stream, 0, 0);
 }
 
 #pragma GCC visibility pop

@@ -70,7 +70,8 @@ pn_status pn_sequence_create(int n, pn_graph_t* const* graphs, const void* const
   if (!s) return fail(PN_ERR_INVALID_ARG, "out of host memory");
   s->device = graphs[0]->device;
   s->n_items = n;
-  cudaError_t e = cudaSetDevice(s->device);
+  DeviceScope scope(s->device);   // the caller's current device is put back on every path out
+  cudaError_t e = scope.err;
   if (e != cudaSuccess) { delete s; return cuda_fail("cudaSetDevice", e); }
 
   Capture c;
@@ -121,6 +122,8 @@ pn_status pn_sequence_create(int n, pn_graph_t* const* graphs, const void* const
 
 pn_status pn_sequence_run(pn_sequence_t* s, void* stream) {
   if (!s || !s->exec) return fail(PN_ERR_INVALID_ARG, "null sequence");
+  DeviceScope scope(s->device);
+  if (scope.err != cudaSuccess) return cuda_fail("cudaSetDevice", scope.err);
   const cudaError_t e = cudaGraphLaunch(s->exec, (cudaStream_t)stream);
   if (e != cudaSuccess) return cuda_fail("cudaGraphLaunch", e);
   return PN_OK;

@@ -5,18 +5,30 @@
 // without the per-instruction decode and with registers allocated by the compiler.
 //
 // NVRTC and the driver API are opened with dlopen, so that the library loads (and the
-// interpreter works) on machines that have neither.
+// interpreter works) on machines that have neither.  NVRTC is looked for at the toolkit's full
+// path first (PN_NVRTC_PATH, then CUDA_HOME / CUDA_PATH, then /usr/local/cuda) and by its bare
+// soname last, and bound locally: a process that has another NVRTC loaded under the same soname
+// (a framework's bundled copy, possibly older) still gets the toolkit's.
+//
+// Loaded kernels live in a process-wide cache keyed by a hash of (device, source, options),
+// reference-counted by the handles that use them; entries nobody uses any more are unloaded,
+// least recently used first, once the cache holds more than kCacheCap modules.  With
+// PN_CACHE_DIR set, compiled cubins are also kept on disk there, keyed by the same hash plus the
+// NVRTC version, so that a second process pays no compilation.
 #include <cuda.h>
 #include <dlfcn.h>
 #include <nvrtc.h>
 #include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
+#include <sys/stat.h>
+#include <unistd.h>
 
 #include <algorithm>
 #include <map>
 #include <mutex>
 #include <string>
+#include <tuple>
 #include <vector>
 
 #include "graph.h"
@@ -56,9 +68,13 @@ struct Api {
   nvrtcResult (*GetCUBINSize)(nvrtcProgram, size_t*) = nullptr;
   nvrtcResult (*GetCUBIN)(nvrtcProgram, char*) = nullptr;
   nvrtcResult (*DestroyProgram)(nvrtcProgram*) = nullptr;
+  nvrtcResult (*Version)(int*, int*) = nullptr;
+  int nvrtc_major = 0, nvrtc_minor = 0;
+  std::string nvrtc_path;
   // driver
   CUresult (*ModuleLoadData)(CUmodule*, const void*) = nullptr;
   CUresult (*ModuleGetFunction)(CUfunction*, CUmodule, const char*) = nullptr;
+  CUresult (*ModuleUnload)(CUmodule) = nullptr;
   CUresult (*FuncSetAttribute)(CUfunction, CUfunction_attribute, int) = nullptr;
   CUresult (*LaunchKernelEx)(const CUlaunchConfig*, CUfunction, void**, void**) = nullptr;
   CUresult (*OccupancyMaxActiveBlocks)(int*, CUfunction, int, size_t) = nullptr;
@@ -76,23 +92,31 @@ const Api& api() {
   static Api a;
   static std::once_flag once;
   std::call_once(once, [] {
-    const char* builtins[] = {"libnvrtc-builtins.so.12.9", "/usr/local/cuda/lib64/libnvrtc-builtins.so.12.9",
-                              "libnvrtc-builtins.so.12.8", "libnvrtc-builtins.so"};
-    const char* names[] = {"libnvrtc.so.12", "/usr/local/cuda/lib64/libnvrtc.so.12", "libnvrtc.so"};
-    void* rt = nullptr;
-    for (const char* n : names) {
-      for (const char* b : builtins) if (dlopen(b, RTLD_NOW | RTLD_GLOBAL)) break;   // best effort
-      if ((rt = dlopen(n, RTLD_NOW | RTLD_GLOBAL))) break;
+    // where to look for NVRTC: an explicit path (then nothing else), the toolkit's directories, the soname
+    std::vector<std::string> names;
+    if (const char* e = getenv("PN_NVRTC_PATH")) names.push_back(e);
+    else {
+      for (const char* var : {"CUDA_HOME", "CUDA_PATH"})
+        if (const char* e = getenv(var)) names.push_back(std::string(e) + "/lib64/libnvrtc.so.12");
+      names.push_back("/usr/local/cuda/lib64/libnvrtc.so.12");
+      names.push_back("libnvrtc.so.12");
+      names.push_back("libnvrtc.so");
     }
-    if (!rt) { a.why = "libnvrtc.so.12 not found"; return; }
+    void* rt = nullptr;
+    for (const std::string& n : names)
+      if ((rt = dlopen(n.c_str(), RTLD_NOW | RTLD_LOCAL))) { a.nvrtc_path = n; break; }
+    if (!rt) { a.why = "NVRTC not found (tried " + names.front() + (names.size() > 1 ? " and " + std::to_string(names.size() - 1) + " more" : std::string()) + ")"; return; }
     bool ok = sym(rt, "nvrtcCreateProgram", a.CreateProgram, a.why) && sym(rt, "nvrtcCompileProgram", a.CompileProgram, a.why) &&
               sym(rt, "nvrtcGetProgramLogSize", a.GetProgramLogSize, a.why) && sym(rt, "nvrtcGetProgramLog", a.GetProgramLog, a.why) &&
               sym(rt, "nvrtcGetCUBINSize", a.GetCUBINSize, a.why) && sym(rt, "nvrtcGetCUBIN", a.GetCUBIN, a.why) &&
-              sym(rt, "nvrtcDestroyProgram", a.DestroyProgram, a.why);
+              sym(rt, "nvrtcDestroyProgram", a.DestroyProgram, a.why) && sym(rt, "nvrtcVersion", a.Version, a.why);
     if (!ok) { a.CreateProgram = nullptr; return; }
-    void* cu = dlopen("libcuda.so.1", RTLD_NOW | RTLD_GLOBAL);   // absent on machines without a GPU
-    if (!cu) { a.why = "libcuda.so.1 not found"; return; }
+    a.Version(&a.nvrtc_major, &a.nvrtc_minor);
+    const char* cu_name = getenv("PN_LIBCUDA_PATH") ? getenv("PN_LIBCUDA_PATH") : "libcuda.so.1";
+    void* cu = dlopen(cu_name, RTLD_NOW | RTLD_LOCAL);   // absent on machines without a GPU
+    if (!cu) { a.why = std::string(cu_name) + " not found (the CUDA driver library)"; return; }
     ok = sym(cu, "cuModuleLoadData", a.ModuleLoadData, a.why) && sym(cu, "cuModuleGetFunction", a.ModuleGetFunction, a.why) &&
+              sym(cu, "cuModuleUnload", a.ModuleUnload, a.why) &&
               sym(cu, "cuFuncSetAttribute", a.FuncSetAttribute, a.why) && sym(cu, "cuLaunchKernelEx", a.LaunchKernelEx, a.why) &&
               sym(cu, "cuOccupancyMaxActiveBlocksPerMultiprocessor", a.OccupancyMaxActiveBlocks, a.why) &&
               sym(cu, "cuGetErrorString", a.GetErrorString, a.why);
@@ -322,9 +346,65 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
   return true;
 }
 
-struct Compiled { CUmodule mod = nullptr; CUfunction fn = nullptr; };
+struct Compiled { CUmodule mod = nullptr; CUfunction fn = nullptr; int refs = 0; uint64_t used = 0; };
+struct Key {
+  int device; uint64_t h1, h2; size_t len;
+  bool operator<(const Key& o) const { return std::tie(device, h1, h2, len) < std::tie(o.device, o.h1, o.h2, o.len); }
+};
+constexpr size_t kCacheCap = 256;   // loaded modules kept although no handle uses them
 std::mutex g_cache_mutex;
-std::map<std::pair<int, std::string>, Compiled> g_cache;   // (device, source) -> loaded kernel; lives until exit
+std::map<Key, Compiled> g_cache;
+uint64_t g_cache_clock = 0;
+
+uint64_t fnv(const std::string& s, uint64_t h) { for (unsigned char c : s) { h ^= c; h *= 1099511628211ull; } return h; }
+Key key_of(int device, const std::string& src) { return Key{device, fnv(src, 1469598103934665603ull), fnv(src, 0x9E3779B97F4A7C15ull), src.size()}; }
+
+// unload modules nobody holds, least recently used first, down to the cap (call with the lock held)
+void evict_unused() {
+  while (g_cache.size() > kCacheCap) {
+    auto victim = g_cache.end();
+    for (auto it = g_cache.begin(); it != g_cache.end(); ++it)
+      if (it->second.refs == 0 && (victim == g_cache.end() || it->second.used < victim->second.used)) victim = it;
+    if (victim == g_cache.end()) return;
+    if (api().ModuleUnload) api().ModuleUnload(victim->second.mod);
+    g_cache.erase(victim);
+  }
+}
+
+// ---- the optional cubin cache on disk ------------------------------------------------------------
+struct DiskHeader { uint32_t magic; int32_t nvrtc_major, nvrtc_minor; uint64_t h1, h2, src_len, cubin_len; };
+constexpr uint32_t kDiskMagic = 0x42434E50u;   // 'PNCB'
+std::string disk_path(const Key& k) {
+  const char* dir = getenv("PN_CACHE_DIR");
+  if (!dir || !*dir) return std::string();
+  char name[96];
+  snprintf(name, sizeof(name), "/pn_%016llx%016llx_sm100a.cubin", (unsigned long long)k.h1, (unsigned long long)k.h2);
+  return std::string(dir) + name;
+}
+bool disk_load(const Key& k, std::vector<char>& cubin) {
+  const std::string path = disk_path(k);
+  if (path.empty()) return false;
+  FILE* f = fopen(path.c_str(), "rb");
+  if (!f) return false;
+  DiskHeader h;
+  bool ok = fread(&h, sizeof(h), 1, f) == 1 && h.magic == kDiskMagic && h.nvrtc_major == api().nvrtc_major && h.nvrtc_minor == api().nvrtc_minor &&
+            h.h1 == k.h1 && h.h2 == k.h2 && h.src_len == k.len && h.cubin_len > 0 && h.cubin_len < (64u << 20);
+  if (ok) { cubin.resize(h.cubin_len); ok = fread(cubin.data(), 1, cubin.size(), f) == cubin.size(); }
+  fclose(f);
+  return ok;
+}
+void disk_store(const Key& k, const std::vector<char>& cubin) {
+  const std::string path = disk_path(k);
+  if (path.empty()) return;
+  mkdir(getenv("PN_CACHE_DIR"), 0777);   // best effort; an existing directory is fine
+  const std::string tmp = path + "." + std::to_string((long)getpid()) + ".tmp";
+  FILE* f = fopen(tmp.c_str(), "wb");
+  if (!f) return;
+  const DiskHeader h{kDiskMagic, api().nvrtc_major, api().nvrtc_minor, k.h1, k.h2, (uint64_t)k.len, (uint64_t)cubin.size()};
+  const bool ok = fwrite(&h, sizeof(h), 1, f) == 1 && fwrite(cubin.data(), 1, cubin.size(), f) == cubin.size();
+  fclose(f);
+  if (ok) rename(tmp.c_str(), path.c_str()); else remove(tmp.c_str());   // rename: readers never see half a file
+}
 
 }  // namespace
 
@@ -366,42 +446,56 @@ bool spec_compile(LaunchPlan& lp, int device, int sm_count, SpecKernel& out, std
   std::string src;
   if (!generate_source(lp, src, err)) return false;
   { std::string key; for (const std::string& x : nvrtc_options()) key += x + " "; src += "\n// " + key + "\n"; }
+  const Key key = key_of(device, src);
   Compiled cmp;
   {
     std::lock_guard<std::mutex> lock(g_cache_mutex);
-    auto it = g_cache.find(std::make_pair(device, src));
-    if (it != g_cache.end()) cmp = it->second;
+    auto it = g_cache.find(key);
+    if (it != g_cache.end()) { it->second.refs++; it->second.used = ++g_cache_clock; cmp = it->second; }
   }
   if (!cmp.fn) {
-    nvrtcProgram prog;
-    if (a.CreateProgram(&prog, src.c_str(), "pn_spec.cu", 0, nullptr, nullptr) != NVRTC_SUCCESS) { err = "nvrtcCreateProgram failed"; return false; }
-    const std::vector<std::string> ov = nvrtc_options();
-    std::vector<const char*> opts;
-    for (const std::string& x : ov) opts.push_back(x.c_str());
-    const nvrtcResult r = a.CompileProgram(prog, (int)opts.size(), opts.data());
-    if (r != NVRTC_SUCCESS) {
-      size_t n = 0; a.GetProgramLogSize(prog, &n);
-      std::string log(n, '\0');
-      if (n) a.GetProgramLog(prog, &log[0]);
+    std::vector<char> cubin;
+    if (!disk_load(key, cubin)) {
+      nvrtcProgram prog;
+      if (a.CreateProgram(&prog, src.c_str(), "pn_spec.cu", 0, nullptr, nullptr) != NVRTC_SUCCESS) { err = "nvrtcCreateProgram failed"; return false; }
+      const std::vector<std::string> ov = nvrtc_options();
+      std::vector<const char*> opts;
+      for (const std::string& x : ov) opts.push_back(x.c_str());
+      const nvrtcResult r = a.CompileProgram(prog, (int)opts.size(), opts.data());
+      if (r != NVRTC_SUCCESS) {
+        size_t n = 0; a.GetProgramLogSize(prog, &n);
+        std::string log(n, '\0');
+        if (n) a.GetProgramLog(prog, &log[0]);
+        a.DestroyProgram(&prog);
+        err = "run-time compilation failed: " + log.substr(0, 2000);
+        return false;
+      }
+      size_t n = 0;
+      a.GetCUBINSize(prog, &n);
+      cubin.resize(n);
+      a.GetCUBIN(prog, cubin.data());
       a.DestroyProgram(&prog);
-      err = "run-time compilation failed: " + log.substr(0, 2000);
-      return false;
+      disk_store(key, cubin);
     }
-    size_t n = 0;
-    a.GetCUBINSize(prog, &n);
-    std::vector<char> cubin(n);
-    a.GetCUBIN(prog, cubin.data());
-    a.DestroyProgram(&prog);
     CUresult cr = a.ModuleLoadData(&cmp.mod, cubin.data());
     if (cr != CUDA_SUCCESS) { err = "cuModuleLoadData: " + cu_err(cr); return false; }
     cr = a.ModuleGetFunction(&cmp.fn, cmp.mod, kernel_name(lp).c_str());
-    if (cr != CUDA_SUCCESS) { err = "cuModuleGetFunction: " + cu_err(cr); return false; }
+    if (cr != CUDA_SUCCESS) { a.ModuleUnload(cmp.mod); err = "cuModuleGetFunction: " + cu_err(cr); return false; }
     std::lock_guard<std::mutex> lock(g_cache_mutex);
-    g_cache[std::make_pair(device, src)] = cmp;
+    auto it = g_cache.find(key);
+    if (it != g_cache.end()) {   // another thread loaded the same kernel meanwhile: keep that one
+      a.ModuleUnload(cmp.mod);
+      it->second.refs++; it->second.used = ++g_cache_clock;
+      cmp = it->second;
+    } else {
+      cmp.refs = 1; cmp.used = ++g_cache_clock;
+      g_cache[key] = cmp;
+      evict_unused();
+    }
   }
   if (lp.smem_bytes > 48 * 1024) {
     const CUresult cr = a.FuncSetAttribute(cmp.fn, CU_FUNC_ATTRIBUTE_MAX_DYNAMIC_SHARED_SIZE_BYTES, lp.smem_bytes);
-    if (cr != CUDA_SUCCESS) { err = "cuFuncSetAttribute: " + cu_err(cr); return false; }
+    if (cr != CUDA_SUCCESS) { spec_release(cmp.fn); err = "cuFuncSetAttribute: " + cu_err(cr); return false; }
   }
   int occ = 0;
   if (a.OccupancyMaxActiveBlocks(&occ, cmp.fn, lp.block, (size_t)lp.smem_bytes) != CUDA_SUCCESS) occ = 0;
@@ -410,6 +504,21 @@ bool spec_compile(LaunchPlan& lp, int device, int sm_count, SpecKernel& out, std
   lp.specialised = 1;
   size_grid(lp, sm_count, occ);
   return true;
+}
+
+void spec_release(void* fn) {
+  if (!fn) return;
+  std::lock_guard<std::mutex> lock(g_cache_mutex);
+  for (auto& kv : g_cache)
+    if (kv.second.fn == (CUfunction)fn) { if (kv.second.refs > 0) kv.second.refs--; break; }
+  evict_unused();
+}
+
+void spec_cache_stats(int64_t* modules, int64_t* in_use) {
+  std::lock_guard<std::mutex> lock(g_cache_mutex);
+  *modules = (int64_t)g_cache.size();
+  *in_use = 0;
+  for (auto& kv : g_cache) *in_use += kv.second.refs > 0;
 }
 
 bool spec_launch(const SpecKernel& k, const LaunchPlan& lp, void* stream, std::string& err) {

@@ -19,6 +19,12 @@ bool spec_available(std::string* why, bool compile_only = false);
 // current device and re-size the plan's grid from the kernel's occupancy.
 bool spec_compile(LaunchPlan& lp, int device, int sm_count, SpecKernel& out, std::string& err);
 
+// A handle that goes away gives its kernel back: the cache may then unload it.
+void spec_release(void* fn);
+
+// Loaded modules in the cache, and how many of them a live handle uses.
+void spec_cache_stats(int64_t* modules, int64_t* in_use);
+
 // Enqueue the specialised kernel of a plan on a stream.
 bool spec_launch(const SpecKernel& k, const LaunchPlan& lp, void* stream, std::string& err);
 

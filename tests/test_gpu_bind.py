@@ -1,0 +1,76 @@
+"""pn_graph_bind / pn_bound_run: the same results as pn_graph_run, from a handle that is only read
+(two bound objects of one handle on different buffers stay independent), and the calling
+thread's current device is what it was."""
+import numpy as np
+import pytest
+
+import paper_2605_29357_b200 as pn
+from pn_workloads import configs as C
+from pn_workloads import descriptor as D
+
+from gpu_util import check_against_oracle, device_bytes, poisoned
+
+pytestmark = pytest.mark.gpu
+
+
+def _buffers(w):
+    d_in = [device_bytes(a) for a in w.inputs]
+    sizes = [D.DTYPE_BYTES[dt] * int(np.prod(dims, dtype=np.int64)) for dt, dims in w.output_meta]
+    return d_in, [poisoned(s) for s in sizes], sizes
+
+
+def _host(d_out, sizes, metas):
+    return [t.cpu().numpy()[:s].view(C.NP_STORAGE[dt]).reshape(dims) for t, s, (dt, dims) in zip(d_out, sizes, metas)]
+
+
+@pytest.mark.parametrize("cfg", ["c1", "c2", "c3", "c4", "c5", "n1", "n2"])
+@pytest.mark.parametrize("flags", [0, pn.FLAG_UNFUSED, pn.FLAG_INTERPRET])
+def test_bound_launches_equal_direct_runs_and_do_not_disturb_each_other(cfg, flags):
+    import torch
+    makers = {**C.CONFIGS, **C.EXTENDED}
+    wa, wb = makers[cfg](seed=1, **C.SMALL[cfg]), makers[cfg](seed=2, **C.SMALL[cfg])
+    g = pn.Graph(wa.desc, 0, flags)
+    stream = torch.cuda.current_stream().cuda_stream
+    ina, outa, sizes = _buffers(wa)
+    inb, outb, _ = _buffers(wb)
+    fa = g.bind([t.data_ptr() for t in ina], [t.data_ptr() for t in outa])
+    fb = g.bind([t.data_ptr() for t in inb], [t.data_ptr() for t in outb])
+    before = torch.cuda.current_device()
+    fa(stream); fb(stream); fa(stream)          # interleaved: neither sees the other's pointers
+    torch.cuda.synchronize()
+    assert torch.cuda.current_device() == before
+    got_a, got_b = _host(outa, sizes, wa.output_meta), _host(outb, sizes, wb.output_meta)
+    check_against_oracle(wa.desc, wa.inputs, got_a, wa.output_meta, wa.output_names)
+    check_against_oracle(wb.desc, wb.inputs, got_b, wb.output_meta, wb.output_names)
+    # bit for bit what the checked entry point gives
+    _, outc, _ = _buffers(wa)
+    g.run([t.data_ptr() for t in ina], [t.data_ptr() for t in outc], stream)
+    torch.cuda.synchronize()
+    for x, y in zip(got_a, _host(outc, sizes, wa.output_meta)):
+        assert np.array_equal(x.view(np.uint8), y.view(np.uint8))
+    fa.close(); fb.close(); g.close()
+
+
+def test_bind_runs_the_argument_checks_once_and_for_all():
+    import torch
+    w = C.c3(**C.SMALL["c3"])
+    g = pn.Graph(w.desc, 0, 0)
+    d_in, d_out, _ = _buffers(w)
+    ins, outs = [t.data_ptr() for t in d_in], [t.data_ptr() for t in d_out]
+    with pytest.raises(pn.PnError) as e:
+        g.bind(ins[:-1], outs)
+    assert e.value.status == -7
+    with pytest.raises(pn.PnError) as e:
+        g.bind([ins[0] + 2] + ins[1:], outs)
+    assert e.value.status == -6
+    with pytest.raises(pn.PnError) as e:
+        g.bind(ins, [outs[0]] * len(outs))      # outputs over one another
+    assert e.value.status == -1
+    with pytest.raises(pn.PnError) as e:
+        g.bind(ins, [ins[0]] + outs[1:])        # an output over an input, exactly
+    assert e.value.status == -1
+    st = pn.Graph(w.desc, 0, pn.FLAG_UNFUSED | pn.FLAG_STATIC_SCRATCH)
+    with pytest.raises(pn.PnError) as e:
+        st.bind(ins, outs)
+    assert e.value.status == -1
+    torch.cuda.synchronize()

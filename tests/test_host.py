@@ -6,6 +6,7 @@ import ctypes
 import os
 import re
 import struct
+import sys
 
 import pytest
 
@@ -283,3 +284,36 @@ def test_checked_accessors_are_compiled_in_only_on_request():
     checked = pn.Graph(w.desc, 0, PLAN | pn.FLAG_BOUNDS)
     assert plain.codegen(0, compile=True) == checked.codegen(0, compile=True)   # same program; the switch is a macro
     assert _status(w.desc, PLAN | pn.FLAG_BOUNDS | pn.FLAG_UNFUSED | pn.FLAG_STATIC_SCRATCH) == -1
+
+
+def _create_in_child(env_extra, flags):
+    """pn_graph_create (plan only) in a fresh process, so that the library resolves NVRTC under the
+    given environment.  Returns (status, detail, specialised)."""
+    import subprocess
+    code = (
+        "import sys; sys.path.insert(0, %r)\n"
+        "import paper_2605_29357_b200 as pn\n"
+        "from pn_workloads import configs as C\n"
+        "w = C.c1(M=4, N=64)\n"
+        "try:\n"
+        "    g = pn.Graph(w.desc, 0, %d)\n"
+        "    print('OK', g.kernel_info[0]['specialised'])\n"
+        "except pn.PnError as e:\n"
+        "    print('ERR', e.status, e.detail)\n" % (ROOT, flags))
+    env = dict(os.environ, **env_extra)
+    r = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    return r.stdout.strip().splitlines()[-1]
+
+
+def test_a_create_that_cannot_specialise_fails_loudly_unless_the_interpreter_is_asked_for():
+    missing = {"PN_NVRTC_PATH": "/nonexistent/libnvrtc.so.12"}
+    out = _create_in_child(missing, pn.FLAG_PLAN_ONLY)
+    assert out.startswith("ERR -8") and "NVRTC not found" in out and "PN_FLAG_ALLOW_INTERPRET" in out
+    # asked for by name, or allowed: the handle is lowered for the interpreter kernels
+    assert _create_in_child(missing, pn.FLAG_PLAN_ONLY | pn.FLAG_ALLOW_INTERPRET) == "OK 0"
+    assert _create_in_child(missing, pn.FLAG_PLAN_ONLY | pn.FLAG_INTERPRET) == "OK 0"
+    # with NVRTC where the toolkit puts it, the same create succeeds (plan-only handles report 0: nothing is loaded)
+    assert _create_in_child({}, pn.FLAG_PLAN_ONLY).startswith("OK")
+    # a run-time library that is there but is not NVRTC is refused as well
+    assert _create_in_child({"PN_NVRTC_PATH": pn.library_path()}, pn.FLAG_PLAN_ONLY).startswith("ERR -8")

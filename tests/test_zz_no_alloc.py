@@ -59,6 +59,36 @@ def test_static_scratch_matches_the_allocating_path_twice_in_a_row(interpret):
         assert bad.value.status == -1
 
 
+def test_a_run_from_the_static_scratch_leaves_free_memory_alone_and_checks_pointers_like_run():
+    """The set-up (the lookup of the array's address, which is what makes the device reserve it)
+    belongs to the create; the runs themselves must not change the free device memory.  And the
+    pointer rules are those of pn_graph_run, checked by the same code: outputs over one another
+    are refused here too, and the host-memory entry point refuses such a handle before it would
+    allocate its staging buffers."""
+    import torch
+    w = C.c5(**C.SMALL["c5"])
+    g = pn.Graph(w.desc, 0, pn.FLAG_UNFUSED | pn.FLAG_STATIC_SCRATCH)
+    d_in = [device_bytes(a) for a in w.inputs]
+    sizes = [D.DTYPE_BYTES[dt] * int(np.prod(dims, dtype=np.int64)) for dt, dims in g.output_meta]
+    d_out = [poisoned(s) for s in sizes]
+    ins, outs = [t.data_ptr() for t in d_in], [t.data_ptr() for t in d_out]
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    for _ in range(3):
+        g.run_static(ins, outs, torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before
+    with pytest.raises(pn.PnError) as aliased:
+        g.run_static(ins, [outs[0]] * len(outs), 0)
+    assert aliased.value.status == -1 and "overlap" in aliased.value.detail
+    host_in = [np.ascontiguousarray(a) for a in w.inputs]
+    host_out = [np.empty(s, np.uint8) for s in sizes]
+    with pytest.raises(pn.PnError) as host:
+        g.run_host([a.ctypes.data for a in host_in], [a.ctypes.data for a in host_out], 0)
+    assert host.value.status == -1
+    assert torch.cuda.mem_get_info()[0] == free_before      # and it allocated nothing on the way
+
+
 def test_static_scratch_rejects_what_does_not_fit():
     w = C.c2(B=64, Q=256, K=512)          # fp32 intermediates of 8.4 M elements each: far above 32 MiB
     g = pn.Graph(w.desc, 0, pn.FLAG_UNFUSED | pn.FLAG_STATIC_SCRATCH)
