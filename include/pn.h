@@ -107,6 +107,9 @@ enum {
                                      ahead (costs registers; off by default)                 */
   PN_FLAG_STATIC_SCRATCH = 1u << 12,/* with PN_FLAG_UNFUSED: allocate no workspace; the handle
                                      is run with pn_graph_run_static only                    */
+  PN_FLAG_FORCE_SPLIT = 1u << 15, /* row kernels: independent blocks over slices of a row, combined
+                                     through partials in a workspace of the handle (single-stage
+                                     graphs, generated kernels)                               */
   PN_FLAG_ALLOW_INTERPRET = 1u << 14,/* a create that cannot specialise kernels (NVRTC or the driver
                                      library cannot be opened) normally fails with PN_ERR_DEVICE;
                                      with this flag it runs on the interpreter kernels instead  */
@@ -141,7 +144,7 @@ enum {
   PN_Q_KERNEL_CACHE = 11,   /* 2 values, process-wide: generated kernels now loaded, and how many of
                                them a live handle uses                                      */
   PN_Q_KERNEL_INFO = 9      /* per kernel 13 values: family (0 pointwise, 1 warp-per-row,
-                               2 block-per-row, 3 cluster-per-row, 4 column-reduce: rows =
+                               2 block-per-row, 3 cluster-per-row, 5 split-row, 4 column-reduce: rows =
                                the dimensions before the reduced one, row length = those after
                                it), grid, block, cluster,
                                dynamic smem bytes, vector length, groups per tile, chunks
@@ -378,12 +381,13 @@ enum {
 typedef struct pn_probe_config {
   int loader;           /* PN_PROBE_*                                                         */
   int streaming_stores; /* 1: stores carry the evict-first hint                               */
-  int layout;           /* direct loaders: 0 grid-stride over units, 1 a contiguous range per block */
+  int layout;           /* direct loaders: 0 grid-stride over units, 1 a contiguous range per block,
+                           2 runs of tile_units units taken by the blocks in turn (read-only path) */
   int block;            /* threads that load / store per block (multiple of 32, <= 992)       */
   int unroll;           /* direct loaders: units in flight per thread (1, 2, 4, 8)            */
   int grid;             /* blocks                                                             */
   int stages;           /* bulk loader: ring depth (2..16)                                    */
-  int tile_units;       /* bulk loader: units per array per stage (32..4096)                  */
+  int tile_units;       /* bulk loader: units per array per stage (32..4096); layout 2: the run length */
 } pn_probe_config;
 pn_status pn_stream_probe(int mix, const pn_probe_config* cfg, const void* a, const void* b, void* c, void* d,
                           size_t units, void* status_word, void* stream);

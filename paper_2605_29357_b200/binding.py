@@ -28,6 +28,7 @@ FLAG_PREFETCH = 1 << 11
 FLAG_STATIC_SCRATCH = 1 << 12
 FLAG_BOUNDS = 1 << 13
 FLAG_ALLOW_INTERPRET = 1 << 14
+FLAG_FORCE_SPLIT = 1 << 15
 STATIC_SCRATCH_BYTES = 32 << 20
 
 
@@ -40,7 +41,7 @@ def tune(cluster: int = 0, block: int = 0, groups: int = 0, waves: int = 0) -> i
 Q_N_INPUTS, Q_N_OUTPUTS, Q_INPUT_META, Q_OUTPUT_META, Q_COMPULSORY_BYTES = 1, 2, 3, 4, 5
 Q_N_KERNELS, Q_N_NODES, Q_WORKSPACE_BYTES, Q_KERNEL_INFO = 6, 7, 8, 9
 
-FAMILY_NAMES = {0: "pointwise", 1: "warp-per-row", 2: "block-per-row", 3: "cluster-per-row", 4: "column-reduce"}
+FAMILY_NAMES = {0: "pointwise", 1: "warp-per-row", 2: "block-per-row", 3: "cluster-per-row", 4: "column-reduce", 5: "split-row"}
 EXPORTS = ["pn_graph_create", "pn_graph_run", "pn_graph_run_host", "pn_graph_run_static", "pn_graph_destroy",
            "pn_graph_bind", "pn_bound_run", "pn_bound_destroy",
            "pn_graph_query", "pn_graph_codegen", "pn_status_string", "pn_last_error",

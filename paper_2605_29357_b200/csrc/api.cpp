@@ -290,6 +290,32 @@ pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsig
         return fail(PN_ERR_CUDA, err);
       }
   }
+  // split-row launches: partials and arrival counters in device memory of the handle, the counters
+  // zero at rest
+  {
+    auto sizes = [](const LaunchPlan& lp, size_t& part_bytes, size_t& ticket_bytes) {
+      const KernelParams& P = lp.p;
+      part_bytes = ((size_t)P.rows * P.splits * P.stage[0].n_red * 3 * sizeof(float) + 255) / 256 * 256;
+      ticket_bytes = ((size_t)P.rows * sizeof(uint32_t) + 255) / 256 * 256;
+    };
+    size_t need = 0;
+    for (PlannedLaunch& pl : h->launches)
+      if (pl.plan.family == FAM_SPLIT) { size_t a = 0, b = 0; sizes(pl.plan, a, b); need += a + b; }
+    if (need > 0 && !h->plan_only) {
+      cudaError_t e = cudaMalloc(&h->split_ws, need);
+      if (e == cudaSuccess) e = cudaMemset(h->split_ws, 0, need);
+      if (e != cudaSuccess) { pn_graph_destroy(h); return fail(PN_ERR_CUDA, std::string("split-row workspace: ") + cudaGetErrorString(e)); }
+      size_t off = 0;
+      for (PlannedLaunch& pl : h->launches)
+        if (pl.plan.family == FAM_SPLIT) {
+          size_t a = 0, b = 0;
+          sizes(pl.plan, a, b);
+          pl.plan.p.split_part = reinterpret_cast<float*>((char*)h->split_ws + off); off += a;
+          pl.plan.p.split_ticket = reinterpret_cast<uint32_t*>((char*)h->split_ws + off); off += b;
+        }
+    }
+    h->workspace_bytes += need;
+  }
   *out = h;
   return PN_OK;
 }
@@ -381,7 +407,7 @@ pn_status pn_graph_run_host(pn_graph_t* h, const void* const* inputs, int n_inpu
   if (h->launches.size() == 1 && in_bytes >= (8ll << 20)) {
     const LaunchPlan& lp = h->launches[0].plan;
     const KernelParams& P = lp.p;
-    bool ok = P.cluster >= 1;
+    bool ok = P.cluster >= 1 && P.family != FAM_SPLIT;
     for (int q = 0; q < P.n_io; ++q) ok = ok && !P.io[q].mapped;
     cut.stride.assign(P.n_io, 0);
     if (ok && P.family == FAM_COLUMN) {
@@ -488,6 +514,7 @@ pn_status pn_graph_destroy(pn_graph_t* h) {
     DeviceScope scope(h->device);
     for (PlannedLaunch& pl : h->launches) spec_release(pl.spec.fn);   // the kernel cache may unload what nobody uses
     if (h->workspace) cudaFree(h->workspace);
+    if (h->split_ws) cudaFree(h->split_ws);
     if (h->status) cudaFree(h->status);
     if (h->copy_in) cudaStreamDestroy((cudaStream_t)h->copy_in);
     if (h->copy_out) cudaStreamDestroy((cudaStream_t)h->copy_out);

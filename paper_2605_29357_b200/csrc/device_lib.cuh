@@ -612,29 +612,32 @@ template <int VL, int NG, bool FULL = false>
 PN_DEV void op_red(const TileCtx& cx, int kind, Part& st, float (&acc)[VL * NG], float& ts) {
   constexpr int V = VL * NG;
   if (kind == RED_ARGMAX || kind == RED_ARGMIN) {
-    // Branch-free: the tile extreme by a fold, then its first holder by a descending scan of
-    // equality tests (the lowest slot is written last), then one predicated update of the
-    // running (extreme, column).  Ties keep the earlier, lower-index holder; a NaN beats every
-    // number, which only the rarely taken branch below has to know about.
+    // The tile extreme by a fold; if it replaces the running extreme, its first holder by a
+    // descending scan of equality tests (the lowest slot is written last).  Ties keep the earlier,
+    // lower-index holder; a NaN beats every number.
     const bool mx = kind == RED_ARGMAX;
     const float m = mx ? tile_fold<VL, NG, FULL>(cx, acc, -PN_INF, FoldMaxNan()) : tile_fold<VL, NG, FULL>(cx, acc, PN_INF, FoldMinNan());
-    int slot = 0;
-    PN_UNROLL for (int j = NG - 1; j >= 0; --j) {
-      const bool ok = FULL || cx.col0 + j * cx.gstride < cx.col_end;
-      PN_UNROLL for (int i = VL - 1; i >= 0; --i) slot = (ok && acc[j * VL + i] == m) ? j * VL + i : slot;
-    }
     const bool m_nan = m != m, s_nan = st.a != st.a;
-    if (m_nan) {   // the fold returns NaN when the tile holds one: find the first
+    const bool take = cx.chunk == 0 || (m_nan ? !s_nan : (!s_nan && (mx ? m > st.a : m < st.a)));
+    // the holder of the extreme is looked for only when the tile's extreme replaces the running one:
+    // always in the first tile of a row, rarely afterwards (a tie keeps the earlier, lower column)
+    if (take) {
+      int slot = 0;
       PN_UNROLL for (int j = NG - 1; j >= 0; --j) {
         const bool ok = FULL || cx.col0 + j * cx.gstride < cx.col_end;
-        PN_UNROLL for (int i = VL - 1; i >= 0; --i) slot = (ok && acc[j * VL + i] != acc[j * VL + i]) ? j * VL + i : slot;
+        PN_UNROLL for (int i = VL - 1; i >= 0; --i) slot = (ok && acc[j * VL + i] == m) ? j * VL + i : slot;
       }
+      if (m_nan) {   // the fold returns NaN when the tile holds one: find the first
+        PN_UNROLL for (int j = NG - 1; j >= 0; --j) {
+          const bool ok = FULL || cx.col0 + j * cx.gstride < cx.col_end;
+          PN_UNROLL for (int i = VL - 1; i >= 0; --i) slot = (ok && acc[j * VL + i] != acc[j * VL + i]) ? j * VL + i : slot;
+        }
+      }
+      // a thread whose tile lies wholly outside the row keeps the sentinel column, which loses every tie
+      const int bi = (FULL || cx.col0 < cx.col_end) ? cx.col0 + (slot / VL) * cx.gstride + (slot % VL) : 0x7FFFFFFF;
+      st.a = m;
+      st.b = bits_f(static_cast<uint32_t>(bi));
     }
-    const bool take = cx.chunk == 0 || (m_nan ? !s_nan : (!s_nan && (mx ? m > st.a : m < st.a)));
-    // a thread whose tile lies wholly outside the row keeps the sentinel column, which loses every tie
-    const int bi = (FULL || cx.col0 < cx.col_end) ? cx.col0 + (slot / VL) * cx.gstride + (slot % VL) : 0x7FFFFFFF;
-    st.a = take ? m : st.a;
-    st.b = take ? bits_f(static_cast<uint32_t>(bi)) : st.b;
     return;
   }
   Part t = red_identity(kind);
@@ -838,6 +841,7 @@ struct Interp {
   static PN_DEV int split_chunks(const KernelParams& p) { return p.split_chunks; }
   static PN_DEV int row_len(const KernelParams& p) { return p.row_len; }
   static PN_DEV int team_lanes(const KernelParams&) { return 32; }   // short rows sharing a warp: generated kernels only
+  static PN_DEV int splits(const KernelParams& p) { return p.splits; }
   static PN_DEV int slice_len(const KernelParams& p) { return p.slice_len; }
   static PN_DEV int n_stages(const KernelParams& p) { return p.n_stages; }
   static PN_DEV int n_io(const KernelParams& p) { return p.n_io; }
@@ -1127,6 +1131,151 @@ PN_DEV void fused_body(const KernelParams& p, unsigned char* smem) {
   }
   // a CTA's shared memory may still be read by its cluster peers until they pass this point
   if (cluster > 1) cluster_sync_all();
+}
+
+// ---------------------------------------------------------------------------------------
+// the kernel body of the split-row family: very few, very long rows whose graph needs each element once
+// ---------------------------------------------------------------------------------------
+// A handful of long rows cannot fill 148 SMs in whole rows or in clusters of at most 8 blocks per
+// row.  Here a row is cut into `splits` slices of slice_len columns and thread block b reduces slice
+// b % splits of row b / splits: one short-lived block per slice, in memory order, so that the
+// hardware's block scheduler spreads the slices over the SMs as they become free and the blocks in
+// flight read one compact window of memory (measured on B200 with the stream probe, 256 MB read-only:
+// resident blocks that each stream through a contiguous range of their own reach 5.0 TB/s, blocks
+// that take 16 - 32 KB pieces in memory order 6.2 - 6.8 TB/s).  A block leaves its partial of every
+// reduction in device memory (split_part) and takes a ticket: one atomic add on the row's counter.
+// Nobody waits for anybody: the block that draws the last ticket of a row finds all partials of that
+// row written (each writer fenced before its ticket), combines them in slice order -- a fixed order,
+// whichever block happens to be last, so results repeat bit for bit -- runs the per-row scalar
+// program, stores the row's results and puts the counter back to zero for the next launch.
+// Generated kernels only; the graph has a single stage (no tile value is needed again after the
+// reductions).
+//
+// Tried on B200 and dropped, each passing the same parity tests (long-row logsumexp + argmax,
+// [64, 262144] and [256, 262144] fp32; clusters of 4 / 2 blocks per row take 16.3 / 51.2 us): resident
+// blocks over contiguous ranges of tiles, loads one tile ahead in registers or four tiles ahead in
+// shared memory by bulk copies (18.6 / 51 us either way: the access pattern, not the bytes in flight,
+// is the limit); resident blocks taking tiles in turn with a partial per warp and tile, tickets at the
+// end of the block (72 / 306 us: every row is completed, and combined, by the few blocks that end
+// last) or one tile later (63 / 263 us: a fence per tile among loads in flight stalls the warp, and
+// the slowest warp draws every last ticket and so falls further behind).
+PN_DEV float ld_cg(const float* p) { float v; asm("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p) : "memory"); return v; }
+
+template <class Prog>
+PN_DEV void split_body(const KernelParams& p, unsigned char* smem) {
+  constexpr int VL = Prog::VL, NG = Prog::NG, K = Prog::K, V = VL * NG;
+  const int bdim = Prog::block_threads();
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = bdim >> 5;
+  const int S = Prog::splits(p);
+  const int chunks = Prog::chunks(p);
+  const int n_red = Prog::n_red(p, 0);
+  const long long row = blockIdx.x / S;
+  const int split = (int)(blockIdx.x - row * S);
+  const int part_floats = n_red * 3;
+
+  long long rowoff_reg[Prog::kNumIo];
+  long long rowoff_nxt[1];
+  float slots_reg[kMaxSlots];
+  float* wpart = reinterpret_cast<float*>(smem + p.sm_wpart);
+
+  TileCtx cx;
+  cx.rowoff = rowoff_reg;
+  cx.part = nullptr; cx.stash = nullptr;
+  cx.part_stride = bdim;
+  cx.slots = slots_reg;
+  cx.gstride = bdim * VL;
+  cx.chunks = chunks;
+  cx.chunk = 0;
+  cx.leader = false;
+  const int slice_lo = split * Prog::slice_len(p);
+  cx.col_end = min(Prog::row_len(p), slice_lo + Prog::slice_len(p));
+  TileCtx nx = cx;
+  nx.rowoff = rowoff_nxt;
+
+  float acc[V];
+  float reg[K][V];
+  float raw[1][V];
+  float ts = 0.f;
+  Part parts[kMaxRed];
+  PN_UNROLL for (int e = 0; e < V; ++e) acc[e] = 0.f;
+  PN_UNROLL for (int k = 0; k < K; ++k) { PN_UNROLL for (int e = 0; e < V; ++e) reg[k][e] = 0.f; }
+  PN_UNROLL for (int r = 0; r < kMaxRed; ++r) parts[r] = Part{0.f, 0.f, 0.f};
+
+  {   // element offset of the row in every input / output
+    const unsigned long long r0 = (unsigned long long)row;
+    const unsigned d2 = Prog::lead_dim(p, 2), d1 = Prog::lead_dim(p, 1);
+    const unsigned long long q2 = r0 / d2;
+    const long long i2 = (long long)(r0 - q2 * d2);
+    const unsigned long long q1 = q2 / d1;
+    const long long i1 = (long long)(q2 - q1 * d1);
+    PN_UNROLL for (int q = 0; q < Prog::kNumIo; ++q) {
+      if (Prog::io_mapped(p, q)) rowoff_reg[q] = mapped_row_offset(r0, Prog::io_map(p, q));
+      else rowoff_reg[q] = (long long)q1 * Prog::lead_stride(p, q, 0) + i1 * Prog::lead_stride(p, q, 1) + i2 * Prog::lead_stride(p, q, 2);
+    }
+  }
+  const int chunk_cols = bdim * V;
+  for (int c = 0; c < chunks; ++c) {
+    cx.chunk = c;
+    cx.col0 = slice_lo + c * chunk_cols + tid * VL;
+    Prog::tile(p, 0, cx, acc, reg, ts, parts, raw, nx, false);
+  }
+  // the block's partial of every reduction: warps through shared memory, then the first warp
+  PN_UNROLL for (int r = 0; r < kMaxRed; ++r) {
+    if (r < n_red) {
+      const Part v = warp_combine(Prog::red_kind(p, 0, r), parts[r]);
+      if (lane == 0) { float* w = wpart + (warp * kMaxRed + r) * 3; w[0] = v.a; w[1] = v.b; w[2] = v.c; }
+    }
+  }
+  __syncthreads();
+  if (warp != 0) return;
+  float* mine = p.split_part + ((size_t)row * S + split) * part_floats;
+  PN_UNROLL for (int r = 0; r < kMaxRed; ++r) {
+    if (r < n_red) {
+      const int kind = Prog::red_kind(p, 0, r);
+      Part v = red_identity(kind);
+      if (lane < nwarps) { const float* w = wpart + (lane * kMaxRed + r) * 3; v = Part{w[0], w[1], w[2]}; }
+      v = warp_combine(kind, v);
+      if (lane == 0) { mine[r * 3] = v.a; mine[r * 3 + 1] = v.b; mine[r * 3 + 2] = v.c; }
+    }
+  }
+  unsigned ticket = 0;
+  if (lane == 0) {
+    __threadfence();                                 // the partial is visible before the ticket is
+    ticket = atomicAdd(p.split_ticket + row, 1u);
+  }
+  ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
+  if (ticket != (unsigned)(S - 1)) return;
+  // the last block of this row: everyone else has written
+  __threadfence();
+  const float* all = p.split_part + (size_t)row * S * part_floats;
+  // a lane takes the slices lane, lane + 32, ... in that order (then the lanes are combined): the loads
+  // of four slices at a time are issued together, the combining stays in slice order
+  Part v[kMaxRed];
+  PN_UNROLL for (int r = 0; r < kMaxRed; ++r) v[r] = red_identity(r < n_red ? Prog::red_kind(p, 0, r) : RED_SUM);
+  for (int s0 = lane; s0 < S; s0 += 32 * 4) {
+    Part q[4][kMaxRed];
+    PN_UNROLL for (int u = 0; u < 4; ++u) {
+      const int s = s0 + 32 * u;
+      PN_UNROLL for (int r = 0; r < kMaxRed; ++r) {
+        if (r < n_red) {
+          const float* w = all + (size_t)s * part_floats + r * 3;
+          q[u][r] = s < S ? Part{ld_cg(w), ld_cg(w + 1), ld_cg(w + 2)} : red_identity(Prog::red_kind(p, 0, r));
+        }
+      }
+    }
+    PN_UNROLL for (int u = 0; u < 4; ++u) {
+      PN_UNROLL for (int r = 0; r < kMaxRed; ++r) { if (r < n_red) v[r] = red_combine(Prog::red_kind(p, 0, r), v[r], q[u][r]); }
+    }
+  }
+  PN_UNROLL for (int r = 0; r < kMaxRed; ++r) {
+    if (r < n_red) {
+      const Part c = warp_combine(Prog::red_kind(p, 0, r), v[r]);
+      float* d = slots_reg + Prog::red_slot(p, 0, r); d[0] = c.a; d[1] = c.b; d[2] = c.c;
+    }
+  }
+  cx.leader = lane == 0;
+  Prog::scalar(p, 0, cx);
+  if (lane == 0) p.split_ticket[row] = 0u;           // ready for the next launch
 }
 
 // ---------------------------------------------------------------------------------------

@@ -69,6 +69,7 @@ struct pn_graph {
   std::vector<pn::PlannedLaunch> launches;
   void* workspace = nullptr;
   size_t workspace_bytes = 0;
+  void* split_ws = nullptr;                 // partials and arrival counters of split-row launches
   int64_t compulsory_bytes = 0;
   std::vector<void*> stage_in, stage_out;   // device staging of pn_graph_run_host
   void* copy_in = nullptr;                  // streams and events of the pipelined pn_graph_run_host

@@ -39,6 +39,7 @@ void size_grid(LaunchPlan& lp, int sms, int occ) {
   if (lp.grid_waves > 0) waves = lp.grid_waves;
   if (lp.grid_waves < 0) waves = int64_t(1) << 40;
   int64_t grid;
+  if (lp.family == FAM_SPLIT) { lp.grid = (int)lp.items; return; }   // one block per slice of a row, always
   if (lp.family <= FAM_WARP) grid = std::min<int64_t>((lp.items + lp.teams_per_cta - 1) / lp.teams_per_cta, resident * waves);
   else if (lp.family == FAM_BLOCK) grid = std::min<int64_t>(lp.items, resident * waves);
   else grid = std::min<int64_t>(lp.items, std::max<int64_t>(1, resident * waves / cluster)) * cluster;
@@ -50,7 +51,7 @@ int tune_waves(unsigned flags) { const int w = (flags >> 29) & 7; return w == 0 
 
 namespace {
 
-struct Config { int family, vl, ng, k, block, cluster, chunks, slice_len; bool multichunk; int lanes; };
+struct Config { int family, vl, ng, k, block, cluster, chunks, slice_len; bool multichunk; int lanes; int splits; };
 
 }  // namespace
 
@@ -493,7 +494,8 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
   } else {
     const bool fw = flags & PN_FLAG_FORCE_WARP, fb = flags & PN_FLAG_FORCE_BLOCK, fc = flags & PN_FLAG_FORCE_CLUSTER;
     const bool fm = flags & PN_FLAG_FORCE_MULTICHUNK;
-    const bool any_force = fw || fb || fc;
+    const bool fs = flags & PN_FLAG_FORCE_SPLIT;
+    const bool any_force = fw || fb || fc || fs;
     const bool few_rows = eff_rows < 2ll * sms;
     // the interpreter's 16-element-tile instances are built for at most 256 threads
     auto tile_ok = [&](int T, int ng) { return spec || !(T > 256 && VL * ng > 8); };
@@ -501,7 +503,7 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     // LayerNorm and softmax graphs): a warp per row while the row fits in 64 two-byte (32
     // four-byte) elements per lane -- no block barrier at all -- and beyond that a block of
     // N / 32 threads holding 32 (16) elements each, when the epilogue needs the row again.
-    if (spec && !fm && !fc && VL > 1) {
+    if (spec && !fm && !fc && !fs && VL > 1) {
       const int v_warp = min_esize <= 2 ? 64 : 32, v_block = min_esize <= 2 ? 32 : 16;
       if (!fb)
         for (int ng = 1; VL * ng <= v_warp; ng *= 2)
@@ -515,8 +517,31 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
         for (int T : {64, 128, 256, 512})
           if ((int64_t)T * v_block >= eff_N) { cands.push_back(Config{FAM_BLOCK, VL, v_block / VL, kSpecRegs, T, 1, 1, (int)eff_N, false}); break; }
     }
+    // Few long rows whose elements are needed once (a single stage): independent blocks over slices
+    // of the rows, in memory order, meeting per row through partials in device memory (generated
+    // kernels; needs a workspace, so not for handles that may not allocate).  About 32 KB of a
+    // four-byte input per block (128 bytes in flight per thread) measured best on B200; smaller
+    // slices when the rows are so few that the SMs would not all get several blocks.
+    if (spec && VL > 1 && n_stages == 1 && !cross_stage && !(flags & PN_FLAG_STATIC_SCRATCH) &&
+        ((!any_force && !fm && few_rows && cands.empty()) || fs)) {   // (rows short enough for a warp stay with it)
+      const int T = 256;
+      for (int ng : {8, 4, 2, 1}) {
+        if (VL * ng > 32) continue;
+        const int64_t tile = (int64_t)T * VL * ng;
+        int seg_chunks = 1;
+        while ((eff_N + tile * seg_chunks - 1) / (tile * seg_chunks) > 1024) seg_chunks *= 2;   // at most 1024 partials per row
+        const int64_t slice = tile * seg_chunks;
+        const int64_t S = (eff_N + slice - 1) / slice;
+        if (S < 2 && !fs) continue;
+        if (eff_rows * S > (int64_t(1) << 30)) continue;
+        if (eff_rows * S < 4ll * sms && ng > 1) continue;   // too few blocks: smaller slices
+        Config c{FAM_SPLIT, VL, ng, kSpecRegs, T, 1, seg_chunks, (int)slice, false, 32, (int)S};
+        cands.push_back(c);
+        break;
+      }
+    }
     // the smallest team that holds the row in one of the interpreter's tile shapes
-    if (!fm && !fc) {
+    if (!fm && !fc && !fs) {
       for (int T : {32, 64, 128, 256, 512}) {
         if ((fw && T != 32) || (fb && T == 32)) continue;
         for (auto o : ng_opts)
@@ -587,6 +612,17 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
         if (t_cluster && c.family == FAM_BLOCK && has_red) { c.family = FAM_CLUSTER; c.cluster = t_cluster; }
         if (c.block < 32 || c.block > 1024 || (c.cluster != 1 && c.cluster != 2 && c.cluster != 4 && c.cluster != 8)) continue;
         if (!spec && c.block > 256 && c.vl * c.ng > 8) continue;
+        if (c.family == FAM_SPLIT) {   // PN_TUNE_CLUSTER(n) on a split-row kernel: n tiles per slice
+          const int64_t tile = (int64_t)c.block * VL * c.ng;
+          int seg_chunks = t_cluster ? t_cluster : 1;
+          while ((eff_N + tile * seg_chunks - 1) / (tile * seg_chunks) > 1024) seg_chunks *= 2;
+          c.cluster = 1; c.chunks = seg_chunks; c.slice_len = (int)(tile * seg_chunks);
+          c.splits = (int)((eff_N + c.slice_len - 1) / c.slice_len);
+          c.multichunk = false;
+          if (eff_rows * c.splits > (int64_t(1) << 30)) continue;
+          extra.push_back(c);
+          continue;
+        }
         const int team = c.family <= FAM_WARP ? 32 : c.block;
         int64_t slice = (eff_N + c.cluster - 1) / c.cluster;
         slice = (slice + VL - 1) / VL * VL;
@@ -648,7 +684,7 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     auto take = [&](int bytes) { const int o = off; off += (bytes + 15) / 16 * 16; return o; };
     P.sm_rowoff = take(teams * kMaxIo * 8);
     P.sm_slots = take(teams * kMaxSlots * 4);
-    P.sm_part = take(has_red ? kMaxRed * 3 * cf.block * 4 : 0);
+    P.sm_part = take(has_red && !spec ? kMaxRed * 3 * cf.block * 4 : 0);   // generated kernels keep their partials in registers
     P.sm_wpart = take(has_red ? 2 * 32 * kMaxRed * 3 * 4 : 0);   // two alternating buffers
     P.sm_ctapart = take(cf.cluster > 1 ? 2 * kMaxRed * 3 * 4 : 0);
     const int64_t stash_floats = (int64_t)n_stash * cf.chunks * cf.vl * cf.ng * cf.block;
@@ -665,17 +701,18 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     P.split_chunks = cf.family == FAM_POINTWISE;
     P.cluster = cf.cluster;
     P.team_lanes = lanes;
+    P.splits = cf.family == FAM_SPLIT ? cf.splits : 0;
     lp.family = cf.family; lp.vl = cf.vl; lp.ng = cf.ng; lp.k = cf.k;
     lp.block = cf.block; lp.smem_bytes = off; lp.code_words = (int)code.size();
     P.family = cf.family;
-    lp.items = P.split_chunks ? eff_rows * cf.chunks : eff_rows;
+    lp.items = P.split_chunks ? eff_rows * cf.chunks : (cf.family == FAM_SPLIT ? eff_rows * cf.splits : eff_rows);
     lp.teams_per_cta = teams;
     lp.specialised = 0;
     lp.persistent = persistent ? 1 : 0;
     lp.grid_waves = tune_waves(flags);
     // long rows split over a cluster run few, long-lived threads: there the first stage's loads
     // are issued one tile ahead (elsewhere the extra registers cost more than they bring)
-    lp.no_prefetch = ((flags & PN_FLAG_PREFETCH) || (cf.family == FAM_CLUSTER && cf.chunks > 1 && !(flags & PN_FLAG_NO_HOIST))) ? 0 : 1;
+    lp.no_prefetch = cf.family == FAM_SPLIT ? 1 : ((flags & PN_FLAG_PREFETCH) || (cf.family == FAM_CLUSTER && cf.chunks > 1 && !(flags & PN_FLAG_NO_HOIST))) ? 0 : 1;
     int occ = (dev.have_device && !spec) ? instance_occupancy(cf.vl, cf.ng, cf.k, cf.block, off) : 0;
     size_grid(lp, sms, occ);
     return PN_OK;

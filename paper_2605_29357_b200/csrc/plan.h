@@ -91,7 +91,7 @@ enum RedKind : uint8_t {
   RED_MEANVAR      // a = count, b = mean, c = sum of squared deviations
 };
 
-enum Family : int32_t { FAM_POINTWISE = 0, FAM_WARP = 1, FAM_BLOCK = 2, FAM_CLUSTER = 3, FAM_COLUMN = 4 };
+enum Family : int32_t { FAM_POINTWISE = 0, FAM_WARP = 1, FAM_BLOCK = 2, FAM_CLUSTER = 3, FAM_COLUMN = 4, FAM_SPLIT = 5 };
 
 struct IoDesc {
   void* base;              // device pointer; filled in per run
@@ -150,7 +150,11 @@ struct KernelParams {
   uint32_t* status;        // checked accessors (PN_FLAG_BOUNDS): bit q is set when an access to io entry q
                            // fell outside its tensor; null when checking is off
   int32_t team_lanes;      // warp-per-row kernels: lanes per row (32, or 16 / 8 when short rows share a warp)
-  int32_t pad1;
+  int32_t splits;          // FAM_SPLIT: independent thread blocks per row, each reducing slice_len columns; their
+                           // partials meet in split_part and the block that arrives last at a row combines them
+  int32_t pad1[3];
+  float* split_part;       // FAM_SPLIT: [rows][splits][reductions of stage 0][3] floats, device memory of the handle
+  uint32_t* split_ticket;  // FAM_SPLIT: [rows] arrival counters, zero between launches
   uint16_t pro_begin, pro_end;   // tile program run once per thread before the row loop: loads of
                                  // operands that are the same for every row (generated kernels only)
   // shared-memory layout, byte offsets into dynamic shared memory

@@ -49,17 +49,22 @@ __device__ __forceinline__ void emit(uint4 x, uint4* c, uint2* d, size_t idx, ui
 }
 
 // Loads straight into registers.  LAYOUT 0: grid-stride over units; 1: every block owns one
-// contiguous range of the arrays.  U units per thread are in flight together.
+// contiguous range of the arrays; 2: the arrays are cut into runs of `run` units, the blocks take
+// the runs in turn and walk each from its start to its end.  U units per thread are in flight
+// together.
 template <int NR, int NW16, int NW8, int U, bool NOALLOC, bool CS, int LAYOUT>
 __global__ void probe_direct(const uint4* __restrict__ a, const uint4* __restrict__ b, uint4* __restrict__ c,
-                             uint2* __restrict__ d, size_t units, unsigned* status) {
+                             uint2* __restrict__ d, size_t units, size_t run, unsigned* status) {
   uint4 sink = make_uint4(0, 0, 0, 0);
   size_t begin, end, step;
   if (LAYOUT == 0) { begin = (size_t)blockIdx.x * blockDim.x + threadIdx.x; end = units; step = (size_t)gridDim.x * blockDim.x; }
-  else {
+  else if (LAYOUT == 1) {
     const size_t per = (units + gridDim.x - 1) / gridDim.x;
     begin = per * blockIdx.x + threadIdx.x; end = min(units, per * (blockIdx.x + 1)); step = blockDim.x;
-  }
+  } else { begin = 0; end = 0; step = blockDim.x; }
+  const size_t n_runs = LAYOUT == 2 ? (units + run - 1) / run : 1;
+  for (size_t r = LAYOUT == 2 ? blockIdx.x : 0; r < n_runs; r += LAYOUT == 2 ? gridDim.x : n_runs) {
+  if (LAYOUT == 2) { begin = r * run + threadIdx.x; end = min(units, (r + 1) * run); }
   for (size_t i = begin; i < end; i += step * U) {
     uint4 va[U], vb[U];
 #pragma unroll
@@ -76,6 +81,7 @@ __global__ void probe_direct(const uint4* __restrict__ a, const uint4* __restric
       const size_t idx = i + u * step;
       if (idx < end) emit<NW16, NW8, CS>(mix4(va[u], vb[u]), c, d, idx, sink);
     }
+  }
   }
   // a read-only probe must keep its loads alive: the store below never happens in practice
   if (NW16 == 0 && NW8 == 0 && (sink.x ^ sink.y ^ sink.z ^ sink.w) == 0x9E3779B9u && sink.x == 0x7F4A7C15u) atomicOr(status, 0x80000000u);
@@ -181,7 +187,7 @@ cudaError_t launch_mix(int loader, int store, int layout, int block, int unroll,
     k<<<grid, block + 32, smem, s>>>(a, b, c, d, units, stages, tile_units, status);
     return cudaGetLastError();
   }
-#define PN_PROBE_GO(U, NA, CS, LY) probe_direct<NR, NW16, NW8, U, NA, CS, LY><<<grid, block, 0, s>>>(a, b, c, d, units, status)
+#define PN_PROBE_GO(U, NA, CS, LY) probe_direct<NR, NW16, NW8, U, NA, CS, LY><<<grid, block, 0, s>>>(a, b, c, d, units, (size_t)tile_units, status)
 #define PN_PROBE_U(NA, CS, LY)                                                            \
   switch (unroll) {                                                                       \
     case 1: PN_PROBE_GO(1, NA, CS, LY); break;                                            \
@@ -192,6 +198,7 @@ cudaError_t launch_mix(int loader, int store, int layout, int block, int unroll,
   }
   const bool na = loader == PN_PROBE_LDG_NOALLOC;
   if (layout == 0) { if (na) { if (store) { PN_PROBE_U(true, true, 0) } else { PN_PROBE_U(true, false, 0) } } else { if (store) { PN_PROBE_U(false, true, 0) } else { PN_PROBE_U(false, false, 0) } } }
+  else if (layout == 2) { if (store) { PN_PROBE_U(false, true, 2) } else { PN_PROBE_U(false, false, 2) } }
   else { if (na) { if (store) { PN_PROBE_U(true, true, 1) } else { PN_PROBE_U(true, false, 1) } } else { if (store) { PN_PROBE_U(false, true, 1) } else { PN_PROBE_U(false, false, 1) } } }
 #undef PN_PROBE_U
 #undef PN_PROBE_GO
@@ -219,7 +226,10 @@ pn_status pn_stream_probe(int mix, const pn_probe_config* cfg, const void* a, co
     if (cfg->stages < 2 || cfg->stages > 16 || cfg->tile_units < 32 || cfg->tile_units > 4096)
       return fail(PN_ERR_INVALID_ARG, "bulk loader: 2..16 stages of 32..4096 units");
     if (1024 + (size_t)cfg->stages * cfg->tile_units * 16 * nr > 227 * 1024) return fail(PN_ERR_TOO_LARGE, "the ring does not fit in shared memory");
-  } else if (cfg->unroll != 1 && cfg->unroll != 2 && cfg->unroll != 4 && cfg->unroll != 8) return fail(PN_ERR_INVALID_ARG, "unroll must be 1, 2, 4 or 8");
+  } else {
+    if (cfg->unroll != 1 && cfg->unroll != 2 && cfg->unroll != 4 && cfg->unroll != 8) return fail(PN_ERR_INVALID_ARG, "unroll must be 1, 2, 4 or 8");
+    if (cfg->layout < 0 || cfg->layout > 2 || (cfg->layout == 2 && cfg->tile_units < 1)) return fail(PN_ERR_INVALID_ARG, "layout must be 0, 1 or 2 (2 with tile_units > 0 as the run length)");
+  }
   if (units == 0) return PN_OK;
   const uint4* pa = (const uint4*)a; const uint4* pb = (const uint4*)b; uint4* pc = (uint4*)c; uint2* pd = (uint2*)d;
   cudaError_t e;

@@ -208,20 +208,20 @@ bool emit_program(const KernelParams& P, int pc, int end, bool scalar, int vl, i
 // Name of the kernel generated for a plan: family, tile shape and a hash of the program and
 // its shape constants, so that profiler listings tell the kernels of different graphs apart.
 std::string kernel_name(const LaunchPlan& lp) {
-  static const char* fam[] = {"pointwise", "warp_row", "block_row", "cluster_row", "column_red"};
+  static const char* fam[] = {"pointwise", "warp_row", "block_row", "cluster_row", "column_red", "split_row"};
   uint64_t h = 1469598103934665603ull;
   auto mix = [&](uint64_t v) { for (int i = 0; i < 8; ++i) { h ^= (v >> (8 * i)) & 0xFF; h *= 1099511628211ull; } };
   for (int i = 0; i < lp.code_words; ++i) mix(lp.p.code[i]);
   mix((uint64_t)lp.p.row_len); mix((uint64_t)lp.p.rows); mix((uint64_t)lp.block); mix((uint64_t)lp.p.cluster);
-  mix((uint64_t)lp.p.red_len); mix((uint64_t)lp.p.col_tx); mix((uint64_t)lp.p.team_lanes);
+  mix((uint64_t)lp.p.red_len); mix((uint64_t)lp.p.col_tx); mix((uint64_t)lp.p.team_lanes); mix((uint64_t)lp.p.splits); mix((uint64_t)lp.p.slice_len);
   for (int q = 0; q < lp.p.n_io; ++q) {
     const IoDesc& io = lp.p.io[q];
     mix(io.dtype); mix((uint64_t)io.col_stride); mix(io.mapped); mix((uint64_t)io.red_stride);
     for (int i = 0; i < 3; ++i) { mix((uint64_t)io.lead_stride[i]); mix((uint64_t)io.map_dim[i]); mix((uint64_t)io.map_add[i]); mix((uint64_t)io.map_mod[i]); }
   }
   char b[96];
-  snprintf(b, sizeof(b), "pn_spec_%s_v%dx%d_%08x", fam[lp.family >= 0 && lp.family <= FAM_COLUMN ? lp.family : 0], lp.vl, lp.ng, (unsigned)(h ^ (h >> 32)));
-  static_assert(FAM_COLUMN == 4, "family names");
+  snprintf(b, sizeof(b), "pn_spec_%s_v%dx%d_%08x", fam[lp.family >= 0 && lp.family <= FAM_SPLIT ? lp.family : 0], lp.vl, lp.ng, (unsigned)(h ^ (h >> 32)));
+  static_assert(FAM_SPLIT == 5, "family names");
   return b;
 }
 
@@ -269,14 +269,14 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
   const int team_lanes = (P.family == FAM_WARP && (P.team_lanes == 16 || P.team_lanes == 8)) ? P.team_lanes : 32;
   // (teams that share a warp may be switched off for a row: their accesses keep their validity tests)
   const bool full = team_lanes == 32 && (long long)P.chunks * team_threads * lp.vl * lp.ng == P.slice_len &&
-                    (long long)P.slice_len * P.cluster == P.row_len;
+                    (long long)P.slice_len * (P.family == FAM_SPLIT ? P.splits : P.cluster) == P.row_len;
   const bool reg_slots = true;   // generated programs keep the per-row scalars in registers
   auto konst = [&](const char* name, long long v) {
     s += std::string("  static PN_DEV int ") + name + "(const KernelParams&) { return " + I(v) + "; }\n";
   };
   konst("family", P.family); konst("cluster", P.cluster); konst("chunks", P.chunks); konst("split_chunks", P.split_chunks);
   konst("row_len", P.row_len); konst("slice_len", P.slice_len); konst("n_stages", P.n_stages); konst("n_io", P.n_io);
-  konst("col_tx", P.col_tx); konst("red_len", P.red_len); konst("team_lanes", team_lanes);
+  konst("col_tx", P.col_tx); konst("red_len", P.red_len); konst("team_lanes", team_lanes); konst("splits", P.splits);
   auto table = [&](const char* name, const char* type, auto get) {
     s += std::string("  static PN_DEV ") + type + " " + name + "(const KernelParams&, int s, int r) {\n    switch (s * " + I(kMaxRed) + " + r) {\n";
     for (int st = 0; st < P.n_stages; ++st)
@@ -341,7 +341,7 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
   s += "#if PN_MIN_BLOCKS > 1\n#define PN_LAUNCH_BOUNDS __launch_bounds__(" + I(lp.block) + ", PN_MIN_BLOCKS)\n#else\n"
        "#define PN_LAUNCH_BOUNDS __launch_bounds__(" + I(lp.block) + ")\n#endif\n";
   s += "extern \"C\" __global__ void PN_LAUNCH_BOUNDS " + kernel_name(lp) + "(const __grid_constant__ pn::KernelParams p) {\n"
-       "  extern __shared__ __align__(16) unsigned char smem[];\n  pn::" + std::string(P.family == FAM_COLUMN ? "column_body" : "fused_body") + "<pn::Spec>(p, smem);\n}\n";
+       "  extern __shared__ __align__(16) unsigned char smem[];\n  pn::" + std::string(P.family == FAM_COLUMN ? "column_body" : P.family == FAM_SPLIT ? "split_body" : "fused_body") + "<pn::Spec>(p, smem);\n}\n";
   src.swap(s);
   return true;
 }

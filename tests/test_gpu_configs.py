@@ -26,6 +26,7 @@ FORCES = {
     "block_multichunk": pn.FLAG_FORCE_BLOCK | pn.FLAG_FORCE_MULTICHUNK,
     "cluster_multichunk": pn.FLAG_FORCE_CLUSTER | pn.FLAG_FORCE_MULTICHUNK,
     "warp_scalar": pn.FLAG_FORCE_WARP | pn.FLAG_FORCE_SCALAR,
+    "split": pn.FLAG_FORCE_SPLIT,
 }
 
 

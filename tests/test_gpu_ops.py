@@ -146,7 +146,7 @@ def test_all_reductions_over_row_lengths(n, mode):
 
 @pytest.mark.parametrize("force", [0, pn.FLAG_FORCE_WARP, pn.FLAG_FORCE_BLOCK, pn.FLAG_FORCE_CLUSTER,
                                    pn.FLAG_FORCE_BLOCK | pn.FLAG_FORCE_MULTICHUNK, pn.FLAG_FORCE_SCALAR,
-                                   pn.FLAG_PREFETCH, pn.FLAG_PREFETCH | pn.FLAG_FORCE_CLUSTER])
+                                   pn.FLAG_PREFETCH, pn.FLAG_PREFETCH | pn.FLAG_FORCE_CLUSTER, pn.FLAG_FORCE_SPLIT])
 def test_reductions_with_nan_and_infinities_in_every_family(force):
     x = rnd((6, 2048), 13, 2.0)
     x[0, 100] = np.nan; x[0, 1500] = np.nan              # first NaN wins argmax / argmin; sums are NaN

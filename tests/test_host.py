@@ -92,7 +92,7 @@ def test_shape_and_support_errors():
     assert _status(g.build(), PLAN | pn.FLAG_UNFUSED) == 0      # one node at a time still fits
 
 
-FAMILY = {"c1": "pointwise", "c2": "warp-per-row", "c3": "block-per-row", "c4": "cluster-per-row",
+FAMILY = {"c1": "pointwise", "c2": "warp-per-row", "c3": "block-per-row", "c4": "split-row",
           "c5": "block-per-row"}
 FULL = {"c1": dict(M=1024, N=1024), "c2": dict(B=512, Q=512, K=512), "c3": dict(M=16384, N=4096),
         "c4": dict(M=64, N=262144), "c5": dict(M=8192, N=14336)}
@@ -123,12 +123,15 @@ def test_lowering_of_the_benchmark_graphs(cfg):
         assert k["vl"] == 4 and k["ng"] == 8
     else:
         assert k["vl"] * (2 if cfg in ("c2", "c5") else 4) == 16           # 128-bit accesses
-    if cfg == "c4":   # 64 rows: split over clusters so that every SM gets work
-        assert k["cluster"] in (2, 4, 8) and k["grid"] % k["cluster"] == 0 and 64 * k["cluster"] >= 148
+    if cfg == "c4":   # 64 long rows, a single stage: independent blocks over slices of the rows
+        assert k["grid"] % 64 == 0 and k["grid"] >= 8 * 148 and g.workspace_bytes > 0
+        gc = pn.Graph(w.desc, 0, PLAN | pn.FLAG_FORCE_CLUSTER)   # clusters when asked for: every SM still gets work
+        kc = gc.kernel_info[0]
+        assert kc["cluster"] in (2, 4, 8) and kc["grid"] % kc["cluster"] == 0 and 64 * kc["cluster"] >= 148
     if cfg in ("c2", "c3"):
         assert k["chunks"] == 1                                             # row resident in registers
     gu = pn.Graph(w.desc, 0, PLAN | pn.FLAG_UNFUSED)
-    assert gu.n_kernels == w.n_nodes and (gu.workspace_bytes > 0 or cfg == "c4")
+    assert gu.n_kernels == w.n_nodes and gu.workspace_bytes > 0
     assert [m for m in g.input_meta] == [(dt, tuple(d)) for dt, d in w.input_meta]
     assert [m for m in g.output_meta] == [(dt, tuple(d)) for dt, d in w.output_meta]
 
