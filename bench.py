@@ -167,6 +167,25 @@ def time_graph(torch, g, sets, steps, warmup, flush=None):
     return evs[0].elapsed_time(evs[steps]), per
 
 
+def time_host_launched(torch, g, sets, steps, warmup):
+    """K launches through bound launch objects (pn_bound_run: one launch call each) rotating over the
+    buffer sets, one pair of events around all of them: what a caller who launches from the host
+    pays per launch, without an event record between the launches.  Returns ms per launch."""
+    stream = torch.cuda.current_stream()
+    launch = [g.bind([t.data_ptr() for t in a], [t.data_ptr() for t in b]) for a, b in sets]
+    for i in range(max(warmup, 3)):
+        launch[i % len(launch)](stream.cuda_stream)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n, s = len(launch), stream.cuda_stream
+    e0.record(stream)
+    for i in range(steps):
+        launch[i % n](s)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps
+
+
 def time_graph_replay(torch, g, sets, steps, warmup):
     """The same launches recorded once into a CUDA graph (one launch per buffer set) and
     replayed: the device-side time per launch, free of the host's launch rate.  Used for the
@@ -245,13 +264,13 @@ class StreamProbe:
         for cfg in self._configs(mix, units):
             for _ in range(3):
                 self._launch(mix, cfg, units, 0, s.cuda_stream)
-            ev = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
-            ev[0].record(s)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(s)
             for i in range(reps):
                 self._launch(mix, cfg, units, 0, s.cuda_stream)
-                ev[i + 1].record(s)
+            e1.record(s)
             torch.cuda.synchronize()
-            ms = float(np.median([ev[i].elapsed_time(ev[i + 1]) for i in range(reps)]))
+            ms = e0.elapsed_time(e1) / reps   # (single launches are timed in steps of a microsecond or two: take the mean)
             gbs = units * MIX_UNIT_BYTES[mix] / (ms * 1e-3) / 1e9
             if best is None or gbs > best["gbs"]:
                 best = {"gbs": gbs, "block": cfg.block, "unroll": cfg.unroll, "streaming_stores": cfg.streaming_stores,
@@ -662,6 +681,7 @@ def main():
             ms_roof, timing = sti["median_ms"], "CUDA events around each host launch, median"
             if ns > 1:   # kernels shorter than a host launch: also the device-side time per launch
                 ms_r = time_graph_replay(torch, gi, si, max(args.steps, 10 * ns), warmup)
+                entry["host_launched_ms"] = time_host_launched(torch, gi, si, max(200, args.steps), warmup)
                 entry["graph_replay_ms"] = ms_r
                 entry["graph_replay_gbs"] = cb / (ms_r * 1e-3) / 1e9
                 entry["graph_replay_frac_of_measured_peak"] = entry["graph_replay_gbs"] / peak

@@ -22,7 +22,7 @@ constexpr int kMaxIo = 12;      // graph inputs + outputs of one kernel
 constexpr int kMaxCode = 224;   // 32-bit bytecode words of one kernel
 constexpr int kMaxStages = 4;   // reduction-separated stages
 constexpr int kMaxRed = 4;      // reductions accumulated in one stage
-constexpr int kMaxSlots = 24;   // per-row scalar slots
+constexpr int kMaxSlots = 48;   // per-row scalar slots
 constexpr int kMaxStash = 6;    // tile values parked in shared memory across stages
 constexpr int kAccReg = 31;     // register operand id that names the accumulator tile
 constexpr int kSpecRegs = 12;   // tile registers of a generated kernel (only live ones cost anything)
