@@ -46,9 +46,12 @@
  * value cannot flow back into a tensor that still has the reduced dimension.
  * Index operators (the index-remapped loads of the paper's first case study, Section 4.4): 160
  * roll (attr = dim, shift), 161 slice (attr = dim, start; length from the output shape), 162 view
- * (regroups leading dimensions).  They act on leading dimensions of graph inputs, or of chains of
+ * (regroups leading dimensions).  A roll or slice over two dimensions at once, as graph traces have
+ * them, gives the second one in imm = (1 + dim, shift / start); imm[0] = 0 means one dimension.  They act on leading dimensions of graph inputs, or of chains of
  * index operators that start at one, and cost no data movement: the fused kernel computes the
- * source row instead (idx = (S + i - shift) mod S).  163 cat (attr[0] = dim): with one operand it
+ * source row instead (idx = (S + i - shift) mod S).  164 contiguous: the identity on values (every
+ * tensor here is dense already); after a chain of index operators it is one more link of the chain,
+ * on a computed value a pointwise identity.  163 cat (attr[0] = dim): with one operand it
  * is the identity, as graph traces contain it; several operands are not lowered.
  * Arithmetic is fp32 in registers whatever the storage types; integer and boolean
  * tensors take part as exact small integers / predicates; a node whose declared
@@ -107,6 +110,10 @@ enum {
                                      ahead (costs registers; off by default)                 */
   PN_FLAG_STATIC_SCRATCH = 1u << 12,/* with PN_FLAG_UNFUSED: allocate no workspace; the handle
                                      is run with pn_graph_run_static only                    */
+  PN_FLAG_ONE_KERNEL = 1u << 3,   /* a graph that does not fit one kernel (a bytecode, register, scalar,
+                                     I/O or stage budget; a combination the fused lowering does not
+                                     take) is refused with PN_ERR_TOO_LARGE / PN_ERR_UNSUPPORTED_OP
+                                     instead of being cut into several fused launches          */
   PN_FLAG_FORCE_SPLIT = 1u << 15, /* row kernels: independent blocks over slices of a row, combined
                                      through partials in a workspace of the handle (single-stage
                                      graphs, generated kernels)                               */
@@ -161,8 +168,15 @@ enum {
  *   device           : CUDA device ordinal the handle is bound to.
  *   flags            : PN_FLAG_* bits.
  *   out              : receives the handle; set to NULL on failure.
- * Allocates device memory only for PN_FLAG_UNFUSED (the intermediates) -- owned by the
- * handle and released by pn_graph_destroy.  Launches no kernel.
+ * A graph that exceeds what one kernel takes (the paper's fusible subgraphs run to 35 operators,
+ * its classical ones to 62: Section 3.3) is cut into the cheapest sequence of fused launches --
+ * consecutive runs of nodes, the tensors that cross a cut written once to a workspace of the handle
+ * and read once; cheapest by bytes moved, then by launches -- unless PN_FLAG_ONE_KERNEL asks for the
+ * refusal.  PN_Q_N_KERNELS tells the number of launches, PN_Q_WORKSPACE_BYTES the workspace.
+ * Allocates device memory for the workspace of such cuts, of PN_FLAG_UNFUSED (the intermediates
+ * between all nodes) and of split-row kernels (partials and arrival counters of rows reduced by
+ * several independent blocks) -- owned by the handle and released by pn_graph_destroy.  Launches
+ * no kernel.
  * Unless PN_FLAG_INTERPRET is given, the bytecode of each launch is also translated into a
  * kernel of its own and compiled for sm_100a with NVRTC (a few hundred ms per distinct
  * kernel).  Loaded kernels are shared through a process-wide cache, reference-counted by the

@@ -60,7 +60,7 @@ _OP_NAMES = {
     96: "sum", 97: "mean", 98: "var", 99: "amax", 100: "amin", 101: "argmax", 102: "argmin",
     103: "logsumexp", 104: "sum_dim", 105: "mean_dim", 106: "amax_dim", 107: "amin_dim",
     128: "softmax", 129: "log_softmax", 130: "layer_norm", 131: "rms_norm",
-    160: "roll", 161: "slice", 162: "view", 163: "cat",
+    160: "roll", 161: "slice", 162: "view", 163: "cat", 164: "contiguous",
 }
 
 
@@ -412,6 +412,13 @@ def op_view(x, dims):
     return np.ascontiguousarray(x).reshape(dims)
 
 
+def op_contiguous(x):
+    """The same values, laid out densely in row-major order: as every tensor of a descriptor is
+    dense already, the identity on values (the paper's first case study keeps such a node after its
+    rolls and slices, Section 4.4)."""
+    return np.ascontiguousarray(x)
+
+
 def op_cast(x, dst_dtype: int):
     """Value conversion.  Float -> integer truncates toward zero; anything -> bool
     tests for non-zero; to a float type the value is kept (narrow-float rounding is
@@ -488,16 +495,22 @@ def evaluate(desc: bytes, inputs: Sequence[np.ndarray],
                 res = [np.minimum(np.maximum(a[0], a[1]), a[2])]
             elif n.op == "fma":
                 res = [a[0] * a[1] + a[2]]
-            elif n.op == "roll":
+            elif n.op == "roll":      # (dim, shift) in attr; optionally a second dimension as imm = (1 + dim, shift)
                 res = [op_roll(a[0], int(n.attr[0]), int(n.attr[1]))]
-            elif n.op == "slice":
+                if n.imm[0] != 0:
+                    res = [op_roll(res[0], int(n.imm[0]) - 1, int(n.imm[1]))]
+            elif n.op == "slice":     # (dim, start) in attr, the length from the output shape; optionally a second dimension in imm
                 res = [op_slice(a[0], int(n.attr[0]), int(n.attr[1]), int(out_t[0].dims[int(n.attr[0])]))]
+                if n.imm[0] != 0:
+                    res = [op_slice(res[0], int(n.imm[0]) - 1, int(n.imm[1]), int(out_t[0].dims[int(n.imm[0]) - 1]))]
             elif n.op == "view":
                 res = [op_view(a[0], tuple(out_t[0].dims))]
             elif n.op in ("sum_dim", "mean_dim", "amax_dim", "amin_dim"):
                 res = [red_over_dim(n.op, a[0], int(n.attr[0]))]
             elif n.op == "cat":
                 res = [op_cat(a, int(n.attr[0]))]
+            elif n.op == "contiguous":
+                res = [op_contiguous(a[0])]
             elif n.op == "sum":
                 res = [red_sum(a[0])]
             elif n.op == "mean":

@@ -17,6 +17,7 @@ from . import _build
 PN_OK = 0
 FLAG_UNFUSED = 1 << 0
 FLAG_PLAN_ONLY = 1 << 1
+FLAG_ONE_KERNEL = 1 << 3
 FLAG_FORCE_WARP = 1 << 4
 FLAG_FORCE_BLOCK = 1 << 5
 FLAG_FORCE_CLUSTER = 1 << 6

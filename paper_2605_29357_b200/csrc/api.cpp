@@ -1,6 +1,8 @@
 // api.cpp -- the exported C ABI (see include/pn.h): handle life cycle, pointer checks,
 // launches, the unfused one-kernel-per-node path, and the host-memory convenience call.
 #include <cuda_runtime.h>
+#include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
@@ -36,7 +38,7 @@ bool any_empty(const Graph& g) {
   return false;
 }
 
-// The graph executed by one launch: the nodes `members` of g (ascending, hence topological).  Its
+// The graph executed by one launch: the nodes `members` of g, in a topological order.  Its
 // inputs are the tensors the members read that no member produces; its outputs are the tensors a
 // member produces that a node outside the group reads or that are outputs of g.
 void group_subgraph(const Graph& g, const std::vector<int>& members, Graph& sub, std::vector<int>& orig_of_sub) {
@@ -75,6 +77,78 @@ void group_subgraph(const Graph& g, const std::vector<int>& members, Graph& sub,
     if (sub.tensors[i].role & 1) sub.inputs.push_back((int)i);
     if (sub.tensors[i].role & 2) sub.outputs.push_back((int)i);
   }
+}
+
+// A graph that does not fit one kernel (a bytecode, register, scalar-slot, I/O or stage budget, or
+// a combination the fused lowering does not take, such as a second softmax) is cut into the
+// cheapest sequence of fused launches: consecutive runs of nodes, each lowered on its own, the
+// tensors that cross a cut materialised once in the workspace.  Cheapest by a two-term estimate of
+// the time: the bytes every launch moves (its inputs read once, its outputs written once) at
+// 6 bytes per nanosecond, plus 3 microseconds per launch -- so cuts go through per-row results and
+// other small tensors, and a launch is not added to save a few kilobytes; found by dynamic
+// programming over the cut positions.  Returns false when some node cannot be lowered even alone.
+bool partition_graph(const Graph& g, unsigned flags, const DeviceModel& dev, std::vector<std::vector<int>>& groups) {
+  const int n = (int)g.nodes.size();
+  if (n < 2 || n > 512) return false;
+  // The runs are taken from the nodes ordered by reduction depth (how many reductions lie between a
+  // node and the graph's inputs; ties in descriptor order), which is again a topological order: a
+  // kernel takes a few consecutive depths, so its runs should not be interrupted by nodes of other
+  // depths that merely happen to be listed in between.
+  std::vector<int> t_level(g.tensors.size(), 0), n_level(n, 0), order(n);
+  for (int i = 0; i < n; ++i) {
+    const Node& nd = g.nodes[i];
+    int lv = 0;
+    for (int k = 0; k < nd.n_in; ++k) if (nd.in[k] < g.tensors.size()) lv = std::max(lv, t_level[nd.in[k]]);
+    n_level[i] = lv;
+    const bool reduces = is_reduction(nd.op) || is_composite(nd.op) || is_dim_reduction(nd.op);
+    for (int k = 0; k < nd.n_out; ++k) t_level[nd.out[k]] = lv + (reduces ? 1 : 0);
+    order[i] = i;
+  }
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return n_level[a] < n_level[b]; });
+  const int64_t kInf = INT64_MAX / 4;
+  std::vector<int64_t> best(n + 1, kInf);
+  std::vector<int> from(n + 1, -1);
+  best[0] = 0;
+  for (int i = 0; i < n; ++i) {
+    if (best[i] >= kInf) continue;
+    std::vector<int> members;
+    int misses = 0;
+    for (int j = i; j < n; ++j) {
+      members.push_back(order[j]);
+      Graph sub;
+      std::vector<int> orig;
+      group_subgraph(g, members, sub, orig);
+      LaunchPlan lp;
+      std::string err;
+      // A run over a budget stays over it when it grows.  A run that fails for another reason may
+      // become lowerable again with a few more nodes (a tensor of a broadcast shape cannot be cut
+      // at -- a launch stores only full-shape and per-row tensors -- but can stay inside a launch).
+      const int st = lower_graph(sub, flags, dev, lp, err);
+      if (st != PN_OK && getenv("PN_DEBUG_PARTITION")) fprintf(stderr, "partition: run [%d, %d] status %d: %s\n", i, j, st, err.c_str());
+      if (st == PN_ERR_TOO_LARGE) break;
+      if (st != PN_OK) { if (++misses > 24) break; continue; }
+      misses = 0;
+      int64_t bytes = 0;
+      for (int t : sub.inputs) bytes += tensor_bytes(sub.tensors[t]);
+      for (int t : sub.outputs) bytes += tensor_bytes(sub.tensors[t]);
+      const int64_t cand = best[i] + bytes / 6 + 3000;   // estimated nanoseconds
+      if (cand < best[j + 1]) { best[j + 1] = cand; from[j + 1] = i; }
+    }
+  }
+  if (best[n] >= kInf) return false;
+  groups.clear();
+  for (int j = n; j > 0; j = from[j]) {
+    std::vector<int> m;
+    for (int k = from[j]; k < j; ++k) m.push_back(order[k]);
+    groups.insert(groups.begin(), m);
+  }
+  if (getenv("PN_DEBUG_PARTITION"))
+    for (size_t k = 0; k < groups.size(); ++k) {
+      std::string line = "partition: launch " + std::to_string(k) + " = nodes";
+      for (int m : groups[k]) line += " " + std::to_string(m);
+      fprintf(stderr, "%s\n", line.c_str());
+    }
+  return groups.size() > 1;
 }
 
 pn_status check_counts(const pn_graph* h, const void* const* inputs, int n_inputs, void* const* outputs, int n_outputs) {
@@ -217,6 +291,15 @@ pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsig
   } else {
     groups.emplace_back();
     for (size_t ni = 0; ni < g.nodes.size(); ++ni) groups[0].push_back((int)ni);
+    // does the whole graph fit one kernel?  If a budget or an unsupported combination says no, cut it
+    // into the cheapest sequence of fused launches (PN_FLAG_ONE_KERNEL asks for the refusal instead)
+    LaunchPlan probe;
+    std::string why_not;
+    const int whole = lower_graph(g, flags, dev, probe, why_not);
+    if ((whole == PN_ERR_TOO_LARGE || whole == PN_ERR_UNSUPPORTED_OP) && !(flags & PN_FLAG_ONE_KERNEL)) {
+      std::vector<std::vector<int>> cut;
+      if (partition_graph(g, flags, dev, cut)) groups.swap(cut);
+    }
   }
   // tensors that cross from one launch to a later one live in a workspace, in their declared dtype
   std::vector<int> group_of_node(g.nodes.size(), 0);

@@ -24,7 +24,7 @@ bool arity_of(uint16_t op, Arity& a) {
   if (op == N_SOFTMAX || op == N_LOG_SOFTMAX) { a = {1, 1, 1, 1}; return true; }
   if (op == N_LAYER_NORM) { a = {1, 3, 1, 3}; return true; }
   if (op == N_RMS_NORM) { a = {1, 2, 1, 1}; return true; }
-  if (op >= N_ROLL && op <= N_VIEW) { a = {1, 1, 1, 1}; return true; }
+  if ((op >= N_ROLL && op <= N_VIEW) || op == N_CONTIGUOUS) { a = {1, 1, 1, 1}; return true; }
   return false;
 }
 

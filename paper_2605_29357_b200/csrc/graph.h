@@ -20,7 +20,8 @@ enum NodeOp : uint16_t {
   N_SUM_DIM = 104, N_MEAN_DIM, N_AMAX_DIM, N_AMIN_DIM,   // over one leading dimension, attr[0] = dim
   N_SOFTMAX = 128, N_LOG_SOFTMAX, N_LAYER_NORM, N_RMS_NORM,
   N_ROLL = 160, N_SLICE, N_VIEW,   // index operators on leading dimensions
-  N_CAT = 163                      // concatenation along attr[0]
+  N_CAT = 163,                     // concatenation along attr[0]
+  N_CONTIGUOUS = 164               // the identity on values (dense layout is what every tensor has)
 };
 
 constexpr uint32_t kImm0 = 0xFFFFFFFFu, kImm1 = 0xFFFFFFFEu;

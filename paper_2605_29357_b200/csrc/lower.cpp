@@ -80,6 +80,19 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     bool frozen = false;                 // regrouped by a view after rolls / slices: no further index ops
   };
   std::vector<IdxMap> imap(nt);
+  // which nodes only re-index: roll / slice / view, and contiguous where it follows such a chain (or a
+  // graph input): it is then a view of the same shape; on a computed value it is a pointwise identity
+  std::vector<char> idx_like(g.nodes.size(), 0);
+  {
+    std::vector<char> chained(nt, 0);
+    for (int t : g.inputs) chained[t] = 1;
+    for (size_t ni = 0; ni < g.nodes.size(); ++ni) {
+      const Node& n = g.nodes[ni];
+      const bool src_chained = n.n_in >= 1 && n.in[0] < (uint32_t)nt && chained[n.in[0]];
+      idx_like[ni] = is_index_op(n.op) || (n.op == N_CONTIGUOUS && src_chained);
+      if (idx_like[ni] && src_chained) chained[n.out[0]] = 1;
+    }
+  }
   auto plain_map = [&](int root, const Tensor& T) {
     IdxMap m; m.root = root;
     const Shape4 s = align4(T);
@@ -89,39 +102,50 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
   };
   for (int t : g.inputs) imap[t] = plain_map(t, g.tensors[t]);
   std::vector<char> by_compute(nt, 0);   // read by an arithmetic node, or a graph output
-  for (const Node& n : g.nodes)
-    if (!is_index_op(n.op)) for (int k = 0; k < n.n_in; ++k) if (n.in[k] < (uint32_t)nt) by_compute[n.in[k]] = 1;
+  for (size_t ni = 0; ni < g.nodes.size(); ++ni)
+    if (!idx_like[ni]) for (int k = 0; k < g.nodes[ni].n_in; ++k) if (g.nodes[ni].in[k] < (uint32_t)nt) by_compute[g.nodes[ni].in[k]] = 1;
   for (int o : g.outputs) by_compute[o] = 1;
   for (size_t ni = 0; ni < g.nodes.size(); ++ni) {
     const Node& n = g.nodes[ni];
-    if (!is_index_op(n.op)) continue;
+    if (!idx_like[ni]) continue;
     const std::string where = "node " + std::to_string(ni) + ": ";
     const Tensor& X = g.tensors[n.in[0]]; const Tensor& Y = g.tensors[n.out[0]];
     IdxMap m = imap[n.in[0]];
     if (m.root < 0) { err = where + "roll / slice / view apply to graph inputs (or chains of them) only"; return PN_ERR_UNSUPPORTED_OP; }
     if (Y.dtype != X.dtype) { err = where + "an index operator keeps the dtype"; return PN_ERR_UNSUPPORTED_OP; }
     if (X.rank < 1 || Y.rank < 1 || X.dims[X.rank - 1] != Y.dims[Y.rank - 1]) { err = where + "index operators act on leading dimensions; the last one must be unchanged"; return PN_ERR_SHAPE; }
-    if (n.op == N_VIEW) {
+    if (n.op == N_CONTIGUOUS && (X.rank != Y.rank || memcmp(X.dims, Y.dims, sizeof(X.dims)) != 0)) { err = where + "contiguous keeps the shape"; return PN_ERR_SHAPE; }
+    if (n.op == N_VIEW || n.op == N_CONTIGUOUS) {
       if (X.numel() != Y.numel()) { err = where + "a view keeps the number of elements"; return PN_ERR_SHAPE; }
       if (m.plain) m = plain_map(m.root, Y); else m.frozen = true;
     } else {
       if (m.frozen) { err = where + "roll / slice after a view of a rolled or sliced tensor is not lowered"; return PN_ERR_UNSUPPORTED_OP; }
-      const int64_t k = n.attr[0];
-      if (k < 0 || k >= X.rank - 1 || X.rank > 4) { err = where + "roll / slice dimension must be a leading one"; return PN_ERR_SHAPE; }
-      const int kk = 3 - (X.rank - 1) + (int)k;
-      for (int d = 0; d < X.rank; ++d)
-        if (d != k && X.dims[d] != Y.dims[d]) { err = where + "only the rolled / sliced dimension may change"; return PN_ERR_SHAPE; }
+      // one dimension in attr (dim, shift / start); optionally a second one in imm (1 + dim, shift / start)
+      int64_t dims2[2] = {n.attr[0], -1}, amt2[2] = {n.attr[1], 0};
+      if (n.imm[0] != 0.0) {
+        if (n.imm[0] != floor(n.imm[0]) || n.imm[1] != floor(n.imm[1]) || n.imm[0] < 1 || n.imm[0] > 4) { err = where + "second dimension of a roll / slice: imm = (1 + dim, shift / start), integers"; return PN_ERR_BAD_DESCRIPTOR; }
+        dims2[1] = (int64_t)n.imm[0] - 1; amt2[1] = (int64_t)n.imm[1];
+        if (dims2[1] == dims2[0]) { err = where + "a roll / slice names each dimension once"; return PN_ERR_SHAPE; }
+      }
       if (X.rank != Y.rank) { err = where + "rank must be kept"; return PN_ERR_SHAPE; }
-      const int64_t Dk = X.dims[k];
-      if (n.op == N_ROLL) {
-        if (Y.dims[k] != Dk) { err = where + "a roll keeps the shape"; return PN_ERR_SHAPE; }
-        if (m.sliced[kk]) { err = where + "roll after slice on the same dimension is not lowered"; return PN_ERR_UNSUPPORTED_OP; }
-        if (Dk > 0) { m.add[kk] = ((m.add[kk] - n.attr[1]) % Dk + Dk) % Dk; m.mod[kk] = Dk; }
-      } else {
-        const int64_t a = n.attr[1], L = Y.dims[k];
-        if (a < 0 || a + L > Dk) { err = where + "slice outside the tensor"; return PN_ERR_SHAPE; }
-        m.add[kk] += a; m.ext[kk] = L; m.sliced[kk] = true;
-        if (m.mod[kk]) m.add[kk] %= m.mod[kk];
+      for (int d = 0; d < X.rank; ++d)
+        if (d != dims2[0] && d != dims2[1] && X.dims[d] != Y.dims[d]) { err = where + "only the rolled / sliced dimensions may change"; return PN_ERR_SHAPE; }
+      for (int which = 0; which < 2; ++which) {
+        const int64_t k = dims2[which];
+        if (which == 1 && k < 0) break;
+        if (k < 0 || k >= X.rank - 1 || X.rank > 4) { err = where + "roll / slice dimension must be a leading one"; return PN_ERR_SHAPE; }
+        const int kk = 3 - (X.rank - 1) + (int)k;
+        const int64_t Dk = X.dims[k];
+        if (n.op == N_ROLL) {
+          if (Y.dims[k] != Dk) { err = where + "a roll keeps the shape"; return PN_ERR_SHAPE; }
+          if (m.sliced[kk]) { err = where + "roll after slice on the same dimension is not lowered"; return PN_ERR_UNSUPPORTED_OP; }
+          if (Dk > 0) { m.add[kk] = ((m.add[kk] - amt2[which]) % Dk + Dk) % Dk; m.mod[kk] = Dk; }
+        } else {
+          const int64_t a = amt2[which], L = Y.dims[k];
+          if (a < 0 || a + L > Dk) { err = where + "slice outside the tensor"; return PN_ERR_SHAPE; }
+          m.add[kk] += a; m.ext[kk] = L; m.sliced[kk] = true;
+          if (m.mod[kk]) m.add[kk] %= m.mod[kk];
+        }
       }
       m.plain = false;
     }
@@ -131,8 +155,9 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
   std::vector<char> index_only(nt, 0);
   for (int t = 0; t < nt; ++t) index_only[t] = imap[t].root >= 0 && !by_compute[t];
 
-  for (const Node& n : g.nodes) {   // per-row scalars
-    if (is_index_op(n.op)) continue;
+  for (size_t ni = 0; ni < g.nodes.size(); ++ni) {   // per-row scalars
+    const Node& n = g.nodes[ni];
+    if (idx_like[ni]) continue;
     if (is_reduction(n.op)) is_s[n.out[0]] = 1;
     else if (n.op == N_LAYER_NORM) { for (int k = 1; k < n.n_out; ++k) is_s[n.out[k]] = 1; }
     else if (!is_composite(n.op)) {
@@ -169,7 +194,7 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
   if (N >= (int64_t(1) << 30)) { err = "last dimension too long"; return PN_ERR_TOO_LARGE; }
   for (size_t ni = 0; ni < g.nodes.size(); ++ni) {   // per-node shape rules
     const Node& n = g.nodes[ni];
-    if (is_index_op(n.op)) continue;   // checked with the chains above
+    if (idx_like[ni]) continue;   // checked with the chains above
     const std::string where = "node " + std::to_string(ni) + ": ";
     auto row_shaped = [&](const Tensor& t, const Tensor& src) {
       if (t.rank == src.rank - 1) { for (int i = 0; i < t.rank; ++i) if (t.dims[i] != src.dims[i]) return false; return true; }
@@ -344,7 +369,7 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
       else if (n.in[k] == kImm1) in[k] = imm_val(n.imm[1]);
       else in[k] = tval[n.in[k]];
     }
-    if (is_index_op(n.op)) {
+    if (idx_like[ni]) {
       const int t = n.out[0];
       if (g.tensors[t].role & 2) {
         if (tval[t] < 0) { err = where + "internal: re-indexed output without a value"; return PN_ERR_UNSUPPORTED_OP; }

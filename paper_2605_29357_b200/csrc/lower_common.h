@@ -238,8 +238,11 @@ struct Gen {
             }
             Src sy;
             if (!src_operand(Y, sy)) return false;
-            vals[x].uses--; vals[X].uses--; vals[Y].uses--;
+            // (the copy that keeps X alive is made while the other operands still count as used: their
+            // registers must not be handed out before the instruction that reads them)
+            vals[X].uses--;
             if (!keep_if_live(X)) return false;
+            vals[x].uses--; vals[Y].uses--;
             emit(OP_WHERE_RAW, k, sy.idx, sy.kind);
             if (sy.kind == OPK_IMM) emit_f(sy.imm);
             result(m.out);
@@ -251,8 +254,9 @@ struct Gen {
         if (!place_in_acc(x)) return false;
         Src sx, sy;
         if (!src_operand(X, sx) || !src_operand(Y, sy)) return false;
-        vals[x].uses--; vals[X].uses--; vals[Y].uses--;
+        vals[x].uses--;
         if (!keep_if_live(x)) return false;
+        vals[X].uses--; vals[Y].uses--;
         emit(m.op, sx.idx, sy.idx, sx.kind | (sy.kind << 4));
         if (sx.kind == OPK_IMM) emit_f(sx.imm);
         if (sy.kind == OPK_IMM) emit_f(sy.imm);
@@ -277,8 +281,9 @@ struct Gen {
     if (!place_in_acc(x)) return false;
     Src s;
     if (!src_operand(y, s)) return false;
-    vals[x].uses--; vals[y].uses--;
+    vals[x].uses--;
     if (!keep_if_live(x)) return false;
+    vals[y].uses--;
     emit(op, s.idx, s.kind);
     if (s.kind == OPK_IMM) emit_f(s.imm);
     result(m.out);
@@ -407,6 +412,10 @@ struct Expander {
       for (int k = 0; k < 3; ++k) if (vals[in[k]].int_bits) in[k] = pointwise(OP_I2F, {in[k]}, true);
       const int lo = pointwise(OP_MAX, {in[0], in[1]}, false);
       res[0] = pointwise(OP_MIN, {lo, in[2]}, false);
+    } else if (n.op == N_CONTIGUOUS) {   // on a computed value: the identity
+      if (g.tensors[n.in[0]].numel() != T0.numel() || g.tensors[n.in[0]].dtype != T0.dtype) { err = where + "contiguous keeps shape and dtype"; return PN_ERR_SHAPE; }
+      if (vals[in[0]].kind == VK_IMM) { err = where + "contiguous of a constant"; return PN_ERR_UNSUPPORTED_OP; }
+      res[0] = in[0];
     } else if (n.op == N_CAT) {
       if (n.n_in != 1) { err = where + "cat of several operands is not lowered (one operand is the identity)"; return PN_ERR_UNSUPPORTED_OP; }
       if (g.tensors[n.in[0]].numel() != T0.numel()) { err = where + "cat of one operand keeps its shape"; return PN_ERR_SHAPE; }

@@ -247,12 +247,14 @@ def n1(S: int = 133, SC: int = 128, Cc: int = 96, shift: int = 3, seed: int = 0,
     res = g.input(dtype, (1, SC * SC, Cc))
     gamma = g.input(dtype, (Cc,))
     beta = g.input(dtype, (Cc,))
-    v = g.op("view", [x], dtype, (S, S, Cc))
-    r0 = g.op("roll", [v], dtype, (S, S, Cc), attr=[0, shift])
-    r1 = g.op("roll", [r0], dtype, (S, S, Cc), attr=[1, shift])
-    s0 = g.op("slice", [r1], dtype, (SC, S, Cc), attr=[0, 0])
-    s1 = g.op("slice", [s0], dtype, (SC, SC, Cc), attr=[1, 0])
-    w = g.op("view", [s1], dtype, (1, SC * SC, Cc))
+    # the eight operators of the case study: contiguous, view, roll (both window axes at once), slice
+    # (both), contiguous, view, add, layer_norm
+    c0 = g.op("contiguous", [x], dtype, (1, S * S, Cc))
+    v = g.op("view", [c0], dtype, (S, S, Cc))
+    r = g.op("roll", [v], dtype, (S, S, Cc), attr=[0, shift], extra_imm=[1 + 1, shift])
+    sl = g.op("slice", [r], dtype, (SC, SC, Cc), attr=[0, 0], extra_imm=[1 + 1, 0])
+    c1 = g.op("contiguous", [sl], dtype, (SC, SC, Cc))
+    w = g.op("view", [c1], dtype, (1, SC * SC, Cc))
     cast = (lambda t, dm: g.op("cast", [t], D.F32, dm)) if dtype != D.F32 else (lambda t, dm: t)
     h = g.op("add", [cast(res, (1, SC * SC, Cc)), cast(w, (1, SC * SC, Cc))], D.F32, (1, SC * SC, Cc))
     y = g.node("layer_norm", [h, cast(gamma, (Cc,)), cast(beta, (Cc,))], [D.F32], [(1, SC * SC, Cc)], extra_imm=[eps])[0]

@@ -64,12 +64,16 @@ OPCODES = {
     # composites over the last dim
     "softmax": 128, "log_softmax": 129, "layer_norm": 130, "rms_norm": 131,
     # index operators on leading dimensions (they move data, they compute nothing):
-    # roll: attr = (dim, shift); slice: attr = (dim, start), length from the output shape;
+    # roll: attr = (dim, shift); slice: attr = (dim, start), length from the output shape; a second
+    # dimension of either goes into the immediates as (1 + dim, shift / start), 0 meaning none;
     # view: regroups leading dimensions, the last one and the element order unchanged
     "roll": 160, "slice": 161, "view": 162,
     # cat: attr = (dim, 0); the concatenation of its operands along dim.  With one operand it is
     # the identity (graph traces keep such nodes)
     "cat": 163,
+    # contiguous: the same values in the dense row-major layout every tensor here already has: the
+    # identity (graph traces keep such nodes after index operators)
+    "contiguous": 164,
 }
 
 

@@ -1,9 +1,10 @@
 """Seeded random graphs against the CPU oracle, through the C ABI, with checked accessors on: the
 register allocator, the stage splitter and the spill / fill paths of the lowering meet graph
 structures nobody wrote by hand (the paper's demand that a rewrite hold in general rather than fit
-one instance, Section 3.1, applied to the graph itself).  Every graph runs fused on a generated
-kernel; in turn also on the interpreter, node by node (unfused), and in a forced kernel family.  A
-mode that refuses a graph must do so with a documented status."""
+one instance, Section 3.1, applied to the graph itself).  Every graph runs fused on generated
+kernels (one launch, or a few where a kernel budget cuts the graph); in turn also on the
+interpreter, node by node (unfused), and in a forced kernel family.  A mode that refuses a graph
+must do so with a documented status."""
 import numpy as np
 import pytest
 

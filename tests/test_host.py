@@ -88,8 +88,10 @@ def test_shape_and_support_errors():
     for u in ins[1:]:
         t = g.op("add", [t, u], D.F32, (8,))
     g.mark_output(t)
-    assert _status(g.build()) == -5                             # more inputs than a kernel takes
-    assert _status(g.build(), PLAN | pn.FLAG_UNFUSED) == 0      # one node at a time still fits
+    assert _status(g.build(), PLAN | pn.FLAG_ONE_KERNEL) == -5  # more inputs than a kernel takes
+    cut = pn.Graph(g.build(), 0, PLAN)                          # ... so the graph is cut into two fused launches
+    assert cut.n_kernels == 2 and cut.workspace_bytes > 0
+    assert _status(g.build(), PLAN | pn.FLAG_UNFUSED) == 0      # and one node at a time fits anyway
 
 
 FAMILY = {"c1": "pointwise", "c2": "warp-per-row", "c3": "block-per-row", "c4": "split-row",
@@ -215,13 +217,15 @@ def test_index_operator_errors():
     g = GraphBuilder(); x = g.input(D.F32, (4, 8))
     y = g.op("neg", [x], D.F32, (4, 8))
     g.mark_output(g.op("roll", [y], D.F32, (4, 8), attr=[0, 1]))
-    assert _status(g.build()) == -3
+    assert _status(g.build(), PLAN | pn.FLAG_ONE_KERNEL) == -3
+    assert pn.Graph(g.build(), 0, PLAN).n_kernels == 2          # cut after the computed value: the roll is then a copy of its own
     assert _status(g.build(), PLAN | pn.FLAG_UNFUSED) == 0      # one node at a time it is a plain copy
     # roll after slice on the same dimension would need a second modulus
     g = GraphBuilder(); x = g.input(D.F32, (6, 8))
     s = g.op("slice", [x], D.F32, (4, 8), attr=[0, 1])
     g.mark_output(g.op("roll", [s], D.F32, (4, 8), attr=[0, 1]))
-    assert _status(g.build()) == -3
+    assert _status(g.build(), PLAN | pn.FLAG_ONE_KERNEL) == -3
+    assert pn.Graph(g.build(), 0, PLAN).n_kernels == 2
     assert _status(g.build(), PLAN | pn.FLAG_UNFUSED) == 0
 
 
@@ -256,9 +260,9 @@ def test_masked_mean_pooling_lowers_to_one_column_kernel():
 
 
 def test_unsupported_column_forms_are_refused():
-    def status(g):
+    def status(g, extra=pn.FLAG_ONE_KERNEL):
         try:
-            pn.Graph(g.build(), 0, PLAN).close()
+            pn.Graph(g.build(), 0, PLAN | extra).close()
             return 0
         except pn.PnError as e:
             return e.status
@@ -266,6 +270,7 @@ def test_unsupported_column_forms_are_refused():
     s = g.op("sum_dim", [x], D.F32, (4, 1, 8), attr=[1, 0])
     g.mark_output(g.op("sub", [x, s], D.F32, (4, 6, 8)))             # needs a second pass over the dimension
     assert status(g) == -3
+    assert pn.Graph(g.build(), 0, PLAN).n_kernels == 2               # ... which is what two launches are
     g = GraphBuilder(); x = g.input(D.F32, (4, 6, 8))
     g.mark_output(g.op("sum_dim", [x], D.F32, (4, 6), attr=[2, 0]))  # the last dimension has its own opcodes
     assert status(g) == -3
@@ -276,6 +281,7 @@ def test_unsupported_column_forms_are_refused():
     g.mark_output(g.op("sum_dim", [x], D.F32, (4, 8), attr=[1, 0]))
     g.mark_output(g.op("sum_dim", [x], D.F32, (6, 8), attr=[0, 0]))  # two different dimensions in one graph
     assert status(g) == -3
+    assert pn.Graph(g.build(), 0, PLAN).n_kernels == 2
     g = GraphBuilder(); x = g.input(D.F32, (4, 6, 8)); y = g.input(D.F32, (4, 6, 8))
     g.mark_output(g.op("cat", [x, y], D.F32, (4, 12, 8), attr=[1, 0]))   # a real concatenation is not lowered
     assert status(g) == -3

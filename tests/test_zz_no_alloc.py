@@ -51,8 +51,8 @@ def test_static_scratch_matches_the_allocating_path_twice_in_a_row(interpret):
             got = _run(g, w.inputs, static=True)
             for a, b, (dt, _dims) in zip(got, want, w.output_meta):
                 res = E.compare(E.widen(a, dt), E.widen(b, dt), dt)   # same tolerance rule as every GPU test
-                assert res["ok"], res
-                assert np.array_equal(a, b)                             # same kernels, same order: same bits
+                assert res["ok"], res        # (not the same bits: a handle that may not allocate never takes the
+                                             #  kernel family that needs a workspace, so sums may be taken in another order)
             check_against_oracle(w.desc, w.inputs, got, w.output_meta, w.output_names)
         with pytest.raises(pn.PnError) as bad:                       # the ordinary entry point refuses the handle
             _run(g, w.inputs, static=False)
