@@ -51,8 +51,11 @@
  * index operators that start at one, and cost no data movement: the fused kernel computes the
  * source row instead (idx = (S + i - shift) mod S).  164 contiguous: the identity on values (every
  * tensor here is dense already); after a chain of index operators it is one more link of the chain,
- * on a computed value a pointwise identity.  163 cat (attr[0] = dim): with one operand it
- * is the identity, as graph traces contain it; several operands are not lowered.
+ * on a computed value a pointwise identity.  163 cat (attr[0] = dim, up to 4 operands of the
+ * result's dtype): with one operand it is the identity, as graph traces contain it; with several it
+ * is not computed at all: every operand is stored straight into its block of the result by the
+ * kernel that produces it (an output-address remap), operands of different shapes by a launch
+ * each, and a node that reads the result runs in a later launch.
  * Arithmetic is fp32 in registers whatever the storage types; integer and boolean
  * tensors take part as exact small integers / predicates; a node whose declared
  * output dtype is bf16 / f16 is rounded to it (nearest even) for its consumers.
@@ -396,12 +399,19 @@ typedef struct pn_probe_config {
   int loader;           /* PN_PROBE_*                                                         */
   int streaming_stores; /* 1: stores carry the evict-first hint                               */
   int layout;           /* direct loaders: 0 grid-stride over units, 1 a contiguous range per block,
-                           2 runs of tile_units units taken by the blocks in turn (read-only path) */
+                           2 runs of tile_units units taken by the blocks in turn, 3 (PN_MIX_READ only)
+                           strips: the array as rows of tile_units units, a block owning strip_units
+                           units by rows_per_block rows, its block / strip_units walkers going down
+                           the rows (the pattern of a reduction over a leading dimension; the grid
+                           follows from the sizes)                                              */
   int block;            /* threads that load / store per block (multiple of 32, <= 992)       */
   int unroll;           /* direct loaders: units in flight per thread (1, 2, 4, 8)            */
   int grid;             /* blocks                                                             */
   int stages;           /* bulk loader: ring depth (2..16)                                    */
-  int tile_units;       /* bulk loader: units per array per stage (32..4096); layout 2: the run length */
+  int tile_units;       /* bulk loader: units per array per stage (32..4096); layout 2: the run length;
+                           layout 3: units per row                                              */
+  int strip_units;      /* layout 3: units a strip is wide                                    */
+  int rows_per_block;   /* layout 3: rows a strip is long                                     */
 } pn_probe_config;
 pn_status pn_stream_probe(int mix, const pn_probe_config* cfg, const void* a, const void* b, void* c, void* d,
                           size_t units, void* status_word, void* stream);

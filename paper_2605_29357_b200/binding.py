@@ -57,7 +57,8 @@ class ProbeConfig(ctypes.Structure):
     """pn_probe_config: how pn_stream_probe moves its bytes."""
     _fields_ = [("loader", ctypes.c_int), ("streaming_stores", ctypes.c_int), ("layout", ctypes.c_int),
                 ("block", ctypes.c_int), ("unroll", ctypes.c_int), ("grid", ctypes.c_int),
-                ("stages", ctypes.c_int), ("tile_units", ctypes.c_int)]
+                ("stages", ctypes.c_int), ("tile_units", ctypes.c_int), ("strip_units", ctypes.c_int),
+                ("rows_per_block", ctypes.c_int)]
 
 
 class PnError(RuntimeError):

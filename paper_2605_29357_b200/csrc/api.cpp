@@ -14,6 +14,7 @@
 #include "graph.h"
 #include "handle.h"
 #include "spec.h"
+#include "lower_common.h"
 
 namespace pn {
 cudaError_t launch_plan(const LaunchPlan& lp, cudaStream_t stream);   // kernels.cu
@@ -54,7 +55,8 @@ void group_subgraph(const Graph& g, const std::vector<int>& members, Graph& sub,
   auto add = [&](int orig) {
     for (size_t i = 0; i < orig_of_sub.size(); ++i) if (orig_of_sub[i] == orig) return (int)i;
     Tensor t = g.tensors[orig];
-    t.role = made_here[orig] ? (uint8_t)(((g.tensors[orig].role & 2) || read_outside[orig]) ? 2 : 0) : (uint8_t)1;
+    // (a part of a cat result is always stored: that store is what the cat is)
+    t.role = made_here[orig] ? (uint8_t)(((g.tensors[orig].role & 2) || read_outside[orig] || g.tensors[orig].embed_parent >= 0) ? 2 : 0) : (uint8_t)1;
     t.producer = -1;
     sub.tensors.push_back(t);
     orig_of_sub.push_back(orig);
@@ -99,12 +101,50 @@ bool partition_graph(const Graph& g, unsigned flags, const DeviceModel& dev, std
     const Node& nd = g.nodes[i];
     int lv = 0;
     for (int k = 0; k < nd.n_in; ++k) if (nd.in[k] < g.tensors.size()) lv = std::max(lv, t_level[nd.in[k]]);
+    for (int k = 0; k < nd.n_in; ++k)   // (a cat result is as deep as its deepest part)
+      if (nd.in[k] < g.tensors.size() && g.tensors[nd.in[k]].assembled)
+        for (const Tensor& P : g.tensors) if (P.embed_parent == (int)nd.in[k] && P.producer >= 0 && P.producer < i) lv = std::max(lv, n_level[P.producer]);
     n_level[i] = lv;
     const bool reduces = is_reduction(nd.op) || is_composite(nd.op) || is_dim_reduction(nd.op);
     for (int k = 0; k < nd.n_out; ++k) t_level[nd.out[k]] = lv + (reduces ? 1 : 0);
     order[i] = i;
   }
-  std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return n_level[a] < n_level[b]; });
+  // ... and among the nodes that are ready at the same depth, one that works on the shape of the node
+  // listed before it comes first, so that a chain over one shape is not interleaved with a chain
+  // over another (two operands of a cat, say, each with its own producers).
+  {
+    std::vector<int> pending(n, 0);
+    std::vector<std::vector<int>> users(n);
+    for (int i = 0; i < n; ++i)
+      for (int k = 0; k < g.nodes[i].n_in; ++k) {
+        const uint32_t t = g.nodes[i].in[k];
+        if (t >= g.tensors.size()) continue;
+        std::vector<int> producers;
+        if (g.tensors[t].producer >= 0) producers.push_back(g.tensors[t].producer);
+        if (g.tensors[t].assembled) for (const Tensor& P : g.tensors) if (P.embed_parent == (int)t && P.producer >= 0) producers.push_back(P.producer);
+        for (int pr : producers) if (pr != i) { users[pr].push_back(i); pending[i]++; }
+      }
+    using lowering::Shape4;
+    auto shape_of = [&](int i) { return lowering::align4(g.tensors[g.nodes[i].out[0]]); };
+    std::vector<char> done(n, 0);
+    int last = -1;
+    for (int pos = 0; pos < n; ++pos) {
+      int pick = -1;
+      for (int i = 0; i < n; ++i) {
+        if (done[i] || pending[i] > 0) continue;
+        if (pick < 0) { pick = i; continue; }
+        if (n_level[i] != n_level[pick]) { if (n_level[i] < n_level[pick]) pick = i; continue; }
+        if (last >= 0) {
+          const Shape4 sl = shape_of(last), si = shape_of(i), sp = shape_of(pick);
+          const bool mi = memcmp(&sl, &si, sizeof(sl)) == 0, mp = memcmp(&sl, &sp, sizeof(sl)) == 0;
+          if (mi && !mp) pick = i;
+        }
+      }
+      if (pick < 0) return false;   // (cannot happen: the descriptor is in topological order)
+      order[pos] = pick; done[pick] = 1; last = pick;
+      for (int u : users[pick]) pending[u]--;
+    }
+  }
   const int64_t kInf = INT64_MAX / 4;
   std::vector<int64_t> best(n + 1, kInf);
   std::vector<int> from(n + 1, -1);
@@ -115,6 +155,16 @@ bool partition_graph(const Graph& g, unsigned flags, const DeviceModel& dev, std
     int misses = 0;
     for (int j = i; j < n; ++j) {
       members.push_back(order[j]);
+      {   // a launch cannot both store a part of a cat result and read that result
+        bool clash = false;
+        for (int a : members)
+          for (int k = 0; k < g.nodes[a].n_in && !clash; ++k) {
+            const uint32_t t = g.nodes[a].in[k];
+            if (t >= g.tensors.size() || !g.tensors[t].assembled) continue;
+            for (int b : members) if (g.tensors[g.nodes[b].out[0]].embed_parent == (int)t) clash = true;
+          }
+        if (clash) { if (++misses > 24) break; continue; }
+      }
       Graph sub;
       std::vector<int> orig;
       group_subgraph(g, members, sub, orig);
@@ -163,9 +213,10 @@ pn_status check_counts(const pn_graph* h, const void* const* inputs, int n_input
 void fill_pointers(const pn_graph* h, const PlannedLaunch& pl, const void* const* inputs, void* const* outputs, void* workspace, LaunchPlan& lp) {
   for (int q = 0; q < lp.p.n_io; ++q) {
     const IoSource& s = pl.src[q];
-    lp.p.io[q].base = s.kind == 0 ? const_cast<void*>(inputs[s.index])
-                    : s.kind == 1 ? outputs[s.index]
-                                  : (void*)((char*)workspace + s.index);
+    char* base = s.kind == 0 ? (char*)const_cast<void*>(inputs[s.index])
+               : s.kind == 1 ? (char*)outputs[s.index]
+                             : (char*)workspace + s.index;
+    lp.p.io[q].base = base + lp.io_offset[q] * dtype_bytes(lp.p.io[q].dtype);
   }
   (void)h;
 }
@@ -246,6 +297,9 @@ pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsig
   std::string err;
   int st = parse_descriptor(desc, desc_bytes, h->g, err);
   if (st != PN_OK) { delete h; return fail(st, err); }
+  h->n_nodes = (int)h->g.nodes.size();
+  st = expand_concatenations(h->g, err);   // a cat of several operands becomes stores into blocks of its result
+  if (st != PN_OK) { delete h; return fail(st, err); }
   if ((flags & PN_FLAG_BOUNDS) && (flags & PN_FLAG_STATIC_SCRATCH)) { delete h; return fail(PN_ERR_INVALID_ARG, "PN_FLAG_BOUNDS allocates a status word: it cannot be combined with PN_FLAG_STATIC_SCRATCH"); }
   h->flags = flags;
   h->device = device;
@@ -295,7 +349,21 @@ pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsig
     // into the cheapest sequence of fused launches (PN_FLAG_ONE_KERNEL asks for the refusal instead)
     LaunchPlan probe;
     std::string why_not;
-    const int whole = lower_graph(g, flags, dev, probe, why_not);
+    bool any_assembled = false;
+    for (const Tensor& T : g.tensors) any_assembled = any_assembled || T.assembled;
+    int whole;
+    if (any_assembled) {   // (the cat results themselves take no part in a launch: only their parts do)
+      Graph sub;
+      std::vector<int> orig;
+      group_subgraph(g, groups[0], sub, orig);
+      whole = lower_graph(sub, flags, dev, probe, why_not);
+    } else whole = lower_graph(g, flags, dev, probe, why_not);
+    // a cat result is complete only when the launches that store its parts are done: a node that
+    // reads it cannot share a launch with them
+    for (const Node& nd : g.nodes)
+      for (int k = 0; k < nd.n_in; ++k)
+        if (nd.in[k] < g.tensors.size() && g.tensors[nd.in[k]].assembled && whole == PN_OK) { whole = PN_ERR_UNSUPPORTED_OP; why_not = "a cat result is read inside the graph"; }
+    if (whole == PN_ERR_SHAPE && any_assembled) whole = PN_ERR_UNSUPPORTED_OP;   // parts of different shapes: one launch each
     if ((whole == PN_ERR_TOO_LARGE || whole == PN_ERR_UNSUPPORTED_OP) && !(flags & PN_FLAG_ONE_KERNEL)) {
       std::vector<std::vector<int>> cut;
       if (partition_graph(g, flags, dev, cut)) groups.swap(cut);
@@ -306,21 +374,24 @@ pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsig
   for (size_t gi = 0; gi < groups.size(); ++gi) for (int ni : groups[gi]) group_of_node[ni] = (int)gi;
   std::vector<int64_t> ws_off(g.tensors.size(), -1);
   size_t ws = 0;
-  if (groups.size() > 1)
-    for (size_t t = 0; t < g.tensors.size(); ++t) {
-      if (g.tensors[t].role != 0 || g.tensors[t].producer < 0) continue;
-      bool crosses = false;
-      for (size_t ni = 0; ni < g.nodes.size() && !crosses; ++ni)
+  for (size_t t = 0; t < g.tensors.size(); ++t) {
+    const Tensor& T = g.tensors[t];
+    if (T.role != 0 || T.embed_parent >= 0) continue;          // the caller's buffers; parts live in their parent
+    bool stored = T.assembled;                                  // a cat result is always materialised
+    if (!stored && T.producer >= 0 && groups.size() > 1)
+      for (size_t ni = 0; ni < g.nodes.size() && !stored; ++ni)
         for (int k = 0; k < g.nodes[ni].n_in; ++k)
-          if (g.nodes[ni].in[k] == t && group_of_node[ni] != group_of_node[g.tensors[t].producer]) crosses = true;
-      if (!crosses) continue;
-      ws_off[t] = (int64_t)ws;
-      ws += ((size_t)tensor_bytes(g.tensors[t]) + 255) / 256 * 256;
-    }
+          if (g.nodes[ni].in[k] == t && group_of_node[ni] != group_of_node[T.producer]) stored = true;
+    if (!stored) continue;
+    ws_off[t] = (int64_t)ws;
+    ws += ((size_t)tensor_bytes(T) + 255) / 256 * 256;
+  }
   for (size_t gi = 0; gi < groups.size(); ++gi) {
     PlannedLaunch pl;
     std::vector<int> orig;
-    if (groups.size() == 1) {
+    bool plain_whole = groups.size() == 1;
+    for (const Tensor& T : g.tensors) plain_whole = plain_whole && !T.assembled;
+    if (plain_whole) {
       st = lower_graph(g, flags, dev, pl.plan, err);
       for (size_t t = 0; t < g.tensors.size(); ++t) orig.push_back((int)t);
     } else {
@@ -331,8 +402,12 @@ pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsig
     }
     if (st != PN_OK) { delete h; return fail(st, err); }
     for (int q = 0; q < pl.plan.p.n_io; ++q) {
-      const int t = orig[pl.plan.io_tensor[q]];
+      int t = orig[pl.plan.io_tensor[q]];
       pl.plan.p.io[q].numel = g.tensors[t].numel();
+      if (pl.plan.io_is_output[q] && g.tensors[t].embed_parent >= 0) {   // a part of a cat result: stored inside it
+        t = g.tensors[t].embed_parent;
+        pl.plan.p.io[q].numel = g.tensors[t].numel() - pl.plan.io_offset[q];
+      }
       IoSource s{2, ws_off[t]};
       // a tensor that is both read and written by the graph's caller (an input passed through) is
       // looked up on the side this launch uses it on
@@ -627,7 +702,7 @@ pn_status pn_graph_query(const pn_graph_t* h, int what, void* out, size_t out_by
     case PN_Q_OUTPUT_META: meta(g.outputs); break;
     case PN_Q_COMPULSORY_BYTES: v.push_back(h->compulsory_bytes); break;
     case PN_Q_N_KERNELS: v.push_back((int64_t)h->launches.size()); break;
-    case PN_Q_N_NODES: v.push_back((int64_t)g.nodes.size()); break;
+    case PN_Q_N_NODES: v.push_back((int64_t)h->n_nodes); break;
     case PN_Q_WORKSPACE_BYTES: v.push_back((int64_t)h->workspace_bytes); break;
     case PN_Q_KERNEL_INFO:
       for (const PlannedLaunch& pl : h->launches) {

@@ -4,6 +4,7 @@
 #include <string.h>
 
 #include <string>
+#include <vector>
 
 #include "../../include/pn.h"
 #include "graph.h"
@@ -102,6 +103,51 @@ int parse_descriptor(const void* desc, size_t bytes, Graph& g, std::string& err)
   }
   for (int o : g.outputs)
     if (g.tensors[o].producer < 0) { err = "output tensor " + std::to_string(o) + " is never produced"; return PN_ERR_BAD_DESCRIPTOR; }
+  return PN_OK;
+}
+
+int expand_concatenations(Graph& g, std::string& err) {
+  bool any = false;
+  for (const Node& n : g.nodes) any = any || (n.op == N_CAT && n.n_in > 1);
+  if (!any) return PN_OK;
+  std::vector<Node> nodes;
+  for (size_t ni = 0; ni < g.nodes.size(); ++ni) {
+    const Node n = g.nodes[ni];
+    if (!(n.op == N_CAT && n.n_in > 1)) { nodes.push_back(n); continue; }
+    const std::string where = "node " + std::to_string(ni) + ": ";
+    const int y = (int)n.out[0];
+    const Tensor Y = g.tensors[y];
+    const int64_t dim = n.attr[0];
+    if (dim < 0 || dim >= Y.rank) { err = where + "cat dimension outside the tensor"; return PN_ERR_SHAPE; }
+    int64_t pd[4] = {1, 1, 1, 1};
+    for (int i = 0; i < Y.rank; ++i) pd[4 - Y.rank + i] = Y.dims[i];
+    int64_t at = 0;
+    for (int k = 0; k < n.n_in; ++k) {
+      if (n.in[k] >= g.tensors.size()) { err = where + "cat of a constant"; return PN_ERR_UNSUPPORTED_OP; }
+      const Tensor X = g.tensors[n.in[k]];
+      if (X.rank != Y.rank || X.dtype != Y.dtype) { err = where + "the operands of a cat have the rank and dtype of its result"; return X.rank != Y.rank ? PN_ERR_SHAPE : PN_ERR_UNSUPPORTED_OP; }
+      for (int i = 0; i < Y.rank; ++i)
+        if (i != dim && X.dims[i] != Y.dims[i]) { err = where + "the operands of a cat differ from its result in the cat dimension only"; return PN_ERR_SHAPE; }
+      Tensor part = X;
+      part.role = 0; part.producer = (int)nodes.size();
+      part.assembled = false;
+      part.embed_parent = y;
+      for (int i = 0; i < 4; ++i) { part.embed_dims[i] = pd[i]; part.embed_off[i] = 0; }
+      part.embed_off[4 - Y.rank + dim] = at;
+      at += X.dims[dim];
+      g.tensors.push_back(part);
+      Node c;
+      c.op = N_CONTIGUOUS; c.n_in = 1; c.n_out = 1;
+      c.in[0] = n.in[k]; c.out[0] = (uint32_t)g.tensors.size() - 1;
+      nodes.push_back(c);
+    }
+    if (at != Y.dims[dim]) { err = where + "the operands of a cat do not add up to its result along the cat dimension"; return PN_ERR_SHAPE; }
+    g.tensors[y].assembled = true;
+    g.tensors[y].producer = -1;
+  }
+  g.nodes.swap(nodes);
+  for (size_t ni = 0; ni < g.nodes.size(); ++ni)   // producers by the new numbering
+    for (int k = 0; k < g.nodes[ni].n_out; ++k) g.tensors[g.nodes[ni].out[k]].producer = (int)ni;
   return PN_OK;
 }
 

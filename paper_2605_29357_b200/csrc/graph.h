@@ -32,6 +32,14 @@ struct Tensor {
   int rank = 0;
   int64_t dims[4] = {1, 1, 1, 1};
   int producer = -1;       // node index, -1 for graph inputs
+  // A concatenation of several operands is not computed: each operand is stored straight into its
+  // block of the result.  `assembled`: this tensor is such a result (no node of its own produces it;
+  // it is complete once its parts are stored).  `embed_parent` >= 0: this tensor is such a part: it
+  // lives inside tensor embed_parent, whose dims (aligned to 4) are embed_dims, at embed_off.
+  bool assembled = false;
+  int embed_parent = -1;
+  int64_t embed_dims[4] = {1, 1, 1, 1};
+  int64_t embed_off[4] = {0, 0, 0, 0};
   int64_t numel() const { int64_t n = 1; for (int i = 0; i < rank; ++i) n *= dims[i]; return n; }
 };
 
@@ -61,6 +69,10 @@ inline bool is_index_op(uint16_t op) { return op >= N_ROLL && op <= N_VIEW; }
 
 // Returns a pn_status value (see pn.h).
 int parse_descriptor(const void* desc, size_t bytes, Graph& g, std::string& err);
+
+// Replaces every cat of several operands by one `contiguous` node per operand whose result is
+// embedded in the cat's output (see Tensor::embed_parent).  Returns a pn_status value.
+int expand_concatenations(Graph& g, std::string& err);
 
 struct DeviceModel {      // what the lowering needs to know about the GPU
   int sm_count = 148;

@@ -65,6 +65,7 @@ struct pn_graph {
   pn::Graph g;
   unsigned flags = 0;
   int device = 0;
+  int n_nodes = 0;                          // operator nodes of the descriptor (before any rewriting)
   bool plan_only = false;
   std::vector<pn::PlannedLaunch> launches;
   void* workspace = nullptr;

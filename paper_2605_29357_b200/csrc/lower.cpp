@@ -57,8 +57,8 @@ struct Config { int family, vl, ng, k, block, cluster, chunks, slice_len; bool m
 
 // ---------------------------------------------------------------------------------------
 int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPlan& lp, std::string& err) {
-  for (const Node& n : g.nodes)
-    if (n.op == N_CAT && n.n_in != 1) { err = "cat of several operands is not lowered (one operand is the identity)"; return PN_ERR_UNSUPPORTED_OP; }
+  for (const Node& n : g.nodes)   // (a cat of several operands has been rewritten into embedded parts before any lowering)
+    if (n.op == N_CAT && n.n_in != 1) { err = "internal: a cat of several operands reached the lowering"; return PN_ERR_UNSUPPORTED_OP; }
   for (const Node& n : g.nodes) if (is_dim_reduction(n.op)) return lower_column_graph(g, flags, dev, lp, err);
   const int nt = (int)g.tensors.size();
   std::vector<char> is_s(nt, 0);
@@ -261,6 +261,14 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
         io.col_stride = (s.d[3] == 1 && N != 1) ? 0 : 1;
         io_streamed[idx] = full;
       }
+      lp.io_offset[idx] = 0;
+      if (is_out && T.embed_parent >= 0) {   // stored as a block of a larger tensor: the parent's strides, the block's start
+        if (is_s[t]) return false;
+        int64_t st = 1, ps[4];
+        for (int i = 3; i >= 0; --i) { ps[i] = st; st *= T.embed_dims[i]; }
+        for (int i = 0; i < 3; ++i) io.lead_stride[i] = F.d[i] == 1 ? 0 : ps[i];
+        for (int i = 0; i < 4; ++i) lp.io_offset[idx] += T.embed_off[i] * ps[i];
+      }
       if (!is_out && !imap[t].plain) {   // read through rolls / slices: own coordinates, source strides
         const IdxMap& m = imap[t];
         const Shape4 s = align4(T);
@@ -278,7 +286,8 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     };
     for (int t : in_like)
       if (!add_io(t, false)) { err = "tensor " + std::to_string(t) + ": a rolled / sliced input must cover the whole iteration space"; return PN_ERR_UNSUPPORTED_OP; }
-    for (int t : g.outputs) add_io(t, true);
+    for (int t : g.outputs)
+      if (!add_io(t, true)) { err = "tensor " + std::to_string(t) + ": a per-row result cannot be an operand of a cat"; return PN_ERR_UNSUPPORTED_OP; }
   }
   // collapse leading dims that every io walks contiguously (or broadcasts) together
   int64_t lead_dim[3] = {F.d[0], F.d[1], F.d[2]};
@@ -471,7 +480,7 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     if (io.is_row_scalar || io.col_stride == 0) continue;
     if (io_streamed[q]) min_esize = std::min(min_esize, dtype_bytes(io.dtype));
     for (int vl : {8, 4}) {
-      bool ok = eff_N % vl == 0;
+      bool ok = eff_N % vl == 0 && lp.io_offset[q] % vl == 0;
       for (int i = 0; i < 3; ++i) ok = ok && io.lead_stride[i] % vl == 0;
       if (vl == 8) vec8 = vec8 && ok; else vec4 = vec4 && ok;
     }

@@ -53,6 +53,8 @@ int group_state(const int64_t* d, const int64_t* full, int lo, int hi) {
 
 int lower_column_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPlan& lp, std::string& err) {
   const int nt = (int)g.tensors.size();
+  for (int o : g.outputs)
+    if (g.tensors[o].embed_parent >= 0) { err = "a result of a reduction over a leading dimension cannot be stored as an operand of a cat in the same kernel"; return PN_ERR_UNSUPPORTED_OP; }
   // ---- (1) the reduced dimension and the two spaces ----------------------------------------
   int rs = -1, dr = -1;   // rank of the reduced tensors, reduced dimension
   for (size_t ni = 0; ni < g.nodes.size(); ++ni) {

@@ -87,6 +87,33 @@ __global__ void probe_direct(const uint4* __restrict__ a, const uint4* __restric
   if (NW16 == 0 && NW8 == 0 && (sink.x ^ sink.y ^ sink.z ^ sink.w) == 0x9E3779B9u && sink.x == 0x7F4A7C15u) atomicOr(status, 0x80000000u);
 }
 
+// Read-only, the access pattern of a reduction over a leading dimension: the array is rows of C units;
+// a block owns a strip of TX units by RS consecutive rows and its blockDim.x / TX walkers go down the
+// rows, U rows of each in flight together.  Blocks are numbered so that neighbours own neighbouring
+// strips of the same rows.
+template <int U>
+__global__ void probe_strips(const uint4* __restrict__ a, size_t units, int C, int TX, int RS, unsigned* status) {
+  const size_t rows = units / C;
+  const int ctiles = C / TX, TY = blockDim.x / TX;
+  const int ct = blockIdx.x % ctiles;
+  const size_t rb = blockIdx.x / ctiles;
+  const int tx = threadIdx.x % TX, ty = threadIdx.x / TX;
+  const size_t r_end = min(rows, (rb + 1) * (size_t)RS);
+  uint4 sink = make_uint4(0, 0, 0, 0);
+  for (size_t r0 = rb * (size_t)RS + ty; r0 < r_end; r0 += (size_t)TY * U) {
+    uint4 v[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const size_t r = r0 + (size_t)u * TY;
+      v[u] = make_uint4(0, 0, 0, 0);
+      if (r < r_end) v[u] = ld_nc(a + r * C + (size_t)ct * TX + tx);
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) sink = mix4(sink, v[u]);
+  }
+  if ((sink.x ^ sink.y ^ sink.z ^ sink.w) == 0x9E3779B9u && sink.x == 0x7F4A7C15u) atomicOr(status, 0x80000000u);
+}
+
 // ---- bulk copies into a shared-memory ring -----------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
@@ -219,7 +246,7 @@ pn_status pn_stream_probe(int mix, const pn_probe_config* cfg, const void* a, co
   if ((nr >= 1 && !a) || (nr >= 2 && !b) || (w16 && !c) || (w8 && !d)) return fail(PN_ERR_INVALID_ARG, "a buffer of this mix is null");
   for (const void* p : {a, b, (const void*)c, (const void*)d, (const void*)status_word})
     if ((uintptr_t)p & 15) return fail(PN_ERR_ALIGNMENT, "probe buffers must be aligned to 16 bytes");
-  if (cfg->block < 32 || cfg->block > 992 || cfg->block % 32 || cfg->grid < 1) return fail(PN_ERR_INVALID_ARG, "block must be a multiple of 32 up to 992, grid positive");
+  if (cfg->block < 32 || cfg->block > 992 || cfg->block % 32 || (cfg->grid < 1 && cfg->layout != 3)) return fail(PN_ERR_INVALID_ARG, "block must be a multiple of 32 up to 992, grid positive");
   if (cfg->loader < PN_PROBE_LDG || cfg->loader > PN_PROBE_BULK) return fail(PN_ERR_INVALID_ARG, "unknown loader");
   if (cfg->loader == PN_PROBE_BULK) {
     if (nr == 0) return fail(PN_ERR_INVALID_ARG, "a write-only probe has nothing to load");
@@ -228,9 +255,28 @@ pn_status pn_stream_probe(int mix, const pn_probe_config* cfg, const void* a, co
     if (1024 + (size_t)cfg->stages * cfg->tile_units * 16 * nr > 227 * 1024) return fail(PN_ERR_TOO_LARGE, "the ring does not fit in shared memory");
   } else {
     if (cfg->unroll != 1 && cfg->unroll != 2 && cfg->unroll != 4 && cfg->unroll != 8) return fail(PN_ERR_INVALID_ARG, "unroll must be 1, 2, 4 or 8");
-    if (cfg->layout < 0 || cfg->layout > 2 || (cfg->layout == 2 && cfg->tile_units < 1)) return fail(PN_ERR_INVALID_ARG, "layout must be 0, 1 or 2 (2 with tile_units > 0 as the run length)");
+    if (cfg->layout < 0 || cfg->layout > 3 || (cfg->layout == 2 && cfg->tile_units < 1)) return fail(PN_ERR_INVALID_ARG, "layout must be 0 .. 3 (2 with tile_units > 0 as the run length)");
   }
   if (units == 0) return PN_OK;
+  if (cfg->layout == 3) {   // strips: read-only
+    if (mix != PN_MIX_READ || cfg->loader != PN_PROBE_LDG) return fail(PN_ERR_INVALID_ARG, "the strip layout is a read-only probe with plain loads");
+    const int C = cfg->tile_units, TX = cfg->strip_units, RS = cfg->rows_per_block;
+    if (C < 1 || TX < 1 || RS < 1 || C % TX || cfg->block % TX || units % (size_t)C) return fail(PN_ERR_INVALID_ARG, "strips: tile_units (row length) must divide the array and be a multiple of strip_units, which must divide block");
+    const size_t rows = units / C;
+    const size_t blocks = (rows + RS - 1) / RS * (C / TX);
+    if (blocks > (1u << 30)) return fail(PN_ERR_TOO_LARGE, "too many strips");
+    unsigned* st = (unsigned*)status_word;
+    cudaStream_t s = (cudaStream_t)stream;
+    switch (cfg->unroll) {
+      case 1: probe_strips<1><<<(unsigned)blocks, cfg->block, 0, s>>>((const uint4*)a, units, C, TX, RS, st); break;
+      case 2: probe_strips<2><<<(unsigned)blocks, cfg->block, 0, s>>>((const uint4*)a, units, C, TX, RS, st); break;
+      case 4: probe_strips<4><<<(unsigned)blocks, cfg->block, 0, s>>>((const uint4*)a, units, C, TX, RS, st); break;
+      default: probe_strips<8><<<(unsigned)blocks, cfg->block, 0, s>>>((const uint4*)a, units, C, TX, RS, st); break;
+    }
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(PN_ERR_CUDA, std::string("probe launch: ") + cudaGetErrorString(e));
+    return PN_OK;
+  }
   const uint4* pa = (const uint4*)a; const uint4* pb = (const uint4*)b; uint4* pc = (uint4*)c; uint2* pd = (uint2*)d;
   cudaError_t e;
 #define PN_MIX_GO(NR, W16, W8) launch_mix<NR, W16, W8>(cfg->loader, cfg->streaming_stores, cfg->layout, cfg->block, cfg->unroll, cfg->grid, cfg->stages, cfg->tile_units, pa, pb, pc, pd, units, (unsigned*)status_word, (cudaStream_t)stream)

@@ -251,7 +251,11 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
   s += "  static PN_DEV long long red_stride(const KernelParams&, int io) {\n    switch (io) {\n";
   for (int q = 0; q < P.n_io; ++q) if (P.io[q].red_stride != 0) s += "      case " + I(q) + ": return " + I(P.io[q].red_stride) + "ll;\n";
   s += "      default: return 0;\n    }\n  }\n";
-  s += "#ifndef PN_WALK_UNROLL\n#define PN_WALK_UNROLL " + I(P.family == FAM_COLUMN ? 4 : 1) + "\n#endif\n  static constexpr int kWalkUnroll = PN_WALK_UNROLL;\n";
+  // column kernels: steps whose loads are in flight together.  Six under a bound of 7 blocks of 128
+  // threads (72 registers) measured best on the pooling workload (47.2 -> 45.2 us); larger blocks keep
+  // four under 64 registers.
+  const int walk_unroll = P.family == FAM_COLUMN ? (lp.block == 128 ? 6 : 4) : 1;
+  s += "#ifndef PN_WALK_UNROLL\n#define PN_WALK_UNROLL " + I(walk_unroll) + "\n#endif\n  static constexpr int kWalkUnroll = PN_WALK_UNROLL;\n";
   s += "  static PN_DEV bool io_mapped(const KernelParams&, int io) {\n    switch (io) {\n";
   for (int q = 0; q < P.n_io; ++q) if (P.io[q].mapped) s += "      case " + I(q) + ": return true;\n";
   s += "      default: return false;\n    }\n  }\n";
@@ -336,7 +340,8 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
   // Column kernels likewise: their walk keeps several steps of loads in flight per thread, and the
   // bound keeps that from eating the resident warps (measured: 64 registers with 4 steps in flight
   // beats every larger budget on the pooling workload).
-  const int min_blocks = ((P.family == FAM_BLOCK && P.chunks == 1) || P.family == FAM_COLUMN) ? std::max(1, 1024 / lp.block) : 1;
+  const int min_blocks = (P.family == FAM_COLUMN && lp.block == 128) ? 7
+                       : ((P.family == FAM_BLOCK && P.chunks == 1) || P.family == FAM_COLUMN) ? std::max(1, 1024 / lp.block) : 1;
   s += "#ifndef PN_MIN_BLOCKS\n#define PN_MIN_BLOCKS " + I(min_blocks) + "\n#endif\n";
   s += "#if PN_MIN_BLOCKS > 1\n#define PN_LAUNCH_BOUNDS __launch_bounds__(" + I(lp.block) + ", PN_MIN_BLOCKS)\n#else\n"
        "#define PN_LAUNCH_BOUNDS __launch_bounds__(" + I(lp.block) + ")\n#endif\n";

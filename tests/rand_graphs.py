@@ -150,7 +150,7 @@ class RandomGraph:
             v = self._pick(self.tiles + self.scalars, P)
             if not v:
                 return False
-            cands = [("sqrt", math.sqrt(v.lo), math.sqrt(v.hi)), ("sigmoid", 0.5, 1.0), ("tanh", math.tanh(v.lo), 1.0),
+            cands = [("sqrt", math.sqrt(v.lo), math.sqrt(v.hi)), ("sigmoid", 0.5, 1.0), ("contiguous", v.lo, v.hi), ("tanh", math.tanh(v.lo), 1.0),
                      ("relu", v.lo, v.hi), ("abs", v.lo, v.hi), ("erf", math.erf(v.lo), 1.0),
                      ("silu", v.lo / (1 + math.exp(-v.lo)), v.hi), ("gelu_tanh", 0.5 * v.lo, v.hi), ("gelu_erf", 0.5 * v.lo, v.hi)]
             if v.hi * v.hi <= HI_MAX:
@@ -430,7 +430,16 @@ class RandomGraph:
         if not extra and not self.outputs:         # nothing full-shaped was computed: make one value that is
             x = self.tiles[0]
             extra = [self._emit("mul", [x, Imm(1.5)], D.F32, self.full, "P", x.lo * 1.5, x.hi * 1.5)]
-        outs = (self.outputs + extra)[: 12 - len(self.inputs)]
+        if r.random() < 0.25:                      # a concatenation of two or three computed values leaves the graph too
+            parts = [v for v in self.tiles if self._is_full(v) and v.kind in ("P", "S") and v.dtype == D.F32 and v.tid not in self.g.input_ids()]
+            if len(parts) >= 2:
+                k = int(r.integers(2, min(3, len(parts)) + 1))
+                pick = [parts[int(i)] for i in r.choice(len(parts), size=k, replace=False)]
+                dim = int(r.integers(0, len(self.full)))
+                shape = list(self.full); shape[dim] = k * self.full[dim]
+                c = self._emit("cat", pick, D.F32, tuple(shape), "S", attr=(dim, 0))
+                self.g.mark_output(c.tid)
+        outs = (self.outputs + extra)[: 11 - len(self.inputs)]
         seen = set()
         for v in outs:
             if v.tid in seen:

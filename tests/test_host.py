@@ -283,8 +283,11 @@ def test_unsupported_column_forms_are_refused():
     assert status(g) == -3
     assert pn.Graph(g.build(), 0, PLAN).n_kernels == 2
     g = GraphBuilder(); x = g.input(D.F32, (4, 6, 8)); y = g.input(D.F32, (4, 6, 8))
-    g.mark_output(g.op("cat", [x, y], D.F32, (4, 12, 8), attr=[1, 0]))   # a real concatenation is not lowered
-    assert status(g) == -3
+    g.mark_output(g.op("cat", [x, y], D.F32, (4, 12, 8), attr=[1, 0]))   # a concatenation of two inputs: each stored into its block
+    assert status(g, 0) == 0
+    g = GraphBuilder(); x = g.input(D.F32, (4, 6, 8)); y = g.input(D.F32, (4, 5, 8))
+    g.mark_output(g.op("cat", [x, y], D.F32, (4, 12, 8), attr=[1, 0]))   # 6 + 5 is not 12
+    assert status(g, 0) == -4
 
 
 def test_checked_accessors_are_compiled_in_only_on_request():
