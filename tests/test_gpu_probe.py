@@ -65,3 +65,16 @@ def test_probe_rejects_bad_configurations():
     with pytest.raises(B.PnError) as e:
         B.stream_probe(B.MIX_1_1, B.ProbeConfig(0, 0, 0, 128, 1, 1, 0, 0), p + 4, p, p, p, 4, p, 0)
     assert e.value.status == -6
+
+
+def test_probe_command_line(capsys):
+    """`python -m paper_2605_29357_b200.probe`: every mix and access pattern runs, the bounded waits
+    of the bulk loader never run out, and a streaming read is far above anything a broken grid gives."""
+    import json
+    from paper_2605_29357_b200 import probe
+    assert probe.main(["--mb", "64", "--reps", "3"]) == 0
+    out = json.loads(capsys.readouterr().out)
+    assert out["status_word"] == 0
+    assert set(out["mixes"]) == {"read", "write", "1:1", "2:1", "4:3"}
+    assert len(out["read_patterns"]) >= 20 and all(v > 100 for v in out["read_patterns"].values())
+    assert out["mixes"]["read"]["gbs"] > 1000
