@@ -119,7 +119,8 @@ enum {
                                      instead of being cut into several fused launches          */
   PN_FLAG_FORCE_SPLIT = 1u << 15, /* row kernels: independent blocks over slices of a row, combined
                                      through partials in a workspace of the handle (single-stage
-                                     graphs, generated kernels)                               */
+                                     graphs, generated kernels); kernels that reduce over a
+                                     leading dimension: at least two slices of that dimension  */
   PN_FLAG_ALLOW_INTERPRET = 1u << 14,/* a create that cannot specialise kernels (NVRTC or the driver
                                      library cannot be opened) normally fails with PN_ERR_DEVICE;
                                      with this flag it runs on the interpreter kernels instead  */
@@ -133,7 +134,9 @@ enum {
 #define PN_STATIC_SCRATCH_BYTES (32ll << 20)
 /* Tuning overrides of the lowering's own choices, for measurements and tests: OR them into
  * `flags`.  A value of 0 leaves the choice to the lowering; an impossible one is ignored. */
-#define PN_TUNE_CLUSTER(n) (((unsigned)(n) & 15u) << 16)      /* CTAs per cluster: 2, 4, 8      */
+#define PN_TUNE_CLUSTER(n) (((unsigned)(n) & 15u) << 16)      /* CTAs per cluster: 2, 4, 8; split-row kernels: tiles per
+                                                                 slice; column-reduce kernels: slices of the reduced
+                                                                 dimension (2..15)                */
 #define PN_TUNE_BLOCK_LOG2(n) (((unsigned)(n) & 15u) << 20)   /* threads per block = 1 << n     */
 #define PN_TUNE_GROUPS(n) (((unsigned)(n) & 31u) << 24)       /* vector groups per thread tile  */
 #define PN_TUNE_WAVES(n) (((unsigned)(n) & 7u) << 29)         /* grid <= 2^(n-1) x the resident CTAs; 7: one CTA per work item */
@@ -153,13 +156,14 @@ enum {
                                waits for the device                                        */
   PN_Q_KERNEL_CACHE = 11,   /* 2 values, process-wide: generated kernels now loaded, and how many of
                                them a live handle uses                                      */
-  PN_Q_KERNEL_INFO = 9      /* per kernel 13 values: family (0 pointwise, 1 warp-per-row,
+  PN_Q_KERNEL_INFO = 9      /* per kernel 14 values: family (0 pointwise, 1 warp-per-row,
                                2 block-per-row, 3 cluster-per-row, 5 split-row, 4 column-reduce: rows =
                                the dimensions before the reduced one, row length = those after
                                it), grid, block, cluster,
                                dynamic smem bytes, vector length, groups per tile, chunks
                                per row slice, bytecode words, stages, rows, row length,
-                               specialised (1) or interpreted (0)                        */
+                               specialised (1) or interpreted (0), slices (split-row: of a row;
+                               column-reduce: of the reduced dimension; else 0)          */
 };
 
 /*
@@ -208,8 +212,8 @@ pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsig
  * read-only data path, which does not see a kernel's own writes.  The library never retains or
  * frees user memory.  The handle itself is only read, so runs of one fused handle may be issued
  * from several threads and streams at once; runs of a handle that has a workspace
- * (PN_Q_WORKSPACE_BYTES > 0: unfused handles, graphs cut into several launches, rows split over
- * independent blocks) share that workspace and must be stream-ordered by the caller.  The launch
+ * (PN_Q_WORKSPACE_BYTES > 0: unfused handles, graphs cut into several launches, rows or a reduced
+ * leading dimension split over independent blocks) share that workspace and must be stream-ordered by the caller.  The launch
  * goes to the handle's device whatever device the calling thread has current, and that choice
  * is left as it was.  A graph any of whose inputs or outputs has zero elements runs as a no-op.
  */

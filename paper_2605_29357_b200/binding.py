@@ -193,10 +193,10 @@ class Graph:
     @property
     def kernel_info(self) -> List[dict]:
         n = self.n_kernels
-        v = self._query(Q_KERNEL_INFO, 13 * n)
+        v = self._query(Q_KERNEL_INFO, 14 * n)
         keys = ["family", "grid", "block", "cluster", "smem_bytes", "vl", "ng", "chunks",
-                "code_words", "stages", "rows", "row_len", "specialised"]
-        return [dict(zip(keys, v[13 * i: 13 * i + 13])) for i in range(n)]
+                "code_words", "stages", "rows", "row_len", "specialised", "slices"]
+        return [dict(zip(keys, v[14 * i: 14 * i + 14])) for i in range(n)]
 
     def codegen(self, kernel: int = 0, compile: bool = False) -> str:
         """Generated CUDA source of one launch; with compile=True also compiled by NVRTC."""

@@ -451,21 +451,30 @@ pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsig
   // split-row launches: partials and arrival counters in device memory of the handle, the counters
   // zero at rest
   {
+    auto uses_tickets = [](const LaunchPlan& lp) { return lp.family == FAM_SPLIT || (lp.family == FAM_COLUMN && lp.p.splits > 1); };
     auto sizes = [](const LaunchPlan& lp, size_t& part_bytes, size_t& ticket_bytes) {
       const KernelParams& P = lp.p;
-      part_bytes = ((size_t)P.rows * P.splits * P.stage[0].n_red * 3 * sizeof(float) + 255) / 256 * 256;
-      ticket_bytes = ((size_t)P.rows * sizeof(uint32_t) + 255) / 256 * 256;
+      if (lp.family == FAM_SPLIT) {   // a partial (three floats) per reduction, slice and row; a counter per row
+        part_bytes = (size_t)P.rows * P.splits * P.stage[0].n_red * 3 * sizeof(float);
+        ticket_bytes = (size_t)P.rows * sizeof(uint32_t);
+      } else {                        // column family: the accumulators of a column tile per slice; a counter per item
+        const size_t items = (size_t)P.rows * P.chunks;
+        part_bytes = items * P.splits * P.stage[0].n_red * ((size_t)P.col_tx * lp.vl * lp.ng) * sizeof(float);
+        ticket_bytes = items * sizeof(uint32_t);
+      }
+      part_bytes = (part_bytes + 255) / 256 * 256;
+      ticket_bytes = (ticket_bytes + 255) / 256 * 256;
     };
     size_t need = 0;
     for (PlannedLaunch& pl : h->launches)
-      if (pl.plan.family == FAM_SPLIT) { size_t a = 0, b = 0; sizes(pl.plan, a, b); need += a + b; }
+      if (uses_tickets(pl.plan)) { size_t a = 0, b = 0; sizes(pl.plan, a, b); need += a + b; }
     if (need > 0 && !h->plan_only) {
       cudaError_t e = cudaMalloc(&h->split_ws, need);
       if (e == cudaSuccess) e = cudaMemset(h->split_ws, 0, need);
       if (e != cudaSuccess) { pn_graph_destroy(h); return fail(PN_ERR_CUDA, std::string("split-row workspace: ") + cudaGetErrorString(e)); }
       size_t off = 0;
       for (PlannedLaunch& pl : h->launches)
-        if (pl.plan.family == FAM_SPLIT) {
+        if (uses_tickets(pl.plan)) {
           size_t a = 0, b = 0;
           sizes(pl.plan, a, b);
           pl.plan.p.split_part = reinterpret_cast<float*>((char*)h->split_ws + off); off += a;
@@ -565,7 +574,7 @@ pn_status pn_graph_run_host(pn_graph_t* h, const void* const* inputs, int n_inpu
   if (h->launches.size() == 1 && in_bytes >= (8ll << 20)) {
     const LaunchPlan& lp = h->launches[0].plan;
     const KernelParams& P = lp.p;
-    bool ok = P.cluster >= 1 && P.family != FAM_SPLIT;
+    bool ok = P.cluster >= 1 && P.family != FAM_SPLIT && P.splits <= 1;   // (kernels with arrival counters run whole)
     for (int q = 0; q < P.n_io; ++q) ok = ok && !P.io[q].mapped;
     cut.stride.assign(P.n_io, 0);
     if (ok && P.family == FAM_COLUMN) {
@@ -707,9 +716,9 @@ pn_status pn_graph_query(const pn_graph_t* h, int what, void* out, size_t out_by
     case PN_Q_KERNEL_INFO:
       for (const PlannedLaunch& pl : h->launches) {
         const LaunchPlan& p = pl.plan;
-        const int64_t row[13] = {p.family, p.grid, p.block, p.p.cluster, p.smem_bytes, p.vl, p.ng, p.p.chunks,
-                                 p.code_words, p.p.n_stages, p.p.rows, p.p.row_len, p.specialised};
-        v.insert(v.end(), row, row + 13);
+        const int64_t row[14] = {p.family, p.grid, p.block, p.p.cluster, p.smem_bytes, p.vl, p.ng, p.p.chunks,
+                                 p.code_words, p.p.n_stages, p.p.rows, p.p.row_len, p.specialised, p.p.splits};
+        v.insert(v.end(), row, row + 14);
       }
       break;
     case PN_Q_BOUNDS_STATUS: {

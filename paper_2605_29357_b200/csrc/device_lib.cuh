@@ -1291,6 +1291,14 @@ PN_DEV void split_body(const KernelParams& p, unsigned char* smem) {
 // ty = 0 thread, in the fixed order ty = 0, 1, ..., so results repeat bit for bit; that thread
 // runs the stage-1 program (the epilogue on the reduced values) and stores.  Every input element
 // is read once.  Hand-offs are __syncthreads only.
+//
+// With p.splits > 1 the reduced dimension itself is cut into that many slices, one work item per
+// (row, column tile, slice): what fills the GPU when a graph has few columns and a long reduced
+// dimension.  As in the split-row family nobody waits: a block leaves the combined accumulators of
+// its slice in device memory (split_part, [item][slice][reduction][element][tx]), fences, and takes
+// a ticket on the item's counter; the block that draws the item's last ticket reads all slices back
+// in slice order (its own included, so the order of the combine never depends on who is last), runs
+// the epilogue, stores, and puts the counter back to zero.
 template <class Prog>
 PN_DEV void column_body(const KernelParams& p, unsigned char* smem) {
   constexpr int VL = Prog::VL, NG = Prog::NG, K = Prog::K, V = VL * NG;
@@ -1327,8 +1335,13 @@ PN_DEV void column_body(const KernelParams& p, unsigned char* smem) {
   PN_UNROLL for (int u = 0; u < U; ++u) { PN_UNROLL for (int j = 0; j < (kPf > 0 ? kPf : 1); ++j) { PN_UNROLL for (int e = 0; e < V; ++e) raw[u][j][e] = 0.f; } }
   PN_UNROLL for (int r = 0; r < kMaxRed; ++r) parts[r] = Part{0.f, 0.f, 0.f};
 
-  const long long n_items = p.item_end > 0 ? p.item_end : p.rows * n_ctiles;
-  for (long long item = (p.item_end > 0 ? p.item_begin : 0) + blockIdx.x; item < n_items; item += gridDim.x) {
+  const int S = Prog::splits(p) > 1 ? Prog::splits(p) : 1;   // slices of the reduced dimension
+  const int Rs = (R + S - 1) / S;
+  const long long n_items = (p.item_end > 0 ? p.item_end : p.rows * n_ctiles) * S;
+  for (long long it = (p.item_end > 0 ? p.item_begin : 0) * S + blockIdx.x; it < n_items; it += gridDim.x) {
+    const long long item = it / S;
+    const int split = (int)(it - item * S);
+    const int s_lo = split * Rs, s_hi = min(R, s_lo + Rs);
     const long long o = item / n_ctiles;
     const int ct = (int)(item - o * n_ctiles);
     cx.col0 = ct * (TX * V) + tx * VL;
@@ -1347,18 +1360,18 @@ PN_DEV void column_body(const KernelParams& p, unsigned char* smem) {
       // U steps at a time: all their loads are issued, then their arithmetic runs in step order.
       // (Measured on B200: issuing the next batch before the arithmetic of the current one costs
       // more in registers, hence resident warps, than it gains.)
-      for (int s0 = ty; s0 < R; s0 += U * TY) {
+      for (int s0 = s_lo + ty; s0 < s_hi; s0 += U * TY) {
         PN_UNROLL for (int u = 0; u < U; ++u) {
           const int s = s0 + u * TY;
-          if (s < R) { at_step(s); Prog::prefetch(p, cx, raw[u]); }
+          if (s < s_hi) { at_step(s); Prog::prefetch(p, cx, raw[u]); }
         }
         PN_UNROLL for (int u = 0; u < U; ++u) {
           const int s = s0 + u * TY;
-          if (s < R) { at_step(s); Prog::tile(p, 0, cx, acc, reg, ts, parts, raw[u], cx, false); }
+          if (s < s_hi) { at_step(s); Prog::tile(p, 0, cx, acc, reg, ts, parts, raw[u], cx, false); }
         }
       }
     } else {
-      for (int s = ty; s < R; s += TY) {
+      for (int s = s_lo + ty; s < s_hi; s += TY) {
         at_step(s);
         Prog::tile(p, 0, cx, acc, reg, ts, parts, raw[0], cx, false);
       }
@@ -1385,7 +1398,43 @@ PN_DEV void column_body(const KernelParams& p, unsigned char* smem) {
         }
       }
     }
-    if (ty == 0) {
+    bool finish = ty == 0;
+    if (S > 1 && tid < 32) {   // the ty = 0 threads are the first TX (<= 32) threads of the block
+      const size_t slice_floats = (size_t)n_red * V * TX;
+      if (ty == 0) {
+        float* mine = p.split_part + (size_t)it * slice_floats;
+        PN_UNROLL for (int r = 0; r < kAcc; ++r) {
+          if (r < n_red) { PN_UNROLL for (int e = 0; e < V; ++e) mine[(r * V + e) * TX + tx] = reg[r][e]; }
+        }
+        __threadfence();                               // the slice is visible before the ticket is
+      }
+      __syncwarp();
+      unsigned ticket = 0;
+      if (tid == 0) ticket = atomicAdd(p.split_ticket + item, 1u);
+      ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
+      finish = finish && ticket == (unsigned)(S - 1);
+      if (finish) {   // the item's last block: every other slice has been written
+        __threadfence();
+        const float* all = p.split_part + (size_t)item * S * slice_floats;
+        PN_UNROLL for (int r = 0; r < kAcc; ++r) {
+          if (r < n_red) {
+            const int kind = Prog::red_kind(p, 0, r);
+            PN_UNROLL for (int e = 0; e < V; ++e) {
+              const float* col = all + (r * V + e) * TX + tx;
+              float v = ld_cg(col);
+              for (int s1 = 1; s1 < S; s1 += 4) {        // four slices' loads together, combined in slice order
+                float q4[4];
+                PN_UNROLL for (int u = 0; u < 4; ++u) q4[u] = s1 + u < S ? ld_cg(col + (size_t)(s1 + u) * slice_floats) : 0.f;
+                PN_UNROLL for (int u = 0; u < 4; ++u) { if (s1 + u < S) v = accum_combine(kind, v, q4[u]); }
+              }
+              reg[r][e] = v;
+            }
+          }
+        }
+        if (tid == 0) p.split_ticket[item] = 0u;       // ready for the next launch
+      }
+    }
+    if (finish) {
       PN_UNROLL for (int q = 0; q < Prog::kNumIo; ++q) rowoff[q] = item_off[q];
       Prog::tile(p, 1, cx, acc, reg, ts, parts, raw[0], cx, false);
     }

@@ -321,18 +321,40 @@ int lower_column_graph(const Graph& g, unsigned flags, const DeviceModel& dev, L
   while (TX < 32 && (int64_t)TX * VL * NG < C) TX *= 2;
   // Few (row, column tile) items for the size of the GPU: more walkers per item first (blocks of up
   // to 512 threads, while every walker keeps a batch of steps), then narrower column tiles (down to
-  // 8 threads: 128 contiguous bytes per step and item), then blocks of 1024.  This is what keeps a
-  // small batch of long sequences from running on a handful of SMs.
-  if (spec && !t_block) {
+  // 8 threads: 128 contiguous bytes per step and item), then slices of the reduced dimension itself
+  // -- a block per (item, slice), combined by the block that arrives last; partials and arrival
+  // counters live in a workspace of the handle, so not for handles that may not have one -- and only
+  // then blocks of 1024.  This is what keeps a small batch of long sequences, or a few columns under
+  // a very long reduced dimension, from running on a handful of SMs.  Measured on B200 (bf16 sums,
+  // L2-cold): [1,1M,8] 43.8 -> 26.6 us, [4,16384,64] 12.3 -> 10.3, [1,8192,4096] 24.1 -> 16.4;
+  // slices where blocks of 512 already fill the GPU only cost ([64,512,1024] 14.4 -> 18.0 with two).
+  // PN_TUNE_CLUSTER(n) asks for n slices, PN_FLAG_FORCE_SPLIT for at least two.
+  const bool may_slice = !(flags & PN_FLAG_STATIC_SCRATCH);
+  const int t_slices = may_slice ? (int)((flags >> 16) & 15) : 0;   // PN_TUNE_CLUSTER on a column kernel
+  int splits = 1;
+  if (spec && !t_block && t_slices <= 1) {
     const int64_t want = (int64_t)dev.sm_count * 512;   // threads for a quarter of the resident capacity
     auto threads = [&](int tx, int blk) { return O * ((C + (int64_t)tx * VL * NG - 1) / ((int64_t)tx * VL * NG)) * blk; };
     auto steps_ok = [&](int tx, int blk) { return R / (blk / tx) >= 8; };
     while (threads(TX, block) < want && block < 512 && steps_ok(TX, block * 2)) block *= 2;
     while (threads(TX, block) < want && TX > 8 && (int64_t)(TX / 2) * VL * NG * 2 <= C * 2 && steps_ok(TX / 2, block)) TX /= 2;
-    while (threads(TX, block) < want && block < 1024 && steps_ok(TX, block * 2)) block *= 2;
+    if (may_slice && threads(TX, block) < want) {
+      const int64_t per_walker = R / (block / TX);      // steps a walker takes over the whole of R
+      int64_t s = 1;
+      while (s * threads(TX, block) < want) s *= 2;     // (a power of two: [1,8192,4096] 18.5 us in 3 slices, 16.4 in 4)
+      s = std::min<int64_t>(std::min<int64_t>(s, per_walker / 8), 64);
+      if (s >= 2) splits = (int)s;
+    }
+    while (splits == 1 && threads(TX, block) < want && block < 1024 && steps_ok(TX, block * 2)) block *= 2;
   }
   const int64_t ctile = (int64_t)TX * VL * NG;
   const int64_t n_ctiles = (C + ctile - 1) / ctile;
+  if (may_slice) {
+    const int64_t per_walker = std::max<int64_t>(1, R / (block / TX));
+    if (t_slices > 1) splits = (int)std::min<int64_t>(t_slices, per_walker);
+    if ((flags & PN_FLAG_FORCE_SPLIT) && splits < 2 && per_walker >= 2) splits = 2;
+    if (splits < 2 || O * n_ctiles * splits > (int64_t(1) << 30)) splits = 1;
+  } else splits = 1;
 
   // ---- (4) code generation ----------------------------------------------------------------------
   std::vector<uint32_t> code;
@@ -372,10 +394,11 @@ int lower_column_graph(const Graph& g, unsigned flags, const DeviceModel& dev, L
   P.split_chunks = 0;
   P.cluster = 1;
   P.col_tx = TX;
+  P.splits = splits > 1 ? splits : 0;
   P.family = FAM_COLUMN;
   lp.family = FAM_COLUMN; lp.vl = VL; lp.ng = NG; lp.k = K;
   lp.block = block; lp.smem_bytes = off; lp.code_words = (int)code.size();
-  lp.items = O * n_ctiles;
+  lp.items = O * n_ctiles * (splits > 1 ? splits : 1);
   lp.teams_per_cta = 1;
   // generated kernels issue the loads of several steps of the walk before the arithmetic of the first
   lp.specialised = 0; lp.persistent = 0; lp.grid_waves = tune_waves(flags); lp.no_prefetch = (flags & PN_FLAG_NO_HOIST) ? 1 : 0;

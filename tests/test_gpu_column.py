@@ -163,3 +163,65 @@ def test_values_before_and_after_the_reduction(flags):
     gr, _ = _run(g, [x, w, c, bias, scale], flags)
     if not flags & pn.FLAG_UNFUSED:
         assert gr.n_kernels == 1
+
+
+SLICED = {
+    "default": 0,
+    "two": pn.FLAG_FORCE_SPLIT,
+    "three": pn.tune(cluster=3),
+    "fifteen": pn.tune(cluster=15),
+    "five_block64": pn.tune(cluster=5, block=64),
+    "interpret_four": pn.FLAG_INTERPRET | pn.tune(cluster=4),
+    "scalar_two": pn.FLAG_FORCE_SCALAR | pn.FLAG_FORCE_SPLIT,
+    "bounds_seven": pn.FLAG_BOUNDS | pn.tune(cluster=7),
+}
+
+
+@pytest.mark.parametrize("force", list(SLICED))
+@pytest.mark.parametrize("shape,dim", [((1, 5000, 40), 1), ((3, 2500, 7), 1), ((4099, 24), 0), ((2, 700, 3, 16), 1),
+                                       ((2, 129, 1), 1), ((1, 64, 300), 1), ((1, 65536, 64), 1)])
+def test_reduced_dimension_cut_into_slices(shape, dim, force):
+    """Few columns under a long reduced dimension: blocks over slices of that dimension, combined by
+    whichever block arrives last, in slice order.  Sums of quarters are exact in fp32, so they also
+    judge that every step is folded exactly once; extremes judge the identity of empty slices."""
+    flags = SLICED[force]
+    x = _quarters(shape, 40 + dim + len(shape))
+    drop = shape[:dim] + shape[dim + 1:]
+    for ops in (("sum_dim", "amax_dim"), ("mean_dim", "amin_dim")):
+        g = GraphBuilder(); xi = g.input(D.F32, shape)
+        t = g.op("mul", [xi, Imm(0.5)], D.F32, shape)
+        outs_t = [g.op(op, [t], D.F32, drop, attr=[dim, 0]) for op in ops]
+        for o in outs_t:
+            g.mark_output(o)
+        g.mark_output(g.op("sub", outs_t, D.F32, drop))           # an epilogue on the combined values
+        gr, outs = _run(g, [x], flags)
+        info = gr.kernel_info[0]
+        assert gr.n_kernels == 1 and pn.FAMILY_NAMES[info["family"]] == "column-reduce"
+        R = shape[dim]
+        if force != "default":
+            want = {"two": 2, "three": 3, "fifteen": 15, "five_block64": 5, "interpret_four": 4, "scalar_two": 2, "bounds_seven": 7}[force]
+            at_least = "two" in force                                 # PN_FLAG_FORCE_SPLIT: two or whatever the lowering wants
+            assert at_least or 0 <= info["slices"] <= want
+            if R >= 2048:
+                assert (info["slices"] >= want if at_least else info["slices"] == want) and gr.workspace_bytes > 0
+        elif shape == (1, 65536, 64):
+            assert info["slices"] > 8                                 # the lowering's own choice fills the GPU
+        if ops[0] == "sum_dim":
+            assert np.array_equal(outs[0], (x.astype(np.float64) * 0.5).sum(axis=dim).astype(np.float32))
+        again = run_graph(gr, [x])                                    # counters back at zero; same bits
+        for a, b in zip(outs, again):
+            assert np.array_equal(a, b)
+        if flags & pn.FLAG_BOUNDS:
+            assert gr.bounds_status == 0
+
+
+def test_masked_mean_pooling_in_slices():
+    """The pooling subgraph of the second case study with a small batch of long sequences, the
+    sequence dimension cut into slices: the mask count (a reduction carried by one element of the
+    tile) and the masked sum go through the same partials."""
+    w = C.n2(B=2, S=4096, Dh=256)
+    for flags in (0, pn.tune(cluster=6), pn.FLAG_INTERPRET | pn.FLAG_FORCE_SPLIT):
+        g = pn.Graph(w.desc, 0, flags)
+        outs = run_graph(g, w.inputs)
+        check_against_oracle(w.desc, w.inputs, outs, w.output_meta, w.output_names)
+        assert g.n_kernels == 1 and g.kernel_info[0]["slices"] >= 2
