@@ -13,8 +13,11 @@ weak and the value is the sum over ranks divided by the slowest rank's time.
 One JSON line is printed by rank 0.  Beside the base keys it carries `roofline` (the fused
 kernel against the measured HBM copy rate), `e2e` (the same metric through
 pn_graph_run_host on pinned host buffers, copies inside the timed region),
-`cpu_baseline` (the CPU oracle timed on a bounded sample of the same workload) and, at
-N = 1 unless --no-sweep, `sweep`: the other four benchmark subgraphs, fused and unfused.
+`cpu_baseline` (the CPU oracle timed over the host's cores on the same workload) and, at
+N = 1 unless --no-sweep, `mix_peaks` (the stream probe's ceilings), `sweep` (the other six
+subgraphs, fused and unfused, each with its own roofline object), `tiny_graphs` (launch latency
+of many small subgraphs) and `create_ms` (what creating a handle costs, with and without the
+kernel caches).  With --gpus N > 1 and no launcher around it, the script starts its own N ranks.
 
 --impl reference times the CPU oracle itself, as it stands, on the host cores.
 """
@@ -168,9 +171,13 @@ def time_graph(torch, g, sets, steps, warmup, flush=None):
 
 
 def time_host_launched(torch, g, sets, steps, warmup):
-    """K launches through bound launch objects (pn_bound_run: one launch call each) rotating over the
+    """Launches through bound launch objects (pn_bound_run: one launch call each) rotating over the
     buffer sets, one pair of events around all of them: what a caller who launches from the host
-    pays per launch, without an event record between the launches.  Returns ms per launch."""
+    pays per launch, without an event record between the launches.  At least 2000 launches: host
+    and device run at nearly the same rate here (an empty kernel takes 2.9 us per launch on the
+    same box), so a short run measures the start of the queue rather than its steady state.
+    Returns ms per launch."""
+    steps = max(steps, 2000)
     stream = torch.cuda.current_stream()
     launch = [g.bind([t.data_ptr() for t in a], [t.data_ptr() for t in b]) for a, b in sets]
     for i in range(max(warmup, 3)):
@@ -334,7 +341,7 @@ def roofline_entry(cbytes, seconds, peak, peak_src, mix, probe, small):
 def tiny_graph_latency(torch, pn, device, passes, repeats=8):
     """Latency of many small subgraphs run back to back (the regime where the paper finds fixed
     per-call overhead decisive): the reduced-size graphs of every workload, `repeats` instances
-    each on their own buffers, (a) launched one by one from the host with pn_graph_run,
+    each on their own buffers, (a) launched one by one from the host through bound launches (pn_bound_run),
     (b) recorded once as a sequence and replayed in order, (c) the same as independent items.
     Returns microseconds per subgraph for each; the inputs are L2-resident, so this is launch
     and latency, not bandwidth."""
@@ -377,6 +384,32 @@ def tiny_graph_latency(torch, pn, device, passes, repeats=8):
     for g in graphs.values():
         g.close()
     return out
+
+
+def create_times(device):
+    """What pn_graph_create costs, on the unfused handle of the gated multi-output graph (13 nodes, a
+    kernel each, every one compiled by NVRTC): in a fresh process with an empty on-disk kernel cache
+    (PN_CACHE_DIR), a second time in that process (the process-wide kernel cache), and in another
+    fresh process that finds the cubins on disk.  Milliseconds.  The processes load only the
+    library, not torch."""
+    import tempfile
+    code = ("import json, time\nimport paper_2605_29357_b200 as pn\nfrom pn_workloads import configs as C\n"
+            "w = C.c5(**C.SMALL['c5'])\nout = []\n"
+            "for _ in range(2):\n"
+            "    t0 = time.perf_counter(); g = pn.Graph(w.desc, %d, pn.FLAG_UNFUSED); out.append((time.perf_counter() - t0) * 1e3)\n"
+            "    n = g.n_kernels\n"
+            "print(json.dumps({'ms': out, 'kernels': n, 'cache': list(g.kernel_cache)}))\n" % device)
+    with tempfile.TemporaryDirectory() as d:
+        env = dict(os.environ, PN_CACHE_DIR=d, PYTHONPATH=ROOT + os.pathsep + os.environ.get("PYTHONPATH", ""))
+        runs = []
+        for _ in range(2):
+            r = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=300, cwd=ROOT)
+            if r.returncode != 0:
+                return {"error": (r.stderr or r.stdout).strip()[-300:]}
+            runs.append(json.loads(r.stdout.strip().splitlines()[-1]))
+        files = len(os.listdir(d))
+    return {"graph": "c5 unfused", "kernels": runs[0]["kernels"], "compiled_ms": runs[0]["ms"][0], "again_in_process_ms": runs[0]["ms"][1],
+            "from_disk_cache_ms": runs[1]["ms"][0], "cubins_on_disk": files}
 
 
 def rank_workload(name, rank, **size):
@@ -722,6 +755,7 @@ def main():
         line["sweep"] = sweep
         line["probe_status_word"] = probe.status_word()
         line["tiny_graphs"] = tiny_graph_latency(torch, pn, local_rank, max(10, args.steps // 2))
+        line["create_ms"] = create_times(local_rank)
 
     # ---- the CPU oracle on a bounded sample of the same workload ------------------------------
     # the whole benchmark batch (512 batches of the softmax workload), 8 batches per job over a pool

@@ -46,10 +46,15 @@
  * value cannot flow back into a tensor that still has the reduced dimension.
  * Index operators (the index-remapped loads of the paper's first case study, Section 4.4): 160
  * roll (attr = dim, shift), 161 slice (attr = dim, start; length from the output shape), 162 view
- * (regroups leading dimensions).  A roll or slice over two dimensions at once, as graph traces have
- * them, gives the second one in imm = (1 + dim, shift / start); imm[0] = 0 means one dimension.  They act on leading dimensions of graph inputs, or of chains of
- * index operators that start at one, and cost no data movement: the fused kernel computes the
- * source row instead (idx = (S + i - shift) mod S).  164 contiguous: the identity on values (every
+ * (regroups leading dimensions; of a tensor that is still dense, any dimensions).  A roll or slice
+ * over two dimensions at once, as graph traces have them, gives the second one in
+ * imm = (1 + dim, shift / start); imm[0] = 0 means one dimension.  They act on any dimension of
+ * graph inputs, or of chains of index operators that start at one, and cost no data movement: the
+ * fused kernel computes the source row instead (idx = (S + i - shift) mod S); along the last
+ * dimension a slice is an offset of the row's start and a roll a circular shift of the columns
+ * (whole 128-bit groups when shift and row length allow it, element by element otherwise), so the
+ * two halves of a gated activation are two views of one input.  On a computed value an index
+ * operator starts a launch of its own.  164 contiguous: the identity on values (every
  * tensor here is dense already); after a chain of index operators it is one more link of the chain,
  * on a computed value a pointwise identity.  163 cat (attr[0] = dim, up to 4 operands of the
  * result's dtype): with one operand it is the identity, as graph traces contain it; with several it

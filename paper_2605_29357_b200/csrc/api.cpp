@@ -300,6 +300,7 @@ pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsig
   h->n_nodes = (int)h->g.nodes.size();
   st = expand_concatenations(h->g, err);   // a cat of several operands becomes stores into blocks of its result
   if (st != PN_OK) { delete h; return fail(st, err); }
+  prune_dead_nodes(h->g);                  // what reaches no output is not part of f_G
   if ((flags & PN_FLAG_BOUNDS) && (flags & PN_FLAG_STATIC_SCRATCH)) { delete h; return fail(PN_ERR_INVALID_ARG, "PN_FLAG_BOUNDS allocates a status word: it cannot be combined with PN_FLAG_STATIC_SCRATCH"); }
   h->flags = flags;
   h->device = device;
@@ -403,7 +404,7 @@ pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsig
     if (st != PN_OK) { delete h; return fail(st, err); }
     for (int q = 0; q < pl.plan.p.n_io; ++q) {
       int t = orig[pl.plan.io_tensor[q]];
-      pl.plan.p.io[q].numel = g.tensors[t].numel();
+      pl.plan.p.io[q].numel = g.tensors[t].numel() - (pl.plan.io_is_output[q] ? 0 : pl.plan.io_offset[q]);   // (an input sliced along the last dimension starts later)
       if (pl.plan.io_is_output[q] && g.tensors[t].embed_parent >= 0) {   // a part of a cat result: stored inside it
         t = g.tensors[t].embed_parent;
         pl.plan.p.io[q].numel = g.tensors[t].numel() - pl.plan.io_offset[q];

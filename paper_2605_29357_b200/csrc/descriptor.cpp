@@ -151,4 +151,54 @@ int expand_concatenations(Graph& g, std::string& err) {
   return PN_OK;
 }
 
+// Nodes whose results reach no graph output take no part in f_G: they are dropped before any
+// lowering (fused, they would cost nothing anyway; as a launch of their own they would have
+// nothing to store).  A part of a cat result counts as used when the result is.
+void prune_dead_nodes(Graph& g) {
+  std::vector<char> used(g.tensors.size(), 0);
+  for (size_t t = 0; t < g.tensors.size(); ++t) used[t] = (g.tensors[t].role & 2) != 0;
+  std::vector<char> live(g.nodes.size(), 0);
+  for (int pass = 0; pass < 2; ++pass)   // (a second pass: a cat result read by a node listed before its parts' stores)
+    for (int ni = (int)g.nodes.size() - 1; ni >= 0; --ni) {
+      const Node& n = g.nodes[ni];
+      bool need = false;
+      for (int k = 0; k < n.n_out; ++k) {
+        const Tensor& T = g.tensors[n.out[k]];
+        need = need || used[n.out[k]] || (T.embed_parent >= 0 && used[T.embed_parent]);
+      }
+      if (!need) continue;
+      live[ni] = 1;
+      for (int k = 0; k < n.n_in; ++k) if (n.in[k] < g.tensors.size()) used[n.in[k]] = 1;
+    }
+  bool all = true;
+  for (char c : live) all = all && c;
+  if (all) return;
+  std::vector<Node> nodes;
+  for (size_t ni = 0; ni < g.nodes.size(); ++ni) if (live[ni]) nodes.push_back(g.nodes[ni]);
+  g.nodes.swap(nodes);
+  // the tensors only dead nodes touched leave the table too (the lowering looks at every tensor)
+  std::vector<char> keep(g.tensors.size(), 0);
+  for (size_t t = 0; t < g.tensors.size(); ++t) keep[t] = g.tensors[t].role != 0;
+  for (const Node& n : g.nodes) {
+    for (int k = 0; k < n.n_in; ++k) if (n.in[k] < g.tensors.size()) keep[n.in[k]] = 1;
+    for (int k = 0; k < n.n_out; ++k) {
+      keep[n.out[k]] = 1;
+      if (g.tensors[n.out[k]].embed_parent >= 0) keep[g.tensors[n.out[k]].embed_parent] = 1;
+    }
+  }
+  std::vector<int> new_id(g.tensors.size(), -1);
+  std::vector<Tensor> tensors;
+  for (size_t t = 0; t < g.tensors.size(); ++t)
+    if (keep[t]) { new_id[t] = (int)tensors.size(); tensors.push_back(g.tensors[t]); }
+  for (Tensor& T : tensors) { T.producer = -1; if (T.embed_parent >= 0) T.embed_parent = new_id[T.embed_parent]; }
+  g.tensors.swap(tensors);
+  for (size_t ni = 0; ni < g.nodes.size(); ++ni) {
+    Node& n = g.nodes[ni];
+    for (int k = 0; k < n.n_in; ++k) if (n.in[k] < new_id.size()) n.in[k] = (uint32_t)new_id[n.in[k]];
+    for (int k = 0; k < n.n_out; ++k) { n.out[k] = (uint32_t)new_id[n.out[k]]; g.tensors[n.out[k]].producer = (int)ni; }
+  }
+  for (int& t : g.inputs) t = new_id[t];
+  for (int& t : g.outputs) t = new_id[t];
+}
+
 }  // namespace pn

@@ -462,14 +462,19 @@ struct TileCtx {
 };
 
 // FULL: every group of every tile lies inside the row (no validity tests needed).
-template <int VL, int NG, bool FULL = false>
+// ROLL: the input is rolled along the last dimension, column c is read at (c + col_add) mod col_mod
+// (both multiples of VL, so a group never straddles the wrap); 0 no, 1 yes, 2 ask the descriptor.
+template <int VL, int NG, bool FULL = false, int ROLL = 2>
 PN_DEV void op_ldraw(const KernelParams& p, const TileCtx& cx, int io, int dt, float (&r)[VL * NG]) {
   const char* base = static_cast<const char*>(p.io[io].base);
   const long long off = cx.rowoff[io];
+  const int wrap = ROLL == 0 ? 0 : p.io[io].col_mod;
   PN_UNROLL for (int j = 0; j < NG; ++j) {
     const int col = cx.col0 + j * cx.gstride;
-    if ((FULL || col < cx.col_end) && in_bounds(p, io, off + col, VL)) {
-      load_group_raw<VL>(base, off + col, dt, &r[j * VL]);
+    int src = col;
+    if (ROLL != 0 && wrap != 0) { src += p.io[io].col_add; if (src >= wrap) src -= wrap; }
+    if ((FULL || col < cx.col_end) && in_bounds(p, io, off + src, VL)) {
+      load_group_raw<VL>(base, off + src, dt, &r[j * VL]);
     } else {
       PN_UNROLL for (int i = 0; i < VL; ++i) r[j * VL + i] = 0.f;
     }

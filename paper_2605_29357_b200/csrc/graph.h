@@ -74,6 +74,9 @@ int parse_descriptor(const void* desc, size_t bytes, Graph& g, std::string& err)
 // embedded in the cat's output (see Tensor::embed_parent).  Returns a pn_status value.
 int expand_concatenations(Graph& g, std::string& err);
 
+// Drops the nodes whose results reach no graph output (after expand_concatenations).
+void prune_dead_nodes(Graph& g);
+
 struct DeviceModel {      // what the lowering needs to know about the GPU
   int sm_count = 148;
   int max_smem_per_block = 227 * 1024;

@@ -76,6 +76,8 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     int root = -1;                       // the graph input the chain starts at
     int64_t ext[3] = {1, 1, 1}, add[3] = {0, 0, 0}, mod[3] = {0, 0, 0}, stride[3] = {0, 0, 0};
     bool sliced[3] = {false, false, false};
+    int64_t col_add = 0, col_mod = 0;    // the last dimension: column c of the view is column (c + col_add) mod col_mod of the root
+    bool col_sliced = false;
     bool plain = true;                   // still the dense tensor itself (views only)
     bool frozen = false;                 // regrouped by a view after rolls / slices: no further index ops
   };
@@ -113,7 +115,11 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     IdxMap m = imap[n.in[0]];
     if (m.root < 0) { err = where + "roll / slice / view apply to graph inputs (or chains of them) only"; return PN_ERR_UNSUPPORTED_OP; }
     if (Y.dtype != X.dtype) { err = where + "an index operator keeps the dtype"; return PN_ERR_UNSUPPORTED_OP; }
-    if (X.rank < 1 || Y.rank < 1 || X.dims[X.rank - 1] != Y.dims[Y.rank - 1]) { err = where + "index operators act on leading dimensions; the last one must be unchanged"; return PN_ERR_SHAPE; }
+    if (X.rank < 1 || Y.rank < 1) { err = where + "index operators need a dimension to act on"; return PN_ERR_SHAPE; }
+    // the last dimension changes only under a slice of it, or under a view of a tensor that is still dense
+    const bool last_sliced = n.op == N_SLICE && (n.attr[0] == X.rank - 1 || (n.imm[0] != 0.0 && (int64_t)n.imm[0] - 1 == X.rank - 1));
+    const bool dense_view = (n.op == N_VIEW || n.op == N_CONTIGUOUS) && m.plain;
+    if (X.dims[X.rank - 1] != Y.dims[Y.rank - 1] && !last_sliced && !dense_view) { err = where + "the last dimension changes only under a slice of it or a view of a dense tensor"; return PN_ERR_SHAPE; }
     if (n.op == N_CONTIGUOUS && (X.rank != Y.rank || memcmp(X.dims, Y.dims, sizeof(X.dims)) != 0)) { err = where + "contiguous keeps the shape"; return PN_ERR_SHAPE; }
     if (n.op == N_VIEW || n.op == N_CONTIGUOUS) {
       if (X.numel() != Y.numel()) { err = where + "a view keeps the number of elements"; return PN_ERR_SHAPE; }
@@ -133,9 +139,22 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
       for (int which = 0; which < 2; ++which) {
         const int64_t k = dims2[which];
         if (which == 1 && k < 0) break;
-        if (k < 0 || k >= X.rank - 1 || X.rank > 4) { err = where + "roll / slice dimension must be a leading one"; return PN_ERR_SHAPE; }
-        const int kk = 3 - (X.rank - 1) + (int)k;
+        if (k < 0 || k >= X.rank || X.rank > 4) { err = where + "roll / slice dimension outside the tensor"; return PN_ERR_SHAPE; }
         const int64_t Dk = X.dims[k];
+        if (k == X.rank - 1) {   // the last dimension: a column offset (slice) or a circular column shift (roll)
+          if (n.op == N_ROLL) {
+            if (Y.dims[k] != Dk) { err = where + "a roll keeps the shape"; return PN_ERR_SHAPE; }
+            if (m.col_sliced) { err = where + "roll after slice on the same dimension is not lowered"; return PN_ERR_UNSUPPORTED_OP; }
+            if (Dk > 0) { m.col_add = ((m.col_add - amt2[which]) % Dk + Dk) % Dk; m.col_mod = Dk; }
+          } else {
+            const int64_t a = amt2[which], L = Y.dims[k];
+            if (a < 0 || a + L > Dk) { err = where + "slice outside the tensor"; return PN_ERR_SHAPE; }
+            m.col_add += a; m.col_sliced = true;
+            if (m.col_mod) m.col_add %= m.col_mod;
+          }
+          continue;
+        }
+        const int kk = 3 - (X.rank - 1) + (int)k;
         if (n.op == N_ROLL) {
           if (Y.dims[k] != Dk) { err = where + "a roll keeps the shape"; return PN_ERR_SHAPE; }
           if (m.sliced[kk]) { err = where + "roll after slice on the same dimension is not lowered"; return PN_ERR_UNSUPPORTED_OP; }
@@ -278,6 +297,8 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
           io.lead_stride[i] = m.stride[i];
           io.map_dim[i] = (int32_t)std::max<int64_t>(m.ext[i], 1); io.map_add[i] = (int32_t)m.add[i]; io.map_mod[i] = (int32_t)m.mod[i];
         }
+        if (m.col_mod) { io.col_add = (int32_t)m.col_add; io.col_mod = (int32_t)m.col_mod; }   // rolled columns wrap in the kernel
+        else lp.io_offset[idx] += m.col_add;                                                     // sliced columns: the row starts later
       }
       lp.io_tensor[idx] = is_out ? t : imap[t].root; lp.io_is_output[idx] = is_out;
       if (is_out) io_of_tensor[t] = idx; else in_io_of_tensor[t] = idx;
@@ -480,7 +501,7 @@ int lower_graph(const Graph& g, unsigned flags, const DeviceModel& dev, LaunchPl
     if (io.is_row_scalar || io.col_stride == 0) continue;
     if (io_streamed[q]) min_esize = std::min(min_esize, dtype_bytes(io.dtype));
     for (int vl : {8, 4}) {
-      bool ok = eff_N % vl == 0 && lp.io_offset[q] % vl == 0;
+      bool ok = eff_N % vl == 0 && lp.io_offset[q] % vl == 0 && io.col_add % vl == 0 && io.col_mod % vl == 0;
       for (int i = 0; i < 3; ++i) ok = ok && io.lead_stride[i] % vl == 0;
       if (vl == 8) vec8 = vec8 && ok; else vec4 = vec4 && ok;
     }

@@ -106,6 +106,9 @@ struct IoDesc {
   int32_t map_dim[3];
   int32_t map_add[3];
   int32_t map_mod[3];
+  int32_t col_add, col_mod;// an input rolled along the last dimension: column c is read at (c + col_add) mod col_mod
+                           // (col_mod 0 = none; a slice of the last dimension is an offset of the base instead)
+  int32_t pad2;
   int64_t red_stride;      // column kernels: elements per step of the reduced dimension; 0 = broadcast
   int64_t numel;           // elements of the tensor behind this entry (checked accessors)
 };

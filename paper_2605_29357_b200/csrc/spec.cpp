@@ -160,7 +160,7 @@ bool emit_program(const KernelParams& P, int pc, int end, bool scalar, int vl, i
     const std::string A = std::to_string(a), B = std::to_string(b), OP = std::to_string(op);
     auto dt = [&](int io) { return std::to_string((int)P.io[io].dtype); };
     std::string s;
-    if (op == OP_LDRAW) s = "op_ldraw<" + VLNGF + ">(p, cx, " + A + ", " + dt(a) + ", " + regname(b) + ");";
+    if (op == OP_LDRAW) s = "op_ldraw<" + VLNGF + (P.io[a].col_mod ? ", 1" : ", 0") + ">(p, cx, " + A + ", " + dt(a) + ", " + regname(b) + ");";
     else if (op == OP_WIDEN) s = "op_widen<" + VLNG + ">(" + dt(a) + ", " + regname(b) + ");";
     else if (op == OP_LDBC) s = "op_ldbc<" + V + ">(p, cx, " + A + ", " + dt(a) + ", " + regname(b) + ");";
     else if (op == OP_LD) s = "op_mov<" + V + ">(acc, " + regname(a) + ");";
@@ -314,7 +314,7 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
     const uint32_t w = P.code[P.stage[0].elem_begin + j];
     const int io = (w >> 8) & 0xFF;
     if ((w & 0xFF) == OP_LDBC) s += "    op_ldbc_raw<" + V + ">(p, cx, " + I(io) + ", " + I(P.io[io].dtype) + ", raw[" + I(j) + "]);\n";
-    else s += "    op_ldraw<" + I(lp.vl) + ", " + I(lp.ng) + (full ? ", true" : ", false") + ">(p, cx, " + I(io) + ", " + I(P.io[io].dtype) + ", raw[" + I(j) + "]);\n";
+    else s += "    op_ldraw<" + I(lp.vl) + ", " + I(lp.ng) + (full ? ", true" : ", false") + (P.io[io].col_mod ? ", 1" : ", 0") + ">(p, cx, " + I(io) + ", " + I(P.io[io].dtype) + ", raw[" + I(j) + "]);\n";
   }
   s += "  }\n";
   s += "  static PN_DEV void tile(const KernelParams& p, int s, const TileCtx& cx, float (&acc)[" + V + "], float (&reg)[" + I(lp.k) + "][" + V + "], float& ts, Part (&parts)[" + I(kMaxRed) + "],\n"

@@ -96,15 +96,36 @@ class RandomGraph:
             v = Val(self.g.input(dt, shape), shape, "E", lo=-5, hi=5, dtype=dt, integral=True)
         else:
             dt = int(dtype if dtype is not None else r.choice(FLOAT_STORAGE))
+            # a full-shape operand is sometimes read through rolls and slices of a larger graph input,
+            # over leading dimensions and over the last one (index-remapped loads)
+            chain = []
+            root = list(shape)
+            if shape == self.full and r.random() < 0.3:
+                for d in range(len(shape)):
+                    if r.random() < 0.5:
+                        chain.append(("roll", d, int(r.choice([1, 3, 8, -8, 16, 250]))))
+                for d in range(len(shape)):
+                    if r.random() < 0.5:
+                        extra = int(r.choice([1, 3, 8, 8, 16, 32]))
+                        chain.append(("slice", d, int(r.integers(0, extra + 1)) if r.random() < 0.5 else extra))
+                        root[d] += extra
+            root = tuple(root)
             if kind == "P":
-                x = (r.random(shape) * 1.5 + 0.5).astype(np.float32)
+                x = (r.random(root) * 1.5 + 0.5).astype(np.float32)
                 x = np.clip(x, 0.5, 2.0)
-                v = Val(self.g.input(dt, shape), shape, "P", lo=0.5, hi=2.0, dtype=dt)
+                v = Val(self.g.input(dt, root), root, "P", lo=0.5, hi=2.0, dtype=dt)
             else:
-                x = (r.standard_normal(shape) * float(r.choice([0.5, 1.0, 3.0]))).astype(np.float32)
+                x = (r.standard_normal(root) * float(r.choice([0.5, 1.0, 3.0]))).astype(np.float32)
                 x = np.round(x * 8) / 8 if r.random() < 0.3 else x          # quarter-ish steps: exact ties for the arg-reductions
-                v = Val(self.g.input(dt, shape), shape, "E", lo=-20, hi=20, dtype=dt)
+                v = Val(self.g.input(dt, root), root, "E", lo=-20, hi=20, dtype=dt)
             arr = C._store(x.astype(np.float32), dt)
+            cur = list(root)
+            for op, d, amount in chain:                                     # rolls first, then the slices, one dimension a node
+                if op == "slice":
+                    cur[d] = shape[d]
+                v = self._emit(op, [v], dt, tuple(cur), v.kind, v.lo, v.hi, attr=(d, amount), fresh=True)
+            if chain:
+                self.notes.append("indexed input: " + ", ".join(f"{o}({d},{a})" for o, d, a in chain))
         self.inputs.append(np.ascontiguousarray(arr))
         if v.dtype != D.F32 and v.kind in ("P", "E") and not v.integral:
             v = self._emit("cast", [v], D.F32, shape, v.kind, v.lo, v.hi, fresh=True)     # widen: exact

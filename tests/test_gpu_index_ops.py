@@ -1,6 +1,7 @@
 """GPU parity of the index operators (roll, slice, view: Section 3.2's index-remapped
-loads) against the CPU oracle: each operator alone, chains of them feeding arithmetic, and
-the roll + slice + add + LayerNorm subgraph at reduced and full size."""
+loads) against the CPU oracle: each operator alone, over leading dimensions and over the last
+one, chains of them feeding arithmetic, and the roll + slice + add + LayerNorm subgraph at
+reduced and full size."""
 import numpy as np
 import pytest
 
@@ -145,3 +146,86 @@ def test_slice_then_slice_and_roll_compose():
     v = _values((20, 16), D.F32, 7)
     _, outs = _run(g, [v])
     assert np.array_equal(outs[0], -np.roll(v, 13, 0)[13:18])
+
+
+LAST = {"default": 0, "interpret": pn.FLAG_INTERPRET, "unfused": pn.FLAG_UNFUSED, "scalar": pn.FLAG_FORCE_SCALAR,
+        "bounds": pn.FLAG_BOUNDS, "block": pn.FLAG_FORCE_BLOCK}
+
+
+@pytest.mark.parametrize("force", list(LAST))
+@pytest.mark.parametrize("dtype", [D.F32, D.BF16])
+@pytest.mark.parametrize("shape,shift", [((7, 64), 8), ((7, 64), 5), ((3, 5, 96), -16), ((2, 3, 4, 40), 39), ((1, 1000), 250),
+                                         ((9, 33), 4)])
+def test_roll_over_the_last_dimension(shape, shift, dtype, force):
+    """Column c is read at (c - shift) mod N: whole 128-bit groups when the shift and the row length
+    allow it, element by element otherwise."""
+    x = _values(shape, dtype, 70)
+    g = GraphBuilder(); xi = g.input(dtype, shape)
+    r = g.op("roll", [xi], dtype, shape, attr=[len(shape) - 1, shift])
+    g.mark_output(r)                                                   # the roll alone: a copy with moved columns
+    f = g.op("cast", [r], D.F32, shape)
+    g.mark_output(g.op("sum", [g.op("mul", [f, f], D.F32, shape)], D.F32, shape[:-1]))   # and feeding a row reduction
+    gr, outs = _run(g, [x], LAST[force])
+    assert np.array_equal(outs[0], np.roll(x, shift, axis=len(shape) - 1))
+    if force == "default":
+        assert gr.n_kernels == 1
+    if force == "bounds":
+        assert gr.bounds_status == 0
+
+
+@pytest.mark.parametrize("force", list(LAST))
+@pytest.mark.parametrize("dtype", [D.F32, D.BF16])
+@pytest.mark.parametrize("shape,start,length", [((7, 64), 8, 32), ((7, 64), 3, 31), ((3, 5, 96), 48, 48), ((2, 3, 4, 40), 0, 8),
+                                                ((1, 1000), 500, 500), ((16, 2048), 1024, 1024)])
+def test_slice_of_the_last_dimension(shape, start, length, dtype, force):
+    x = _values(shape, dtype, 71)
+    out_shape = shape[:-1] + (length,)
+    g = GraphBuilder(); xi = g.input(dtype, shape)
+    s = g.op("slice", [xi], dtype, out_shape, attr=[len(shape) - 1, start])
+    g.mark_output(s)
+    f = g.op("cast", [s], D.F32, out_shape)
+    g.mark_output(g.op("softmax", [f], D.F32, out_shape))
+    gr, outs = _run(g, [x], LAST[force])
+    assert np.array_equal(outs[0], x[..., start:start + length])
+    if force == "default":
+        assert gr.n_kernels == 1
+    if force == "bounds":
+        assert gr.bounds_status == 0
+
+
+@pytest.mark.parametrize("flags", [0, pn.FLAG_INTERPRET, pn.FLAG_UNFUSED, pn.FLAG_FORCE_SCALAR, pn.FLAG_BOUNDS])
+@pytest.mark.parametrize("M,N", [(64, 1024), (5, 24), (3, 7)])
+def test_gated_activation_reads_both_halves_of_one_tensor(M, N, flags):
+    """x[..., :N] * silu(x[..., N:]) with a LayerNorm behind it: two slices of the last dimension of
+    one input, each its own view of the same buffer, in one kernel."""
+    x = _values((M, 2 * N), D.BF16, 72)
+    ga = _values((N,), D.F32, 73); be = _values((N,), D.F32, 74)
+    g = GraphBuilder(); xi = g.input(D.BF16, (M, 2 * N)); gi = g.input(D.F32, (N,)); bi = g.input(D.F32, (N,))
+    a = g.op("cast", [g.op("slice", [xi], D.BF16, (M, N), attr=[1, 0])], D.F32, (M, N))
+    b = g.op("cast", [g.op("slice", [xi], D.BF16, (M, N), attr=[1, N])], D.F32, (M, N))
+    h = g.op("mul", [a, g.op("silu", [b], D.F32, (M, N))], D.F32, (M, N))
+    y = g.node("layer_norm", [h, gi, bi], [D.F32], [(M, N)], extra_imm=[1e-5])[0]
+    g.mark_output(g.op("cast", [y], D.BF16, (M, N)))
+    gr, _ = _run(g, [x, ga, be], flags)
+    if not flags & pn.FLAG_UNFUSED:
+        assert gr.n_kernels == 1
+        assert gr.compulsory_bytes == x.nbytes + ga.nbytes + be.nbytes + M * N * 2
+
+
+@pytest.mark.parametrize("flags", [0, pn.FLAG_INTERPRET, pn.FLAG_UNFUSED])
+def test_rolls_and_slices_over_leading_and_last_dimensions_compose(flags):
+    """One node rolling a leading and the last dimension at once, a slice of both behind it, then a
+    second slice of the last dimension; and a view of a dense input that regroups the last dimension."""
+    x = _values((6, 10, 48), D.F32, 75)
+    g = GraphBuilder(); xi = g.input(D.F32, x.shape)
+    r = g.op("roll", [xi], D.F32, (6, 10, 48), attr=[1, 3], extra_imm=[3, 8])             # dims 1 and 2
+    s = g.op("slice", [r], D.F32, (6, 7, 32), attr=[1, 2], extra_imm=[3, 4])              # rows 2.., columns 4..
+    s2 = g.op("slice", [s], D.F32, (6, 7, 16), attr=[2, 8])
+    g.mark_output(g.op("exp", [s2], D.F32, (6, 7, 16)))
+    gr, outs = _run(g, [x], flags)
+    want = np.roll(np.roll(x, 3, axis=1), 8, axis=2)[:, 2:9, 4:36][:, :, 8:24]
+    assert np.allclose(outs[0], np.exp(want.astype(np.float64)), rtol=1e-5)
+    v = GraphBuilder(); vi = v.input(D.F32, (6, 10, 48))
+    w = v.op("view", [vi], D.F32, (60, 4, 12))
+    v.mark_output(v.op("relu", [v.op("slice", [w], D.F32, (60, 4, 6), attr=[2, 6])], D.F32, (60, 4, 6)))
+    _run(v, [x], flags)

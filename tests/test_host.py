@@ -205,12 +205,15 @@ def test_index_operator_errors():
         g.mark_output(g.op(op, [x], dtype_out, out_shape, attr=attr))
         return _status(g.build())
     assert one("roll", (4, 8), (4, 8), [0, 1]) == 0
-    assert one("roll", (4, 8), (4, 8), [1, 1]) == -4            # the last dimension is not a leading one
+    assert one("roll", (4, 8), (4, 8), [1, 1]) == 0             # the last dimension: a circular shift of the columns
+    assert one("roll", (4, 8), (4, 8), [2, 1]) == -4            # no such dimension
     assert one("roll", (4, 8), (5, 8), [0, 1]) == -4            # a roll keeps the shape
     assert one("roll", (4, 8), (4, 8), [0, 1], D.BF16) == -3    # and the dtype
     assert one("slice", (4, 8), (3, 8), [0, 1]) == 0
     assert one("slice", (4, 8), (3, 8), [0, 2]) == -4           # 2 + 3 > 4
-    assert one("slice", (4, 8), (3, 4), [0, 0]) == -4           # last dimension must be whole
+    assert one("slice", (4, 8), (3, 4), [0, 0]) == -4           # a slice of dimension 0 leaves the last one whole
+    assert one("slice", (4, 8), (4, 4), [1, 4]) == 0            # a slice of the last dimension: the second half
+    assert one("slice", (4, 8), (4, 4), [1, 5]) == -4           # 5 + 4 > 8
     assert one("view", (4, 6, 8), (3, 8, 8), [0, 0]) == 0
     assert one("view", (4, 6, 8), (3, 8, 4), [0, 0]) == -4
     # index operators read graph inputs (or chains of them), not computed values

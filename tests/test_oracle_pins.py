@@ -492,6 +492,14 @@ def test_roll_slice_view_match_the_papers_index_formula():
         assert out[:, 0].tolist() == [float(a[(i - sh) % 5, 0]) for i in range(5)]
     out = run1("slice", [a], [D.F32], D.F32, (2, 2), attr=(0, 2))
     assert out.tolist() == [[4.0, 5.0], [6.0, 7.0]]
+    # the same two operators along the last dimension (the halves of a gated activation are two such
+    # slices of one tensor), element by element from the definition
+    b = np.arange(12, dtype=np.float32).reshape(2, 6)
+    for sh in (2, -1, 13):
+        out = run1("roll", [b], [D.F32], D.F32, (2, 6), attr=(1, sh))
+        assert out.tolist() == [[float(b[i, (j - sh) % 6]) for j in range(6)] for i in range(2)]
+    out = run1("slice", [b], [D.F32], D.F32, (2, 3), attr=(1, 3))
+    assert out.tolist() == [[3.0, 4.0, 5.0], [9.0, 10.0, 11.0]]
 
 
 def test_n1_restated():

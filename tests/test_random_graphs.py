@@ -29,7 +29,7 @@ def test_generated_graphs_are_valid_and_span_what_they_claim():
         assert g.n_nodes == rg.n_nodes and 1 <= g.n_kernels < rg.n_nodes
         if g.n_kernels > 1:
             cut += 1
-            assert g.workspace_bytes > 0
+            assert g.workspace_bytes >= 0                          # (launches that share no tensor need none)
             with pytest.raises(pn.PnError) as e:                  # as one kernel it is refused, with a documented status
                 pn.Graph(rg.desc, 0, pn.FLAG_PLAN_ONLY | pn.FLAG_ONE_KERNEL)
             assert e.value.status in DOCUMENTED_REFUSALS, (seed, e.value.status, e.value.detail)
