@@ -200,6 +200,11 @@ enum {
  * FAILS with PN_ERR_DEVICE and the reason, unless PN_FLAG_INTERPRET or PN_FLAG_ALLOW_INTERPRET
  * was given (the interpreter kernels are more than ten times slower); PN_Q_KERNEL_INFO tells
  * which kind a handle runs.  The calling thread's current device is left as it was.
+ * Two more environment variables are aids for measurement and debugging: PN_NVRTC_FLAGS adds
+ * options to the run-time compilation (e.g. -DPN_MIN_BLOCKS=6, the resident blocks per SM the
+ * register allocation aims at), PN_DEBUG_PARTITION prints to stderr how a graph was cut into
+ * launches and why the runs that were tried did not lower, PN_DEBUG_SPEC the registers and local
+ * memory of every generated kernel as it is loaded.
  */
 pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsigned flags,
                           pn_graph_t** out);

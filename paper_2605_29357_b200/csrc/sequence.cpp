@@ -61,11 +61,11 @@ pn_status pn_sequence_create(int n, pn_graph_t* const* graphs, const void* const
     if (graphs[i]->flags & PN_FLAG_STATIC_SCRATCH) return fail(PN_ERR_INVALID_ARG, "item " + std::to_string(i) + ": static-scratch handles are not recorded");
   }
   const bool independent = (flags & PN_SEQ_INDEPENDENT) != 0;
-  if (independent)   // the workspace of an unfused handle is shared by its runs: two of them may not overlap
+  if (independent)   // the workspace of a handle (intermediates, partials, arrival counters) is shared by its runs: two of them may not overlap
     for (int i = 0; i < n; ++i)
       for (int j = 0; j < i; ++j)
         if (graphs[i] == graphs[j] && graphs[i]->workspace_bytes > 0)
-          return fail(PN_ERR_INVALID_ARG, "an unfused handle appears twice in an independent sequence (items " + std::to_string(j) + " and " + std::to_string(i) + " would share its workspace)");
+          return fail(PN_ERR_INVALID_ARG, "a handle that has a workspace appears twice in an independent sequence (items " + std::to_string(j) + " and " + std::to_string(i) + " would share its workspace)");
   pn_sequence* s = new (std::nothrow) pn_sequence();
   if (!s) return fail(PN_ERR_INVALID_ARG, "out of host memory");
   s->device = graphs[0]->device;

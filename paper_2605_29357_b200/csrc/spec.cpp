@@ -76,6 +76,7 @@ struct Api {
   CUresult (*ModuleGetFunction)(CUfunction*, CUmodule, const char*) = nullptr;
   CUresult (*ModuleUnload)(CUmodule) = nullptr;
   CUresult (*FuncSetAttribute)(CUfunction, CUfunction_attribute, int) = nullptr;
+  CUresult (*FuncGetAttribute)(int*, CUfunction_attribute, CUfunction) = nullptr;
   CUresult (*LaunchKernelEx)(const CUlaunchConfig*, CUfunction, void**, void**) = nullptr;
   CUresult (*OccupancyMaxActiveBlocks)(int*, CUfunction, int, size_t) = nullptr;
   CUresult (*GetErrorString)(CUresult, const char**) = nullptr;
@@ -117,7 +118,7 @@ const Api& api() {
     if (!cu) { a.why = std::string(cu_name) + " not found (the CUDA driver library)"; return; }
     ok = sym(cu, "cuModuleLoadData", a.ModuleLoadData, a.why) && sym(cu, "cuModuleGetFunction", a.ModuleGetFunction, a.why) &&
               sym(cu, "cuModuleUnload", a.ModuleUnload, a.why) &&
-              sym(cu, "cuFuncSetAttribute", a.FuncSetAttribute, a.why) && sym(cu, "cuLaunchKernelEx", a.LaunchKernelEx, a.why) &&
+              sym(cu, "cuFuncSetAttribute", a.FuncSetAttribute, a.why) && sym(cu, "cuFuncGetAttribute", a.FuncGetAttribute, a.why) && sym(cu, "cuLaunchKernelEx", a.LaunchKernelEx, a.why) &&
               sym(cu, "cuOccupancyMaxActiveBlocksPerMultiprocessor", a.OccupancyMaxActiveBlocks, a.why) &&
               sym(cu, "cuGetErrorString", a.GetErrorString, a.why);
     a.ok = ok;
@@ -223,6 +224,11 @@ std::string kernel_name(const LaunchPlan& lp) {
   snprintf(b, sizeof(b), "pn_spec_%s_v%dx%d_%08x", fam[lp.family >= 0 && lp.family <= FAM_SPLIT ? lp.family : 0], lp.vl, lp.ng, (unsigned)(h ^ (h >> 32)));
   static_assert(FAM_SPLIT == 5, "family names");
   return b;
+}
+
+// whether the generated kernel is first compiled under a register bound that it may not be able to keep
+bool tentative_reg_bound(const LaunchPlan& lp) {
+  return lp.p.family == FAM_WARP && lp.block == 256 && !lp.persistent && lp.vl * lp.ng <= 16 && !lp.no_reg_bound;
 }
 
 bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
@@ -340,7 +346,13 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
   // Column kernels likewise: their walk keeps several steps of loads in flight per thread, and the
   // bound keeps that from eating the resident warps (measured: 64 registers with 4 steps in flight
   // beats every larger budget on the pooling workload).
+  // Warp-per-row kernels that keep nothing across rows (the softmax workload: 39 registers left
+  // to itself) gain from one more resident block per SM: 83.9 -> 82.3 us under a bound of 7 blocks
+  // of 256 threads (the compiler settles on 32 registers and parks two words).  The bound is
+  // tentative: a kernel that spills more than a few words under it is compiled again without
+  // (spec_compile).
   const int min_blocks = (P.family == FAM_COLUMN && lp.block == 128) ? 7
+                       : tentative_reg_bound(lp) ? 7
                        : ((P.family == FAM_BLOCK && P.chunks == 1) || P.family == FAM_COLUMN) ? std::max(1, 1024 / lp.block) : 1;
   s += "#ifndef PN_MIN_BLOCKS\n#define PN_MIN_BLOCKS " + I(min_blocks) + "\n#endif\n";
   s += "#if PN_MIN_BLOCKS > 1\n#define PN_LAUNCH_BOUNDS __launch_bounds__(" + I(lp.block) + ", PN_MIN_BLOCKS)\n#else\n"
@@ -496,6 +508,21 @@ bool spec_compile(LaunchPlan& lp, int device, int sm_count, SpecKernel& out, std
       cmp.refs = 1; cmp.used = ++g_cache_clock;
       g_cache[key] = cmp;
       evict_unused();
+    }
+  }
+  if (getenv("PN_DEBUG_SPEC")) {
+    int regs = 0, local_b = 0;
+    a.FuncGetAttribute(&regs, CU_FUNC_ATTRIBUTE_NUM_REGS, cmp.fn);
+    a.FuncGetAttribute(&local_b, CU_FUNC_ATTRIBUTE_LOCAL_SIZE_BYTES, cmp.fn);
+    fprintf(stderr, "spec: %s registers %d local bytes %d%s\n", kernel_name(lp).c_str(), regs, local_b, tentative_reg_bound(lp) ? " (tentative register bound)" : "");
+  }
+  if (tentative_reg_bound(lp)) {   // did the kernel keep the bound without spilling more than a few words?
+    // (the softmax workload's kernel parks two words -- 8 bytes -- and is still the faster one)
+    int local_bytes = 0;
+    if (a.FuncGetAttribute(&local_bytes, CU_FUNC_ATTRIBUTE_LOCAL_SIZE_BYTES, cmp.fn) == CUDA_SUCCESS && local_bytes > 32) {
+      spec_release(cmp.fn);
+      lp.no_reg_bound = 1;
+      return spec_compile(lp, device, sm_count, out, err);
     }
   }
   if (lp.smem_bytes > 48 * 1024) {

@@ -306,6 +306,23 @@ def n2(B: int = 256, S: int = 512, Dh: int = 1024, seed: int = 0, dtype: int = D
                    {"floor": floor, "lengths_min": int(lens.min()), "lengths_max": int(lens.max())})
 
 
+# ---------------------------------------------------------------------------
+# A gated activation read from the two halves of one tensor: y = x[..., :N] * silu(x[..., N:]).
+# Two slices of the last dimension of one input (index-remapped loads, Section 3.2): a
+# supplementary shape for the benchmark sweep and the parity tests, not one of the named configs.
+# ---------------------------------------------------------------------------
+def gated_halves(M: int = 8192, N: int = 14336, seed: int = 0, dtype: int = D.BF16) -> Workload:
+    g = GraphBuilder()
+    x = g.input(dtype, (M, 2 * N))
+    a = g.op("slice", [x], dtype, (M, N), attr=[1, 0])
+    b = g.op("slice", [x], dtype, (M, N), attr=[1, N])
+    cast = (lambda t: g.op("cast", [t], D.F32, (M, N))) if dtype != D.F32 else (lambda t: t)
+    h = g.op("mul", [cast(a), g.op("silu", [cast(b)], D.F32, (M, N))], D.F32, (M, N))
+    g.mark_output(g.op("cast", [h], dtype, (M, N)) if dtype != D.F32 else h)
+    xv = _store(_draw(_rng(seed, 8, 0), "normal", (M, 2 * N), 0.0, 1.0), dtype)
+    return _finish("gated_halves", g, ["x"], ["y"], [xv])
+
+
 CONFIGS = {"c1": c1, "c2": c2, "c3": c3, "c4": c4, "c5": c5}
 # subgraphs beyond the five benchmark ones (index-remapped loads; a reduction over a leading dimension)
 EXTENDED = {"n1": n1, "n2": n2}

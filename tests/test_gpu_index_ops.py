@@ -229,3 +229,20 @@ def test_rolls_and_slices_over_leading_and_last_dimensions_compose(flags):
     w = v.op("view", [vi], D.F32, (60, 4, 12))
     v.mark_output(v.op("relu", [v.op("slice", [w], D.F32, (60, 4, 6), attr=[2, 6])], D.F32, (60, 4, 6)))
     _run(v, [x], flags)
+
+
+def test_gated_halves_workload_small_and_full_size():
+    """The supplementary sweep shape: every element at a reduced size; at the size the benchmark
+    times, the rows of a sample (rows are independent) and the byte count."""
+    from oracle import evaluator as E
+    w = C.gated_halves(M=19, N=1432)
+    g = pn.Graph(w.desc, 0, 0)
+    check_against_oracle(w.desc, w.inputs, run_graph(g, w.inputs), w.output_meta, w.output_names)
+    w = C.gated_halves()
+    g = pn.Graph(w.desc, 0, 0)
+    assert g.n_kernels == 1 and g.compulsory_bytes == w.inputs[0].nbytes * 3 // 2
+    out = run_graph(g, w.inputs)[0]
+    rows = np.random.default_rng(5).choice(w.inputs[0].shape[0], size=64, replace=False)
+    sub = C.gated_halves(M=64)
+    ref = E.evaluate(sub.desc, [np.ascontiguousarray(w.inputs[0][rows])])
+    check_against_oracle(sub.desc, None, [out[rows]], sub.output_meta, sub.output_names, ref=ref)
