@@ -359,7 +359,8 @@ def roofline_entry(cbytes, seconds, peak, peak_src, mix, probe, small):
 def tiny_graph_latency(torch, pn, device, passes, repeats=8):
     """Latency of many small subgraphs run back to back (the regime where the paper finds fixed
     per-call overhead decisive): the reduced-size graphs of every workload, `repeats` instances
-    each on their own buffers, (a) launched one by one from the host through bound launches (pn_bound_run),
+    each on their own buffers, (a) launched one by one from the host through bound launches (pn_bound_run
+    from a Python loop, and pn_bound_run_many: the same launches issued by one call),
     (b) recorded once as a sequence and replayed in order, (c) the same as independent items.
     Returns microseconds per subgraph for each; the inputs are L2-resident, so this is launch
     and latency, not bandwidth."""
@@ -388,13 +389,17 @@ def tiny_graph_latency(torch, pn, device, passes, repeats=8):
         return e0.elapsed_time(e1) * 1e3 / (passes * len(items))
 
     bound = [g.bind(i, o) for g, i, o in items]
+    many = pn.BoundList(bound)
 
     def host_pass():
         for f in bound:
             f(stream.cuda_stream)
 
+    def host_pass_one_call():
+        many(stream.cuda_stream)
+
     out = {"subgraphs": len(items), "distinct_graphs": len(graphs), "kernels_per_pass": sum(g.n_kernels for g, _, _ in items),
-           "host_launched_us_per_subgraph": timed(host_pass)}
+           "host_launched_us_per_subgraph": timed(host_pass), "host_launched_one_call_us_per_subgraph": timed(host_pass_one_call)}
     for key, indep in (("sequence_us_per_subgraph", False), ("sequence_independent_us_per_subgraph", True)):
         seq = pn.Sequence(items, independent=indep)
         out[key] = timed(lambda: seq.run(stream.cuda_stream))

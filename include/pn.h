@@ -246,11 +246,16 @@ pn_status pn_graph_run(pn_graph_t* g, const void* const* inputs, int n_inputs,
  * object is immutable: pn_bound_run may be called from several threads at once (the workspace
  * rule of pn_graph_run applies).  Asynchronous, no allocation at run time, capturable in a CUDA
  * graph like pn_graph_run.
+ * pn_bound_run_many(bound, n, stream): the launches of n bound objects, in the order of the HOST
+ * array `bound`, on one stream, in one call -- for many small subgraphs whose pointers are known
+ * but which are not worth a CUDA graph; stops at the first failure and returns its status (the
+ * launches before it stay enqueued).  n = 0 is a no-op.
  */
 typedef struct pn_bound pn_bound_t;
 pn_status pn_graph_bind(pn_graph_t* g, const void* const* inputs, int n_inputs, void* const* outputs,
                         int n_outputs, pn_bound_t** out);
 pn_status pn_bound_run(pn_bound_t* b, void* stream);
+pn_status pn_bound_run_many(pn_bound_t* const* bound, int n, void* stream);
 pn_status pn_bound_destroy(pn_bound_t* b);
 
 /*

@@ -44,7 +44,7 @@ Q_N_KERNELS, Q_N_NODES, Q_WORKSPACE_BYTES, Q_KERNEL_INFO = 6, 7, 8, 9
 
 FAMILY_NAMES = {0: "pointwise", 1: "warp-per-row", 2: "block-per-row", 3: "cluster-per-row", 4: "column-reduce", 5: "split-row"}
 EXPORTS = ["pn_graph_create", "pn_graph_run", "pn_graph_run_host", "pn_graph_run_static", "pn_graph_destroy",
-           "pn_graph_bind", "pn_bound_run", "pn_bound_destroy",
+           "pn_graph_bind", "pn_bound_run", "pn_bound_run_many", "pn_bound_destroy",
            "pn_graph_query", "pn_graph_codegen", "pn_status_string", "pn_last_error",
            "pn_sequence_create", "pn_sequence_run", "pn_sequence_query", "pn_sequence_destroy",
            "pn_stream_probe"]
@@ -95,6 +95,8 @@ def load_library() -> ctypes.CDLL:
     lib.pn_graph_bind.argtypes = [vp, vpp, ctypes.c_int, vpp, ctypes.c_int, vpp]
     lib.pn_bound_run.restype = ctypes.c_int
     lib.pn_bound_run.argtypes = [vp, vp]
+    lib.pn_bound_run_many.restype = ctypes.c_int
+    lib.pn_bound_run_many.argtypes = [ctypes.POINTER(vp), ctypes.c_int, vp]
     lib.pn_bound_destroy.restype = ctypes.c_int
     lib.pn_bound_destroy.argtypes = [vp]
     lib.pn_graph_query.restype = ctypes.c_int
@@ -249,6 +251,21 @@ class Graph:
             self.close()
         except Exception:
             pass
+
+
+class BoundList:
+    """Several bound launches run in order by one call (pn_bound_run_many)."""
+
+    def __init__(self, bound: Sequence["Bound"]):
+        self._keep = list(bound)
+        self._n = len(self._keep)
+        self._arr = (ctypes.c_void_p * max(self._n, 1))(*[b._h.value for b in self._keep])
+        self._run = load_library().pn_bound_run_many
+
+    def __call__(self, stream: int = 0) -> None:
+        st = self._run(self._arr, self._n, ctypes.c_void_p(stream))
+        if st != PN_OK:
+            _check(st, "pn_bound_run_many")
 
 
 class Bound:

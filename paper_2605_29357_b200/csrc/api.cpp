@@ -535,6 +535,28 @@ pn_status pn_bound_run(pn_bound_t* b, void* stream) {
   return PN_OK;
 }
 
+pn_status pn_bound_run_many(pn_bound_t* const* bound, int n, void* stream) {
+  if (n < 0 || (n > 0 && !bound)) return fail(PN_ERR_INVALID_ARG, "null argument");
+  for (int i = 0; i < n; ++i)
+    if (!bound[i] || !bound[i]->g) return fail(PN_ERR_INVALID_ARG, "bound object " + std::to_string(i) + " is null");
+  int current = -2;   // the device made current so far (-2: none yet); the caller's is put back at the end
+  int callers = 0;
+  cudaError_t e = n > 0 ? cudaGetDevice(&callers) : cudaSuccess;
+  if (e != cudaSuccess) return fail(PN_ERR_CUDA, std::string("cudaGetDevice: ") + cudaGetErrorString(e));
+  pn_status st = PN_OK;
+  for (int i = 0; i < n && st == PN_OK; ++i) {
+    const pn_graph* h = bound[i]->g;
+    if (h->device != current && !(current == -2 && h->device == callers)) {
+      e = cudaSetDevice(h->device);
+      if (e != cudaSuccess) { st = fail(PN_ERR_CUDA, std::string("cudaSetDevice: ") + cudaGetErrorString(e)); break; }
+    }
+    current = h->device;
+    for (size_t k = 0; k < bound[i]->plans.size() && st == PN_OK; ++k) st = launch_filled(h->launches[k], bound[i]->plans[k], stream);
+  }
+  if (current >= 0 && current != callers) cudaSetDevice(callers);
+  return st;
+}
+
 pn_status pn_bound_destroy(pn_bound_t* b) {
   delete b;
   return PN_OK;

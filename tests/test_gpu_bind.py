@@ -74,3 +74,34 @@ def test_bind_runs_the_argument_checks_once_and_for_all():
         st.bind(ins, outs)
     assert e.value.status == -1
     torch.cuda.synchronize()
+
+
+def test_many_bound_launches_in_one_call():
+    """pn_bound_run_many: the launches of several bound objects (different graphs, fused and cut into
+    several kernels) in the order given, by one call; the same bits as one pn_bound_run each."""
+    import torch
+    makers = {**C.CONFIGS, **C.EXTENDED}
+    stream = torch.cuda.current_stream().cuda_stream
+    graphs, bound, outs_many, outs_one, keep = [], [], [], [], []
+    for cfg, flags in (("c1", 0), ("c3", 0), ("c5", pn.FLAG_UNFUSED), ("n1", 0), ("c4", 0), ("n2", 0)):
+        w = makers[cfg](seed=3, **C.SMALL[cfg])
+        g = pn.Graph(w.desc, 0, flags)
+        d_in, d_out, sizes = _buffers(w)
+        _, d_ref, _ = _buffers(w)
+        ins = [t.data_ptr() for t in d_in]
+        bound.append(g.bind(ins, [t.data_ptr() for t in d_out]))
+        one = g.bind(ins, [t.data_ptr() for t in d_ref])
+        one(stream)
+        graphs.append((g, w, sizes)); outs_many.append(d_out); outs_one.append(d_ref); keep.append((d_in, one))
+    many = pn.BoundList(bound)
+    before = torch.cuda.current_device()
+    many(stream)
+    many(stream)                                   # (arrival counters of split kernels are back at zero)
+    torch.cuda.synchronize()
+    assert torch.cuda.current_device() == before
+    for (g, w, sizes), d_out, d_ref in zip(graphs, outs_many, outs_one):
+        got = _host(d_out, sizes, w.output_meta)
+        check_against_oracle(w.desc, w.inputs, got, w.output_meta, w.output_names)
+        for x, y in zip(got, _host(d_ref, sizes, w.output_meta)):
+            assert np.array_equal(x.view(np.uint8), y.view(np.uint8))
+    pn.BoundList([])(stream)                       # nothing to launch: a no-op
