@@ -118,6 +118,11 @@ enum {
                                      ahead (costs registers; off by default)                 */
   PN_FLAG_STATIC_SCRATCH = 1u << 12,/* with PN_FLAG_UNFUSED: allocate no workspace; the handle
                                      is run with pn_graph_run_static only                    */
+  PN_FLAG_PLAIN_LAUNCH = 1u << 2, /* launch the generated kernels in plain stream order.  By default they
+                                     are launched with programmatic stream serialization: a kernel is
+                                     set up while its predecessor in the stream still runs and waits
+                                     at its head until that one is complete -- the same results, about
+                                     a microsecond less per launch for kernels of a few microseconds */
   PN_FLAG_ONE_KERNEL = 1u << 3,   /* a graph that does not fit one kernel (a bytecode, register, scalar,
                                      I/O or stage budget; a combination the fused lowering does not
                                      take) is refused with PN_ERR_TOO_LARGE / PN_ERR_UNSUPPORTED_OP

@@ -18,6 +18,7 @@ PN_OK = 0
 FLAG_UNFUSED = 1 << 0
 FLAG_PLAN_ONLY = 1 << 1
 FLAG_ONE_KERNEL = 1 << 3
+FLAG_PLAIN_LAUNCH = 1 << 2
 FLAG_FORCE_WARP = 1 << 4
 FLAG_FORCE_BLOCK = 1 << 5
 FLAG_FORCE_CLUSTER = 1 << 6

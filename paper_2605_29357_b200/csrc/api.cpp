@@ -430,6 +430,7 @@ pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsig
     st = static_scratch_address(device, &h->static_scratch);
     if (st != PN_OK) { delete h; return st; }
   }
+  if (flags & PN_FLAG_PLAIN_LAUNCH) for (PlannedLaunch& pl : h->launches) pl.plan.plain_launch = 1;
   // checked accessors: one status word on the device, shared by the launches of the handle
   if (flags & PN_FLAG_BOUNDS) {
     for (PlannedLaunch& pl : h->launches) pl.plan.bounds = 1;

@@ -9,6 +9,7 @@
 // read this GPU's own memory only and are never multicast.  Every mbarrier wait is a try_wait
 // loop with a retry limit: a wait that runs out sets a bit in the status word, the kernel
 // waits (again bounded) for its own copies in flight and returns.
+#include <cstring>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -55,6 +56,9 @@ __device__ __forceinline__ void emit(uint4 x, uint4* c, uint2* d, size_t idx, ui
 template <int NR, int NW16, int NW8, int U, bool NOALLOC, bool CS, int LAYOUT>
 __global__ void probe_direct(const uint4* __restrict__ a, const uint4* __restrict__ b, uint4* __restrict__ c,
                              uint2* __restrict__ d, size_t units, size_t run, unsigned* status) {
+  // launched like the generated graph kernels: set up while the kernel before it in the stream still
+  // runs, and waiting here until that one is complete
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   uint4 sink = make_uint4(0, 0, 0, 0);
   size_t begin, end, step;
   if (LAYOUT == 0) { begin = (size_t)blockIdx.x * blockDim.x + threadIdx.x; end = units; step = (size_t)gridDim.x * blockDim.x; }
@@ -214,7 +218,15 @@ cudaError_t launch_mix(int loader, int store, int layout, int block, int unroll,
     k<<<grid, block + 32, smem, s>>>(a, b, c, d, units, stages, tile_units, status);
     return cudaGetLastError();
   }
-#define PN_PROBE_GO(U, NA, CS, LY) probe_direct<NR, NW16, NW8, U, NA, CS, LY><<<grid, block, 0, s>>>(a, b, c, d, units, (size_t)tile_units, status)
+  cudaLaunchConfig_t lc;
+  memset(&lc, 0, sizeof(lc));
+  lc.gridDim = dim3((unsigned)grid, 1, 1); lc.blockDim = dim3((unsigned)block, 1, 1); lc.dynamicSmemBytes = 0; lc.stream = s;
+  cudaLaunchAttribute overlap;
+  overlap.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  overlap.val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = &overlap; lc.numAttrs = 1;
+  cudaError_t le = cudaSuccess;
+#define PN_PROBE_GO(U, NA, CS, LY) le = cudaLaunchKernelEx(&lc, probe_direct<NR, NW16, NW8, U, NA, CS, LY>, a, b, c, d, units, (size_t)tile_units, status)
 #define PN_PROBE_U(NA, CS, LY)                                                            \
   switch (unroll) {                                                                       \
     case 1: PN_PROBE_GO(1, NA, CS, LY); break;                                            \
@@ -229,7 +241,7 @@ cudaError_t launch_mix(int loader, int store, int layout, int block, int unroll,
   else { if (na) { if (store) { PN_PROBE_U(true, true, 1) } else { PN_PROBE_U(true, false, 1) } } else { if (store) { PN_PROBE_U(false, true, 1) } else { PN_PROBE_U(false, false, 1) } } }
 #undef PN_PROBE_U
 #undef PN_PROBE_GO
-  return cudaGetLastError();
+  return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 }  // namespace

@@ -105,3 +105,34 @@ def test_many_bound_launches_in_one_call():
         for x, y in zip(got, _host(d_ref, sizes, w.output_meta)):
             assert np.array_equal(x.view(np.uint8), y.view(np.uint8))
     pn.BoundList([])(stream)                       # nothing to launch: a no-op
+
+
+def test_overlapped_launches_keep_stream_order():
+    """Generated kernels are launched so that their set-up overlaps the tail of the kernel before
+    them in the stream, and wait at their head for it to complete: a producer of another library
+    right before a launch, and a chain of two handles where the second reads what the first wrote,
+    give the bits of plain stream order (PN_FLAG_PLAIN_LAUNCH)."""
+    import torch
+    from pn_workloads.descriptor import GraphBuilder, Imm
+    M, N = 256, 4096
+    def scale_graph(k):
+        g = GraphBuilder(); x = g.input(D.F32, (M, N))
+        g.mark_output(g.op("mul", [g.op("add", [x, Imm(1.0)], D.F32, (M, N)), Imm(k)], D.F32, (M, N)))
+        return g.build()
+    stream = torch.cuda.current_stream().cuda_stream
+    results = {}
+    for label, flags in (("overlapped", 0), ("plain", pn.FLAG_PLAIN_LAUNCH)):
+        a, b = pn.Graph(scale_graph(0.5), 0, flags), pn.Graph(scale_graph(3.0), 0, flags)
+        x = torch.zeros(M, N, device="cuda"); mid = torch.empty_like(x); out = torch.empty_like(x)
+        fa, fb = a.bind([x.data_ptr()], [mid.data_ptr()]), b.bind([mid.data_ptr()], [out.data_ptr()])
+        got = []
+        for step in range(30):
+            x.fill_(float(step))                  # a kernel of another library writes the input ...
+            fa(stream); fb(stream)                # ... and the two launches follow at once, the second reading the first
+            got.append(out[::37, ::129].clone())
+        torch.cuda.synchronize()
+        results[label] = torch.stack(got).cpu().numpy()
+        for step in range(30):
+            assert np.all(results[label][step] == np.float32((step + 1.0) * 0.5 + 1.0) * np.float32(3.0)), (label, step)
+        a.close(); b.close()
+    assert np.array_equal(results["overlapped"], results["plain"])
