@@ -221,6 +221,9 @@ pn_status pn_graph_create(const void* desc, size_t desc_bytes, int device, unsig
  *             element of every output is overwritten.
  *   stream  : a cudaStream_t (NULL = the default stream).
  * Asynchronous: returns after the launch(es).  No allocation, no host synchronisation.
+ * Stream order holds as for any kernel launch; the generated kernels are, unless
+ * PN_FLAG_PLAIN_LAUNCH was given, set up while the kernel before them in the stream still runs and
+ * touch no memory until that kernel is complete and its writes are visible.
  * Pointers must be aligned to 16 bytes unless the handle was created with
  * PN_FLAG_FORCE_SCALAR (then to the element size); otherwise PN_ERR_ALIGNMENT.  Inputs
  * and outputs must not overlap, not even exactly: the kernels read inputs through the
