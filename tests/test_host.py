@@ -332,3 +332,17 @@ def test_a_create_that_cannot_specialise_fails_loudly_unless_the_interpreter_is_
     assert _create_in_child({}, pn.FLAG_PLAN_ONLY).startswith("OK")
     # a run-time library that is there but is not NVRTC is refused as well
     assert _create_in_child({"PN_NVRTC_PATH": pn.library_path()}, pn.FLAG_PLAN_ONLY).startswith("ERR -8")
+
+
+def test_nodes_that_reach_no_output_are_dropped():
+    """A node whose result no graph output depends on is not part of f_G: it costs no launch on the
+    unfused path, and what it would need (here a second softmax) is not asked of the kernel."""
+    g = GraphBuilder(); x = g.input(D.F32, (4, 64))
+    dead = g.op("softmax", [g.op("softmax", [x], D.F32, (4, 64))], D.F32, (4, 64))
+    live = g.op("exp", [x], D.F32, (4, 64))
+    g.op("add", [dead, live], D.F32, (4, 64))                     # dead as well: nothing reads it
+    g.mark_output(live)
+    fused = pn.Graph(g.build(), 0, PLAN | pn.FLAG_ONE_KERNEL)
+    assert fused.n_kernels == 1 and fused.n_nodes == 4
+    assert pn.FAMILY_NAMES[fused.kernel_info[0]["family"]] == "pointwise"
+    assert pn.Graph(g.build(), 0, PLAN | pn.FLAG_UNFUSED).n_kernels == 1
