@@ -113,7 +113,7 @@ int lower_column_graph(const Graph& g, unsigned flags, const DeviceModel& dev, L
   for (int t = 0; t < nt; ++t) {
     const Tensor& T = g.tensors[t];
     const std::string where = "tensor " + std::to_string(t) + ": ";
-    if (space[t] == SP_NONE) { err = where + "not connected to the computation"; return PN_ERR_UNSUPPORTED_OP; }
+    if (space[t] == SP_NONE) continue;   // a graph input nothing reads (or only nodes that reach no output): takes no part
     int64_t d[4];
     if (space[t] == SP_PRE) {
       if (!right_align(T, rs, d)) { err = where + "rank above that of the reduced tensors"; return PN_ERR_SHAPE; }
@@ -181,7 +181,9 @@ int lower_column_graph(const Graph& g, unsigned flags, const DeviceModel& dev, L
   // ---- io table: graph inputs and outputs as [O, R, C] / [O, C] with strides ----------------
   memset(&lp, 0, sizeof(lp));
   KernelParams& P = lp.p;
-  const int n_io = (int)(g.inputs.size() + g.outputs.size());
+  std::vector<int> read_inputs;   // graph inputs that the computation reads
+  for (int t : g.inputs) if (space[t] != SP_NONE) read_inputs.push_back(t);
+  const int n_io = (int)(read_inputs.size() + g.outputs.size());
   if (n_io > kMaxIo) { err = "more graph inputs + outputs than one kernel takes (" + std::to_string(kMaxIo) + ")"; return PN_ERR_TOO_LARGE; }
   P.n_io = n_io;
   std::vector<int> io_of_tensor(nt, -1);
@@ -189,7 +191,7 @@ int lower_column_graph(const Graph& g, unsigned flags, const DeviceModel& dev, L
   {
     int idx = 0;
     for (int pass = 0; pass < 2; ++pass)
-      for (int t : pass == 0 ? g.inputs : g.outputs) {
+      for (int t : pass == 0 ? read_inputs : g.outputs) {
         IoDesc& io = P.io[idx];
         const std::string where = "tensor " + std::to_string(t) + ": ";
         io.dtype = g.tensors[t].dtype;
@@ -224,7 +226,7 @@ int lower_column_graph(const Graph& g, unsigned flags, const DeviceModel& dev, L
   // ---- (2) micro-operations -----------------------------------------------------------------
   Expander ex;
   std::vector<int> tval(nt, -1);
-  for (int t : g.inputs) {
+  for (int t : read_inputs) {
     const int v = ex.new_val(VK_E, space[t] == SP_POST ? 1 : 0);
     const int q = io_of_tensor[t];
     ex.vals[v].io = q;

@@ -480,3 +480,116 @@ class RandomGraph:
 
 def make(seed: int, max_nodes: Optional[int] = None) -> RandomGraph:
     return RandomGraph(seed, max_nodes)
+
+
+# ---------------------------------------------------------------------------------------------
+# Graphs that reduce over a LEADING dimension (the masked-mean-pooling shape): a pointwise chain
+# with broadcast operands before the reductions, one to three reductions over one dimension, a
+# pointwise chain on the reduced values after them.  Values stay positive where they are summed
+# (no cancellation), so fp32 kernels can be held to the relative tolerance.
+# ---------------------------------------------------------------------------------------------
+class ColumnGraph:
+    def __init__(self, seed: int):
+        r = self.rng = np.random.default_rng([104729, seed])
+        g = self.g = GraphBuilder()
+        self.inputs: List[np.ndarray] = []
+        rank = int(r.choice([2, 3, 3, 4]))
+        C_ = int(r.choice([1, 7, 8, 24, 64, 96, 200, 256, 1000, 1032]))
+        R = int(r.choice([1, 2, 5, 33, 64, 129, 700, 2500]))
+        if R * C_ > 400_000:
+            R = 129
+        lead = {2: (), 3: (int(r.integers(1, 7)),), 4: (int(r.integers(1, 4)), int(r.integers(1, 4)))}[rank]
+        dim = len(lead)                                            # the reduced dimension: the last leading one ...
+        full = tuple(lead) + (R, C_)
+        if rank == 4 and r.random() < 0.5:                         # ... or, at rank 4, the one before it
+            dim = 1
+            full = (lead[0], R, lead[1], C_)
+        self.full, self.dim = full, dim
+        keep = tuple(1 if i == dim else d for i, d in enumerate(full))
+        drop = tuple(d for i, d in enumerate(full) if i != dim)
+        dt = int(r.choice(FLOAT_STORAGE))
+        x = self._input(dt, full, "P")
+        xf = g.op("cast", [x], D.F32, full) if dt != D.F32 else x
+        pre, n_nodes = [xf], (1 if dt != D.F32 else 0)
+        # the chain before the reductions: broadcast operands of every pattern the column family takes
+        for _ in range(int(r.integers(0, 5))):
+            a = pre[int(r.integers(len(pre)))]
+            kind = str(r.choice(["scale", "vec", "mask", "sqrt", "imm_add", "full"]))
+            if kind == "scale":
+                v = g.op("mul", [a, Imm(float(r.choice([0.5, 1.25, 2.0])))], D.F32, full)
+            elif kind == "imm_add":
+                v = g.op("add", [a, Imm(float(r.choice([0.25, 1.0])))], D.F32, full)
+            elif kind == "sqrt":
+                v = g.op("sqrt", [a], D.F32, full)
+            elif kind == "vec":                                    # a vector over the columns
+                w = self._input(D.F32, (C_,), "P")
+                v = g.op("mul", [a, w], D.F32, full)
+            elif kind == "mask":                                   # one value per step of the reduced dimension
+                mshape = tuple(d if i <= dim else 1 for i, d in enumerate(full))
+                mdt = int(r.choice([D.I64, D.I8, D.F32]))
+                m = self._input(mdt, mshape, "M")
+                mf = g.op("cast", [m], D.F32, mshape) if mdt != D.F32 else m
+                n_nodes += 1 if mdt != D.F32 else 0
+                v = g.op("mul", [a, mf], D.F32, full)
+            else:
+                b2 = self._input(int(r.choice(FLOAT_STORAGE)), full, "P")
+                bf = b2 if g.tensor_meta(b2)[0] == D.F32 else g.op("cast", [b2], D.F32, full)
+                n_nodes += 0 if g.tensor_meta(b2)[0] == D.F32 else 1
+                v = g.op(str(r.choice(["add", "mul", "max"])), [a, bf], D.F32, full)
+            pre.append(v); n_nodes += 1
+        self._pre, self._keep, self._drop, self._n = pre, keep, drop, n_nodes
+        self._finish()
+
+    def _input(self, dt, shape, kind):
+        r = self.rng
+        if kind == "M":                                            # 0 / 1 with a run of kept positions
+            arr = (r.random(shape) < 0.7).astype(C.NP_STORAGE[dt])
+        else:
+            arr = C._store((r.random(shape) * 1.5 + 0.5).astype(np.float32), dt)
+        self.inputs.append(np.ascontiguousarray(arr))
+        return self.g.input(dt, shape)
+
+    def _finish(self):
+        r, g = self.rng, self.g
+        pre, keep, drop, dim = self._pre, self._keep, self._drop, self.dim
+        reds = []
+        for _ in range(int(r.integers(1, 4))):
+            src = pre[int(r.integers(len(pre)))]
+            op = str(r.choice(["sum_dim", "sum_dim", "mean_dim", "amax_dim", "amin_dim"]))
+            reds.append(g.op(op, [src], D.F32, keep if r.random() < 0.5 else drop, attr=[dim, 0]))
+            self._n += 1
+        post = list(reds)
+        shape_of = lambda t: tuple(g.tensor_meta(t)[1])
+        for _ in range(int(r.integers(0, 4))):                     # the epilogue on the reduced values
+            a = post[int(r.integers(len(post)))]
+            sh = shape_of(a)
+            kind = str(r.choice(["scale", "clamp", "pair", "input"]))
+            if kind == "scale":
+                v = g.op("mul", [a, Imm(float(r.choice([0.5, 3.0])))], D.F32, sh)
+            elif kind == "clamp":
+                v = g.op("clamp", [a, Imm(0.75), Imm(50.0)], D.F32, sh)
+            elif kind == "pair":
+                same = [t for t in post if shape_of(t) == sh and t != a]
+                if not same:
+                    continue
+                b2 = same[int(r.integers(len(same)))]
+                v = g.op(str(r.choice(["add", "div", "max"])), [a, g.op("add", [b2, Imm(1.0)], D.F32, sh)], D.F32, sh)
+                self._n += 1
+            else:                                                  # a graph input of the reduced shape
+                w = self._input(D.F32, sh, "P")
+                v = g.op("mul", [a, w], D.F32, sh)
+            post.append(v); self._n += 1
+        outs = [post[-1]] + [t for t in post[:-1] if r.random() < 0.4]
+        if len(pre) > 1 and r.random() < 0.3:
+            outs.append(pre[-1])                                   # a full-shape value of the walk leaves the graph too
+        for t in dict.fromkeys(outs):
+            if r.random() < 0.3:
+                t = g.op("cast", [t], int(r.choice([D.BF16, D.F16])), shape_of(t)); self._n += 1
+            g.mark_output(t)
+        self.n_nodes = self._n
+        self.desc = g.build()
+        self.output_meta = [g.tensor_meta(t) for t in g.output_ids()]
+
+
+def make_column(seed: int) -> ColumnGraph:
+    return ColumnGraph(seed)

@@ -56,3 +56,31 @@ def test_random_graph(seed):
         outs = run_graph(g, rg.inputs)
         check_against_oracle(rg.desc, rg.inputs, outs, rg.output_meta, ref=ref)
         assert g.bounds_status == 0
+
+
+COLUMN_MODES = [("generated", 0), ("interpreter", pn.FLAG_INTERPRET), ("slices", pn.FLAG_FORCE_SPLIT),
+                ("three slices", pn.tune(cluster=3)), ("unfused", pn.FLAG_UNFUSED), ("scalar", pn.FLAG_FORCE_SCALAR)]
+
+
+@pytest.mark.parametrize("seed", range(80))
+def test_random_column_graph(seed):
+    """Random graphs that reduce over a leading dimension (chains with broadcast operands before the
+    reductions and on the reduced values after them): generated kernels, and in turn the interpreter,
+    the reduced dimension cut into slices, node by node, element-wise accesses."""
+    rg = rand_graphs.make_column(seed)
+    ref = E.evaluate(rg.desc, rg.inputs)
+    ran = 0
+    for label, flags in [COLUMN_MODES[0], COLUMN_MODES[1 + seed % (len(COLUMN_MODES) - 1)]]:
+        try:
+            g = pn.Graph(rg.desc, 0, flags | pn.FLAG_BOUNDS)
+        except pn.PnError as e:
+            assert e.status in DOCUMENTED_REFUSALS, (seed, label, e.status, e.detail)
+            continue
+        outs = run_graph(g, rg.inputs)
+        check_against_oracle(rg.desc, rg.inputs, outs, rg.output_meta, names=[f"column seed {seed} {label} out {k}" for k in range(len(outs))], ref=ref)
+        again = run_graph(g, rg.inputs)                     # arrival counters back at zero; the same bits
+        assert all(np.array_equal(a.view(np.uint8), b.view(np.uint8)) for a, b in zip(outs, again)), (seed, label)
+        assert g.bounds_status == 0, (seed, label)
+        ran += 1
+        g.close()
+    assert ran >= 1, seed

@@ -47,3 +47,18 @@ def test_generated_graphs_are_valid_and_span_what_they_claim():
 def test_generation_is_reproducible(seed):
     a, b = rand_graphs.make(seed), rand_graphs.make(seed)
     assert a.desc == b.desc and all(np.array_equal(x, y) for x, y in zip(a.inputs, b.inputs))
+
+
+def test_generated_column_graphs_are_valid_and_lower():
+    """The second generator: reductions over a leading dimension with chains before and after."""
+    kernels, sliced = [], 0
+    for seed in range(150):
+        rg = rand_graphs.make_column(seed)
+        ref = E.evaluate(rg.desc, rg.inputs)
+        for r, (dt, dims) in zip(ref, rg.output_meta):
+            assert tuple(r.shape) == tuple(dims) and np.isfinite(np.asarray(r, dtype=np.float64)).all(), seed
+        g = pn.Graph(rg.desc, 0, pn.FLAG_PLAN_ONLY)
+        kernels.append(g.n_kernels)
+        sliced += any(k["slices"] > 1 for k in g.kernel_info)
+        assert any(pn.FAMILY_NAMES[k["family"]] == "column-reduce" for k in g.kernel_info), seed
+    assert sum(k == 1 for k in kernels) >= 140 and sliced >= 3      # nearly all one kernel; some cut the reduced dimension
