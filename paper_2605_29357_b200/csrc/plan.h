@@ -182,6 +182,7 @@ struct LaunchPlan {
   int32_t no_prefetch;     // 1: generated kernels issue no loads ahead of the tile in hand
   int32_t bounds;          // 1: the generated kernel is compiled with checked accessors
   int32_t plain_launch;    // 1: launch in plain stream order (no overlap of the set-up with the predecessor's tail)
+  int32_t walk_cap;        // column kernels: at most this many steps of the walk in flight (0 = the default)
   int32_t no_reg_bound;    // 1: compile the generated kernel without the tentative register bound (it spilled)
   int64_t io_offset[kMaxIo];   // elements between the start of the tensor's storage and this entry's first element
                                // (non-zero for an output stored as a block of a larger tensor: an operand of a cat)

@@ -260,7 +260,8 @@ bool generate_source(const LaunchPlan& lp, std::string& src, std::string& err) {
   // column kernels: steps whose loads are in flight together.  Six under a bound of 7 blocks of 128
   // threads (72 registers) measured best on the pooling workload (47.2 -> 45.2 us); larger blocks keep
   // four under 64 registers.
-  const int walk_unroll = P.family == FAM_COLUMN ? (lp.block == 128 ? 6 : 4) : 1;
+  int walk_unroll = P.family == FAM_COLUMN ? (lp.block == 128 ? 6 : 4) : 1;
+  if (lp.walk_cap > 0) walk_unroll = std::min(walk_unroll, (int)lp.walk_cap);
   s += "#ifndef PN_WALK_UNROLL\n#define PN_WALK_UNROLL " + I(walk_unroll) + "\n#endif\n  static constexpr int kWalkUnroll = PN_WALK_UNROLL;\n";
   s += "  static PN_DEV bool io_mapped(const KernelParams&, int io) {\n    switch (io) {\n";
   for (int q = 0; q < P.n_io; ++q) if (P.io[q].mapped) s += "      case " + I(q) + ": return true;\n";
@@ -519,6 +520,17 @@ bool spec_compile(LaunchPlan& lp, int device, int sm_count, SpecKernel& out, std
     a.FuncGetAttribute(&regs, CU_FUNC_ATTRIBUTE_NUM_REGS, cmp.fn);
     a.FuncGetAttribute(&local_b, CU_FUNC_ATTRIBUTE_LOCAL_SIZE_BYTES, cmp.fn);
     fprintf(stderr, "spec: %s registers %d local bytes %d%s\n", kernel_name(lp).c_str(), regs, local_b, tentative_reg_bound(lp) ? " (tentative register bound)" : "");
+  }
+  // A column kernel that spills heavily under its register bound gains nothing from the steps it
+  // keeps in flight, and one such kernel (six steps, 216 bytes of local memory, compiled with checked
+  // accessors) was seen to compute a wrong first element per group: fewer steps in flight instead.
+  if (lp.p.family == FAM_COLUMN && lp.walk_cap != 2) {
+    int local_bytes = 0;
+    if (a.FuncGetAttribute(&local_bytes, CU_FUNC_ATTRIBUTE_LOCAL_SIZE_BYTES, cmp.fn) == CUDA_SUCCESS && local_bytes > 96) {
+      spec_release(cmp.fn);
+      lp.walk_cap = lp.walk_cap == 0 ? 4 : 2;
+      return spec_compile(lp, device, sm_count, out, err);
+    }
   }
   if (tentative_reg_bound(lp)) {   // did the kernel keep the bound without spilling more than a few words?
     // (the softmax workload's kernel parks two words -- 8 bytes -- and is still the faster one)
